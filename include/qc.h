@@ -1,0 +1,197 @@
+/*
+ * qc.h -- C ABI of the Lazy Attention / Q Cache decode library (sm_100a).
+ *
+ * The library implements the decode-step attention of an MLLM decoder stack whose layers
+ * are either ordinary ("full") or lazy, as defined in the paper's section "Method":
+ *   - Eq. 2   decode attention of an ordinary layer over its KV cache plus the new token;
+ *   - section "Lazy Attention": a lazy block is one ordinary layer l_c followed by lazy
+ *     layers; the Q Cache holds the query of l_c;
+ *   - Eq. 6   GLA decode: Q = Q Cache, K = K cache of l_c, V = the lazy layer's own;
+ *   - Eq. 8   VLA decode: K = [own text K, visual K of l_c, own new k], V = own;
+ *   - section "Efficiency Analysis": what each layer stores (all V; ordinary layers all K;
+ *     VLA lazy layers text K only; GLA lazy layers no K) and the closed-form saving.
+ *
+ * Conventions common to every call
+ *   - Every function returns an int32 status (QC_OK == 0).  Nothing throws, aborts or prints.
+ *     On an error status the cache is unchanged and no output is written.
+ *   - "dev" pointers are CUDA device pointers on the context's device; "host" pointers are
+ *     ordinary host memory.  All device memory is owned by the caller: the pool and the
+ *     workspace are handed in at qc_alloc_cache and must outlive the cache.  The library
+ *     allocates no device memory.  It owns the qc_ctx / qc_cache host objects and a few KiB of
+ *     pinned host memory per cache.
+ *   - Kernels are launched asynchronously on the stream given to qc_init.  Device pointers
+ *     passed to a call must stay valid until that stream has executed the call.  Host arrays
+ *     (seq_ids, n_tokens, kind) are consumed before the call returns.
+ *   - bf16 tensors are dense, row-major in the index order written in brackets.
+ *   - A sequence id is an integer in [0, max_seqs).  The token axis of a sequence is kept as
+ *     two ordered streams, text and visual (the paper's "concatenation" simplification after
+ *     Eq. 8); generated tokens are text.
+ */
+#ifndef QC_H_
+#define QC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct qc_ctx qc_ctx;     /* device, stream, SM count */
+typedef struct qc_cache qc_cache; /* page tables, stream lengths, free list, Q Cache, plans */
+
+enum {
+  QC_OK = 0,
+  QC_ERR_INVALID_ARG = 1, /* null pointer, out-of-range id or size, misaligned pointer */
+  QC_ERR_UNSUPPORTED = 2, /* shape the kernels do not cover */
+  QC_ERR_OOM_PAGES = 3,   /* the pool has too few free pages for this call */
+  QC_ERR_STATE = 4,       /* lazy layer 0, decode on an unknown sequence, duplicate id, ... */
+  QC_ERR_CUDA = 5,        /* a CUDA runtime call failed */
+  QC_ERR_TIMEOUT = 6      /* a bounded wait inside a kernel ran out (device error word) */
+};
+
+enum { QC_LAYER_FULL = 0, QC_LAYER_LAZY = 1 };
+
+/* Which query scores which keys in a lazy layer (one mode per cache; the paper's overview
+ * states that a model is optimised for a single mode).
+ *   QC_MODE_VLA_QC  : text keys = own text K scored by the own q; visual keys = leader's
+ *                     visual K scored by the Q Cache (the leader's q of the same token).
+ *   QC_MODE_VLA_EQ8 : Eq. 8 as printed: the own q scores own text K and leader's visual K.
+ *   QC_MODE_GLA     : Eq. 6: the Q Cache scores all of the leader's K.
+ * V is always the lazy layer's own. */
+enum { QC_MODE_VLA_QC = 0, QC_MODE_VLA_EQ8 = 1, QC_MODE_GLA = 2 };
+
+/* Streams of one (layer, sequence), in allocation order. */
+enum { QC_STREAM_K_TEXT = 0, QC_STREAM_K_VISUAL = 1, QC_STREAM_V_TEXT = 2, QC_STREAM_V_VISUAL = 3 };
+
+enum { QC_KIND_TEXT = 0, QC_KIND_VISUAL = 1 };
+
+typedef struct qc_config {
+  int32_t n_layers;            /* 1..127 */
+  int32_t n_q_heads;           /* multiple of n_kv_heads; query head h reads KV head h / group */
+  int32_t n_kv_heads;
+  int32_t head_dim;            /* 64 or 128 */
+  int32_t page_size;           /* 16 = paged; 0 = contiguous: every stream owns a fixed extent of
+                                  the pool (no allocator, no OOM), index
+                                  ((layer*4 + stream)*max_seqs + seq) */
+  int32_t max_seqs;            /* 1..4096 */
+  int32_t max_tokens_per_seq;  /* bound on text tokens and on visual tokens of one sequence */
+  int64_t n_pages;             /* pool capacity in pages (paged mode); ignored when contiguous */
+  float softmax_scale;         /* 0 => 1/sqrt(head_dim) (Eq. 2) */
+  int32_t lazy_mode;           /* QC_MODE_* */
+  int32_t split_tokens;        /* keys per split-KV work item, a multiple of 16 in 16..512;
+                                  0 => 128.  Every stream is cut into ceil(len/split_tokens)
+                                  chunks whose partial results are merged by log-sum-exp. */
+  const uint8_t* layer_kind;   /* host, [n_layers], QC_LAYER_*; layer 0 must be FULL; copied */
+} qc_config;
+
+typedef struct qc_stats {
+  int64_t pages_total;            /* pool capacity in pages */
+  int64_t pages_in_use;
+  int64_t page_bytes;             /* bytes of one page: n_kv_heads * 16 * head_dim * 2 */
+  int64_t kv_bytes_stored;        /* token-exact bytes of K and V rows held */
+  int64_t kv_bytes_all_full;      /* token-exact bytes if every layer were ordinary */
+  int64_t kv_bytes_stored_paged;  /* pages_in_use * page_bytes */
+  int64_t kv_bytes_all_full_paged;/* page-rounded bytes if every layer were ordinary */
+  int64_t qcache_bytes;           /* bytes of the Q Cache buffer */
+  int64_t decode_steps;           /* qc_decode_step calls completed (enqueued) */
+  int64_t attend_launches;        /* launches of the attention kernel so far */
+  int32_t device_error;           /* 0, or the QC_ERR_* code the device error word holds */
+  int32_t n_active_seqs;
+} qc_stats;
+
+/* Per-step kernel timing (CUDA events on the library's stream), for roofline accounting. */
+typedef struct qc_profile {
+  int64_t steps;              /* decode steps covered */
+  double attend_ms;           /* summed duration of the attention (split-KV partial) kernel */
+  double step_ms;             /* summed duration of whole steps (setup+append+attend+merge) */
+  int64_t kv_bytes_read;      /* algorithmic K/V bytes those steps had to read: every stored
+                                 row of the listed sequences once, per step */
+  int64_t items;              /* split-KV work items executed */
+} qc_profile;
+
+/* Create a context on `device` that launches on `cuda_stream` (a cudaStream_t; NULL is the
+ * legacy default stream).  Host object only. */
+int32_t qc_init(int32_t device, void* cuda_stream, qc_ctx** out);
+
+/* Bytes the caller must provide for a cache of this configuration.  pool_bytes covers the
+ * K/V pages, workspace_bytes the page tables, Q Cache, split-KV partials, plans and staging. */
+int32_t qc_cache_bytes_required(const qc_config* cfg, size_t* pool_bytes, size_t* workspace_bytes);
+
+/* Build a cache over caller-owned device memory (both 256-byte aligned).  Page layout: one
+ * page holds 16 tokens of ONE tensor (K or V) for all KV heads, [n_kv_heads][16][head_dim] bf16.
+ * A lazy layer gets no visual-K pages (and in GLA no K pages at all): its reads go to the
+ * leader's pages.  The pool contents are not initialised. */
+int32_t qc_alloc_cache(qc_ctx* ctx, const qc_config* cfg, void* pool_dev, size_t pool_bytes,
+                       void* workspace_dev, size_t workspace_bytes, qc_cache** out);
+
+/* Append prompt tokens (Eq. 1: K and V of the prompt go to the KV cache).  Sequence seq_ids[i]
+ * receives n_tokens[i] tokens; `kind` (host, QC_KIND_*, concatenated per sequence in call
+ * order) routes each token to the text or the visual stream.  k_dev, v_dev:
+ * bf16 [n_layers][sum n_tokens][n_kv_heads][head_dim].  K rows that the mode does not store
+ * are ignored.  New sequences become active.  No attention is computed.  The call returns
+ * after the copies have been enqueued and the host arrays consumed. */
+int32_t qc_prefill_append(qc_cache* cache, int32_t n_seqs, const int32_t* seq_ids,
+                          const int32_t* n_tokens, const uint8_t* kind, const void* k_dev,
+                          const void* v_dev);
+
+/* One generated (text) token for each listed sequence through all layers (Eq. 2, 6, 8):
+ * appends k/v, refreshes the Q Cache from every ordinary layer's q, computes split-KV partial
+ * attention and merges the partials by log-sum-exp.
+ *   q_dev   bf16 [n_layers][n_seqs][n_q_heads][head_dim]
+ *   k_dev   bf16 [n_layers][n_seqs][n_kv_heads][head_dim]  (rows of GLA lazy layers ignored)
+ *   v_dev   bf16 [n_layers][n_seqs][n_kv_heads][head_dim]
+ *   out_dev bf16 [n_layers][n_seqs][n_q_heads][head_dim]
+ *   lse_out_dev  optional fp32 [n_layers][n_seqs][n_q_heads], natural-log sum of exp; may be NULL
+ * seq_ids (host) must be distinct active sequences.  The call is asynchronous. */
+int32_t qc_decode_step(qc_cache* cache, int32_t n_seqs, const int32_t* seq_ids, const void* q_dev,
+                       const void* k_dev, const void* v_dev, void* out_dev, float* lse_out_dev);
+
+/* Same step with HOST buffers of the same layouts: copies q, k, v to staging in the
+ * workspace, runs the step, copies out (and lse if not NULL) back and waits for the stream.
+ * Pinned host buffers make the copies asynchronous; pageable ones also work. */
+int32_t qc_decode_step_host(qc_cache* cache, int32_t n_seqs, const int32_t* seq_ids,
+                            const void* q_host, const void* k_host, const void* v_host,
+                            void* out_host, float* lse_out_host);
+
+/* Release a sequence: its pages return to the free list in reverse order of allocation. */
+int32_t qc_free_seq(qc_cache* cache, int32_t seq_id);
+
+/* Destroy a cache and/or a context (either may be NULL).  Waits for the stream first.
+ * Caller-owned device memory is not touched. */
+int32_t qc_free(qc_ctx* ctx, qc_cache* cache);
+
+/* Accounting for the "KV bytes saved" metric (section "Efficiency Analysis").  Also reads the
+ * device error word (this synchronises the stream). */
+int32_t qc_get_stats(qc_cache* cache, qc_stats* out);
+
+/* Page table of one stream, from the host mirror.  Writes up to `cap` page ids, the page
+ * count, the stream length in tokens and the layer that owns the pages: `layer` itself, the
+ * leader if the stream is an alias, -1 (and zero pages) if the sequence is not active. */
+int32_t qc_debug_page_table(const qc_cache* cache, int32_t layer, int32_t stream, int32_t seq_id,
+                            int32_t* page_ids, int32_t cap, int32_t* n_pages, int32_t* n_tokens,
+                            int32_t* owner_layer);
+
+/* Copy the Q Cache entry a lazy layer reads (its leader's latest queries) to the host:
+ * bf16 [max_seqs][n_q_heads][head_dim].  Synchronises the stream. */
+int32_t qc_debug_read_qcache(qc_cache* cache, int32_t layer, void* host_bf16);
+
+/* Copy one stored row (bf16 [head_dim]) of a stream to the host; aliases resolve to the
+ * leader's pages.  Synchronises the stream.  For tests of the append path. */
+int32_t qc_debug_read_row(qc_cache* cache, int32_t layer, int32_t stream, int32_t seq_id,
+                          int32_t token, int32_t kv_head, void* host_bf16);
+
+/* Tuning knobs (all optional).  key: "split_tokens" (as in qc_config), "layers_per_launch"
+ * (0 = one attention launch for the whole step; k>0 = one launch per k consecutive lazy
+ * blocks, in layer order), "profile" (1 = record CUDA events per step). */
+int32_t qc_set_option(qc_cache* cache, const char* key, int64_t value);
+
+/* Sum the recorded kernel times since the last call (synchronises), then reset them. */
+int32_t qc_get_profile(qc_cache* cache, qc_profile* out);
+
+const char* qc_status_string(int32_t status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QC_H_ */

@@ -1,0 +1,100 @@
+// Structures shared by the host runtime (qc_runtime.cu) and the kernels (qc_kernels.cu).
+// Not part of the public ABI.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace qc {
+
+constexpr int kPage = 16;      // tokens per page
+constexpr int kMaxCons = 4;    // V streams (output layers) one K sweep can feed
+constexpr int kMaxChunkPages = 32;
+
+// flags of Job / Item
+constexpr uint8_t kFlagShared = 1;      // one query scores for every consumer (same weights)
+constexpr int kFlagCachedShift = 4;     // bit (4 + x): consumer x's query is read from the Q Cache
+
+// layer flags
+constexpr uint8_t kLayerOwnsTextK = 1;
+constexpr uint8_t kLayerWritesQCache = 2;
+
+// One K sweep: the keys of (k_layer, stream) scored by up to kMaxCons queries, each set of
+// weights applied to the V stream of one output layer.
+struct Job {
+  uint8_t k_layer, stream, n_cons, flags;
+  uint8_t v_layer[kMaxCons];
+  uint8_t q_layer[kMaxCons];
+  uint32_t pad;
+};
+static_assert(sizeof(Job) == 16, "Job layout");
+
+// (job, sequence) of one step; built on the host.
+struct __align__(16) Seg {
+  int32_t job, seq_idx, seq_id, len;        // len: tokens in the stream after this step's append
+  int32_t item_base, n_chunks, slot_base, pad;
+};
+static_assert(sizeof(Seg) == 32, "Seg layout");
+
+// One split-KV work item: a chunk of pages of one (job, sequence, head).
+struct __align__(16) Item {
+  uint8_t k_layer, stream, n_cons, flags;
+  uint8_t v_layer[kMaxCons];
+  uint8_t q_layer[kMaxCons];
+  uint16_t seq_id, seq_idx;
+  uint16_t head, slot;
+  uint16_t first_page, n_pages;
+  uint16_t n_valid_last, kv_head;
+  uint32_t pad1;
+};
+static_assert(sizeof(Item) == 32, "Item layout");
+
+struct StepSeq {
+  int32_t seq_id, len_text, len_vis, n_slots;
+};
+
+struct Patch {
+  int32_t index, page;
+};
+
+// Kernel parameter block.
+struct Params {
+  // cache-lifetime
+  uint16_t* pool;          // bf16 pages
+  int32_t* table;          // [n_layers][4][max_seqs][max_pages]
+  uint16_t* qcache;        // bf16 [n_layers][max_seqs][hq][d]
+  float* part_acc;         // [n_layers][max_seqs][max_slots][hq][d]
+  float2* part_ml;         // [n_layers][max_seqs][max_slots][hq]  (max, sum) in the log2 domain
+  Item* items;
+  const Seg* segs;
+  const Job* jobs;
+  const StepSeq* seqs;
+  const Patch* patches;
+  const uint8_t* layer_flags;
+  int32_t* err;
+  int64_t n_pool_pages;    // bound for page ids (reads never leave the pool)
+  int32_t n_layers, hq, hkv, d, group, max_seqs, max_pages, max_slots, chunk_pages;
+  int32_t heads_per_item_dim;   // hq: one item per query head
+  float scale_log2;             // softmax scale * log2(e)
+  // per step
+  const uint16_t* q;
+  const uint16_t* k;
+  const uint16_t* v;
+  uint16_t* out;
+  float* lse;
+  int32_t n_seqs, n_segs, n_items, n_patches;
+  int32_t item_begin, item_end;      // range handled by one attention launch
+  int32_t layer_begin, layer_end;    // range handled by one merge launch
+};
+
+// launchers (qc_kernels.cu); all asynchronous on `stream`
+cudaError_t launch_setup(const Params& p, cudaStream_t stream);
+cudaError_t launch_append(const Params& p, cudaStream_t stream);
+cudaError_t launch_attend(const Params& p, int n_sms, cudaStream_t stream);
+cudaError_t launch_merge(const Params& p, cudaStream_t stream);
+cudaError_t launch_prefill_scatter(const Params& p, const int32_t* tok_seq, const int32_t* tok_stream,
+                                   const int32_t* tok_ord, int32_t n_tokens, int32_t tok_stride,
+                                   int32_t tok_offset, cudaStream_t stream);
+cudaError_t configure_kernels(int* attend_smem_bytes);
+
+}  // namespace qc

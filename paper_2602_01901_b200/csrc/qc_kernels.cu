@@ -1,0 +1,668 @@
+// CUDA kernels of the Lazy Attention decode path (sm_100a).
+//
+//   setup_kernel    applies this step's page-table patches and expands (job, sequence)
+//                   segments into split-KV work items
+//   append_kernel   writes the new token's k / v rows into the text streams and every
+//                   ordinary layer's q into the Q Cache
+//   attend_kernel   persistent split-KV partial attention: each warp is an independent
+//                   worker that streams K/V page tiles through its own shared-memory ring
+//                   with bulk asynchronous copies and keeps an online softmax in registers
+//   merge_kernel    log-sum-exp merge of the partials, bf16 output
+//   prefill_scatter_kernel  stores prompt K/V rows into their pages
+//
+// Attention arithmetic: scores are kept in the log2 domain (q is pre-multiplied by
+// scale * log2 e), accumulation is fp32, inputs and outputs are bf16.
+
+#include "qc_internal.h"
+
+#include <math.h>
+
+namespace qc {
+namespace {
+
+constexpr int kWarps = 8;
+constexpr int kThreads = kWarps * 32;
+constexpr int kRing = 6;                  // tiles in flight per warp
+constexpr uint32_t kSpinLimit = 1u << 22; // bounded mbarrier wait
+
+constexpr int kErrTimeout = 6;
+constexpr int kErrBadPage = 5;
+
+// ------------------------------------------------------------------------------------------
+// PTX helpers
+// ------------------------------------------------------------------------------------------
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void fence_mbar_init() {
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok;
+}
+// 1-D bulk copy global -> this CTA's shared memory, completion counted on an mbarrier.
+// Source, destination and size are multiples of 16 bytes by construction (whole page tiles).
+__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_u32(dst)),
+               "l"(src), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+
+__device__ __forceinline__ void bf16x8_to_f32(const uint4& r, float* f) {
+  f[0] = __uint_as_float(r.x << 16);
+  f[1] = __uint_as_float(r.x & 0xffff0000u);
+  f[2] = __uint_as_float(r.y << 16);
+  f[3] = __uint_as_float(r.y & 0xffff0000u);
+  f[4] = __uint_as_float(r.z << 16);
+  f[5] = __uint_as_float(r.z & 0xffff0000u);
+  f[6] = __uint_as_float(r.w << 16);
+  f[7] = __uint_as_float(r.w & 0xffff0000u);
+}
+
+__device__ __forceinline__ uint16_t f32_to_bf16_rne(float x) {
+  uint32_t u = __float_as_uint(x);
+  if ((u & 0x7fffffffu) > 0x7f800000u) return static_cast<uint16_t>((u >> 16) | 0x40);   // NaN
+  u += 0x7fffu + ((u >> 16) & 1u);
+  return static_cast<uint16_t>(u >> 16);
+}
+
+__device__ __forceinline__ size_t table_row(const Params& P, int layer, int stream, int seq_id) {
+  return ((static_cast<size_t>(layer) * 4 + stream) * P.max_seqs + seq_id) * P.max_pages;
+}
+
+// ------------------------------------------------------------------------------------------
+// setup: page-table patches + item expansion
+// ------------------------------------------------------------------------------------------
+
+__global__ void setup_kernel(Params P) {
+  const int b = blockIdx.x;
+  if (b >= P.n_segs) {   // patch blocks
+    const int i = (b - P.n_segs) * blockDim.x + threadIdx.x;
+    if (i < P.n_patches) P.table[P.patches[i].index] = P.patches[i].page;
+    return;
+  }
+  const Seg sg = P.segs[b];
+  const Job jb = P.jobs[sg.job];
+  const int n_heads = P.heads_per_item_dim;
+  const int total_pages = (sg.len + kPage - 1) / kPage;
+  const int n = sg.n_chunks * n_heads;
+  for (int t = threadIdx.x; t < n; t += blockDim.x) {
+    const int chunk = t / n_heads;
+    const int head = t - chunk * n_heads;
+    Item it;
+    it.k_layer = jb.k_layer;
+    it.stream = jb.stream;
+    it.n_cons = jb.n_cons;
+    it.flags = jb.flags;
+#pragma unroll
+    for (int x = 0; x < kMaxCons; ++x) {
+      it.v_layer[x] = jb.v_layer[x];
+      it.q_layer[x] = jb.q_layer[x];
+    }
+    it.seq_id = static_cast<uint16_t>(sg.seq_id);
+    it.seq_idx = static_cast<uint16_t>(sg.seq_idx);
+    it.head = static_cast<uint16_t>(head);
+    it.slot = static_cast<uint16_t>(sg.slot_base + chunk);
+    const int first = chunk * P.chunk_pages;
+    const int np = min(P.chunk_pages, total_pages - first);
+    it.first_page = static_cast<uint16_t>(first);
+    it.n_pages = static_cast<uint16_t>(np);
+    const bool last = (first + np == total_pages);
+    it.n_valid_last = static_cast<uint16_t>(last ? sg.len - (total_pages - 1) * kPage : kPage);
+    it.kv_head = static_cast<uint16_t>(head / P.group);
+    it.pad1 = 0;
+    P.items[sg.item_base + t] = it;
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// append: new token's k, v rows and the Q Cache refresh
+// ------------------------------------------------------------------------------------------
+
+__global__ void append_kernel(Params P) {
+  const int si = blockIdx.x;
+  const int layer = blockIdx.y;
+  const StepSeq sq = P.seqs[si];
+  const int pos = sq.len_text - 1;          // ordinal of the new token in the text stream
+  const int pg = pos / kPage, slot = pos % kPage;
+  const uint8_t lf = P.layer_flags[layer];
+  const int vec_per_row = P.d / 8;          // uint4 per head row
+  const int n_kv_vec = P.hkv * vec_per_row;
+  const size_t in_kv = (static_cast<size_t>(layer) * P.n_seqs + si) * P.hkv * P.d;
+
+  const int pid_v = P.table[table_row(P, layer, 2, sq.seq_id) + pg];
+  const int pid_k = (lf & kLayerOwnsTextK) ? P.table[table_row(P, layer, 0, sq.seq_id) + pg] : -1;
+  for (int e = threadIdx.x; e < n_kv_vec; e += blockDim.x) {
+    const int head = e / vec_per_row, j = e - head * vec_per_row;
+    const size_t src = in_kv + static_cast<size_t>(head) * P.d + j * 8;
+    const size_t dst_v = ((static_cast<size_t>(pid_v) * P.hkv + head) * kPage + slot) * P.d + j * 8;
+    *reinterpret_cast<uint4*>(P.pool + dst_v) = *reinterpret_cast<const uint4*>(P.v + src);
+    if (pid_k >= 0) {
+      const size_t dst_k = ((static_cast<size_t>(pid_k) * P.hkv + head) * kPage + slot) * P.d + j * 8;
+      *reinterpret_cast<uint4*>(P.pool + dst_k) = *reinterpret_cast<const uint4*>(P.k + src);
+    }
+  }
+  if (lf & kLayerWritesQCache) {
+    const int n_q_vec = P.hq * vec_per_row;
+    const size_t src0 = (static_cast<size_t>(layer) * P.n_seqs + si) * P.hq * P.d;
+    const size_t dst0 = (static_cast<size_t>(layer) * P.max_seqs + sq.seq_id) * P.hq * P.d;
+    for (int e = threadIdx.x; e < n_q_vec; e += blockDim.x)
+      reinterpret_cast<uint4*>(P.qcache + dst0)[e] = reinterpret_cast<const uint4*>(P.q + src0)[e];
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// prefill scatter
+// ------------------------------------------------------------------------------------------
+
+__global__ void prefill_scatter_kernel(Params P, const int32_t* tok_seq, const int32_t* tok_stream,
+                                       const int32_t* tok_ord, int32_t tok_stride, int32_t tok_offset) {
+  const int t = blockIdx.x;
+  const int layer = blockIdx.y;
+  const int seq = tok_seq[t], stream = tok_stream[t], ord = tok_ord[t];
+  const int pg = ord / kPage, slot = ord % kPage;
+  const uint8_t lf = P.layer_flags[layer];
+  // K of a lazy layer: visual rows are never kept; text rows only where the mode keeps them
+  const bool keep_k = (lf & kLayerWritesQCache) || (stream == 0 && (lf & kLayerOwnsTextK));
+  const int pid_v = P.table[table_row(P, layer, 2 + stream, seq) + pg];
+  const int pid_k = keep_k ? P.table[table_row(P, layer, stream, seq) + pg] : -1;
+  const int vec_per_row = P.d / 8;
+  const int n_vec = P.hkv * vec_per_row;
+  const size_t in = (static_cast<size_t>(layer) * tok_stride + tok_offset + t) * P.hkv * P.d;
+  for (int e = threadIdx.x; e < n_vec; e += blockDim.x) {
+    const int head = e / vec_per_row, j = e - head * vec_per_row;
+    const size_t src = in + static_cast<size_t>(head) * P.d + j * 8;
+    const size_t dst_v = ((static_cast<size_t>(pid_v) * P.hkv + head) * kPage + slot) * P.d + j * 8;
+    *reinterpret_cast<uint4*>(P.pool + dst_v) = *reinterpret_cast<const uint4*>(P.v + src);
+    if (pid_k >= 0) {
+      const size_t dst_k = ((static_cast<size_t>(pid_k) * P.hkv + head) * kPage + slot) * P.d + j * 8;
+      *reinterpret_cast<uint4*>(P.pool + dst_k) = *reinterpret_cast<const uint4*>(P.k + src);
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// attend: persistent split-KV partial attention, one independent worker per warp
+// ------------------------------------------------------------------------------------------
+
+template <int D>
+struct WarpCtx {
+  Item item;
+  int32_t pages[1 + kMaxCons][kMaxChunkPages];   // [0]: K pages, [1 + x]: V pages of consumer x
+  uint4 qraw[kMaxCons][D / 8];
+};
+
+struct WorkerState {
+  int n_my;            // items this worker owns
+  int cons_k;          // item being consumed
+  int iss_k;           // item being fetched (cons_k or cons_k + 1)
+  int iss_page, iss_which;
+  int iss_slot, cons_slot;
+  uint32_t cons_phase;
+  int in_flight;
+  bool dead;           // a bounded wait ran out: stop fetching, drain, leave
+};
+
+template <int D>
+__device__ __forceinline__ bool issue_one(WorkerState& st, const WarpCtx<D>* ctx, uint8_t* ring, uint64_t* full,
+                                          const Params& P, int lane) {
+  constexpr uint32_t kTile = kPage * D * 2;
+  if (st.dead || st.iss_k >= st.n_my || st.iss_k > st.cons_k + 1) return false;
+  const WarpCtx<D>& c = ctx[st.iss_k & 1];
+  const int n_cons = c.item.n_cons;
+  int pid = c.pages[st.iss_which][st.iss_page];
+  if (static_cast<uint32_t>(pid) >= static_cast<uint64_t>(P.n_pool_pages)) {   // never read outside the pool
+    if (lane == 0) atomicMax(P.err, kErrBadPage);
+    pid = 0;
+  }
+  if (lane == 0) {
+    const uint16_t* src = P.pool + (static_cast<size_t>(pid) * P.hkv + c.item.kv_head) * (kPage * D);
+    uint64_t* bar = &full[st.iss_slot];
+    fence_proxy_async();   // the slot's earlier generic-proxy reads precede this async write
+    mbar_expect_tx(bar, kTile);
+    bulk_g2s(ring + st.iss_slot * kTile, src, kTile, bar);
+  }
+  st.iss_slot = (st.iss_slot + 1 == kRing) ? 0 : st.iss_slot + 1;
+  st.in_flight++;
+  if (++st.iss_which > n_cons) {
+    st.iss_which = 0;
+    if (++st.iss_page == c.item.n_pages) {
+      st.iss_page = 0;
+      st.iss_k++;
+    }
+  }
+  return true;
+}
+
+template <int D>
+__device__ __forceinline__ void fill_ring(WorkerState& st, const WarpCtx<D>* ctx, uint8_t* ring, uint64_t* full,
+                                          const Params& P, int lane) {
+  while (st.in_flight < kRing) {
+    if (!issue_one<D>(st, ctx, ring, full, P, lane)) break;
+  }
+}
+
+// Wait until the oldest tile in flight has landed; returns its shared-memory address.
+template <int D>
+__device__ __forceinline__ const uint8_t* wait_tile(WorkerState& st, uint8_t* ring, uint64_t* full, const Params& P,
+                                                    int lane) {
+  constexpr uint32_t kTile = kPage * D * 2;
+  uint64_t* bar = &full[st.cons_slot];
+  uint32_t done = mbar_try_wait(bar, st.cons_phase);
+  for (uint32_t spin = 0; !done && spin < kSpinLimit; ++spin) done = mbar_try_wait(bar, st.cons_phase);
+  if (!done) {
+    if (lane == 0) atomicMax(P.err, kErrTimeout);
+    st.dead = true;
+  }
+  return ring + st.cons_slot * kTile;
+}
+
+__device__ __forceinline__ void release_tile(WorkerState& st) {
+  __syncwarp();
+  st.in_flight--;
+  if (++st.cons_slot == kRing) {
+    st.cons_slot = 0;
+    st.cons_phase ^= 1u;
+  }
+}
+
+// Fetch an item's descriptor, page ids and raw queries into the warp's context slot.
+template <int D>
+__device__ __forceinline__ void load_ctx(WarpCtx<D>& c, const Params& P, int item_idx, int lane) {
+  const uint4* ip = reinterpret_cast<const uint4*>(P.items + item_idx);
+  uint4 a = __ldg(ip), b = __ldg(ip + 1);
+  __syncwarp();
+  if (lane == 0) {
+    reinterpret_cast<uint4*>(&c.item)[0] = a;
+    reinterpret_cast<uint4*>(&c.item)[1] = b;
+  }
+  Item it;
+  reinterpret_cast<uint4*>(&it)[0] = a;
+  reinterpret_cast<uint4*>(&it)[1] = b;
+  if (lane < it.n_pages) {
+    c.pages[0][lane] = P.table[table_row(P, it.k_layer, it.stream, it.seq_id) + it.first_page + lane];
+    for (int x = 0; x < it.n_cons; ++x)
+      c.pages[1 + x][lane] = P.table[table_row(P, it.v_layer[x], 2 + it.stream, it.seq_id) + it.first_page + lane];
+  }
+  const int nq = (it.flags & kFlagShared) ? 1 : it.n_cons;
+  if (lane < D / 8) {
+    for (int x = 0; x < nq; ++x) {
+      const bool cached = (it.flags >> (kFlagCachedShift + x)) & 1;
+      const uint16_t* src =
+          cached ? P.qcache + ((static_cast<size_t>(it.q_layer[x]) * P.max_seqs + it.seq_id) * P.hq + it.head) * D
+                 : P.q + ((static_cast<size_t>(it.q_layer[x]) * P.n_seqs + it.seq_idx) * P.hq + it.head) * D;
+      c.qraw[x][lane] = reinterpret_cast<const uint4*>(src)[lane];
+    }
+  }
+  __syncwarp();
+}
+
+// One item: NQ queries score the K tiles, NV value streams are accumulated.
+// NQ == 1: every consumer shares the weights; NQ == NV: consumer x has its own query.
+template <int D, int NQ, int NV>
+__device__ __forceinline__ void process_item(WorkerState& st, const WarpCtx<D>* ctx, uint8_t* ring, uint64_t* full,
+                                             const Params& P, int lane) {
+  constexpr int EPL = D / 8;    // elements of a row held by one lane
+  constexpr int LPR = D / 64;   // 16-byte loads per lane per row
+  const WarpCtx<D>& c = ctx[st.cons_k & 1];
+  const int kg = lane >> 3;     // which of 4 keys of a pass
+  const int c8 = lane & 7;      // which 16-byte chunk of the row (and of its second half)
+
+  float qf[NQ][EPL];
+#pragma unroll
+  for (int x = 0; x < NQ; ++x) {
+#pragma unroll
+    for (int j = 0; j < LPR; ++j) {
+      const uint4 raw = c.qraw[x][c8 + 8 * j];
+      bf16x8_to_f32(raw, &qf[x][8 * j]);
+    }
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) qf[x][e] *= P.scale_log2;
+  }
+
+  float m[NQ], l[NQ], acc[NV][EPL];
+#pragma unroll
+  for (int x = 0; x < NQ; ++x) {
+    m[x] = -INFINITY;
+    l[x] = 0.f;
+  }
+#pragma unroll
+  for (int v = 0; v < NV; ++v)
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) acc[v][e] = 0.f;
+
+  const int n_pages = c.item.n_pages;
+  const int n_valid_last = c.item.n_valid_last;
+
+  for (int pg = 0; pg < n_pages && !st.dead; ++pg) {
+    const int nvalid = (pg == n_pages - 1) ? n_valid_last : kPage;
+    float p[NQ][4];
+    // ---- K tile: scores of 16 keys
+    {
+      const uint8_t* tile = wait_tile<D>(st, ring, full, P, lane);
+      if (st.dead) break;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int r = 4 * i + kg;
+        const uint4* row = reinterpret_cast<const uint4*>(tile + r * (D * 2));
+        float kf[EPL];
+#pragma unroll
+        for (int j = 0; j < LPR; ++j) bf16x8_to_f32(row[c8 + 8 * j], &kf[8 * j]);
+#pragma unroll
+        for (int x = 0; x < NQ; ++x) {
+          float a0 = 0.f, a1 = 0.f;
+#pragma unroll
+          for (int e = 0; e < EPL; e += 2) {
+            a0 = fmaf(kf[e], qf[x][e], a0);
+            a1 = fmaf(kf[e + 1], qf[x][e + 1], a1);
+          }
+          p[x][i] = a0 + a1;
+        }
+      }
+      release_tile(st);
+      fill_ring<D>(st, ctx, ring, full, P, lane);
+    }
+#pragma unroll
+    for (int x = 0; x < NQ; ++x) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        float s = p[x][i];
+        s += __shfl_xor_sync(0xffffffffu, s, 1);
+        s += __shfl_xor_sync(0xffffffffu, s, 2);
+        s += __shfl_xor_sync(0xffffffffu, s, 4);
+        p[x][i] = (4 * i + kg < nvalid) ? s : -INFINITY;
+      }
+      float tmax = fmaxf(fmaxf(p[x][0], p[x][1]), fmaxf(p[x][2], p[x][3]));
+      tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 8));
+      tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 16));
+      const float m_new = fmaxf(m[x], tmax);
+      const float corr = exp2f(m[x] - m_new);
+      float psum = 0.f;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        p[x][i] = exp2f(p[x][i] - m_new);
+        psum += p[x][i];
+      }
+      l[x] = l[x] * corr + psum;
+      m[x] = m_new;
+      if (corr != 1.f) {
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+          if (NQ == 1 || v == x) {
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) acc[v][e] *= corr;
+          }
+        }
+      }
+    }
+    // ---- V tiles: weighted sums for each consumer
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+      const uint8_t* tile = wait_tile<D>(st, ring, full, P, lane);
+      if (st.dead) break;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int r = 4 * i + kg;
+        if (r < nvalid) {
+          const uint4* row = reinterpret_cast<const uint4*>(tile + r * (D * 2));
+          float vf[EPL];
+#pragma unroll
+          for (int j = 0; j < LPR; ++j) bf16x8_to_f32(row[c8 + 8 * j], &vf[8 * j]);
+          const float pv = p[NQ == 1 ? 0 : v][i];
+#pragma unroll
+          for (int e = 0; e < EPL; ++e) acc[v][e] = fmaf(pv, vf[e], acc[v][e]);
+        }
+      }
+      release_tile(st);
+      fill_ring<D>(st, ctx, ring, full, P, lane);
+    }
+  }
+  if (st.dead) return;
+
+  // ---- partial results: sum over the 4 key groups, then lanes 0..7 store
+#pragma unroll
+  for (int x = 0; x < NQ; ++x) {
+    l[x] += __shfl_xor_sync(0xffffffffu, l[x], 8);
+    l[x] += __shfl_xor_sync(0xffffffffu, l[x], 16);
+  }
+#pragma unroll
+  for (int v = 0; v < NV; ++v) {
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) {
+      acc[v][e] += __shfl_xor_sync(0xffffffffu, acc[v][e], 8);
+      acc[v][e] += __shfl_xor_sync(0xffffffffu, acc[v][e], 16);
+    }
+  }
+  if (kg == 0) {
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+      const size_t row =
+          ((static_cast<size_t>(c.item.v_layer[v]) * P.max_seqs + c.item.seq_idx) * P.max_slots + c.item.slot) *
+              P.hq + c.item.head;
+      float* dst = P.part_acc + row * D;
+#pragma unroll
+      for (int j = 0; j < LPR; ++j) {
+        float4* d4 = reinterpret_cast<float4*>(dst + 64 * j + 8 * c8);
+        d4[0] = make_float4(acc[v][8 * j + 0], acc[v][8 * j + 1], acc[v][8 * j + 2], acc[v][8 * j + 3]);
+        d4[1] = make_float4(acc[v][8 * j + 4], acc[v][8 * j + 5], acc[v][8 * j + 6], acc[v][8 * j + 7]);
+      }
+      if (c8 == 0) P.part_ml[row] = make_float2(m[NQ == 1 ? 0 : v], l[NQ == 1 ? 0 : v]);
+    }
+  }
+}
+
+template <int D>
+__global__ void __launch_bounds__(kThreads, 1) attend_kernel(Params P) {
+  constexpr uint32_t kTile = kPage * D * 2;
+  extern __shared__ __align__(128) uint8_t smem[];
+  __shared__ __align__(8) uint64_t full_all[kWarps][kRing];
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  uint8_t* ring = smem + static_cast<size_t>(warp) * kRing * kTile;
+  WarpCtx<D>* ctx = reinterpret_cast<WarpCtx<D>*>(smem + static_cast<size_t>(kWarps) * kRing * kTile) + warp * 2;
+  uint64_t* full = full_all[warp];
+
+  if (lane == 0) {
+    for (int s = 0; s < kRing; ++s) mbar_init(&full[s], 1);
+    fence_mbar_init();
+  }
+  __syncthreads();
+
+  const int n_workers = gridDim.x * kWarps;
+  const int worker = blockIdx.x * kWarps + warp;   // consecutive warps take consecutive items
+  const int n_items = P.item_end - P.item_begin;
+  WorkerState st;
+  st.n_my = (worker < n_items) ? (n_items - worker + n_workers - 1) / n_workers : 0;
+  st.cons_k = 0;
+  st.iss_k = 0;
+  st.iss_page = st.iss_which = 0;
+  st.iss_slot = st.cons_slot = 0;
+  st.cons_phase = 0;
+  st.in_flight = 0;
+  st.dead = false;
+  if (st.n_my == 0) return;
+
+  auto item_index = [&](int k) { return P.item_begin + worker + k * n_workers; };
+  load_ctx<D>(ctx[0], P, item_index(0), lane);
+  if (st.n_my > 1) load_ctx<D>(ctx[1], P, item_index(1), lane);
+  fill_ring<D>(st, ctx, ring, full, P, lane);
+
+  for (int k = 0; k < st.n_my && !st.dead; ++k) {
+    const Item& it = ctx[k & 1].item;
+    const int nc = it.n_cons;
+    const bool shared = it.flags & kFlagShared;
+    if (nc == 1) process_item<D, 1, 1>(st, ctx, ring, full, P, lane);
+    else if (shared && nc == 2) process_item<D, 1, 2>(st, ctx, ring, full, P, lane);
+    else if (shared && nc == 3) process_item<D, 1, 3>(st, ctx, ring, full, P, lane);
+    else if (shared) process_item<D, 1, 4>(st, ctx, ring, full, P, lane);
+    else if (nc == 2) process_item<D, 2, 2>(st, ctx, ring, full, P, lane);
+    else if (nc == 3) process_item<D, 3, 3>(st, ctx, ring, full, P, lane);
+    else process_item<D, 4, 4>(st, ctx, ring, full, P, lane);
+    if (st.dead) break;
+    __syncwarp();
+    if (k + 2 < st.n_my) load_ctx<D>(ctx[k & 1], P, item_index(k + 2), lane);
+    st.cons_k = k + 1;
+    fill_ring<D>(st, ctx, ring, full, P, lane);
+  }
+
+  if (st.dead) {
+    // copies still in flight write into this CTA's shared memory: give them a bounded
+    // chance to land before the warp leaves
+    while (st.in_flight > 0) {
+      uint64_t* bar = &full[st.cons_slot];
+      uint32_t done = 0;
+      for (uint32_t spin = 0; !done && spin < kSpinLimit; ++spin) done = mbar_try_wait(bar, st.cons_phase);
+      st.in_flight--;
+      if (++st.cons_slot == kRing) {
+        st.cons_slot = 0;
+        st.cons_phase ^= 1u;
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// merge: log-sum-exp combination of the partials of one (layer, sequence, head) per warp
+// ------------------------------------------------------------------------------------------
+
+template <int D>
+__global__ void merge_kernel(Params P) {
+  constexpr int VPL = D / 32;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n_layers = P.layer_end - P.layer_begin;
+  const int idx = blockIdx.x * (blockDim.x >> 5) + warp;
+  if (idx >= n_layers * P.n_seqs * P.hq) return;
+  const int head = idx % P.hq;
+  const int si = (idx / P.hq) % P.n_seqs;
+  const int layer = P.layer_begin + idx / (P.hq * P.n_seqs);
+  const int n_slots = P.seqs[si].n_slots;
+  const size_t base = (static_cast<size_t>(layer) * P.max_seqs + si) * P.max_slots;
+
+  float mmax = -INFINITY;
+  for (int s = lane; s < n_slots; s += 32) mmax = fmaxf(mmax, P.part_ml[(base + s) * P.hq + head].x);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xffffffffu, mmax, o));
+
+  float lsum = 0.f;
+  float acc[VPL];
+#pragma unroll
+  for (int e = 0; e < VPL; ++e) acc[e] = 0.f;
+  for (int s = 0; s < n_slots; ++s) {
+    const size_t row = (base + s) * P.hq + head;
+    const float2 ml = P.part_ml[row];
+    const float w = exp2f(ml.x - mmax);
+    lsum = fmaf(ml.y, w, lsum);
+    const float* src = P.part_acc + row * D + lane * VPL;
+    if (VPL == 4) {
+      const float4 a = *reinterpret_cast<const float4*>(src);
+      acc[0] = fmaf(a.x, w, acc[0]);
+      acc[1] = fmaf(a.y, w, acc[1]);
+      acc[2 % VPL] = fmaf(a.z, w, acc[2 % VPL]);
+      acc[3 % VPL] = fmaf(a.w, w, acc[3 % VPL]);
+    } else {
+      const float2 a = *reinterpret_cast<const float2*>(src);
+      acc[0] = fmaf(a.x, w, acc[0]);
+      acc[1] = fmaf(a.y, w, acc[1]);
+    }
+  }
+  const float inv = 1.f / lsum;
+  const size_t orow = ((static_cast<size_t>(layer) * P.n_seqs + si) * P.hq + head);
+  uint16_t* dst = P.out + orow * D + lane * VPL;
+  if (VPL == 4) {
+    uint2 o;
+    o.x = f32_to_bf16_rne(acc[0] * inv) | (static_cast<uint32_t>(f32_to_bf16_rne(acc[1] * inv)) << 16);
+    o.y = f32_to_bf16_rne(acc[2 % VPL] * inv) | (static_cast<uint32_t>(f32_to_bf16_rne(acc[3 % VPL] * inv)) << 16);
+    *reinterpret_cast<uint2*>(dst) = o;
+  } else {
+    const uint32_t o = f32_to_bf16_rne(acc[0] * inv) | (static_cast<uint32_t>(f32_to_bf16_rne(acc[1] * inv)) << 16);
+    *reinterpret_cast<uint32_t*>(dst) = o;
+  }
+  if (P.lse != nullptr && lane == 0) P.lse[orow] = (mmax + log2f(lsum)) * 0.6931471805599453f;
+}
+
+template <int D>
+constexpr int attend_smem_bytes() {
+  return kWarps * kRing * kPage * D * 2 + kWarps * 2 * static_cast<int>(sizeof(WarpCtx<D>));
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------------
+// launchers
+// ------------------------------------------------------------------------------------------
+
+cudaError_t configure_kernels(int* attend_smem) {
+  cudaError_t e = cudaFuncSetAttribute(attend_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       attend_smem_bytes<128>());
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(attend_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, attend_smem_bytes<64>());
+  if (attend_smem) *attend_smem = attend_smem_bytes<128>();
+  return e;
+}
+
+cudaError_t launch_setup(const Params& p, cudaStream_t stream) {
+  const int blocks = p.n_segs + (p.n_patches + 255) / 256;
+  if (blocks == 0) return cudaSuccess;
+  setup_kernel<<<blocks, 256, 0, stream>>>(p);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_append(const Params& p, cudaStream_t stream) {
+  dim3 grid(p.n_seqs, p.n_layers);
+  append_kernel<<<grid, 128, 0, stream>>>(p);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_attend(const Params& p, int n_sms, cudaStream_t stream) {
+  const int n_items = p.item_end - p.item_begin;
+  if (n_items <= 0) return cudaSuccess;
+  const int grid = min(n_sms, (n_items + kWarps - 1) / kWarps);
+  if (p.d == 128)
+    attend_kernel<128><<<grid, kThreads, attend_smem_bytes<128>(), stream>>>(p);
+  else
+    attend_kernel<64><<<grid, kThreads, attend_smem_bytes<64>(), stream>>>(p);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_merge(const Params& p, cudaStream_t stream) {
+  const int n = (p.layer_end - p.layer_begin) * p.n_seqs * p.hq;
+  if (n <= 0) return cudaSuccess;
+  const int warps_per_block = 8;
+  const int blocks = (n + warps_per_block - 1) / warps_per_block;
+  if (p.d == 128)
+    merge_kernel<128><<<blocks, warps_per_block * 32, 0, stream>>>(p);
+  else
+    merge_kernel<64><<<blocks, warps_per_block * 32, 0, stream>>>(p);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_prefill_scatter(const Params& p, const int32_t* tok_seq, const int32_t* tok_stream,
+                                   const int32_t* tok_ord, int32_t n_tokens, int32_t tok_stride,
+                                   int32_t tok_offset, cudaStream_t stream) {
+  if (n_tokens <= 0) return cudaSuccess;
+  dim3 grid(n_tokens, p.n_layers);
+  prefill_scatter_kernel<<<grid, 128, 0, stream>>>(p, tok_seq, tok_stream, tok_ord, tok_stride, tok_offset);
+  return cudaGetLastError();
+}
+
+}  // namespace qc

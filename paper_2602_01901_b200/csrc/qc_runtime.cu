@@ -1,0 +1,869 @@
+// Host runtime behind the C ABI of include/qc.h: context, cache object, paged allocator,
+// page tables, per-step planning and kernel launches.  No device memory is allocated here:
+// everything lives in the pool and the workspace the caller hands to qc_alloc_cache.
+
+#include "../../include/qc.h"
+#include "qc_internal.h"
+
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+using namespace qc;
+
+namespace {
+
+constexpr int kStageSlots = 8;       // pinned step-descriptor ring
+constexpr int kMaxProfileSteps = 16384;
+constexpr int kPrefillBatchTokens = 1 << 16;
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct SeqState {
+  bool active = false;
+  int32_t len_text = 0, len_vis = 0;
+  std::vector<int32_t> alloc_order;
+};
+
+// One attention launch: a run of consecutive lazy blocks.
+struct LaunchGroup {
+  int job_begin, job_end, layer_begin, layer_end;
+};
+
+struct Layout {   // byte offsets into the workspace
+  size_t table, layer_flags, jobs, qcache, part_acc, part_ml, items, step, err, stage_q, stage_k, stage_v,
+      stage_out, stage_lse, tok, total;
+  size_t step_seqs, step_patches, step_segs, step_bytes;   // offsets inside the step block
+};
+
+}  // namespace
+
+struct qc_ctx {
+  int device = 0;
+  cudaStream_t stream = nullptr;
+  int n_sms = 0;
+};
+
+struct qc_cache {
+  qc_ctx* ctx = nullptr;
+  qc_config cfg{};
+  std::vector<uint8_t> kind;
+  std::vector<int> leader;
+  std::vector<uint8_t> layer_flags;
+  int D = 0, hq = 0, hkv = 0, group = 0;
+  bool paged = true;
+  int max_pages = 0;       // per stream
+  int chunk_pages = 0, min_chunk_pages = 0, max_slots = 0;
+  int64_t n_pool_pages = 0;
+  int layers_per_launch = 0;
+  float scale = 0.f;
+
+  uint8_t* ws = nullptr;
+  uint16_t* pool = nullptr;
+  Layout lay{};
+  size_t max_items = 0, max_segs = 0, max_patches = 0;
+
+  std::vector<int32_t> table;          // host mirror
+  std::vector<int32_t> free_stack;
+  std::vector<SeqState> seqs;
+  std::vector<Job> jobs;
+  std::vector<std::pair<int, int>> block_jobs;   // per lazy block: [job_begin, job_end)
+  std::vector<std::pair<int, int>> block_layers; // per lazy block: [layer_begin, layer_end)
+  int text_streams_per_seq = 0;        // pages a sequence needs when its text crosses a page
+
+  // pinned staging ring for step descriptors
+  uint8_t* pinned = nullptr;
+  cudaEvent_t stage_done[kStageSlots]{};
+  bool stage_used[kStageSlots]{};
+  int stage_next = 0;
+
+  // profiling
+  bool profile = false;
+  std::vector<cudaEvent_t> ev;         // 4 per step: step begin, attend begin, attend end, step end
+  int ev_steps = 0;
+  int64_t prof_bytes = 0, prof_items = 0;
+
+  int64_t decode_steps = 0, attend_launches = 0;
+};
+
+namespace {
+
+inline bool owns(const qc_cache* c, int layer, int stream) {
+  if (stream >= 2 || c->kind[layer] == QC_LAYER_FULL) return true;
+  if (stream == QC_STREAM_K_TEXT) return c->cfg.lazy_mode != QC_MODE_GLA;
+  return false;
+}
+
+inline size_t trow(const qc_cache* c, int layer, int stream, int seq) {
+  return ((static_cast<size_t>(layer) * 4 + stream) * c->cfg.max_seqs + seq) * c->max_pages;
+}
+
+int validate_config(const qc_config* cfg) {
+  if (!cfg || !cfg->layer_kind) return QC_ERR_INVALID_ARG;
+  if (cfg->n_layers < 1 || cfg->n_layers > 127) return QC_ERR_INVALID_ARG;
+  if (cfg->n_kv_heads < 1 || cfg->n_q_heads < 1 || cfg->n_q_heads % cfg->n_kv_heads) return QC_ERR_INVALID_ARG;
+  if (cfg->n_q_heads > 65535) return QC_ERR_INVALID_ARG;
+  if (cfg->head_dim != 64 && cfg->head_dim != 128) return QC_ERR_UNSUPPORTED;
+  if (cfg->page_size != 16 && cfg->page_size != 0) return QC_ERR_UNSUPPORTED;
+  if (cfg->max_seqs < 1 || cfg->max_seqs > 4096) return QC_ERR_INVALID_ARG;
+  if (cfg->max_tokens_per_seq < 1 || cfg->max_tokens_per_seq > (1 << 20) - 16) return QC_ERR_INVALID_ARG;
+  if (cfg->page_size == 16 && (cfg->n_pages < 1 || cfg->n_pages > 0x7fffffffLL)) return QC_ERR_INVALID_ARG;
+  if (cfg->lazy_mode < 0 || cfg->lazy_mode > 2) return QC_ERR_INVALID_ARG;
+  if (cfg->split_tokens != 0 &&
+      (cfg->split_tokens % 16 || cfg->split_tokens < 16 || cfg->split_tokens > 16 * kMaxChunkPages))
+    return QC_ERR_INVALID_ARG;
+  if (!(cfg->softmax_scale >= 0.f) || !std::isfinite(cfg->softmax_scale)) return QC_ERR_INVALID_ARG;
+  for (int l = 0; l < cfg->n_layers; ++l)
+    if (cfg->layer_kind[l] != QC_LAYER_FULL && cfg->layer_kind[l] != QC_LAYER_LAZY) return QC_ERR_INVALID_ARG;
+  if (cfg->layer_kind[0] != QC_LAYER_FULL) return QC_ERR_STATE;
+  return QC_OK;
+}
+
+// Jobs of the whole stack, lazy block by lazy block.
+void build_jobs(const qc_config* cfg, std::vector<Job>& jobs, std::vector<std::pair<int, int>>& block_jobs,
+                std::vector<std::pair<int, int>>& block_layers) {
+  const int N = cfg->n_layers;
+  int l = 0;
+  while (l < N) {
+    const int c = l;
+    int e = l + 1;
+    while (e < N && cfg->layer_kind[e] == QC_LAYER_LAZY) ++e;   // followers c+1 .. e-1
+    const int job0 = static_cast<int>(jobs.size());
+    auto shared_jobs = [&](int stream, bool cached) {
+      // the leader's query scores once; weights applied to the V of the leader and followers
+      for (int first = c; first < e; first += kMaxCons) {
+        Job j{};
+        j.k_layer = static_cast<uint8_t>(c);
+        j.stream = static_cast<uint8_t>(stream);
+        j.n_cons = static_cast<uint8_t>(std::min(kMaxCons, e - first));
+        j.flags = kFlagShared;
+        for (int x = 0; x < j.n_cons; ++x) {
+          j.v_layer[x] = static_cast<uint8_t>(first + x);
+          j.q_layer[x] = static_cast<uint8_t>(c);
+        }
+        if (cached && e - c > 1) j.flags |= static_cast<uint8_t>(1u << kFlagCachedShift);
+        jobs.push_back(j);
+      }
+    };
+    auto own_query_jobs_on_leader_keys = [&](int stream) {   // Eq. 8: own q on the leader's visual K
+      for (int first = c; first < e; first += kMaxCons) {
+        Job j{};
+        j.k_layer = static_cast<uint8_t>(c);
+        j.stream = static_cast<uint8_t>(stream);
+        j.n_cons = static_cast<uint8_t>(std::min(kMaxCons, e - first));
+        j.flags = (j.n_cons == 1) ? kFlagShared : 0;
+        for (int x = 0; x < j.n_cons; ++x) {
+          j.v_layer[x] = static_cast<uint8_t>(first + x);
+          j.q_layer[x] = static_cast<uint8_t>(first + x);
+        }
+        jobs.push_back(j);
+      }
+    };
+    auto own_jobs = [&](int stream) {   // every layer of the block: own q, own K, own V
+      for (int x = c; x < e; ++x) {
+        Job j{};
+        j.k_layer = static_cast<uint8_t>(x);
+        j.stream = static_cast<uint8_t>(stream);
+        j.n_cons = 1;
+        j.flags = kFlagShared;
+        j.v_layer[0] = static_cast<uint8_t>(x);
+        j.q_layer[0] = static_cast<uint8_t>(x);
+        jobs.push_back(j);
+      }
+    };
+    switch (cfg->lazy_mode) {
+      case QC_MODE_VLA_QC:
+        shared_jobs(1, true);
+        own_jobs(0);
+        break;
+      case QC_MODE_VLA_EQ8:
+        own_query_jobs_on_leader_keys(1);
+        own_jobs(0);
+        break;
+      default:   // GLA
+        shared_jobs(1, true);
+        shared_jobs(0, true);
+        break;
+    }
+    block_jobs.emplace_back(job0, static_cast<int>(jobs.size()));
+    block_layers.emplace_back(c, e);
+    l = e;
+  }
+}
+
+struct Sizes {
+  int D, hq, hkv, max_pages, chunk_pages, max_slots;
+  int64_t n_pool_pages;
+  size_t page_bytes, pool_bytes, max_items, max_segs, max_patches;
+  Layout lay;
+};
+
+int compute_sizes(const qc_config* cfg, Sizes* s) {
+  int st = validate_config(cfg);
+  if (st != QC_OK) return st;
+  s->D = cfg->head_dim;
+  s->hq = cfg->n_q_heads;
+  s->hkv = cfg->n_kv_heads;
+  s->max_pages = (cfg->max_tokens_per_seq + kPage - 1) / kPage;
+  const int split = cfg->split_tokens ? cfg->split_tokens : 128;
+  s->chunk_pages = split / kPage;
+  s->max_slots = 2 * ((s->max_pages + s->chunk_pages - 1) / s->chunk_pages);
+  s->page_bytes = static_cast<size_t>(s->hkv) * kPage * s->D * 2;
+  if (cfg->page_size == 0)
+    s->n_pool_pages = static_cast<int64_t>(cfg->n_layers) * 4 * cfg->max_seqs * s->max_pages;
+  else
+    s->n_pool_pages = cfg->n_pages;
+  if (s->n_pool_pages > 0x7fffffffLL) return QC_ERR_INVALID_ARG;
+  s->pool_bytes = static_cast<size_t>(s->n_pool_pages) * s->page_bytes;
+
+  std::vector<Job> jobs;
+  std::vector<std::pair<int, int>> bj, bl;
+  build_jobs(cfg, jobs, bj, bl);
+  const size_t chunks_per_stream = (s->max_pages + s->chunk_pages - 1) / s->chunk_pages;
+  s->max_segs = jobs.size() * cfg->max_seqs;
+  s->max_items = s->max_segs * chunks_per_stream * s->hq;
+  s->max_patches = static_cast<size_t>(cfg->n_layers) * 2 * cfg->max_seqs;
+
+  Layout& L = s->lay;
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    size_t o = off;
+    off = align_up(off + bytes, 256);
+    return o;
+  };
+  const size_t N = cfg->n_layers, S = cfg->max_seqs;
+  L.table = take(N * 4 * S * s->max_pages * sizeof(int32_t));
+  L.layer_flags = take(N);
+  L.jobs = take(jobs.size() * sizeof(Job));
+  L.qcache = take(N * S * s->hq * s->D * 2);
+  L.part_acc = take(N * S * s->max_slots * s->hq * s->D * sizeof(float));
+  L.part_ml = take(N * S * s->max_slots * s->hq * sizeof(float2));
+  L.items = take(s->max_items * sizeof(Item));
+  // step block: header-free arrays at fixed offsets
+  L.step_seqs = 0;
+  L.step_patches = align_up(L.step_seqs + S * sizeof(StepSeq), 16);
+  L.step_segs = align_up(L.step_patches + s->max_patches * sizeof(Patch), 16);
+  L.step_bytes = align_up(L.step_segs + s->max_segs * sizeof(Seg), 256);
+  L.step = take(L.step_bytes);
+  L.err = take(256);
+  L.stage_q = take(N * S * s->hq * s->D * 2);
+  L.stage_k = take(N * S * s->hkv * s->D * 2);
+  L.stage_v = take(N * S * s->hkv * s->D * 2);
+  L.stage_out = take(N * S * s->hq * s->D * 2);
+  L.stage_lse = take(N * S * s->hq * sizeof(float));
+  L.tok = take(static_cast<size_t>(kPrefillBatchTokens) * 3 * sizeof(int32_t));
+  L.total = off;
+  return QC_OK;
+}
+
+#define QC_CUDA(expr)                            \
+  do {                                           \
+    cudaError_t e__ = (expr);                    \
+    if (e__ != cudaSuccess) return QC_ERR_CUDA;  \
+  } while (0)
+
+Params base_params(const qc_cache* c) {
+  Params p{};
+  p.pool = c->pool;
+  p.table = reinterpret_cast<int32_t*>(c->ws + c->lay.table);
+  p.qcache = reinterpret_cast<uint16_t*>(c->ws + c->lay.qcache);
+  p.part_acc = reinterpret_cast<float*>(c->ws + c->lay.part_acc);
+  p.part_ml = reinterpret_cast<float2*>(c->ws + c->lay.part_ml);
+  p.items = reinterpret_cast<Item*>(c->ws + c->lay.items);
+  p.segs = reinterpret_cast<const Seg*>(c->ws + c->lay.step + c->lay.step_segs);
+  p.jobs = reinterpret_cast<const Job*>(c->ws + c->lay.jobs);
+  p.seqs = reinterpret_cast<const StepSeq*>(c->ws + c->lay.step + c->lay.step_seqs);
+  p.patches = reinterpret_cast<const Patch*>(c->ws + c->lay.step + c->lay.step_patches);
+  p.layer_flags = c->ws + c->lay.layer_flags;
+  p.err = reinterpret_cast<int32_t*>(c->ws + c->lay.err);
+  p.n_pool_pages = c->n_pool_pages;
+  p.n_layers = c->cfg.n_layers;
+  p.hq = c->hq;
+  p.hkv = c->hkv;
+  p.d = c->D;
+  p.group = c->group;
+  p.max_seqs = c->cfg.max_seqs;
+  p.max_pages = c->max_pages;
+  p.max_slots = c->max_slots;
+  p.chunk_pages = c->chunk_pages;
+  p.heads_per_item_dim = c->hq;
+  p.scale_log2 = c->scale * 1.4426950408889634f;
+  return p;
+}
+
+// Pop pages for `n_new` more pages of (layer, stream, seq); records them in the host mirror.
+void grow_stream(qc_cache* c, int layer, int stream, int seq, int have, int n_new, std::vector<Patch>* patches) {
+  for (int i = 0; i < n_new; ++i) {
+    const int32_t pid = c->free_stack.back();
+    c->free_stack.pop_back();
+    const size_t idx = trow(c, layer, stream, seq) + have + i;
+    c->table[idx] = pid;
+    c->seqs[seq].alloc_order.push_back(pid);
+    if (patches) patches->push_back(Patch{static_cast<int32_t>(idx), pid});
+  }
+}
+
+inline int pages_for(int tokens) { return (tokens + kPage - 1) / kPage; }
+
+int sync_and_check(qc_cache* c) {
+  QC_CUDA(cudaStreamSynchronize(c->ctx->stream));
+  return QC_OK;
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------------
+// C ABI
+// ------------------------------------------------------------------------------------------
+
+extern "C" {
+
+const char* qc_status_string(int32_t s) {
+  switch (s) {
+    case QC_OK: return "ok";
+    case QC_ERR_INVALID_ARG: return "invalid argument";
+    case QC_ERR_UNSUPPORTED: return "unsupported configuration";
+    case QC_ERR_OOM_PAGES: return "out of pages";
+    case QC_ERR_STATE: return "invalid state";
+    case QC_ERR_CUDA: return "CUDA error";
+    case QC_ERR_TIMEOUT: return "device wait timed out";
+    default: return "unknown status";
+  }
+}
+
+int32_t qc_init(int32_t device, void* cuda_stream, qc_ctx** out) {
+  if (!out || device < 0) return QC_ERR_INVALID_ARG;
+  *out = nullptr;
+  int n_dev = 0;
+  QC_CUDA(cudaGetDeviceCount(&n_dev));
+  if (device >= n_dev) return QC_ERR_INVALID_ARG;
+  QC_CUDA(cudaSetDevice(device));
+  cudaDeviceProp prop;
+  QC_CUDA(cudaGetDeviceProperties(&prop, device));
+  if (prop.major < 10) return QC_ERR_UNSUPPORTED;
+  int smem = 0;
+  QC_CUDA(configure_kernels(&smem));
+  if (static_cast<size_t>(smem) > prop.sharedMemPerBlockOptin) return QC_ERR_UNSUPPORTED;
+  qc_ctx* ctx = new (std::nothrow) qc_ctx();
+  if (!ctx) return QC_ERR_INVALID_ARG;
+  ctx->device = device;
+  ctx->stream = static_cast<cudaStream_t>(cuda_stream);
+  ctx->n_sms = prop.multiProcessorCount;
+  *out = ctx;
+  return QC_OK;
+}
+
+int32_t qc_cache_bytes_required(const qc_config* cfg, size_t* pool_bytes, size_t* workspace_bytes) {
+  Sizes s;
+  int st = compute_sizes(cfg, &s);
+  if (st != QC_OK) return st;
+  if (pool_bytes) *pool_bytes = s.pool_bytes;
+  if (workspace_bytes) *workspace_bytes = s.lay.total;
+  return QC_OK;
+}
+
+int32_t qc_alloc_cache(qc_ctx* ctx, const qc_config* cfg, void* pool_dev, size_t pool_bytes, void* workspace_dev,
+                       size_t workspace_bytes, qc_cache** out) {
+  if (!ctx || !out || !pool_dev || !workspace_dev) return QC_ERR_INVALID_ARG;
+  *out = nullptr;
+  Sizes s;
+  int st = compute_sizes(cfg, &s);
+  if (st != QC_OK) return st;
+  if (pool_bytes < s.pool_bytes || workspace_bytes < s.lay.total) return QC_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(pool_dev) & 255) || (reinterpret_cast<uintptr_t>(workspace_dev) & 255))
+    return QC_ERR_INVALID_ARG;
+  QC_CUDA(cudaSetDevice(ctx->device));
+
+  qc_cache* c = new (std::nothrow) qc_cache();
+  if (!c) return QC_ERR_INVALID_ARG;
+  c->ctx = ctx;
+  c->cfg = *cfg;
+  c->kind.assign(cfg->layer_kind, cfg->layer_kind + cfg->n_layers);
+  c->cfg.layer_kind = c->kind.data();
+  c->D = s.D;
+  c->hq = s.hq;
+  c->hkv = s.hkv;
+  c->group = s.hq / s.hkv;
+  c->paged = cfg->page_size == 16;
+  c->max_pages = s.max_pages;
+  c->chunk_pages = c->min_chunk_pages = s.chunk_pages;
+  c->max_slots = s.max_slots;
+  c->n_pool_pages = s.n_pool_pages;
+  c->scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / std::sqrt(static_cast<float>(s.D));
+  c->ws = static_cast<uint8_t*>(workspace_dev);
+  c->pool = static_cast<uint16_t*>(pool_dev);
+  c->lay = s.lay;
+  c->max_items = s.max_items;
+  c->max_segs = s.max_segs;
+  c->max_patches = s.max_patches;
+  c->leader.resize(cfg->n_layers);
+  c->layer_flags.resize(cfg->n_layers);
+  int last = 0;
+  c->text_streams_per_seq = 0;
+  for (int l = 0; l < cfg->n_layers; ++l) {
+    if (c->kind[l] == QC_LAYER_FULL) last = l;
+    c->leader[l] = last;
+    uint8_t f = 0;
+    if (owns(c, l, QC_STREAM_K_TEXT)) f |= kLayerOwnsTextK;
+    if (c->kind[l] == QC_LAYER_FULL) f |= kLayerWritesQCache;
+    c->layer_flags[l] = f;
+    c->text_streams_per_seq += 1 + (owns(c, l, QC_STREAM_K_TEXT) ? 1 : 0);
+  }
+  build_jobs(&c->cfg, c->jobs, c->block_jobs, c->block_layers);
+  c->seqs.resize(cfg->max_seqs);
+  c->table.assign(static_cast<size_t>(cfg->n_layers) * 4 * cfg->max_seqs * c->max_pages, -1);
+  if (c->paged) {
+    c->free_stack.resize(s.n_pool_pages);
+    for (int64_t i = 0; i < s.n_pool_pages; ++i) c->free_stack[i] = static_cast<int32_t>(s.n_pool_pages - 1 - i);
+  } else {
+    // contiguous: stream (layer, stream, seq) owns pages [extent*max_pages, (extent+1)*max_pages)
+    for (size_t i = 0; i < c->table.size(); ++i) c->table[i] = static_cast<int32_t>(i);
+  }
+
+  cudaStream_t stream = ctx->stream;
+  bool ok = cudaHostAlloc(reinterpret_cast<void**>(&c->pinned), kStageSlots * c->lay.step_bytes,
+                          cudaHostAllocDefault) == cudaSuccess;
+  for (int i = 0; ok && i < kStageSlots; ++i)
+    ok = cudaEventCreateWithFlags(&c->stage_done[i], cudaEventDisableTiming) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(c->ws + c->lay.table, c->table.data(), c->table.size() * sizeof(int32_t),
+                             cudaMemcpyHostToDevice, stream) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(c->ws + c->lay.layer_flags, c->layer_flags.data(), c->layer_flags.size(),
+                             cudaMemcpyHostToDevice, stream) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(c->ws + c->lay.jobs, c->jobs.data(), c->jobs.size() * sizeof(Job),
+                             cudaMemcpyHostToDevice, stream) == cudaSuccess;
+  ok = ok && cudaMemsetAsync(c->ws + c->lay.err, 0, 256, stream) == cudaSuccess;
+  ok = ok && cudaMemsetAsync(c->ws + c->lay.qcache, 0, c->lay.part_acc - c->lay.qcache, stream) == cudaSuccess;
+  ok = ok && cudaStreamSynchronize(stream) == cudaSuccess;
+  if (!ok) {
+    qc_free(nullptr, c);
+    return QC_ERR_CUDA;
+  }
+  *out = c;
+  return QC_OK;
+}
+
+int32_t qc_free(qc_ctx* ctx, qc_cache* cache) {
+  if (cache) {
+    if (cache->ctx) {
+      cudaSetDevice(cache->ctx->device);
+      cudaStreamSynchronize(cache->ctx->stream);
+    }
+    for (int i = 0; i < kStageSlots; ++i)
+      if (cache->stage_done[i]) cudaEventDestroy(cache->stage_done[i]);
+    for (cudaEvent_t e : cache->ev) cudaEventDestroy(e);
+    if (cache->pinned) cudaFreeHost(cache->pinned);
+    delete cache;
+  }
+  if (ctx) delete ctx;
+  return QC_OK;
+}
+
+int32_t qc_prefill_append(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, const int32_t* n_tokens,
+                          const uint8_t* kind, const void* k_dev, const void* v_dev) {
+  if (!c || n_seqs < 0 || (n_seqs > 0 && (!seq_ids || !n_tokens))) return QC_ERR_INVALID_ARG;
+  if (n_seqs == 0) return QC_OK;
+  if (!k_dev || !v_dev) return QC_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(k_dev) & 15) || (reinterpret_cast<uintptr_t>(v_dev) & 15)) return QC_ERR_INVALID_ARG;
+  const int N = c->cfg.n_layers;
+  // ---- validate and plan without touching the state
+  int64_t total = 0, need = 0;
+  std::vector<uint8_t> seen(c->cfg.max_seqs, 0);
+  std::vector<int32_t> add_t(n_seqs), add_v(n_seqs);
+  for (int i = 0; i < n_seqs; ++i) {
+    const int s = seq_ids[i];
+    if (s < 0 || s >= c->cfg.max_seqs || n_tokens[i] < 0) return QC_ERR_INVALID_ARG;
+    if (seen[s]) return QC_ERR_STATE;
+    seen[s] = 1;
+    if (n_tokens[i] > 0 && !kind) return QC_ERR_INVALID_ARG;
+    int nt = 0, nv = 0;
+    for (int t = 0; t < n_tokens[i]; ++t) {
+      const uint8_t kd = kind[total + t];
+      if (kd == QC_KIND_TEXT) ++nt;
+      else if (kd == QC_KIND_VISUAL) ++nv;
+      else return QC_ERR_INVALID_ARG;
+    }
+    add_t[i] = nt;
+    add_v[i] = nv;
+    const SeqState& st = c->seqs[s];
+    if (st.len_text + nt > c->cfg.max_tokens_per_seq || st.len_vis + nv > c->cfg.max_tokens_per_seq)
+      return QC_ERR_INVALID_ARG;
+    if (c->paged) {
+      const int dt = pages_for(st.len_text + nt) - pages_for(st.len_text);
+      const int dv = pages_for(st.len_vis + nv) - pages_for(st.len_vis);
+      for (int l = 0; l < N; ++l)
+        for (int stream = 0; stream < 4; ++stream)
+          if (owns(c, l, stream)) need += (stream & 1) ? dv : dt;
+    }
+    total += n_tokens[i];
+  }
+  if (total > 0x7fffffffLL) return QC_ERR_INVALID_ARG;
+  if (c->paged && need > static_cast<int64_t>(c->free_stack.size())) return QC_ERR_OOM_PAGES;
+  QC_CUDA(cudaSetDevice(c->ctx->device));
+  cudaStream_t stream = c->ctx->stream;
+
+  // ---- commit: pages (sequence -> layer -> stream order), token routing
+  std::vector<int32_t> tok_seq(total), tok_stream(total), tok_ord(total);
+  int64_t t0 = 0;
+  for (int i = 0; i < n_seqs; ++i) {
+    const int s = seq_ids[i];
+    SeqState& st = c->seqs[s];
+    if (c->paged) {
+      const int have_t = pages_for(st.len_text), have_v = pages_for(st.len_vis);
+      const int dt = pages_for(st.len_text + add_t[i]) - have_t;
+      const int dv = pages_for(st.len_vis + add_v[i]) - have_v;
+      for (int l = 0; l < N; ++l)
+        for (int sm = 0; sm < 4; ++sm)
+          if (owns(c, l, sm)) grow_stream(c, l, sm, s, (sm & 1) ? have_v : have_t, (sm & 1) ? dv : dt, nullptr);
+    }
+    int ot = st.len_text, ov = st.len_vis;
+    for (int t = 0; t < n_tokens[i]; ++t) {
+      const bool vis = kind[t0 + t] == QC_KIND_VISUAL;
+      tok_seq[t0 + t] = s;
+      tok_stream[t0 + t] = vis ? 1 : 0;
+      tok_ord[t0 + t] = vis ? ov++ : ot++;
+    }
+    st.len_text = ot;
+    st.len_vis = ov;
+    st.active = true;
+    t0 += n_tokens[i];
+  }
+  // the whole host mirror goes to the device (prefill is not the hot path)
+  if (c->paged)
+    QC_CUDA(cudaMemcpyAsync(c->ws + c->lay.table, c->table.data(), c->table.size() * sizeof(int32_t),
+                            cudaMemcpyHostToDevice, stream));
+  Params p = base_params(c);
+  p.k = static_cast<const uint16_t*>(k_dev);
+  p.v = static_cast<const uint16_t*>(v_dev);
+  int32_t* tok_dev = reinterpret_cast<int32_t*>(c->ws + c->lay.tok);
+  for (int64_t off = 0; off < total; off += kPrefillBatchTokens) {
+    const int n = static_cast<int>(std::min<int64_t>(kPrefillBatchTokens, total - off));
+    QC_CUDA(cudaMemcpyAsync(tok_dev, tok_seq.data() + off, n * sizeof(int32_t), cudaMemcpyHostToDevice, stream));
+    QC_CUDA(cudaMemcpyAsync(tok_dev + kPrefillBatchTokens, tok_stream.data() + off, n * sizeof(int32_t),
+                            cudaMemcpyHostToDevice, stream));
+    QC_CUDA(cudaMemcpyAsync(tok_dev + 2 * kPrefillBatchTokens, tok_ord.data() + off, n * sizeof(int32_t),
+                            cudaMemcpyHostToDevice, stream));
+    QC_CUDA(launch_prefill_scatter(p, tok_dev, tok_dev + kPrefillBatchTokens, tok_dev + 2 * kPrefillBatchTokens, n,
+                                   static_cast<int32_t>(total), static_cast<int32_t>(off), stream));
+    // the host vectors and the device token arrays are reused by the next batch
+    QC_CUDA(cudaStreamSynchronize(stream));
+  }
+  return QC_OK;
+}
+
+int32_t qc_decode_step(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, const void* q_dev, const void* k_dev,
+                       const void* v_dev, void* out_dev, float* lse_out_dev) {
+  if (!c || n_seqs < 0 || (n_seqs > 0 && !seq_ids)) return QC_ERR_INVALID_ARG;
+  if (n_seqs == 0) return QC_OK;
+  if (!q_dev || !k_dev || !v_dev || !out_dev) return QC_ERR_INVALID_ARG;
+  if (n_seqs > c->cfg.max_seqs) return QC_ERR_INVALID_ARG;
+  const void* ptrs[4] = {q_dev, k_dev, v_dev, out_dev};
+  for (const void* ptr : ptrs)
+    if (reinterpret_cast<uintptr_t>(ptr) & 15) return QC_ERR_INVALID_ARG;
+  const int N = c->cfg.n_layers;
+  // ---- validate, count pages
+  int64_t need = 0;
+  {
+    std::vector<uint8_t> seen(c->cfg.max_seqs, 0);
+    for (int i = 0; i < n_seqs; ++i) {
+      const int s = seq_ids[i];
+      if (s < 0 || s >= c->cfg.max_seqs) return QC_ERR_INVALID_ARG;
+      if (!c->seqs[s].active || seen[s]) return QC_ERR_STATE;
+      seen[s] = 1;
+      if (c->seqs[s].len_text + 1 > c->cfg.max_tokens_per_seq) return QC_ERR_INVALID_ARG;
+      if (c->paged && c->seqs[s].len_text % kPage == 0) need += c->text_streams_per_seq;
+    }
+  }
+  if (c->paged && need > static_cast<int64_t>(c->free_stack.size())) return QC_ERR_OOM_PAGES;
+  QC_CUDA(cudaSetDevice(c->ctx->device));
+  cudaStream_t stream = c->ctx->stream;
+
+  // ---- a pinned descriptor slot (wait if the copy that last used it has not run yet)
+  const int slot = c->stage_next;
+  c->stage_next = (c->stage_next + 1) % kStageSlots;
+  if (c->stage_used[slot]) QC_CUDA(cudaEventSynchronize(c->stage_done[slot]));
+  uint8_t* hb = c->pinned + static_cast<size_t>(slot) * c->lay.step_bytes;
+  StepSeq* h_seqs = reinterpret_cast<StepSeq*>(hb + c->lay.step_seqs);
+  Patch* h_patches = reinterpret_cast<Patch*>(hb + c->lay.step_patches);
+  Seg* h_segs = reinterpret_cast<Seg*>(hb + c->lay.step_segs);
+
+  // ---- page planning (sequence -> layer -> K_T, V_T) and lengths
+  int n_patches = 0;
+  std::vector<Patch> patches;
+  int64_t step_rows = 0;   // K/V rows the step has to read (for the profile)
+  for (int i = 0; i < n_seqs; ++i) {
+    const int s = seq_ids[i];
+    SeqState& st = c->seqs[s];
+    if (c->paged && st.len_text % kPage == 0) {
+      const int have = st.len_text / kPage;
+      for (int l = 0; l < N; ++l) {
+        if (owns(c, l, QC_STREAM_K_TEXT)) grow_stream(c, l, QC_STREAM_K_TEXT, s, have, 1, &patches);
+        grow_stream(c, l, QC_STREAM_V_TEXT, s, have, 1, &patches);
+      }
+    }
+    st.len_text += 1;
+    const int ncv = (pages_for(st.len_vis) + c->chunk_pages - 1) / c->chunk_pages;
+    const int nct = (pages_for(st.len_text) + c->chunk_pages - 1) / c->chunk_pages;
+    h_seqs[i] = StepSeq{s, st.len_text, st.len_vis, ncv + nct};
+  }
+  n_patches = static_cast<int>(patches.size());
+  if (n_patches) std::memcpy(h_patches, patches.data(), n_patches * sizeof(Patch));
+
+  // ---- segments, launch group by launch group
+  std::vector<LaunchGroup> groups;
+  {
+    const int nb = static_cast<int>(c->block_jobs.size());
+    const int per = c->layers_per_launch <= 0 ? nb : c->layers_per_launch;
+    for (int b = 0; b < nb; b += per) {
+      const int e = std::min(nb, b + per);
+      groups.push_back(LaunchGroup{c->block_jobs[b].first, c->block_jobs[e - 1].second, c->block_layers[b].first,
+                                   c->block_layers[e - 1].second});
+    }
+  }
+  int n_segs = 0, n_items = 0;
+  std::vector<std::pair<int, int>> group_items;
+  for (const LaunchGroup& g : groups) {
+    const int begin = n_items;
+    for (int j = g.job_begin; j < g.job_end; ++j) {
+      const Job& jb = c->jobs[j];
+      for (int i = 0; i < n_seqs; ++i) {
+        const StepSeq& sq = h_seqs[i];
+        const int len = jb.stream ? sq.len_vis : sq.len_text;
+        if (len == 0) continue;
+        const int nch = (pages_for(len) + c->chunk_pages - 1) / c->chunk_pages;
+        const int ncv = (pages_for(sq.len_vis) + c->chunk_pages - 1) / c->chunk_pages;
+        h_segs[n_segs++] = Seg{j, i, sq.seq_id, len, n_items, nch, jb.stream ? 0 : ncv, 0};
+        n_items += nch * c->hq;
+        step_rows += static_cast<int64_t>(len) * (1 + jb.n_cons);
+      }
+    }
+    group_items.emplace_back(begin, n_items);
+  }
+
+  // ---- enqueue
+  QC_CUDA(cudaMemcpyAsync(c->ws + c->lay.step, hb, c->lay.step_bytes, cudaMemcpyHostToDevice, stream));
+  QC_CUDA(cudaEventRecord(c->stage_done[slot], stream));
+  c->stage_used[slot] = true;
+
+  Params p = base_params(c);
+  p.q = static_cast<const uint16_t*>(q_dev);
+  p.k = static_cast<const uint16_t*>(k_dev);
+  p.v = static_cast<const uint16_t*>(v_dev);
+  p.out = static_cast<uint16_t*>(out_dev);
+  p.lse = lse_out_dev;
+  p.n_seqs = n_seqs;
+  p.n_segs = n_segs;
+  p.n_items = n_items;
+  p.n_patches = n_patches;
+
+  cudaEvent_t* ev = nullptr;
+  if (c->profile && c->ev_steps < kMaxProfileSteps) {
+    if (static_cast<int>(c->ev.size()) < 4 * (c->ev_steps + 1)) {
+      for (int i = 0; i < 4; ++i) {
+        cudaEvent_t e;
+        QC_CUDA(cudaEventCreate(&e));
+        c->ev.push_back(e);
+      }
+    }
+    ev = &c->ev[4 * c->ev_steps];
+    QC_CUDA(cudaEventRecord(ev[0], stream));
+  }
+  QC_CUDA(launch_setup(p, stream));
+  QC_CUDA(launch_append(p, stream));
+  for (size_t gi = 0; gi < groups.size(); ++gi) {
+    p.item_begin = group_items[gi].first;
+    p.item_end = group_items[gi].second;
+    p.layer_begin = groups[gi].layer_begin;
+    p.layer_end = groups[gi].layer_end;
+    if (ev && gi == 0) QC_CUDA(cudaEventRecord(ev[1], stream));
+    QC_CUDA(launch_attend(p, c->ctx->n_sms, stream));
+    if (ev && gi + 1 == groups.size()) QC_CUDA(cudaEventRecord(ev[2], stream));
+    QC_CUDA(launch_merge(p, stream));
+    c->attend_launches++;
+  }
+  if (ev) {
+    QC_CUDA(cudaEventRecord(ev[3], stream));
+    c->ev_steps++;
+    c->prof_bytes += step_rows * c->hkv * c->D * 2;
+    c->prof_items += n_items;
+  }
+  c->decode_steps++;
+  return QC_OK;
+}
+
+int32_t qc_decode_step_host(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, const void* q_host,
+                            const void* k_host, const void* v_host, void* out_host, float* lse_out_host) {
+  if (!c || n_seqs < 0) return QC_ERR_INVALID_ARG;
+  if (n_seqs == 0) return QC_OK;
+  if (!q_host || !k_host || !v_host || !out_host || n_seqs > c->cfg.max_seqs) return QC_ERR_INVALID_ARG;
+  QC_CUDA(cudaSetDevice(c->ctx->device));
+  cudaStream_t stream = c->ctx->stream;
+  const size_t N = c->cfg.n_layers;
+  const size_t qb = N * n_seqs * c->hq * c->D * 2, kb = N * n_seqs * c->hkv * c->D * 2;
+  uint8_t* dq = c->ws + c->lay.stage_q;
+  uint8_t* dk = c->ws + c->lay.stage_k;
+  uint8_t* dv = c->ws + c->lay.stage_v;
+  uint8_t* dout = c->ws + c->lay.stage_out;
+  float* dlse = reinterpret_cast<float*>(c->ws + c->lay.stage_lse);
+  QC_CUDA(cudaMemcpyAsync(dq, q_host, qb, cudaMemcpyHostToDevice, stream));
+  QC_CUDA(cudaMemcpyAsync(dk, k_host, kb, cudaMemcpyHostToDevice, stream));
+  QC_CUDA(cudaMemcpyAsync(dv, v_host, kb, cudaMemcpyHostToDevice, stream));
+  int st = qc_decode_step(c, n_seqs, seq_ids, dq, dk, dv, dout, lse_out_host ? dlse : nullptr);
+  if (st != QC_OK) {
+    cudaStreamSynchronize(stream);
+    return st;
+  }
+  QC_CUDA(cudaMemcpyAsync(out_host, dout, qb, cudaMemcpyDeviceToHost, stream));
+  if (lse_out_host)
+    QC_CUDA(cudaMemcpyAsync(lse_out_host, dlse, N * n_seqs * c->hq * sizeof(float), cudaMemcpyDeviceToHost, stream));
+  QC_CUDA(cudaStreamSynchronize(stream));
+  return QC_OK;
+}
+
+int32_t qc_free_seq(qc_cache* c, int32_t seq_id) {
+  if (!c || seq_id < 0 || seq_id >= c->cfg.max_seqs) return QC_ERR_INVALID_ARG;
+  SeqState& st = c->seqs[seq_id];
+  if (!st.active) return QC_ERR_STATE;
+  if (c->paged) {
+    for (auto it = st.alloc_order.rbegin(); it != st.alloc_order.rend(); ++it) c->free_stack.push_back(*it);
+    for (int l = 0; l < c->cfg.n_layers; ++l)
+      for (int sm = 0; sm < 4; ++sm) {
+        const size_t r = trow(c, l, sm, seq_id);
+        std::fill(c->table.begin() + r, c->table.begin() + r + c->max_pages, -1);
+      }
+  }
+  st = SeqState();
+  return QC_OK;
+}
+
+int32_t qc_get_stats(qc_cache* c, qc_stats* out) {
+  if (!c || !out) return QC_ERR_INVALID_ARG;
+  std::memset(out, 0, sizeof(*out));
+  const int N = c->cfg.n_layers;
+  const int64_t row = static_cast<int64_t>(c->hkv) * c->D * 2;
+  out->page_bytes = row * kPage;
+  out->pages_total = c->n_pool_pages;
+  int64_t rows = 0, rows_full = 0, pages = 0, pages_full = 0;
+  for (const SeqState& st : c->seqs) {
+    if (!st.active) continue;
+    out->n_active_seqs++;
+    for (int l = 0; l < N; ++l)
+      for (int sm = 0; sm < 4; ++sm) {
+        const int len = (sm & 1) ? st.len_vis : st.len_text;
+        if (owns(c, l, sm)) {
+          rows += len;
+          pages += pages_for(len);
+        }
+        rows_full += len;
+        pages_full += pages_for(len);
+      }
+  }
+  out->pages_in_use = c->paged ? c->n_pool_pages - static_cast<int64_t>(c->free_stack.size()) : pages;
+  out->kv_bytes_stored = rows * row;
+  out->kv_bytes_all_full = rows_full * row;
+  out->kv_bytes_stored_paged = pages * out->page_bytes;
+  out->kv_bytes_all_full_paged = pages_full * out->page_bytes;
+  out->qcache_bytes = static_cast<int64_t>(N) * c->cfg.max_seqs * c->hq * c->D * 2;
+  out->decode_steps = c->decode_steps;
+  out->attend_launches = c->attend_launches;
+  QC_CUDA(cudaSetDevice(c->ctx->device));
+  int32_t err = 0;
+  QC_CUDA(cudaMemcpyAsync(&err, c->ws + c->lay.err, sizeof(err), cudaMemcpyDeviceToHost, c->ctx->stream));
+  QC_CUDA(cudaStreamSynchronize(c->ctx->stream));
+  out->device_error = err;
+  return QC_OK;
+}
+
+int32_t qc_debug_page_table(const qc_cache* c, int32_t layer, int32_t stream, int32_t seq_id, int32_t* page_ids,
+                            int32_t cap, int32_t* n_pages, int32_t* n_tokens, int32_t* owner_layer) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers || stream < 0 || stream > 3 || seq_id < 0 ||
+      seq_id >= c->cfg.max_seqs || cap < 0 || (cap > 0 && !page_ids))
+    return QC_ERR_INVALID_ARG;
+  const SeqState& st = c->seqs[seq_id];
+  int owner = -1, np = 0, nt = 0;
+  if (st.active) {
+    owner = owns(c, layer, stream) ? layer : c->leader[layer];
+    nt = (stream & 1) ? st.len_vis : st.len_text;
+    np = pages_for(nt);
+    const size_t r = trow(c, owner, stream, seq_id);
+    for (int i = 0; i < np && i < cap; ++i) page_ids[i] = c->table[r + i];
+  }
+  if (n_pages) *n_pages = np;
+  if (n_tokens) *n_tokens = nt;
+  if (owner_layer) *owner_layer = owner;
+  return QC_OK;
+}
+
+int32_t qc_debug_read_qcache(qc_cache* c, int32_t layer, void* host_bf16) {
+  if (!c || !host_bf16 || layer < 0 || layer >= c->cfg.n_layers) return QC_ERR_INVALID_ARG;
+  QC_CUDA(cudaSetDevice(c->ctx->device));
+  const size_t bytes = static_cast<size_t>(c->cfg.max_seqs) * c->hq * c->D * 2;
+  const uint8_t* src = c->ws + c->lay.qcache + static_cast<size_t>(c->leader[layer]) * bytes;
+  QC_CUDA(cudaMemcpyAsync(host_bf16, src, bytes, cudaMemcpyDeviceToHost, c->ctx->stream));
+  return sync_and_check(c);
+}
+
+int32_t qc_debug_read_row(qc_cache* c, int32_t layer, int32_t stream, int32_t seq_id, int32_t token,
+                          int32_t kv_head, void* host_bf16) {
+  if (!c || !host_bf16 || layer < 0 || layer >= c->cfg.n_layers || stream < 0 || stream > 3 || seq_id < 0 ||
+      seq_id >= c->cfg.max_seqs || kv_head < 0 || kv_head >= c->hkv)
+    return QC_ERR_INVALID_ARG;
+  const SeqState& st = c->seqs[seq_id];
+  if (!st.active) return QC_ERR_STATE;
+  const int len = (stream & 1) ? st.len_vis : st.len_text;
+  if (token < 0 || token >= len) return QC_ERR_INVALID_ARG;
+  const int owner = owns(c, layer, stream) ? layer : c->leader[layer];
+  const int32_t pid = c->table[trow(c, owner, stream, seq_id) + token / kPage];
+  if (pid < 0 || pid >= c->n_pool_pages) return QC_ERR_STATE;
+  const size_t off = ((static_cast<size_t>(pid) * c->hkv + kv_head) * kPage + token % kPage) * c->D;
+  QC_CUDA(cudaSetDevice(c->ctx->device));
+  QC_CUDA(cudaMemcpyAsync(host_bf16, c->pool + off, c->D * 2, cudaMemcpyDeviceToHost, c->ctx->stream));
+  return sync_and_check(c);
+}
+
+int32_t qc_set_option(qc_cache* c, const char* key, int64_t value) {
+  if (!c || !key) return QC_ERR_INVALID_ARG;
+  const std::string k(key);
+  if (k == "split_tokens") {
+    if (value % 16 || value < 16 || value > 16 * kMaxChunkPages) return QC_ERR_INVALID_ARG;
+    const int cp = static_cast<int>(value / 16);
+    if (cp < c->min_chunk_pages) return QC_ERR_INVALID_ARG;   // the workspace was sized for the initial split
+    c->chunk_pages = cp;
+    return QC_OK;
+  }
+  if (k == "layers_per_launch") {
+    if (value < 0 || value > c->cfg.n_layers) return QC_ERR_INVALID_ARG;
+    c->layers_per_launch = static_cast<int>(value);
+    return QC_OK;
+  }
+  if (k == "profile") {
+    c->profile = value != 0;
+    return QC_OK;
+  }
+  return QC_ERR_INVALID_ARG;
+}
+
+int32_t qc_get_profile(qc_cache* c, qc_profile* out) {
+  if (!c || !out) return QC_ERR_INVALID_ARG;
+  std::memset(out, 0, sizeof(*out));
+  QC_CUDA(cudaSetDevice(c->ctx->device));
+  QC_CUDA(cudaStreamSynchronize(c->ctx->stream));
+  for (int s = 0; s < c->ev_steps; ++s) {
+    float a = 0.f, t = 0.f;
+    QC_CUDA(cudaEventElapsedTime(&a, c->ev[4 * s + 1], c->ev[4 * s + 2]));
+    QC_CUDA(cudaEventElapsedTime(&t, c->ev[4 * s + 0], c->ev[4 * s + 3]));
+    out->attend_ms += a;
+    out->step_ms += t;
+  }
+  out->steps = c->ev_steps;
+  out->kv_bytes_read = c->prof_bytes;
+  out->items = c->prof_items;
+  c->ev_steps = 0;
+  c->prof_bytes = 0;
+  c->prof_items = 0;
+  return QC_OK;
+}
+
+}  // extern "C"

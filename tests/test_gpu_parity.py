@@ -1,0 +1,324 @@
+"""GPU parity: the CUDA library through its C ABI against the fp64 oracle, same seeded inputs.
+
+Bars (written here, from the task's stated tolerances): every output element within 2e-2 of
+the oracle and relative L2 error <= 5e-3 (bf16 storage, fp32 accumulation); page tables,
+stream lengths, owner layers and Q Cache contents bit-exact.
+"""
+
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import paging as pg
+from oracle.lazy_attention import LazyAttentionOracle
+from paper_2602_01901_b200 import binding as qc
+from paper_2602_01901_b200 import workloads as W
+from paper_2602_01901_b200.session import Session, bits_of
+
+from parity_util import MAX_ABS, REL_L2, SampledOracle, assert_close, f64, full_oracle, step_schedule
+
+pytestmark = pytest.mark.gpu
+
+MODES = [qc.QC_MODE_VLA_QC, qc.QC_MODE_VLA_EQ8, qc.QC_MODE_GLA]
+MODE_IDS = ["vla_qc", "vla_eq8", "gla"]
+
+
+def _outputs(w, dev):
+    out = torch.empty((w.n_layers, w.batch, w.n_q_heads, w.head_dim), dtype=torch.bfloat16, device=dev)
+    lse = torch.empty((w.n_layers, w.batch, w.n_q_heads), dtype=torch.float32, device=dev)
+    return out, lse
+
+
+# ------------------------------------------------------------------------------------------
+# tiny: every step, every element, every mode (contiguous KV)
+# ------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("mode", MODES, ids=MODE_IDS)
+def test_tiny_every_step(mode):
+    w = W.get_workload("tiny")
+    s = Session.for_workload(w, lazy_mode=mode, poison_pool=True)
+    s.prefill_workload(w)
+    o = full_oracle(w, mode)
+    out, lse = _outputs(w, s.device)
+    ids = list(range(w.batch))
+    for step in range(w.decode_steps):
+        q, k, v = W.decode_qkv_torch(w, step, s.device)
+        s.decode_step(ids, q, k, v, out, lse)
+        qn, kn, vn = W.decode_qkv_np(w, step)
+        got, got_lse = bits_of(out), lse.cpu().numpy()
+        for b in range(w.batch):
+            ref, ref_lse = o.decode_step(b, f64(qn[:, b]), f64(kn[:, b]), f64(vn[:, b]))
+            for l in range(w.n_layers):
+                assert_close(got[l, b], ref[l], f"tiny step {step} layer {l}")
+            np.testing.assert_allclose(got_lse[:, b], ref_lse, atol=2e-3, rtol=0)
+        # Q Cache: the lazy layer reads exactly the leader's q bits
+        assert np.array_equal(s.read_qcache(1)[0], qn[0, 0])
+        # appended rows: own text K of the lazy layer (VLA) and V
+        pos = w.n_text_prompt + step
+        assert np.array_equal(s.read_row(1, qc.QC_STREAM_V_TEXT, 0, pos, 3), vn[1, 0, 3])
+        want_k = kn[0, 0, 3] if mode == qc.QC_MODE_GLA else kn[1, 0, 3]   # GLA aliases the leader's text K
+        assert np.array_equal(s.read_row(1, qc.QC_STREAM_K_TEXT, 0, pos, 3), want_k)
+    # contiguous layout: stream (layer, stream, seq) owns extent ((layer*4 + stream)*max_seqs + seq)
+    max_pages = (w.max_tokens + 15) // 16
+    ids_, n_tok, owner = s.page_table(1, qc.QC_STREAM_V_VISUAL, 0)
+    assert owner == 1 and n_tok == 576
+    assert ids_ == [((1 * 4 + 3) * 1 + 0) * max_pages + i for i in range(36)]
+    ids_, n_tok, owner = s.page_table(1, qc.QC_STREAM_K_VISUAL, 0)
+    assert owner == 0 and ids_[0] == ((0 * 4 + 1) * 1 + 0) * max_pages
+    st = s.stats()
+    assert st.device_error == 0
+    row = w.n_kv_heads * w.head_dim * 2
+    assert st.kv_bytes_stored == o.rows_stored() * row and st.kv_bytes_all_full == o.rows_all_full() * row
+    s.close()
+
+
+# ------------------------------------------------------------------------------------------
+# small paged case: ragged batch, GQA, several lazy-block shapes, split sizes, D in {64, 128}
+# ------------------------------------------------------------------------------------------
+
+def _small_workload(head_dim, group, layer_kind, index):
+    lazy = tuple(i for i, k in enumerate(layer_kind) if k)
+    return W.Workload(index, f"small{index}", len(layer_kind), 2 * group, 2, head_dim, 16, 3, 5, 150, 150, 22, 24, lazy)
+
+
+SMALL = [
+    # (head_dim, group, layer_kind, split_tokens)
+    (128, 1, [0, 1, 0, 1, 1], 64),
+    (128, 2, [0, 1, 1, 1, 1, 1, 0], 32),     # a block of six: more consumers than one sweep feeds
+    (64, 1, [0, 0, 1], 16),
+    (128, 4, [0, 1], 512),
+    (64, 3, [0, 1, 0, 1], 128),
+]
+
+
+@pytest.mark.parametrize("mode", MODES, ids=MODE_IDS)
+@pytest.mark.parametrize("case", range(len(SMALL)))
+def test_small_paged_ragged(mode, case):
+    head_dim, group, layer_kind, split = SMALL[case]
+    w = _small_workload(head_dim, group, layer_kind, 10 + case)
+    trunc = [w.n_prompt, 9, 70]      # sequence 1: text only (5 text + 4 visual dropped below), sequence 2: ragged
+    s = Session(w.n_layers, w.n_q_heads, w.n_kv_heads, head_dim, layer_kind, max_seqs=4, max_tokens_per_seq=256,
+                n_pages=w.n_layers * 4 * 3 * 17, lazy_mode=mode, split_tokens=split, poison_pool=True)
+    o = LazyAttentionOracle(w.n_layers, w.n_q_heads, w.n_kv_heads, head_dim, layer_kind, mode, n_seqs=3)
+    model = pg.PagedCacheModel(layer_kind, mode, 16, w.n_layers * 4 * 3 * 17, 4)
+    seq_ids = [2, 0, 3]              # library sequence ids differ from the batch index on purpose
+    for b, sid in enumerate(seq_ids):
+        kind, k, v = W.prefill_kv_np(w, b)
+        T = trunc[b]
+        kind, k, v = kind[:T].copy(), k[:, :T], v[:, :T]
+        if b == 1:
+            kind[:] = 0              # a sequence without any visual token
+        kt = torch.from_numpy(k.astype(np.int16)).view(torch.bfloat16).to(s.device).contiguous()
+        vt = torch.from_numpy(v.astype(np.int16)).view(torch.bfloat16).to(s.device).contiguous()
+        s.prefill_append([sid], [T], kind, kt, vt)
+        o.prefill_append(b, kind.tolist(), f64(k), f64(v))
+        model.prefill_append([sid], [int((kind == 0).sum())], [int((kind == 1).sum())])
+    _compare_tables(s, model, w.n_layers, seq_ids)
+    out = torch.empty((w.n_layers, 3, w.n_q_heads, head_dim), dtype=torch.bfloat16, device=s.device)
+    lse = torch.empty((w.n_layers, 3, w.n_q_heads), dtype=torch.float32, device=s.device)
+    for step in range(w.decode_steps):
+        qn, kn, vn = W.decode_qkv_np(w, step)
+        dev = lambda a: torch.from_numpy(a.astype(np.int16)).view(torch.bfloat16).to(s.device).contiguous()
+        s.decode_step(seq_ids, dev(qn), dev(kn), dev(vn), out, lse)
+        model.decode_step(seq_ids)
+        got, got_lse = bits_of(out), lse.cpu().numpy()
+        for b in range(3):
+            ref, ref_lse = o.decode_step(b, f64(qn[:, b]), f64(kn[:, b]), f64(vn[:, b]))
+            for l in range(w.n_layers):
+                assert_close(got[l, b], ref[l], f"case {case} step {step} seq {b} layer {l}")
+            np.testing.assert_allclose(got_lse[:, b], ref_lse, atol=2e-3, rtol=0)
+        if step in (0, 10, 11, w.decode_steps - 1):
+            _compare_tables(s, model, w.n_layers, seq_ids)
+    st = s.stats()
+    assert st.device_error == 0
+    assert st.pages_in_use == model.pages_in_use()
+    row = w.n_kv_heads * head_dim * 2
+    assert st.kv_bytes_stored == model.rows_stored() * row
+    assert st.kv_bytes_all_full == model.rows_all_full() * row
+    # freeing returns pages in the model's order: the next prefill must pop the same ids
+    s_free = seq_ids[0]
+    qc.qc_free_seq(s.cache, s_free)
+    model.free_seq(s_free)
+    kind, k, v = W.prefill_kv_np(w, 0)
+    kt = torch.from_numpy(k[:, :40].astype(np.int16)).view(torch.bfloat16).to(s.device).contiguous()
+    s.prefill_append([1], [40], kind[:40], kt, kt)
+    model.prefill_append([1], [int((kind[:40] == 0).sum())], [int((kind[:40] == 1).sum())])
+    _compare_tables(s, model, w.n_layers, [1, seq_ids[1], seq_ids[2], s_free])
+    s.close()
+
+
+def _compare_tables(s, model, n_layers, seq_ids):
+    for sid in seq_ids:
+        for l in range(n_layers):
+            for stream in range(4):
+                got = s.page_table(l, stream, sid)
+                want = model.page_table(l, stream, sid)
+                assert got == (want[0], want[1], want[2]), f"page table layer {l} stream {stream} seq {sid}"
+
+
+# ------------------------------------------------------------------------------------------
+# schedules and entry points that must not change the result
+# ------------------------------------------------------------------------------------------
+
+def test_launch_grouping_and_host_entry_give_identical_bits():
+    w = _small_workload(128, 1, [0, 1, 0, 0, 1, 1], 20)
+    results = []
+    for variant in ("one_launch", "per_block", "host_buffers"):
+        s = Session.for_workload(w, lazy_mode=qc.QC_MODE_VLA_QC, split_tokens=64)
+        s.prefill_workload(w)
+        if variant == "per_block":
+            s.set_option("layers_per_launch", 1)
+        out, lse = _outputs(w, s.device)
+        outs = []
+        for step in range(6):
+            q, k, v = W.decode_qkv_torch(w, step, s.device)
+            if variant == "host_buffers":
+                hq, hk, hv = q.cpu().pin_memory(), k.cpu().pin_memory(), v.cpu().pin_memory()
+                ho = torch.empty(out.shape, dtype=torch.bfloat16).pin_memory()
+                s.decode_step_host(list(range(w.batch)), hq, hk, hv, ho)
+                outs.append(ho.view(torch.int16).numpy().copy())
+            else:
+                s.decode_step(list(range(w.batch)), q, k, v, out, lse)
+                outs.append(out.view(torch.int16).cpu().numpy())
+        assert s.stats().device_error == 0
+        results.append(np.stack(outs))
+        s.close()
+    assert np.array_equal(results[0], results[1])
+    assert np.array_equal(results[0], results[2])
+
+
+def test_split_size_changes_only_rounding():
+    w = _small_workload(128, 1, [0, 1], 21)
+    o = full_oracle(w, qc.QC_MODE_VLA_QC)
+    qn, kn, vn = W.decode_qkv_np(w, 0)
+    refs = [o.decode_step(b, f64(qn[:, b]), f64(kn[:, b]), f64(vn[:, b]))[0] for b in range(w.batch)]
+    for split in (16, 48, 112, 512):
+        s = Session.for_workload(w, split_tokens=16)
+        s.set_option("split_tokens", split)
+        s.prefill_workload(w)
+        out, lse = _outputs(w, s.device)
+        q, k, v = W.decode_qkv_torch(w, 0, s.device)
+        s.decode_step(list(range(w.batch)), q, k, v, out, lse)
+        got = bits_of(out)
+        for b in range(w.batch):
+            for l in range(w.n_layers):
+                assert_close(got[l, b], refs[b][l], f"split {split} seq {b} layer {l}")
+        s.close()
+
+
+# ------------------------------------------------------------------------------------------
+# error behaviour: status codes, cache unchanged
+# ------------------------------------------------------------------------------------------
+
+def test_errors_leave_the_cache_unchanged():
+    w = _small_workload(128, 1, [0, 1], 22)
+    # lazy layer 0 is refused at allocation
+    with pytest.raises(qc.QcError) as e:
+        Session(2, 2, 2, 128, [1, 0], max_seqs=1, max_tokens_per_seq=64, n_pages=64)
+    assert e.value.status == qc.QC_ERR_STATE
+    # a pool with room for the prompt (177 tokens -> 2 text + 10 visual pages per stream) but not one more page
+    prompt_pages = (2 + 10) * 2 + (2 + 2 + 10)
+    s = Session(2, 2, 2, 128, [0, 1], max_seqs=2, max_tokens_per_seq=256, n_pages=prompt_pages + 2)
+    kind, k, v = W.prefill_kv_np(w, 0)
+    kt = torch.from_numpy(k.astype(np.int16)).view(torch.bfloat16).to(s.device).contiguous()
+    s.prefill_append([0], [len(kind)], kind, kt, kt)
+    out = torch.empty((2, 1, 2, 128), dtype=torch.bfloat16, device=s.device)
+    q, kk, vv = (t[:, :1].contiguous() for t in W.decode_qkv_torch(w, 0, s.device))
+    # unknown sequence, duplicate ids, bad id
+    for ids, status in (([1], qc.QC_ERR_STATE), ([0, 0], qc.QC_ERR_STATE), ([7], qc.QC_ERR_INVALID_ARG)):
+        with pytest.raises(qc.QcError) as e:
+            s.decode_step(ids, q, kk, vv, out)
+        assert e.value.status == status
+    before = [s.page_table(l, st, 0) for l in range(2) for st in range(4)]
+    # text length 27 -> steps at lengths 27..31 fit the last page; the step at length 32 needs 4 pages, 2 free
+    for step in range(5):
+        s.decode_step([0], q, kk, vv, out)
+    mid = [s.page_table(l, st, 0) for l in range(2) for st in range(4)]
+    with pytest.raises(qc.QcError) as e:
+        s.decode_step([0], q, kk, vv, out)
+    assert e.value.status == qc.QC_ERR_OOM_PAGES
+    assert [s.page_table(l, st, 0) for l in range(2) for st in range(4)] == mid
+    assert mid[0][1] == before[0][1] + 5
+    with pytest.raises(qc.QcError) as e:
+        s.prefill_append([1], [len(kind)], kind, kt, kt)
+    assert e.value.status == qc.QC_ERR_OOM_PAGES
+    assert s.page_table(0, 0, 1) == ([], 0, -1)
+    assert s.stats().device_error == 0
+    s.close()
+
+
+# ------------------------------------------------------------------------------------------
+# full-size configurations, launched as the benchmark launches them; sampled outputs
+# ------------------------------------------------------------------------------------------
+
+def _samples(w, n, rng):
+    lazy = list(w.lazy_layers)
+    fixed = [(0, 0, 0), (w.n_layers - 1, w.batch - 1, w.n_q_heads - 1), (lazy[0], 0, 1), (lazy[0] - 1, 0, 1),
+             (lazy[-1], w.batch - 1, 0), (1, w.batch // 2, w.n_q_heads // 2)]
+    out = list(dict.fromkeys(fixed))
+    while len(out) < n:
+        t = (int(rng.integers(w.n_layers)), int(rng.integers(w.batch)), int(rng.integers(w.n_q_heads)))
+        if t not in out:
+            out.append(t)
+    return out
+
+
+FULL_CASES = [
+    ("llava15_7b", qc.QC_MODE_VLA_QC, 40),
+    ("llava15_7b", qc.QC_MODE_VLA_EQ8, 16),
+    ("llava15_7b", qc.QC_MODE_GLA, 16),
+    ("llava_next_anyres", qc.QC_MODE_VLA_QC, 32),
+    ("qwen2vl_gqa", qc.QC_MODE_VLA_QC, 40),
+    ("long_video_pruned", qc.QC_MODE_VLA_QC, 24),
+]
+
+
+@pytest.mark.parametrize("name,mode,n_samples", FULL_CASES, ids=[f"{c[0]}-{MODE_IDS[c[1]]}" for c in FULL_CASES])
+def test_full_size_sampled(name, mode, n_samples):
+    w = W.get_workload(name)
+    rng = np.random.default_rng(w.seed)
+    samples = _samples(w, n_samples, rng)
+    oracles = [SampledOracle(w, mode, *t) for t in samples]
+    schedule = set(step_schedule(w.decode_steps))
+    s = Session.for_workload(w, lazy_mode=mode)
+    s.prefill_workload(w)
+    model = pg.PagedCacheModel(w.layer_kind().tolist(), mode, 16, s.cfg.n_pages, w.batch)
+    for b in range(w.batch):
+        model.prefill_append([b], [w.n_text_prompt], [w.n_visual_kept])
+    _compare_tables(s, model, w.n_layers, [0, w.batch - 1])
+    out, lse = _outputs(w, s.device)
+    ids = qc._i32_array(list(range(w.batch)))
+    li = torch.tensor([t[0] for t in samples], device=s.device)
+    bi = torch.tensor([t[1] for t in samples], device=s.device)
+    hi = torch.tensor([t[2] for t in samples], device=s.device)
+    worst = (0.0, 0.0)
+    for step in range(w.decode_steps):
+        q, k, v = W.decode_qkv_torch(w, step, s.device)
+        s.decode_step(ids, q, k, v, out, lse)
+        model.decode_step(list(range(w.batch)))
+        refs = [o.advance() for o in oracles]
+        if step in schedule:
+            got = bits_of(out[li, bi, hi])
+            got_lse = lse[li, bi, hi].cpu().numpy()
+            assert np.all(np.isfinite(f64(bits_of(out)))), f"step {step}: non-finite output somewhere"
+            for i, (ref, ref_lse) in enumerate(refs):
+                e, r = assert_close(got[i], ref, f"{name} step {step} sample {samples[i]}")
+                worst = (max(worst[0], e), max(worst[1], r))
+                assert abs(got_lse[i] - ref_lse) <= 2e-3
+    st = s.stats()
+    assert st.device_error == 0
+    assert st.pages_in_use == model.pages_in_use()
+    for sid in (0, w.batch // 2, w.batch - 1):
+        _compare_tables(s, model, w.n_layers, [sid])
+    # Q Cache after the last step: leader's q bits of that step
+    lazy_layer = w.lazy_layers[0]
+    q_last = W.decode_qkv_np(w, w.decode_steps - 1, layers=[lazy_layer - 1])[0][0]
+    assert np.array_equal(s.read_qcache(lazy_layer)[: w.batch], q_last)
+    # KV-saving metric: token-exact bytes against the integer model
+    row = w.n_kv_heads * w.head_dim * 2
+    assert st.kv_bytes_stored == model.rows_stored() * row
+    assert st.kv_bytes_all_full == model.rows_all_full() * row
+    print(f"{name} mode {mode}: worst max-abs {worst[0]:.3e} (bar {MAX_ABS}), worst rel-L2 {worst[1]:.3e} (bar {REL_L2})")
+    s.close()
