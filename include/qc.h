@@ -189,6 +189,43 @@ int32_t qc_set_option(qc_cache* cache, const char* key, int64_t value);
 /* Sum the recorded kernel times since the last call (synchronises), then reset them. */
 int32_t qc_get_profile(qc_cache* cache, qc_profile* out);
 
+/* ---- A call for callers that cannot allocate ------------------------------------------------
+ *
+ * The paper has no counterpart to this call; it exists for deployment reasons.  Everything
+ * above works on memory the caller allocates and hands over.  Some callers cannot do even
+ * that at the moment they need attention computed: a serving process whose device memory
+ * was partitioned at start-up and whose allocator is frozen afterwards, or code running
+ * inside another framework's callback where device allocation is forbidden.  For them
+ * qc_attend_static computes plain decode attention (Eq. 2) using only the tensors passed in
+ * plus a fixed scratch array that is part of the library image.
+ *
+ *   q_dev   bf16 [n_seqs][n_q_heads][head_dim]              one query token per sequence
+ *   k_dev   bf16 [n_seqs][n_tokens][n_kv_heads][head_dim]   keys, the new token's included
+ *   v_dev   bf16 [n_seqs][n_tokens][n_kv_heads][head_dim]
+ *   out_dev bf16 [n_seqs][n_q_heads][head_dim]
+ *   softmax_scale 0 => 1/sqrt(head_dim)
+ *
+ * The key axis is cut into QC_STATIC_SPLITS ranges whose partial softmax results are kept in
+ * the scratch array and merged by log-sum-exp.  The array holds QC_STATIC_MAX_ROWS *
+ * QC_STATIC_SPLITS * 130 floats (about 2 MiB) on every GPU that loads the library, for the
+ * life of the process.  Limits: n_seqs * n_q_heads <= QC_STATIC_MAX_ROWS, n_tokens <=
+ * QC_STATIC_MAX_TOKENS, head_dim 64 or 128; anything larger returns QC_ERR_INVALID_ARG and
+ * launches nothing.
+ *
+ * The call performs no device or pinned-host allocation and frees nothing.  Its first call
+ * on a device looks up the scratch array's device address (once per device); make that first
+ * call outside any stream capture.  All calls share the one array, and it keeps whatever
+ * the previous call left there: each call overwrites every entry it later reads, so nothing
+ * needs clearing, but two calls whose kernels overlap on the GPU (different streams, or
+ * different host threads) race on it.  Serialise them on one stream.  Asynchronous on
+ * `cuda_stream`; pointers must be 16-byte aligned. */
+#define QC_STATIC_MAX_ROWS 512
+#define QC_STATIC_SPLITS 8
+#define QC_STATIC_MAX_TOKENS 65536
+int32_t qc_attend_static(int32_t device, void* cuda_stream, const void* q_dev, const void* k_dev,
+                         const void* v_dev, void* out_dev, int32_t n_seqs, int32_t n_tokens,
+                         int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim, float softmax_scale);
+
 const char* qc_status_string(int32_t status);
 
 #ifdef __cplusplus

@@ -31,6 +31,7 @@ EXPORTS = (
     "qc_init", "qc_cache_bytes_required", "qc_alloc_cache", "qc_prefill_append", "qc_decode_step",
     "qc_decode_step_host", "qc_free_seq", "qc_free", "qc_get_stats", "qc_debug_page_table",
     "qc_debug_read_qcache", "qc_debug_read_row", "qc_set_option", "qc_get_profile", "qc_status_string",
+    "qc_attend_static",
 )
 
 
@@ -97,6 +98,7 @@ def load() -> C.CDLL:
         "qc_debug_read_row": [vp, i32, i32, i32, i32, i32, vp],
         "qc_set_option": [vp, C.c_char_p, i64],
         "qc_get_profile": [vp, C.POINTER(qc_profile)],
+        "qc_attend_static": [i32, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, C.c_float],
     }
     for name, args in sig.items():
         fn = getattr(lib, name)
@@ -211,3 +213,17 @@ def qc_get_profile(cache) -> qc_profile:
     pr = qc_profile()
     _check(load().qc_get_profile(cache, C.byref(pr)), "qc_get_profile")
     return pr
+
+
+QC_STATIC_MAX_ROWS = 512
+QC_STATIC_SPLITS = 8
+QC_STATIC_MAX_TOKENS = 65536
+
+
+def qc_attend_static(device: int, cuda_stream: int, q_ptr: int, k_ptr: int, v_ptr: int, out_ptr: int, n_seqs: int,
+                     n_tokens: int, n_q_heads: int, n_kv_heads: int, head_dim: int, softmax_scale: float = 0.0) -> None:
+    """Decode attention with the library's built-in scratch array: for callers that cannot
+    allocate device memory (see include/qc.h).  Raises QcError for sizes beyond the fixed limits."""
+    _check(load().qc_attend_static(device, C.c_void_p(cuda_stream), C.c_void_p(q_ptr), C.c_void_p(k_ptr),
+                                   C.c_void_p(v_ptr), C.c_void_p(out_ptr), n_seqs, n_tokens, n_q_heads, n_kv_heads,
+                                   head_dim, softmax_scale), "qc_attend_static")
