@@ -304,6 +304,8 @@ def main():
     ap.add_argument("--mode", default="vla_qc", choices=sorted(MODES))
     ap.add_argument("--e2e-steps", type=int, default=64)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", type=int, default=0, help="cut the stack to its first N layers (profiling-size case)")
+    ap.add_argument("--batch", type=int, default=0, help="override the batch (profiling-size case)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -311,6 +313,14 @@ def main():
     from paper_2602_01901_b200 import workloads as W
 
     w = W.get_workload(args.workload)
+    if args.layers or args.batch:
+        # a smaller case of the same shape, e.g. for a profiler capture that must stay a few GB
+        import dataclasses
+
+        n_layers = args.layers or w.n_layers
+        batch = args.batch or w.batch
+        w = dataclasses.replace(w, name=f"{w.name}[layers={n_layers},batch={batch}]", n_layers=n_layers, batch=batch,
+                                lazy_layers=tuple(l for l in w.lazy_layers if l < n_layers))
     mode = MODES[args.mode]
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
