@@ -10,8 +10,8 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libqcache.so")
-SOURCES = ["qc_runtime.cu", "qc_kernels.cu", "qc_static.cu"]
-HEADERS = ["qc_internal.h", os.path.join("..", "..", "include", "qc.h")]
+SOURCES = ["qc_runtime.cu", "qc_kernels.cu", "qc_attend_tc.cu", "qc_static.cu"]
+HEADERS = ["qc_internal.h", "qc_device.cuh", os.path.join("..", "..", "include", "qc.h")]
 
 
 def _nvcc() -> str:

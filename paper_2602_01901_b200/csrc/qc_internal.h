@@ -2,6 +2,7 @@
 // Not part of the public ABI.
 #pragma once
 
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -45,7 +46,7 @@ struct __align__(16) Item {
   uint16_t head, slot;
   uint16_t first_page, n_pages;
   uint16_t n_valid_last, kv_head;
-  uint32_t pad1;
+  uint16_t n_heads, pad1;       // query heads head .. head + n_heads - 1 share the KV head (1 without GQA)
 };
 static_assert(sizeof(Item) == 32, "Item layout");
 
@@ -60,6 +61,8 @@ struct Patch {
 // Kernel parameter block.
 struct Params {
   // cache-lifetime
+  CUtensorMap tmap;        // the pool as a 2-D bf16 tensor [pages * hkv * 16 rows][d], box 16 x min(d, 64),
+                           // 128-byte swizzle (used by the tensor-core kernel only)
   uint16_t* pool;          // bf16 pages
   int32_t* table;          // [n_layers][4][max_seqs][max_pages]
   uint16_t* qcache;        // bf16 [n_layers][max_seqs][hq][d]
@@ -74,7 +77,8 @@ struct Params {
   int32_t* err;
   int64_t n_pool_pages;    // bound for page ids (reads never leave the pool)
   int32_t n_layers, hq, hkv, d, group, max_seqs, max_pages, max_slots, chunk_pages;
-  int32_t heads_per_item_dim;   // hq: one item per query head
+  int32_t heads_per_item_dim;   // work items per (chunk, sequence): hq, or with GQA hkv * ceil(group / 8)
+  int32_t heads_per_item;       // query heads one item covers: 1, or with GQA up to 8 heads of one KV head
   float scale_log2;             // softmax scale * log2(e)
   // per step
   const uint16_t* q;
@@ -90,11 +94,13 @@ struct Params {
 // launchers (qc_kernels.cu); all asynchronous on `stream`
 cudaError_t launch_setup(const Params& p, cudaStream_t stream);
 cudaError_t launch_append(const Params& p, cudaStream_t stream);
-cudaError_t launch_attend(const Params& p, int n_sms, cudaStream_t stream);
+cudaError_t launch_attend(const Params& p, int n_sms, cudaStream_t stream);      // one query head per item
+cudaError_t launch_attend_tc(const Params& p, int n_sms, cudaStream_t stream);   // query-group items (GQA)
 cudaError_t launch_merge(const Params& p, cudaStream_t stream);
 cudaError_t launch_prefill_scatter(const Params& p, const int32_t* tok_seq, const int32_t* tok_stream,
                                    const int32_t* tok_ord, int32_t n_tokens, int32_t tok_stride,
                                    int32_t tok_offset, cudaStream_t stream);
 cudaError_t configure_kernels(int* attend_smem_bytes);
+cudaError_t configure_kernels_tc(int* attend_smem_bytes);
 
 }  // namespace qc

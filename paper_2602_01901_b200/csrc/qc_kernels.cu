@@ -13,82 +13,10 @@
 // Attention arithmetic: scores are kept in the log2 domain (q is pre-multiplied by
 // scale * log2 e), accumulation is fp32, inputs and outputs are bf16.
 
-#include "qc_internal.h"
-
-#include <math.h>
+#include "qc_device.cuh"
 
 namespace qc {
 namespace {
-
-constexpr int kWarps = 8;
-constexpr int kThreads = kWarps * 32;
-constexpr int kRing = 6;                  // tiles in flight per warp
-constexpr uint32_t kSpinLimit = 1u << 22; // bounded mbarrier wait
-
-constexpr int kErrTimeout = 6;
-constexpr int kErrBadPage = 5;
-
-// ------------------------------------------------------------------------------------------
-// PTX helpers
-// ------------------------------------------------------------------------------------------
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void fence_mbar_init() {
-  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-}
-__device__ __forceinline__ void fence_proxy_async() {
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
-               : "memory");
-}
-__device__ __forceinline__ uint32_t mbar_try_wait(uint64_t* bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
-      : "memory");
-  return ok;
-}
-// 1-D bulk copy global -> this CTA's shared memory, completion counted on an mbarrier.
-// Source, destination and size are multiples of 16 bytes by construction (whole page tiles).
-__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                   smem_u32(dst)),
-               "l"(src), "r"(bytes), "r"(smem_u32(bar))
-               : "memory");
-}
-
-__device__ __forceinline__ void bf16x8_to_f32(const uint4& r, float* f) {
-  f[0] = __uint_as_float(r.x << 16);
-  f[1] = __uint_as_float(r.x & 0xffff0000u);
-  f[2] = __uint_as_float(r.y << 16);
-  f[3] = __uint_as_float(r.y & 0xffff0000u);
-  f[4] = __uint_as_float(r.z << 16);
-  f[5] = __uint_as_float(r.z & 0xffff0000u);
-  f[6] = __uint_as_float(r.w << 16);
-  f[7] = __uint_as_float(r.w & 0xffff0000u);
-}
-
-__device__ __forceinline__ uint16_t f32_to_bf16_rne(float x) {
-  uint32_t u = __float_as_uint(x);
-  if ((u & 0x7fffffffu) > 0x7f800000u) return static_cast<uint16_t>((u >> 16) | 0x40);   // NaN
-  u += 0x7fffu + ((u >> 16) & 1u);
-  return static_cast<uint16_t>(u >> 16);
-}
-
-__device__ __forceinline__ size_t table_row(const Params& P, int layer, int stream, int seq_id) {
-  return ((static_cast<size_t>(layer) * 4 + stream) * P.max_seqs + seq_id) * P.max_pages;
-}
 
 // ------------------------------------------------------------------------------------------
 // setup: page-table patches + item expansion
@@ -103,12 +31,15 @@ __global__ void setup_kernel(Params P) {
   }
   const Seg sg = P.segs[b];
   const Job jb = P.jobs[sg.job];
-  const int n_heads = P.heads_per_item_dim;
+  const int per_chunk = P.heads_per_item_dim;   // items per chunk
+  const int hpi = P.heads_per_item;
+  const int n_sub = (P.group + hpi - 1) / hpi;  // items per KV head
   const int total_pages = (sg.len + kPage - 1) / kPage;
-  const int n = sg.n_chunks * n_heads;
+  const int n = sg.n_chunks * per_chunk;
   for (int t = threadIdx.x; t < n; t += blockDim.x) {
-    const int chunk = t / n_heads;
-    const int head = t - chunk * n_heads;
+    const int chunk = t / per_chunk;
+    const int u = t - chunk * per_chunk;
+    const int kv_head = u / n_sub, sub = u - kv_head * n_sub;
     Item it;
     it.k_layer = jb.k_layer;
     it.stream = jb.stream;
@@ -121,7 +52,7 @@ __global__ void setup_kernel(Params P) {
     }
     it.seq_id = static_cast<uint16_t>(sg.seq_id);
     it.seq_idx = static_cast<uint16_t>(sg.seq_idx);
-    it.head = static_cast<uint16_t>(head);
+    it.head = static_cast<uint16_t>(kv_head * P.group + sub * hpi);
     it.slot = static_cast<uint16_t>(sg.slot_base + chunk);
     const int first = chunk * P.chunk_pages;
     const int np = min(P.chunk_pages, total_pages - first);
@@ -129,7 +60,8 @@ __global__ void setup_kernel(Params P) {
     it.n_pages = static_cast<uint16_t>(np);
     const bool last = (first + np == total_pages);
     it.n_valid_last = static_cast<uint16_t>(last ? sg.len - (total_pages - 1) * kPage : kPage);
-    it.kv_head = static_cast<uint16_t>(head / P.group);
+    it.kv_head = static_cast<uint16_t>(kv_head);
+    it.n_heads = static_cast<uint16_t>(min(hpi, P.group - sub * hpi));
     it.pad1 = 0;
     P.items[sg.item_base + t] = it;
   }
@@ -205,105 +137,18 @@ __global__ void prefill_scatter_kernel(Params P, const int32_t* tok_seq, const i
 // attend: persistent split-KV partial attention, one independent worker per warp
 // ------------------------------------------------------------------------------------------
 
+constexpr int kRing = 6;                  // tiles in flight per warp
+
 template <int D>
 struct WarpCtx {
-  Item item;
-  int32_t pages[1 + kMaxCons][kMaxChunkPages];   // [0]: K pages, [1 + x]: V pages of consumer x
+  ItemPages ip;
   uint4 qraw[kMaxCons][D / 8];
 };
-
-struct WorkerState {
-  int n_my;            // items this worker owns
-  int cons_k;          // item being consumed
-  int iss_k;           // item being fetched (cons_k or cons_k + 1)
-  int iss_page, iss_which;
-  int iss_slot, cons_slot;
-  uint32_t cons_phase;
-  int in_flight;
-  bool dead;           // a bounded wait ran out: stop fetching, drain, leave
-};
-
-template <int D>
-__device__ __forceinline__ bool issue_one(WorkerState& st, const WarpCtx<D>* ctx, uint8_t* ring, uint64_t* full,
-                                          const Params& P, int lane) {
-  constexpr uint32_t kTile = kPage * D * 2;
-  if (st.dead || st.iss_k >= st.n_my || st.iss_k > st.cons_k + 1) return false;
-  const WarpCtx<D>& c = ctx[st.iss_k & 1];
-  const int n_cons = c.item.n_cons;
-  int pid = c.pages[st.iss_which][st.iss_page];
-  if (static_cast<uint32_t>(pid) >= static_cast<uint64_t>(P.n_pool_pages)) {   // never read outside the pool
-    if (lane == 0) atomicMax(P.err, kErrBadPage);
-    pid = 0;
-  }
-  if (lane == 0) {
-    const uint16_t* src = P.pool + (static_cast<size_t>(pid) * P.hkv + c.item.kv_head) * (kPage * D);
-    uint64_t* bar = &full[st.iss_slot];
-    fence_proxy_async();   // the slot's earlier generic-proxy reads precede this async write
-    mbar_expect_tx(bar, kTile);
-    bulk_g2s(ring + st.iss_slot * kTile, src, kTile, bar);
-  }
-  st.iss_slot = (st.iss_slot + 1 == kRing) ? 0 : st.iss_slot + 1;
-  st.in_flight++;
-  if (++st.iss_which > n_cons) {
-    st.iss_which = 0;
-    if (++st.iss_page == c.item.n_pages) {
-      st.iss_page = 0;
-      st.iss_k++;
-    }
-  }
-  return true;
-}
-
-template <int D>
-__device__ __forceinline__ void fill_ring(WorkerState& st, const WarpCtx<D>* ctx, uint8_t* ring, uint64_t* full,
-                                          const Params& P, int lane) {
-  while (st.in_flight < kRing) {
-    if (!issue_one<D>(st, ctx, ring, full, P, lane)) break;
-  }
-}
-
-// Wait until the oldest tile in flight has landed; returns its shared-memory address.
-template <int D>
-__device__ __forceinline__ const uint8_t* wait_tile(WorkerState& st, uint8_t* ring, uint64_t* full, const Params& P,
-                                                    int lane) {
-  constexpr uint32_t kTile = kPage * D * 2;
-  uint64_t* bar = &full[st.cons_slot];
-  uint32_t done = mbar_try_wait(bar, st.cons_phase);
-  for (uint32_t spin = 0; !done && spin < kSpinLimit; ++spin) done = mbar_try_wait(bar, st.cons_phase);
-  if (!done) {
-    if (lane == 0) atomicMax(P.err, kErrTimeout);
-    st.dead = true;
-  }
-  return ring + st.cons_slot * kTile;
-}
-
-__device__ __forceinline__ void release_tile(WorkerState& st) {
-  __syncwarp();
-  st.in_flight--;
-  if (++st.cons_slot == kRing) {
-    st.cons_slot = 0;
-    st.cons_phase ^= 1u;
-  }
-}
 
 // Fetch an item's descriptor, page ids and raw queries into the warp's context slot.
 template <int D>
 __device__ __forceinline__ void load_ctx(WarpCtx<D>& c, const Params& P, int item_idx, int lane) {
-  const uint4* ip = reinterpret_cast<const uint4*>(P.items + item_idx);
-  uint4 a = __ldg(ip), b = __ldg(ip + 1);
-  __syncwarp();
-  if (lane == 0) {
-    reinterpret_cast<uint4*>(&c.item)[0] = a;
-    reinterpret_cast<uint4*>(&c.item)[1] = b;
-  }
-  Item it;
-  reinterpret_cast<uint4*>(&it)[0] = a;
-  reinterpret_cast<uint4*>(&it)[1] = b;
-  if (lane < it.n_pages) {
-    c.pages[0][lane] = P.table[table_row(P, it.k_layer, it.stream, it.seq_id) + it.first_page + lane];
-    for (int x = 0; x < it.n_cons; ++x)
-      c.pages[1 + x][lane] = P.table[table_row(P, it.v_layer[x], 2 + it.stream, it.seq_id) + it.first_page + lane];
-  }
+  const Item it = load_item_pages(c.ip, P, item_idx, lane);
   const int nq = (it.flags & kFlagShared) ? 1 : it.n_cons;
   if (lane < D / 8) {
     for (int x = 0; x < nq; ++x) {
@@ -320,8 +165,9 @@ __device__ __forceinline__ void load_ctx(WarpCtx<D>& c, const Params& P, int ite
 // One item: NQ queries score the K tiles, NV value streams are accumulated.
 // NQ == 1: every consumer shares the weights; NQ == NV: consumer x has its own query.
 template <int D, int NQ, int NV>
-__device__ __forceinline__ void process_item(WorkerState& st, const WarpCtx<D>* ctx, uint8_t* ring, uint64_t* full,
+__device__ __forceinline__ void process_item(WorkerState& st, const WarpCtx<D>* ctx, uint32_t ring, uint64_t* full,
                                              const Params& P, int lane) {
+  auto ctx_of = [ctx](int k) -> const ItemPages& { return ctx[k & 1].ip; };
   constexpr int EPL = D / 8;    // elements of a row held by one lane
   constexpr int LPR = D / 64;   // 16-byte loads per lane per row
   const WarpCtx<D>& c = ctx[st.cons_k & 1];
@@ -351,15 +197,15 @@ __device__ __forceinline__ void process_item(WorkerState& st, const WarpCtx<D>* 
 #pragma unroll
     for (int e = 0; e < EPL; ++e) acc[v][e] = 0.f;
 
-  const int n_pages = c.item.n_pages;
-  const int n_valid_last = c.item.n_valid_last;
+  const int n_pages = c.ip.item.n_pages;
+  const int n_valid_last = c.ip.item.n_valid_last;
 
   for (int pg = 0; pg < n_pages && !st.dead; ++pg) {
     const int nvalid = (pg == n_pages - 1) ? n_valid_last : kPage;
     float p[NQ][4];
     // ---- K tile: scores of 16 keys
     {
-      const uint8_t* tile = wait_tile<D>(st, ring, full, P, lane);
+      const uint8_t* tile = static_cast<const uint8_t*>(__cvta_shared_to_generic(wait_tile<D>(st, ring, full, P, lane)));
       if (st.dead) break;
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
@@ -379,8 +225,8 @@ __device__ __forceinline__ void process_item(WorkerState& st, const WarpCtx<D>* 
           p[x][i] = a0 + a1;
         }
       }
-      release_tile(st);
-      fill_ring<D>(st, ctx, ring, full, P, lane);
+      release_tile<kRing>(st);
+      fill_ring<D, kRing, false>(st, ctx_of, ring, full, P, lane);
     }
 #pragma unroll
     for (int x = 0; x < NQ; ++x) {
@@ -418,7 +264,7 @@ __device__ __forceinline__ void process_item(WorkerState& st, const WarpCtx<D>* 
     // ---- V tiles: weighted sums for each consumer
 #pragma unroll
     for (int v = 0; v < NV; ++v) {
-      const uint8_t* tile = wait_tile<D>(st, ring, full, P, lane);
+      const uint8_t* tile = static_cast<const uint8_t*>(__cvta_shared_to_generic(wait_tile<D>(st, ring, full, P, lane)));
       if (st.dead) break;
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
@@ -433,8 +279,8 @@ __device__ __forceinline__ void process_item(WorkerState& st, const WarpCtx<D>* 
           for (int e = 0; e < EPL; ++e) acc[v][e] = fmaf(pv, vf[e], acc[v][e]);
         }
       }
-      release_tile(st);
-      fill_ring<D>(st, ctx, ring, full, P, lane);
+      release_tile<kRing>(st);
+      fill_ring<D, kRing, false>(st, ctx_of, ring, full, P, lane);
     }
   }
   if (st.dead) return;
@@ -457,8 +303,8 @@ __device__ __forceinline__ void process_item(WorkerState& st, const WarpCtx<D>* 
 #pragma unroll
     for (int v = 0; v < NV; ++v) {
       const size_t row =
-          ((static_cast<size_t>(c.item.v_layer[v]) * P.max_seqs + c.item.seq_idx) * P.max_slots + c.item.slot) *
-              P.hq + c.item.head;
+          ((static_cast<size_t>(c.ip.item.v_layer[v]) * P.max_seqs + c.ip.item.seq_idx) * P.max_slots + c.ip.item.slot) *
+              P.hq + c.ip.item.head;
       float* dst = P.part_acc + row * D;
 #pragma unroll
       for (int j = 0; j < LPR; ++j) {
@@ -472,15 +318,16 @@ __device__ __forceinline__ void process_item(WorkerState& st, const WarpCtx<D>* 
 }
 
 template <int D>
-__global__ void __launch_bounds__(kThreads, 1) attend_kernel(Params P) {
+__global__ void __launch_bounds__(kThreads, 1) attend_kernel(const __grid_constant__ Params P) {
   constexpr uint32_t kTile = kPage * D * 2;
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ __align__(8) uint64_t full_all[kWarps][kRing];
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  uint8_t* ring = smem + static_cast<size_t>(warp) * kRing * kTile;
+  const uint32_t ring = smem_u32(smem) + static_cast<uint32_t>(warp) * kRing * kTile;
   WarpCtx<D>* ctx = reinterpret_cast<WarpCtx<D>*>(smem + static_cast<size_t>(kWarps) * kRing * kTile) + warp * 2;
   uint64_t* full = full_all[warp];
+  auto ctx_of = [ctx](int k) -> const ItemPages& { return ctx[k & 1].ip; };
 
   if (lane == 0) {
     for (int s = 0; s < kRing; ++s) mbar_init(&full[s], 1);
@@ -492,23 +339,16 @@ __global__ void __launch_bounds__(kThreads, 1) attend_kernel(Params P) {
   const int worker = blockIdx.x * kWarps + warp;   // consecutive warps take consecutive items
   const int n_items = P.item_end - P.item_begin;
   WorkerState st;
-  st.n_my = (worker < n_items) ? (n_items - worker + n_workers - 1) / n_workers : 0;
-  st.cons_k = 0;
-  st.iss_k = 0;
-  st.iss_page = st.iss_which = 0;
-  st.iss_slot = st.cons_slot = 0;
-  st.cons_phase = 0;
-  st.in_flight = 0;
-  st.dead = false;
+  worker_init(st, (worker < n_items) ? (n_items - worker + n_workers - 1) / n_workers : 0);
   if (st.n_my == 0) return;
 
   auto item_index = [&](int k) { return P.item_begin + worker + k * n_workers; };
   load_ctx<D>(ctx[0], P, item_index(0), lane);
   if (st.n_my > 1) load_ctx<D>(ctx[1], P, item_index(1), lane);
-  fill_ring<D>(st, ctx, ring, full, P, lane);
+  fill_ring<D, kRing, false>(st, ctx_of, ring, full, P, lane);
 
   for (int k = 0; k < st.n_my && !st.dead; ++k) {
-    const Item& it = ctx[k & 1].item;
+    const Item& it = ctx[k & 1].ip.item;
     const int nc = it.n_cons;
     const bool shared = it.flags & kFlagShared;
     if (nc == 1) process_item<D, 1, 1>(st, ctx, ring, full, P, lane);
@@ -522,23 +362,9 @@ __global__ void __launch_bounds__(kThreads, 1) attend_kernel(Params P) {
     __syncwarp();
     if (k + 2 < st.n_my) load_ctx<D>(ctx[k & 1], P, item_index(k + 2), lane);
     st.cons_k = k + 1;
-    fill_ring<D>(st, ctx, ring, full, P, lane);
+    fill_ring<D, kRing, false>(st, ctx_of, ring, full, P, lane);
   }
-
-  if (st.dead) {
-    // copies still in flight write into this CTA's shared memory: give them a bounded
-    // chance to land before the warp leaves
-    while (st.in_flight > 0) {
-      uint64_t* bar = &full[st.cons_slot];
-      uint32_t done = 0;
-      for (uint32_t spin = 0; !done && spin < kSpinLimit; ++spin) done = mbar_try_wait(bar, st.cons_phase);
-      st.in_flight--;
-      if (++st.cons_slot == kRing) {
-        st.cons_slot = 0;
-        st.cons_phase ^= 1u;
-      }
-    }
-  }
+  if (st.dead) drain_ring<kRing>(st, full);
 }
 
 // ------------------------------------------------------------------------------------------

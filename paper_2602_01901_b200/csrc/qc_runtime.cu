@@ -54,6 +54,9 @@ struct qc_cache {
   std::vector<int> leader;
   std::vector<uint8_t> layer_flags;
   int D = 0, hq = 0, hkv = 0, group = 0;
+  int heads_per_item = 1;  // query heads one work item covers (8 with GQA: one query group, or a slice of it)
+  int items_per_chunk = 0; // work items per (chunk, sequence)
+  CUtensorMap tmap{};      // the pool as a swizzled 2-D tensor (query-group kernel)
   bool paged = true;
   int max_pages = 0;       // per stream
   int chunk_pages = 0, min_chunk_pages = 0, max_slots = 0;
@@ -126,6 +129,9 @@ int validate_config(const qc_config* cfg) {
 void build_jobs(const qc_config* cfg, std::vector<Job>& jobs, std::vector<std::pair<int, int>>& block_jobs,
                 std::vector<std::pair<int, int>>& block_layers) {
   const int N = cfg->n_layers;
+  // own-query sweeps keep one set of query fragments per consumer in registers: the
+  // query-group (tensor-core) kernel feeds two layers per sweep, the one-head kernel four
+  const int max_own = cfg->n_q_heads > cfg->n_kv_heads ? 2 : kMaxCons;
   int l = 0;
   while (l < N) {
     const int c = l;
@@ -149,11 +155,11 @@ void build_jobs(const qc_config* cfg, std::vector<Job>& jobs, std::vector<std::p
       }
     };
     auto own_query_jobs_on_leader_keys = [&](int stream) {   // Eq. 8: own q on the leader's visual K
-      for (int first = c; first < e; first += kMaxCons) {
+      for (int first = c; first < e; first += max_own) {
         Job j{};
         j.k_layer = static_cast<uint8_t>(c);
         j.stream = static_cast<uint8_t>(stream);
-        j.n_cons = static_cast<uint8_t>(std::min(kMaxCons, e - first));
+        j.n_cons = static_cast<uint8_t>(std::min(max_own, e - first));
         j.flags = (j.n_cons == 1) ? kFlagShared : 0;
         for (int x = 0; x < j.n_cons; ++x) {
           j.v_layer[x] = static_cast<uint8_t>(first + x);
@@ -289,7 +295,9 @@ Params base_params(const qc_cache* c) {
   p.max_pages = c->max_pages;
   p.max_slots = c->max_slots;
   p.chunk_pages = c->chunk_pages;
-  p.heads_per_item_dim = c->hq;
+  p.heads_per_item_dim = c->items_per_chunk;
+  p.heads_per_item = c->heads_per_item;
+  p.tmap = c->tmap;
   p.scale_log2 = c->scale * 1.4426950408889634f;
   return p;
 }
@@ -307,6 +315,32 @@ void grow_stream(qc_cache* c, int layer, int stream, int seq, int have, int n_ne
 }
 
 inline int pages_for(int tokens) { return (tokens + kPage - 1) / kPage; }
+
+// The pool seen as a 2-D bf16 tensor [n_pool_pages * hkv * 16 rows][D]: a (page, head) tile is
+// 16 consecutive rows.  Box = 16 rows x 64 elements (128 bytes) with the 128-byte swizzle, so
+// a D = 128 tile is fetched as two column halves.  The driver entry point is looked up at run
+// time; nothing links against the driver library.
+int make_pool_tensor_map(qc_cache* c) {
+  typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                               const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                               CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+      qres != cudaDriverEntryPointSuccess)
+    return QC_ERR_CUDA;
+  const cuuint64_t rows = static_cast<cuuint64_t>(c->n_pool_pages) * c->hkv * kPage;
+  if (rows > 0x7fffffffULL) return QC_ERR_INVALID_ARG;   // tile coordinates are 32-bit
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(c->D), rows};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(c->D) * 2};
+  const cuuint32_t box[2] = {64, kPage};
+  const cuuint32_t elem_strides[2] = {1, 1};
+  const CUresult r = reinterpret_cast<EncodeFn>(fn)(
+      &c->tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, c->pool, dims, strides, box, elem_strides,
+      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? QC_OK : QC_ERR_CUDA;
+}
 
 int sync_and_check(qc_cache* c) {
   QC_CUDA(cudaStreamSynchronize(c->ctx->stream));
@@ -344,9 +378,10 @@ int32_t qc_init(int32_t device, void* cuda_stream, qc_ctx** out) {
   cudaDeviceProp prop;
   QC_CUDA(cudaGetDeviceProperties(&prop, device));
   if (prop.major < 10) return QC_ERR_UNSUPPORTED;
-  int smem = 0;
+  int smem = 0, smem_tc = 0;
   QC_CUDA(configure_kernels(&smem));
-  if (static_cast<size_t>(smem) > prop.sharedMemPerBlockOptin) return QC_ERR_UNSUPPORTED;
+  QC_CUDA(configure_kernels_tc(&smem_tc));
+  if (static_cast<size_t>(std::max(smem, smem_tc)) > prop.sharedMemPerBlockOptin) return QC_ERR_UNSUPPORTED;
   qc_ctx* ctx = new (std::nothrow) qc_ctx();
   if (!ctx) return QC_ERR_INVALID_ARG;
   ctx->device = device;
@@ -387,6 +422,8 @@ int32_t qc_alloc_cache(qc_ctx* ctx, const qc_config* cfg, void* pool_dev, size_t
   c->hq = s.hq;
   c->hkv = s.hkv;
   c->group = s.hq / s.hkv;
+  c->heads_per_item = c->group > 1 ? 8 : 1;
+  c->items_per_chunk = c->group > 1 ? s.hkv * ((c->group + 7) / 8) : s.hq;
   c->paged = cfg->page_size == 16;
   c->max_pages = s.max_pages;
   c->chunk_pages = c->min_chunk_pages = s.chunk_pages;
@@ -421,6 +458,11 @@ int32_t qc_alloc_cache(qc_ctx* ctx, const qc_config* cfg, void* pool_dev, size_t
   } else {
     // contiguous: stream (layer, stream, seq) owns pages [extent*max_pages, (extent+1)*max_pages)
     for (size_t i = 0; i < c->table.size(); ++i) c->table[i] = static_cast<int32_t>(i);
+  }
+
+  if (c->group > 1 && make_pool_tensor_map(c) != QC_OK) {
+    delete c;
+    return QC_ERR_CUDA;
   }
 
   cudaStream_t stream = ctx->stream;
@@ -635,7 +677,7 @@ int32_t qc_decode_step(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, cons
         const int nch = (pages_for(len) + c->chunk_pages - 1) / c->chunk_pages;
         const int ncv = (pages_for(sq.len_vis) + c->chunk_pages - 1) / c->chunk_pages;
         h_segs[n_segs++] = Seg{j, i, sq.seq_id, len, n_items, nch, jb.stream ? 0 : ncv, 0};
-        n_items += nch * c->hq;
+        n_items += nch * c->items_per_chunk;
         step_rows += static_cast<int64_t>(len) * (1 + jb.n_cons);
       }
     }
@@ -678,7 +720,10 @@ int32_t qc_decode_step(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, cons
     p.layer_begin = groups[gi].layer_begin;
     p.layer_end = groups[gi].layer_end;
     if (ev && gi == 0) QC_CUDA(cudaEventRecord(ev[1], stream));
-    QC_CUDA(launch_attend(p, c->ctx->n_sms, stream));
+    if (c->group > 1)
+      QC_CUDA(launch_attend_tc(p, c->ctx->n_sms, stream));
+    else
+      QC_CUDA(launch_attend(p, c->ctx->n_sms, stream));
     if (ev && gi + 1 == groups.size()) QC_CUDA(cudaEventRecord(ev[2], stream));
     QC_CUDA(launch_merge(p, stream));
     c->attend_launches++;

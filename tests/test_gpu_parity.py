@@ -90,6 +90,8 @@ SMALL = [
     (64, 1, [0, 0, 1], 16),
     (128, 4, [0, 1], 512),
     (64, 3, [0, 1, 0, 1], 128),
+    (128, 7, [0, 1, 1], 48),                 # the query-group size of the GQA workload
+    (64, 12, [0, 1, 1, 0], 80),              # a group wider than one tensor-core tile: two slices per KV head
 ]
 
 
