@@ -25,7 +25,7 @@
 namespace qc {
 namespace {
 
-constexpr int kRingTc = 6;
+constexpr int kRingTc = 2;
 
 struct TcCtx {
   ItemPages ip;

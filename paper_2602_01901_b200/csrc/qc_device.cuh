@@ -10,7 +10,7 @@
 namespace qc {
 namespace {
 
-constexpr int kWarps = 8;
+constexpr int kWarps = 12;
 constexpr int kThreads = kWarps * 32;
 constexpr uint32_t kSpinLimit = 1u << 22; // bounded mbarrier wait
 

@@ -137,7 +137,7 @@ __global__ void prefill_scatter_kernel(Params P, const int32_t* tok_seq, const i
 // attend: persistent split-KV partial attention, one independent worker per warp
 // ------------------------------------------------------------------------------------------
 
-constexpr int kRing = 6;                  // tiles in flight per warp
+constexpr int kRing = 2;                  // tiles in flight per warp
 
 template <int D>
 struct WarpCtx {
