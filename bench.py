@@ -205,7 +205,7 @@ def run_gpu(args, w, mode, rank, world, local_rank):
     shape_o = (w.n_layers, w.batch, w.n_q_heads, w.head_dim)
 
     # ---- arm 1: inputs resident in HBM ---------------------------------------------------
-    s = Session.for_workload(w, lazy_mode=mode, device=local_rank)
+    s = Session.for_workload(w, lazy_mode=mode, device=local_rank, split_tokens=args.split_tokens)
     s.prefill_workload(w)
     inputs = _gen_inputs(w, 0, total_steps, dev)
     out = torch.empty(shape_o, dtype=torch.bfloat16, device=dev)
@@ -235,7 +235,7 @@ def run_gpu(args, w, mode, rank, world, local_rank):
 
     # ---- arm 2: host buffers through qc_decode_step_host -----------------------------------
     Ke = min(K, args.e2e_steps)
-    s = Session.for_workload(w, lazy_mode=mode, device=local_rank)
+    s = Session.for_workload(w, lazy_mode=mode, device=local_rank, split_tokens=args.split_tokens)
     s.prefill_workload(w)
     dev_in = _gen_inputs(w, 0, W_ + Ke, dev)
     for i in range(W_):
@@ -304,6 +304,7 @@ def main():
     ap.add_argument("--mode", default="vla_qc", choices=sorted(MODES))
     ap.add_argument("--e2e-steps", type=int, default=64)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--split-tokens", type=int, default=0, help="keys per split-KV work item (0 = library default)")
     ap.add_argument("--layers", type=int, default=0, help="cut the stack to its first N layers (profiling-size case)")
     ap.add_argument("--batch", type=int, default=0, help="override the batch (profiling-size case)")
     args = ap.parse_args()

@@ -79,9 +79,10 @@ typedef struct qc_config {
   int64_t n_pages;             /* pool capacity in pages (paged mode); ignored when contiguous */
   float softmax_scale;         /* 0 => 1/sqrt(head_dim) (Eq. 2) */
   int32_t lazy_mode;           /* QC_MODE_* */
-  int32_t split_tokens;        /* keys per split-KV work item, a multiple of 16 in 16..512;
-                                  0 => 128.  Every stream is cut into ceil(len/split_tokens)
-                                  chunks whose partial results are merged by log-sum-exp. */
+  int32_t split_tokens;        /* keys per split-KV work item, a multiple of 16 in 16..512.  Every
+                                  stream is cut into ceil(len/split_tokens) chunks whose partial
+                                  results are merged by log-sum-exp.  0 => chosen per step among
+                                  128, 256 and 512 from the amount of work (workspace sized for 128). */
   const uint8_t* layer_kind;   /* host, [n_layers], QC_LAYER_*; layer 0 must be FULL; copied */
 } qc_config;
 
@@ -181,7 +182,8 @@ int32_t qc_debug_read_qcache(qc_cache* cache, int32_t layer, void* host_bf16);
 int32_t qc_debug_read_row(qc_cache* cache, int32_t layer, int32_t stream, int32_t seq_id,
                           int32_t token, int32_t kv_head, void* host_bf16);
 
-/* Tuning knobs (all optional).  key: "split_tokens" (as in qc_config), "layers_per_launch"
+/* Tuning knobs (all optional).  key: "split_tokens" (as in qc_config, never below the value
+ * the cache was created with; 0 = per-step choice), "layers_per_launch"
  * (0 = one attention launch for the whole step; k>0 = one launch per k consecutive lazy
  * blocks, in layer order), "profile" (1 = record CUDA events per step). */
 int32_t qc_set_option(qc_cache* cache, const char* key, int64_t value);

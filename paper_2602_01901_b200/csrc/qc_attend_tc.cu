@@ -31,6 +31,10 @@ struct TcCtx {
   ItemPages ip;
 };
 
+__device__ __forceinline__ void load_tc_ctx(TcCtx& c, const Params& P, int item_idx, int lane) {
+  load_item_pages(c.ip, P, item_idx, lane);
+}
+
 // Byte offset of 16-byte chunk `chunk` (0 .. D/8-1) of row `row` inside a swizzled tile:
 // the tile is stored as column halves of 64 elements, each [16 rows][128 bytes], with the
 // chunk index inside a 128-byte row XORed with (row & 7).
@@ -224,16 +228,17 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
   }
   __syncthreads();
 
-  const int n_workers = gridDim.x * kWarps;
-  const int worker = blockIdx.x * kWarps + warp;
-  const int n_items = P.item_end - P.item_begin;
   WorkerState st;
-  worker_init(st, (worker < n_items) ? (n_items - worker + n_workers - 1) / n_workers : 0);
-  if (st.n_my == 0) return;
-
-  auto item_index = [&](int k) { return P.item_begin + worker + k * n_workers; };
-  load_item_pages(ctx[0].ip, P, item_index(0), lane);
-  if (st.n_my > 1) load_item_pages(ctx[1].ip, P, item_index(1), lane);
+  worker_init(st, 0);
+  int next = claim_take(P, claim_issue(P, lane));
+  if (next < 0) return;
+  load_tc_ctx(ctx[0], P, next, lane);
+  st.n_my = 1;
+  next = claim_take(P, claim_issue(P, lane));
+  if (next >= 0) {
+    load_tc_ctx(ctx[1], P, next, lane);
+    st.n_my = 2;
+  }
   __syncwarp();
   fill_ring<D, kRingTc, true>(st, ctx_of, ring, full, P, lane);
 
@@ -241,6 +246,8 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
     const Item& it = ctx[k & 1].ip.item;
     const int nc = it.n_cons;
     const bool shared = it.flags & kFlagShared;
+    // claim the item after next now; the answer is needed only when this item is done
+    const int issued = (next >= 0) ? claim_issue(P, lane) : 0;
     if (nc == 1) process_item_tc<D, 1, 1>(st, ctx, ring, full, P, lane);
     else if (shared && nc == 2) process_item_tc<D, 1, 2>(st, ctx, ring, full, P, lane);
     else if (shared && nc == 3) process_item_tc<D, 1, 3>(st, ctx, ring, full, P, lane);
@@ -248,9 +255,13 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
     else process_item_tc<D, 2, 2>(st, ctx, ring, full, P, lane);   // own-query sweeps feed at most two layers here
     if (st.dead) break;
     __syncwarp();
-    if (k + 2 < st.n_my) {
-      load_item_pages(ctx[k & 1].ip, P, item_index(k + 2), lane);
-      __syncwarp();
+    if (next >= 0) {
+      next = claim_take(P, issued);
+      if (next >= 0) {   // the context slot of the item just finished receives the item after next
+        load_tc_ctx(ctx[k & 1], P, next, lane);
+        __syncwarp();
+        st.n_my = k + 3;
+      }
     }
     st.cons_k = k + 1;
     fill_ring<D, kRingTc, true>(st, ctx_of, ring, full, P, lane);

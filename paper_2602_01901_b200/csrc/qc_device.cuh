@@ -10,7 +10,7 @@
 namespace qc {
 namespace {
 
-constexpr int kWarps = 12;
+constexpr int kWarps = kAttendWarps;
 constexpr int kThreads = kWarps * 32;
 constexpr uint32_t kSpinLimit = 1u << 22; // bounded mbarrier wait
 
@@ -265,6 +265,20 @@ __device__ __forceinline__ Item load_item_pages(ItemPages& c, const Params& P, i
       c.pages[1 + x][lane] = P.table[table_row(P, it.v_layer[x], 2 + it.stream, it.seq_id) + it.first_page + lane];
   }
   return it;
+}
+
+// Items of a launch are handed out in list order (heaviest first, so the work left at the end
+// comes in small pieces).  A claim is an atomic increment issued by lane 0 whose result is only
+// looked at one item later, so its latency never stalls the tile pipeline.
+__device__ __forceinline__ int claim_issue(const Params& P, int lane) {
+  int idx = 0;
+  if (lane == 0) idx = atomicAdd(P.work_counter + P.launch_index, 1);
+  return idx;
+}
+// Turns the value returned by claim_issue into an item index, or -1 when the list is used up.
+__device__ __forceinline__ int claim_take(const Params& P, int issued) {
+  const int idx = __shfl_sync(0xffffffffu, issued, 0);
+  return idx < P.item_end - P.item_begin ? P.item_begin + idx : -1;
 }
 
 }  // namespace

@@ -11,6 +11,7 @@ namespace qc {
 constexpr int kPage = 16;      // tokens per page
 constexpr int kMaxCons = 4;    // V streams (output layers) one K sweep can feed
 constexpr int kMaxChunkPages = 32;
+constexpr int kAttendWarps = 12;   // independent workers (warps) per attention CTA; one CTA per SM
 
 // flags of Job / Item
 constexpr uint8_t kFlagShared = 1;      // one query scores for every consumer (same weights)
@@ -75,6 +76,7 @@ struct Params {
   const Patch* patches;
   const uint8_t* layer_flags;
   int32_t* err;
+  int32_t* work_counter;   // [n_layers] next unclaimed item of each attention launch of a step
   int64_t n_pool_pages;    // bound for page ids (reads never leave the pool)
   int32_t n_layers, hq, hkv, d, group, max_seqs, max_pages, max_slots, chunk_pages;
   int32_t heads_per_item_dim;   // work items per (chunk, sequence): hq, or with GQA hkv * ceil(group / 8)
@@ -88,6 +90,7 @@ struct Params {
   float* lse;
   int32_t n_seqs, n_segs, n_items, n_patches;
   int32_t item_begin, item_end;      // range handled by one attention launch
+  int32_t launch_index;              // which work counter that launch uses
   int32_t layer_begin, layer_end;    // range handled by one merge launch
 };
 

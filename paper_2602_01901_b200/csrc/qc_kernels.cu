@@ -24,9 +24,10 @@ namespace {
 
 __global__ void setup_kernel(Params P) {
   const int b = blockIdx.x;
-  if (b >= P.n_segs) {   // patch blocks
+  if (b >= P.n_segs) {   // housekeeping blocks: page-table patches, work counters
     const int i = (b - P.n_segs) * blockDim.x + threadIdx.x;
     if (i < P.n_patches) P.table[P.patches[i].index] = P.patches[i].page;
+    if (i < P.n_layers) P.work_counter[i] = 0;
     return;
   }
   const Seg sg = P.segs[b];
@@ -335,22 +336,26 @@ __global__ void __launch_bounds__(kThreads, 1) attend_kernel(const __grid_consta
   }
   __syncthreads();
 
-  const int n_workers = gridDim.x * kWarps;
-  const int worker = blockIdx.x * kWarps + warp;   // consecutive warps take consecutive items
-  const int n_items = P.item_end - P.item_begin;
   WorkerState st;
-  worker_init(st, (worker < n_items) ? (n_items - worker + n_workers - 1) / n_workers : 0);
-  if (st.n_my == 0) return;
-
-  auto item_index = [&](int k) { return P.item_begin + worker + k * n_workers; };
-  load_ctx<D>(ctx[0], P, item_index(0), lane);
-  if (st.n_my > 1) load_ctx<D>(ctx[1], P, item_index(1), lane);
+  worker_init(st, 0);
+  int next = claim_take(P, claim_issue(P, lane));
+  if (next < 0) return;
+  load_ctx<D>(ctx[0], P, next, lane);
+  st.n_my = 1;
+  next = claim_take(P, claim_issue(P, lane));
+  if (next >= 0) {
+    load_ctx<D>(ctx[1], P, next, lane);
+    st.n_my = 2;
+  }
+  __syncwarp();
   fill_ring<D, kRing, false>(st, ctx_of, ring, full, P, lane);
 
   for (int k = 0; k < st.n_my && !st.dead; ++k) {
     const Item& it = ctx[k & 1].ip.item;
     const int nc = it.n_cons;
     const bool shared = it.flags & kFlagShared;
+    // claim the item after next now; the answer is needed only when this item is done
+    const int issued = (next >= 0) ? claim_issue(P, lane) : 0;
     if (nc == 1) process_item<D, 1, 1>(st, ctx, ring, full, P, lane);
     else if (shared && nc == 2) process_item<D, 1, 2>(st, ctx, ring, full, P, lane);
     else if (shared && nc == 3) process_item<D, 1, 3>(st, ctx, ring, full, P, lane);
@@ -360,7 +365,14 @@ __global__ void __launch_bounds__(kThreads, 1) attend_kernel(const __grid_consta
     else process_item<D, 4, 4>(st, ctx, ring, full, P, lane);
     if (st.dead) break;
     __syncwarp();
-    if (k + 2 < st.n_my) load_ctx<D>(ctx[k & 1], P, item_index(k + 2), lane);
+    if (next >= 0) {
+      next = claim_take(P, issued);
+      if (next >= 0) {   // the context slot of the item just finished receives the item after next
+        load_ctx<D>(ctx[k & 1], P, next, lane);
+        __syncwarp();
+        st.n_my = k + 3;
+      }
+    }
     st.cons_k = k + 1;
     fill_ring<D, kRing, false>(st, ctx_of, ring, full, P, lane);
   }
@@ -447,8 +459,7 @@ cudaError_t configure_kernels(int* attend_smem) {
 }
 
 cudaError_t launch_setup(const Params& p, cudaStream_t stream) {
-  const int blocks = p.n_segs + (p.n_patches + 255) / 256;
-  if (blocks == 0) return cudaSuccess;
+  const int blocks = p.n_segs + (max(p.n_patches, p.n_layers) + 255) / 256;
   setup_kernel<<<blocks, 256, 0, stream>>>(p);
   return cudaGetLastError();
 }

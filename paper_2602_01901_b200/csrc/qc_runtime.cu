@@ -34,7 +34,7 @@ struct LaunchGroup {
 };
 
 struct Layout {   // byte offsets into the workspace
-  size_t table, layer_flags, jobs, qcache, part_acc, part_ml, items, step, err, stage_q, stage_k, stage_v,
+  size_t table, layer_flags, jobs, qcache, part_acc, part_ml, items, step, err, counters, stage_q, stage_k, stage_v,
       stage_out, stage_lse, tok, total;
   size_t step_seqs, step_patches, step_segs, step_bytes;   // offsets inside the step block
 };
@@ -60,6 +60,8 @@ struct qc_cache {
   bool paged = true;
   int max_pages = 0;       // per stream
   int chunk_pages = 0, min_chunk_pages = 0, max_slots = 0;
+  bool auto_split = false;         // choose chunk_pages per step from the amount of work
+  int n_visual_jobs = 0, n_text_jobs = 0;
   int64_t n_pool_pages = 0;
   int layers_per_launch = 0;
   float scale = 0.f;
@@ -255,6 +257,7 @@ int compute_sizes(const qc_config* cfg, Sizes* s) {
   L.step_bytes = align_up(L.step_segs + s->max_segs * sizeof(Seg), 256);
   L.step = take(L.step_bytes);
   L.err = take(256);
+  L.counters = take(N * sizeof(int32_t));
   L.stage_q = take(N * S * s->hq * s->D * 2);
   L.stage_k = take(N * S * s->hkv * s->D * 2);
   L.stage_v = take(N * S * s->hkv * s->D * 2);
@@ -285,6 +288,7 @@ Params base_params(const qc_cache* c) {
   p.patches = reinterpret_cast<const Patch*>(c->ws + c->lay.step + c->lay.step_patches);
   p.layer_flags = c->ws + c->lay.layer_flags;
   p.err = reinterpret_cast<int32_t*>(c->ws + c->lay.err);
+  p.work_counter = reinterpret_cast<int32_t*>(c->ws + c->lay.counters);
   p.n_pool_pages = c->n_pool_pages;
   p.n_layers = c->cfg.n_layers;
   p.hq = c->hq;
@@ -427,6 +431,7 @@ int32_t qc_alloc_cache(qc_ctx* ctx, const qc_config* cfg, void* pool_dev, size_t
   c->paged = cfg->page_size == 16;
   c->max_pages = s.max_pages;
   c->chunk_pages = c->min_chunk_pages = s.chunk_pages;
+  c->auto_split = cfg->split_tokens == 0;
   c->max_slots = s.max_slots;
   c->n_pool_pages = s.n_pool_pages;
   c->scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / std::sqrt(static_cast<float>(s.D));
@@ -450,6 +455,7 @@ int32_t qc_alloc_cache(qc_ctx* ctx, const qc_config* cfg, void* pool_dev, size_t
     c->text_streams_per_seq += 1 + (owns(c, l, QC_STREAM_K_TEXT) ? 1 : 0);
   }
   build_jobs(&c->cfg, c->jobs, c->block_jobs, c->block_layers);
+  for (const Job& j : c->jobs) (j.stream ? c->n_visual_jobs : c->n_text_jobs)++;
   c->seqs.resize(cfg->max_seqs);
   c->table.assign(static_cast<size_t>(cfg->n_layers) * 4 * cfg->max_seqs * c->max_pages, -1);
   if (c->paged) {
@@ -646,6 +652,34 @@ int32_t qc_decode_step(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, cons
       }
     }
     st.len_text += 1;
+  }
+  if (c->auto_split) {
+    // Larger chunks mean fewer partial results to write and merge; smaller chunks mean more
+    // work items to balance over the workers.  Take the largest chunk that still leaves
+    // every worker several items per launch.
+    const int n_launches =
+        c->layers_per_launch <= 0
+            ? 1
+            : static_cast<int>((c->block_jobs.size() + c->layers_per_launch - 1) / c->layers_per_launch);
+    const int64_t want = 5LL * c->ctx->n_sms * kAttendWarps * n_launches;
+    int pick = c->min_chunk_pages;
+    for (int cp = kMaxChunkPages; cp > c->min_chunk_pages; cp /= 2) {
+      int64_t cv = 0, ct = 0;
+      for (int i = 0; i < n_seqs; ++i) {
+        const SeqState& st = c->seqs[seq_ids[i]];
+        cv += (pages_for(st.len_vis) + cp - 1) / cp;
+        ct += (pages_for(st.len_text) + cp - 1) / cp;
+      }
+      if ((cv * c->n_visual_jobs + ct * c->n_text_jobs) * c->items_per_chunk >= want) {
+        pick = cp;
+        break;
+      }
+    }
+    c->chunk_pages = pick;
+  }
+  for (int i = 0; i < n_seqs; ++i) {
+    const int s = seq_ids[i];
+    const SeqState& st = c->seqs[s];
     const int ncv = (pages_for(st.len_vis) + c->chunk_pages - 1) / c->chunk_pages;
     const int nct = (pages_for(st.len_text) + c->chunk_pages - 1) / c->chunk_pages;
     h_seqs[i] = StepSeq{s, st.len_text, st.len_vis, ncv + nct};
@@ -666,9 +700,19 @@ int32_t qc_decode_step(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, cons
   }
   int n_segs = 0, n_items = 0;
   std::vector<std::pair<int, int>> group_items;
+  std::vector<int> order;
   for (const LaunchGroup& g : groups) {
     const int begin = n_items;
-    for (int j = g.job_begin; j < g.job_end; ++j) {
+    // items are claimed in list order: heaviest sweeps (most tiles per page, visual before
+    // text) first, so that the work left for the end of the launch comes in small pieces
+    order.resize(g.job_end - g.job_begin);
+    for (int j = g.job_begin; j < g.job_end; ++j) order[j - g.job_begin] = j;
+    std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
+      const Job &ja = c->jobs[a], &jb = c->jobs[b];
+      if (ja.n_cons != jb.n_cons) return ja.n_cons > jb.n_cons;
+      return ja.stream > jb.stream;
+    });
+    for (int j : order) {
       const Job& jb = c->jobs[j];
       for (int i = 0; i < n_seqs; ++i) {
         const StepSeq& sq = h_seqs[i];
@@ -719,6 +763,7 @@ int32_t qc_decode_step(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, cons
     p.item_end = group_items[gi].second;
     p.layer_begin = groups[gi].layer_begin;
     p.layer_end = groups[gi].layer_end;
+    p.launch_index = static_cast<int32_t>(gi);
     if (ev && gi == 0) QC_CUDA(cudaEventRecord(ev[1], stream));
     if (c->group > 1)
       QC_CUDA(launch_attend_tc(p, c->ctx->n_sms, stream));
@@ -872,10 +917,15 @@ int32_t qc_set_option(qc_cache* c, const char* key, int64_t value) {
   if (!c || !key) return QC_ERR_INVALID_ARG;
   const std::string k(key);
   if (k == "split_tokens") {
+    if (value == 0) {   // back to the per-step choice
+      c->auto_split = true;
+      return QC_OK;
+    }
     if (value % 16 || value < 16 || value > 16 * kMaxChunkPages) return QC_ERR_INVALID_ARG;
     const int cp = static_cast<int>(value / 16);
     if (cp < c->min_chunk_pages) return QC_ERR_INVALID_ARG;   // the workspace was sized for the initial split
     c->chunk_pages = cp;
+    c->auto_split = false;
     return QC_OK;
   }
   if (k == "layers_per_launch") {
