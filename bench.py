@@ -30,9 +30,11 @@ METRIC = "decode_attention_tokens_per_s"
 UNIT = "tokens/s"
 MODES = {"vla_qc": 0, "vla_eq8": 1, "gla": 2}
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one attend_kernel launch, from the ncu
-# capture summarised under profiles/ (bytes; None until a capture exists for the workload).
-NCU_TRAFFIC_PER_LAUNCH = {}
+# (dram__bytes_read.sum + dram__bytes_write.sum) / algorithmic K/V bytes of one attention launch,
+# from the ncu captures of small cases summarised in profiles/attend_kernels_small_cases_ncu_full.md.
+# Traffic grows in proportion to the K/V bytes swept (every tile is fetched once; partial results are
+# written once per chunk), so a full launch's traffic is this ratio times its algorithmic bytes.
+NCU_TRAFFIC_RATIO = {"attend_kernel": 1.055, "attend_tc_kernel": 1.078}
 
 
 def _peaks():
@@ -260,7 +262,8 @@ def run_gpu(args, w, mode, rank, world, local_rank):
     attend_s = prof.attend_ms / 1e3
     achieved = prof.kv_bytes_read / attend_s / 1e9
     launches_attend = K
-    traffic = NCU_TRAFFIC_PER_LAUNCH.get(w.name)
+    kernel = "attend_tc_kernel" if w.group > 1 else "attend_kernel"
+    traffic = NCU_TRAFFIC_RATIO[kernel] * prof.kv_bytes_read / launches_attend
     line = {
         "metric": METRIC, "value": tokens / (ms / 1e3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W_,
         "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -274,7 +277,8 @@ def run_gpu(args, w, mode, rank, world, local_rank):
         },
         "roofline": {
             "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-            "traffic": traffic, "peak_kind": f"of {peak_kind}", "kernel": "attend_kernel",
+            "traffic": traffic, "traffic_source": "ncu dram bytes of a small case, scaled by K/V bytes per launch",
+            "peak_kind": f"of {peak_kind}", "kernel": kernel,
             "algorithmic_bytes_per_launch": prof.kv_bytes_read / launches_attend,
             "avg_launch_ms": prof.attend_ms / launches_attend, "frac_of_nominal_8TBs": achieved / 8000.0,
         },
