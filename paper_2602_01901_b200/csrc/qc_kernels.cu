@@ -8,6 +8,7 @@
 //                   worker that streams K/V page tiles through its own shared-memory ring
 //                   with bulk asynchronous copies and keeps an online softmax in registers
 //   merge_kernel    log-sum-exp merge of the partials, bf16 output
+// (the grouped-query variant of the attention kernel is in qc_attend_tc.cu)
 //   prefill_scatter_kernel  stores prompt K/V rows into their pages
 //
 // Attention arithmetic: scores are kept in the log2 domain (q is pre-multiplied by
