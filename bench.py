@@ -214,6 +214,7 @@ def run_gpu(args, w, mode, rank, world, local_rank):
     for i in range(W_):
         s.decode_step(ids, *inputs[i], out)
     s.set_option("profile", 1)
+    launches_before = s.stats().kernel_launches
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     with ClockSampler(_physical_gpu_index(local_rank)) as clocks:
@@ -284,7 +285,7 @@ def run_gpu(args, w, mode, rank, world, local_rank):
         },
         "e2e": {"value": w.batch * Ke * world / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "steps": Ke},
-        "gpu_launches": 4 * K,
+        "gpu_launches": int(st.kernel_launches - launches_before),
         "clocks": clocks.summary(),
         "kv_cache": {
             "bytes_stored": st.kv_bytes_stored, "bytes_all_full": st.kv_bytes_all_full,

@@ -99,6 +99,7 @@ typedef struct qc_stats {
   int64_t attend_launches;        /* launches of the attention kernel so far */
   int32_t device_error;           /* 0, or the QC_ERR_* code the device error word holds */
   int32_t n_active_seqs;
+  int64_t kernel_launches;        /* kernels of this library launched for the cache so far */
 } qc_stats;
 
 /* Per-step kernel timing (CUDA events on the library's stream), for roofline accounting. */

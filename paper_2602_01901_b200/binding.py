@@ -51,6 +51,7 @@ class qc_stats(C.Structure):
         ("kv_bytes_stored_paged", C.c_int64), ("kv_bytes_all_full_paged", C.c_int64),
         ("qcache_bytes", C.c_int64), ("decode_steps", C.c_int64), ("attend_launches", C.c_int64),
         ("device_error", C.c_int32), ("n_active_seqs", C.c_int32),
+        ("kernel_launches", C.c_int64),
     ]
 
 

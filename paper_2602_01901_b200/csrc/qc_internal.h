@@ -31,12 +31,13 @@ struct Job {
 };
 static_assert(sizeof(Job) == 16, "Job layout");
 
-// (job, sequence) of one step; built on the host.
-struct __align__(16) Seg {
-  int32_t job, seq_idx, seq_id, len;        // len: tokens in the stream after this step's append
-  int32_t item_base, n_chunks, slot_base, pad;
+// One position of the launch plan: a job plus how many visual-stream and text-stream jobs
+// precede it in the item list (all launches of a step share one list).  Static per cache.
+struct __align__(16) PlanJob {
+  Job job;
+  int32_t vis_before, text_before, pad0, pad1;
 };
-static_assert(sizeof(Seg) == 32, "Seg layout");
+static_assert(sizeof(PlanJob) == 32, "PlanJob layout");
 
 // One split-KV work item: a chunk of pages of one (job, sequence, head).
 struct __align__(16) Item {
@@ -51,8 +52,19 @@ struct __align__(16) Item {
 };
 static_assert(sizeof(Item) == 32, "Item layout");
 
-struct StepSeq {
+// One listed sequence of a step.  Lengths count the new token; ncv chunks of the visual stream
+// come first among the n_slots partial slots of an output row; pre_v / pre_t are the numbers
+// of items that the sequences listed before this one contribute to one visual / text job.
+struct __align__(16) StepSeq {
   int32_t seq_id, len_text, len_vis, n_slots;
+  int32_t pre_v, pre_t, ncv, pad;
+};
+static_assert(sizeof(StepSeq) == 32, "StepSeq layout");
+
+// Step descriptors small enough to travel as a kernel argument instead of a copy.
+constexpr int kInlineSeqs = 64;
+struct StepInline {
+  StepSeq seqs[kInlineSeqs];
 };
 
 struct Patch {
@@ -70,9 +82,9 @@ struct Params {
   float* part_acc;         // [n_layers][max_seqs][max_slots][hq][d]
   float2* part_ml;         // [n_layers][max_seqs][max_slots][hq]  (max, sum) in the log2 domain
   Item* items;
-  const Seg* segs;
+  const PlanJob* plan;
   const Job* jobs;
-  const StepSeq* seqs;
+  StepSeq* seqs;
   const Patch* patches;
   const uint8_t* layer_flags;
   int32_t* err;
@@ -88,14 +100,17 @@ struct Params {
   const uint16_t* v;
   uint16_t* out;
   float* lse;
-  int32_t n_seqs, n_segs, n_items, n_patches;
+  int32_t n_seqs, n_pos, n_items, n_patches;   // n_pos: plan positions (jobs) of the step
+  int32_t tot_v, tot_t;                        // items of one visual / text job over all listed sequences
+  int32_t inline_seqs;                         // 1: the StepSeq array arrives as a kernel argument
+  int32_t fused_append;                        // 1: the set-up launch also does the append
   int32_t item_begin, item_end;      // range handled by one attention launch
   int32_t launch_index;              // which work counter that launch uses
   int32_t layer_begin, layer_end;    // range handled by one merge launch
 };
 
 // launchers (qc_kernels.cu); all asynchronous on `stream`
-cudaError_t launch_setup(const Params& p, cudaStream_t stream);
+cudaError_t launch_setup(const Params& p, const StepInline* inl, cudaStream_t stream);
 cudaError_t launch_append(const Params& p, cudaStream_t stream);
 cudaError_t launch_attend(const Params& p, int n_sms, cudaStream_t stream);      // one query head per item
 cudaError_t launch_attend_tc(const Params& p, int n_sms, cudaStream_t stream);   // query-group items (GQA)

@@ -23,60 +23,8 @@ namespace {
 // setup: page-table patches + item expansion
 // ------------------------------------------------------------------------------------------
 
-__global__ void setup_kernel(Params P) {
-  const int b = blockIdx.x;
-  if (b >= P.n_segs) {   // housekeeping blocks: page-table patches, work counters
-    const int i = (b - P.n_segs) * blockDim.x + threadIdx.x;
-    if (i < P.n_patches) P.table[P.patches[i].index] = P.patches[i].page;
-    if (i < P.n_layers) P.work_counter[i] = 0;
-    return;
-  }
-  const Seg sg = P.segs[b];
-  const Job jb = P.jobs[sg.job];
-  const int per_chunk = P.heads_per_item_dim;   // items per chunk
-  const int hpi = P.heads_per_item;
-  const int n_sub = (P.group + hpi - 1) / hpi;  // items per KV head
-  const int total_pages = (sg.len + kPage - 1) / kPage;
-  const int n = sg.n_chunks * per_chunk;
-  for (int t = threadIdx.x; t < n; t += blockDim.x) {
-    const int chunk = t / per_chunk;
-    const int u = t - chunk * per_chunk;
-    const int kv_head = u / n_sub, sub = u - kv_head * n_sub;
-    Item it;
-    it.k_layer = jb.k_layer;
-    it.stream = jb.stream;
-    it.n_cons = jb.n_cons;
-    it.flags = jb.flags;
-#pragma unroll
-    for (int x = 0; x < kMaxCons; ++x) {
-      it.v_layer[x] = jb.v_layer[x];
-      it.q_layer[x] = jb.q_layer[x];
-    }
-    it.seq_id = static_cast<uint16_t>(sg.seq_id);
-    it.seq_idx = static_cast<uint16_t>(sg.seq_idx);
-    it.head = static_cast<uint16_t>(kv_head * P.group + sub * hpi);
-    it.slot = static_cast<uint16_t>(sg.slot_base + chunk);
-    const int first = chunk * P.chunk_pages;
-    const int np = min(P.chunk_pages, total_pages - first);
-    it.first_page = static_cast<uint16_t>(first);
-    it.n_pages = static_cast<uint16_t>(np);
-    const bool last = (first + np == total_pages);
-    it.n_valid_last = static_cast<uint16_t>(last ? sg.len - (total_pages - 1) * kPage : kPage);
-    it.kv_head = static_cast<uint16_t>(kv_head);
-    it.n_heads = static_cast<uint16_t>(min(hpi, P.group - sub * hpi));
-    it.pad1 = 0;
-    P.items[sg.item_base + t] = it;
-  }
-}
-
-// ------------------------------------------------------------------------------------------
-// append: new token's k, v rows and the Q Cache refresh
-// ------------------------------------------------------------------------------------------
-
-__global__ void append_kernel(Params P) {
-  const int si = blockIdx.x;
-  const int layer = blockIdx.y;
-  const StepSeq sq = P.seqs[si];
+// new token's k, v rows of one (sequence, layer) and the Q Cache refresh
+__device__ __forceinline__ void append_rows(const Params& P, const StepSeq& sq, int si, int layer) {
   const int pos = sq.len_text - 1;          // ordinal of the new token in the text stream
   const int pg = pos / kPage, slot = pos % kPage;
   const uint8_t lf = P.layer_flags[layer];
@@ -103,6 +51,82 @@ __global__ void append_kernel(Params P) {
     for (int e = threadIdx.x; e < n_q_vec; e += blockDim.x)
       reinterpret_cast<uint4*>(P.qcache + dst0)[e] = reinterpret_cast<const uint4*>(P.q + src0)[e];
   }
+}
+
+// Block roles, in grid order: n_pos * n_seqs blocks expand one (plan position, sequence) each
+// into work items; housekeeping blocks apply page-table patches, reset the work counters and
+// store the inline sequence descriptors for the later kernels; with fused_append, n_seqs *
+// n_layers blocks do the append.  (The append reads page ids from the table, so it is only
+// fused on steps without patches.)
+__global__ void setup_kernel(const __grid_constant__ Params P, const __grid_constant__ StepInline inl) {
+  const StepSeq* seqs = P.inline_seqs ? inl.seqs : P.seqs;
+  const int n_expand = P.n_pos * P.n_seqs;
+  const int n_house = (max(max(P.n_patches, P.n_layers), P.n_seqs * 8) + blockDim.x - 1) / blockDim.x;
+  int b = blockIdx.x;
+  if (b >= n_expand + n_house) {   // append blocks
+    b -= n_expand + n_house;
+    const int si = b % P.n_seqs, layer = b / P.n_seqs;
+    append_rows(P, seqs[si], si, layer);
+    return;
+  }
+  if (b >= n_expand) {   // housekeeping blocks
+    const int i = (b - n_expand) * blockDim.x + threadIdx.x;
+    if (i < P.n_patches) P.table[P.patches[i].index] = P.patches[i].page;
+    if (i < P.n_layers) P.work_counter[i] = 0;
+    if (P.inline_seqs && i < P.n_seqs * 8)
+      reinterpret_cast<int32_t*>(P.seqs)[i] = reinterpret_cast<const int32_t*>(inl.seqs)[i];
+    return;
+  }
+  const int pos = b / P.n_seqs, si = b - pos * P.n_seqs;
+  const StepSeq sq = seqs[si];
+  const PlanJob pj = P.plan[pos];
+  const Job jb = pj.job;
+  const int len = jb.stream ? sq.len_vis : sq.len_text;
+  const int n_chunks = jb.stream ? sq.ncv : sq.n_slots - sq.ncv;
+  const int item_base = pj.vis_before * P.tot_v + pj.text_before * P.tot_t + (jb.stream ? sq.pre_v : sq.pre_t);
+  const int slot_base = jb.stream ? 0 : sq.ncv;
+  const int per_chunk = P.heads_per_item_dim;   // items per chunk
+  const int hpi = P.heads_per_item;
+  const int n_sub = (P.group + hpi - 1) / hpi;  // items per KV head
+  const int total_pages = (len + kPage - 1) / kPage;
+  const int n = n_chunks * per_chunk;
+  for (int t = threadIdx.x; t < n; t += blockDim.x) {
+    const int chunk = t / per_chunk;
+    const int u = t - chunk * per_chunk;
+    const int kv_head = u / n_sub, sub = u - kv_head * n_sub;
+    Item it;
+    it.k_layer = jb.k_layer;
+    it.stream = jb.stream;
+    it.n_cons = jb.n_cons;
+    it.flags = jb.flags;
+#pragma unroll
+    for (int x = 0; x < kMaxCons; ++x) {
+      it.v_layer[x] = jb.v_layer[x];
+      it.q_layer[x] = jb.q_layer[x];
+    }
+    it.seq_id = static_cast<uint16_t>(sq.seq_id);
+    it.seq_idx = static_cast<uint16_t>(si);
+    it.head = static_cast<uint16_t>(kv_head * P.group + sub * hpi);
+    it.slot = static_cast<uint16_t>(slot_base + chunk);
+    const int first = chunk * P.chunk_pages;
+    const int np = min(P.chunk_pages, total_pages - first);
+    it.first_page = static_cast<uint16_t>(first);
+    it.n_pages = static_cast<uint16_t>(np);
+    const bool last = (first + np == total_pages);
+    it.n_valid_last = static_cast<uint16_t>(last ? len - (total_pages - 1) * kPage : kPage);
+    it.kv_head = static_cast<uint16_t>(kv_head);
+    it.n_heads = static_cast<uint16_t>(min(hpi, P.group - sub * hpi));
+    it.pad1 = 0;
+    P.items[item_base + t] = it;
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// append: new token's k, v rows and the Q Cache refresh (separate launch on steps with patches)
+// ------------------------------------------------------------------------------------------
+
+__global__ void append_kernel(const __grid_constant__ Params P) {
+  append_rows(P, P.seqs[blockIdx.x], blockIdx.x, blockIdx.y);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -459,9 +483,12 @@ cudaError_t configure_kernels(int* attend_smem) {
   return e;
 }
 
-cudaError_t launch_setup(const Params& p, cudaStream_t stream) {
-  const int blocks = p.n_segs + (max(p.n_patches, p.n_layers) + 255) / 256;
-  setup_kernel<<<blocks, 256, 0, stream>>>(p);
+cudaError_t launch_setup(const Params& p, const StepInline* inl, cudaStream_t stream) {
+  constexpr int kBlock = 256;
+  const int n_house = (max(max(p.n_patches, p.n_layers), p.n_seqs * 8) + kBlock - 1) / kBlock;
+  const int blocks = p.n_pos * p.n_seqs + n_house + (p.fused_append ? p.n_seqs * p.n_layers : 0);
+  static const StepInline kNone{};
+  setup_kernel<<<blocks, kBlock, 0, stream>>>(p, inl ? *inl : kNone);
   return cudaGetLastError();
 }
 

@@ -34,9 +34,9 @@ struct LaunchGroup {
 };
 
 struct Layout {   // byte offsets into the workspace
-  size_t table, layer_flags, jobs, qcache, part_acc, part_ml, items, step, err, counters, stage_q, stage_k, stage_v,
+  size_t table, layer_flags, jobs, plan, qcache, part_acc, part_ml, items, step, err, counters, stage_q, stage_k, stage_v,
       stage_out, stage_lse, tok, total;
-  size_t step_seqs, step_patches, step_segs, step_bytes;   // offsets inside the step block
+  size_t step_seqs, step_patches, step_bytes;   // offsets inside the step block
 };
 
 }  // namespace
@@ -62,6 +62,13 @@ struct qc_cache {
   int chunk_pages = 0, min_chunk_pages = 0, max_slots = 0;
   bool auto_split = false;         // choose chunk_pages per step from the amount of work
   int n_visual_jobs = 0, n_text_jobs = 0;
+  int64_t visual_row_reads = 0, text_row_reads = 0;   // K/V rows read per visual / text token per step
+  // launch plan: jobs in item-list order (launch group by launch group, heaviest first)
+  std::vector<PlanJob> plan;                 // plan[p] for p < n_pos, uploaded to the workspace
+  std::vector<int> plan_vis_before, plan_text_before;   // n_pos + 1 entries
+  std::vector<LaunchGroup> groups;
+  std::vector<std::pair<int, int>> group_pos;           // plan positions [begin, end) of each launch
+  bool plan_dirty = true;
   int64_t n_pool_pages = 0;
   int layers_per_launch = 0;
   float scale = 0.f;
@@ -91,7 +98,7 @@ struct qc_cache {
   int ev_steps = 0;
   int64_t prof_bytes = 0, prof_items = 0;
 
-  int64_t decode_steps = 0, attend_launches = 0;
+  int64_t decode_steps = 0, attend_launches = 0, kernel_launches = 0;
 };
 
 namespace {
@@ -246,6 +253,7 @@ int compute_sizes(const qc_config* cfg, Sizes* s) {
   L.table = take(N * 4 * S * s->max_pages * sizeof(int32_t));
   L.layer_flags = take(N);
   L.jobs = take(jobs.size() * sizeof(Job));
+  L.plan = take(jobs.size() * sizeof(PlanJob));
   L.qcache = take(N * S * s->hq * s->D * 2);
   L.part_acc = take(N * S * s->max_slots * s->hq * s->D * sizeof(float));
   L.part_ml = take(N * S * s->max_slots * s->hq * sizeof(float2));
@@ -253,8 +261,7 @@ int compute_sizes(const qc_config* cfg, Sizes* s) {
   // step block: header-free arrays at fixed offsets
   L.step_seqs = 0;
   L.step_patches = align_up(L.step_seqs + S * sizeof(StepSeq), 16);
-  L.step_segs = align_up(L.step_patches + s->max_patches * sizeof(Patch), 16);
-  L.step_bytes = align_up(L.step_segs + s->max_segs * sizeof(Seg), 256);
+  L.step_bytes = align_up(L.step_patches + s->max_patches * sizeof(Patch), 256);
   L.step = take(L.step_bytes);
   L.err = take(256);
   L.counters = take(N * sizeof(int32_t));
@@ -282,9 +289,9 @@ Params base_params(const qc_cache* c) {
   p.part_acc = reinterpret_cast<float*>(c->ws + c->lay.part_acc);
   p.part_ml = reinterpret_cast<float2*>(c->ws + c->lay.part_ml);
   p.items = reinterpret_cast<Item*>(c->ws + c->lay.items);
-  p.segs = reinterpret_cast<const Seg*>(c->ws + c->lay.step + c->lay.step_segs);
+  p.plan = reinterpret_cast<const PlanJob*>(c->ws + c->lay.plan);
   p.jobs = reinterpret_cast<const Job*>(c->ws + c->lay.jobs);
-  p.seqs = reinterpret_cast<const StepSeq*>(c->ws + c->lay.step + c->lay.step_seqs);
+  p.seqs = reinterpret_cast<StepSeq*>(c->ws + c->lay.step + c->lay.step_seqs);
   p.patches = reinterpret_cast<const Patch*>(c->ws + c->lay.step + c->lay.step_patches);
   p.layer_flags = c->ws + c->lay.layer_flags;
   p.err = reinterpret_cast<int32_t*>(c->ws + c->lay.err);
@@ -344,6 +351,46 @@ int make_pool_tensor_map(qc_cache* c) {
       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? QC_OK : QC_ERR_CUDA;
+}
+
+// Launch groups and the item-list order of the jobs.  Within a launch the heaviest sweeps (most
+// tiles per page, visual before text) come first: items are claimed in list order, so the work
+// left for the end of the launch comes in small pieces.
+int rebuild_plan(qc_cache* c) {
+  c->groups.clear();
+  c->group_pos.clear();
+  c->plan.clear();
+  c->plan_vis_before.assign(1, 0);
+  c->plan_text_before.assign(1, 0);
+  const int nb = static_cast<int>(c->block_jobs.size());
+  const int per = c->layers_per_launch <= 0 ? nb : c->layers_per_launch;
+  std::vector<int> order;
+  for (int b = 0; b < nb; b += per) {
+    const int e = std::min(nb, b + per);
+    const LaunchGroup g{c->block_jobs[b].first, c->block_jobs[e - 1].second, c->block_layers[b].first,
+                        c->block_layers[e - 1].second};
+    c->groups.push_back(g);
+    order.resize(g.job_end - g.job_begin);
+    for (int j = g.job_begin; j < g.job_end; ++j) order[j - g.job_begin] = j;
+    std::stable_sort(order.begin(), order.end(), [&](int x, int y) {
+      const Job &jx = c->jobs[x], &jy = c->jobs[y];
+      if (jx.n_cons != jy.n_cons) return jx.n_cons > jy.n_cons;
+      return jx.stream > jy.stream;
+    });
+    const int begin = static_cast<int>(c->plan.size());
+    for (int j : order) {
+      const int vb = c->plan_vis_before.back(), tb = c->plan_text_before.back();
+      c->plan.push_back(PlanJob{c->jobs[j], vb, tb, 0, 0});
+      c->plan_vis_before.push_back(vb + (c->jobs[j].stream ? 1 : 0));
+      c->plan_text_before.push_back(tb + (c->jobs[j].stream ? 0 : 1));
+    }
+    c->group_pos.emplace_back(begin, static_cast<int>(c->plan.size()));
+  }
+  QC_CUDA(cudaMemcpyAsync(c->ws + c->lay.plan, c->plan.data(), c->plan.size() * sizeof(PlanJob),
+                          cudaMemcpyHostToDevice, c->ctx->stream));
+  QC_CUDA(cudaStreamSynchronize(c->ctx->stream));   // the host vector may be rebuilt later
+  c->plan_dirty = false;
+  return QC_OK;
 }
 
 int sync_and_check(qc_cache* c) {
@@ -455,7 +502,10 @@ int32_t qc_alloc_cache(qc_ctx* ctx, const qc_config* cfg, void* pool_dev, size_t
     c->text_streams_per_seq += 1 + (owns(c, l, QC_STREAM_K_TEXT) ? 1 : 0);
   }
   build_jobs(&c->cfg, c->jobs, c->block_jobs, c->block_layers);
-  for (const Job& j : c->jobs) (j.stream ? c->n_visual_jobs : c->n_text_jobs)++;
+  for (const Job& j : c->jobs) {
+    (j.stream ? c->n_visual_jobs : c->n_text_jobs)++;
+    (j.stream ? c->visual_row_reads : c->text_row_reads) += 1 + j.n_cons;
+  }
   c->seqs.resize(cfg->max_seqs);
   c->table.assign(static_cast<size_t>(cfg->n_layers) * 4 * cfg->max_seqs * c->max_pages, -1);
   if (c->paged) {
@@ -593,6 +643,7 @@ int32_t qc_prefill_append(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, c
                             cudaMemcpyHostToDevice, stream));
     QC_CUDA(cudaMemcpyAsync(tok_dev + 2 * kPrefillBatchTokens, tok_ord.data() + off, n * sizeof(int32_t),
                             cudaMemcpyHostToDevice, stream));
+    c->kernel_launches++;
     QC_CUDA(launch_prefill_scatter(p, tok_dev, tok_dev + kPrefillBatchTokens, tok_dev + 2 * kPrefillBatchTokens, n,
                                    static_cast<int32_t>(total), static_cast<int32_t>(off), stream));
     // the host vectors and the device token arrays are reused by the next batch
@@ -628,19 +679,13 @@ int32_t qc_decode_step(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, cons
   QC_CUDA(cudaSetDevice(c->ctx->device));
   cudaStream_t stream = c->ctx->stream;
 
-  // ---- a pinned descriptor slot (wait if the copy that last used it has not run yet)
-  const int slot = c->stage_next;
-  c->stage_next = (c->stage_next + 1) % kStageSlots;
-  if (c->stage_used[slot]) QC_CUDA(cudaEventSynchronize(c->stage_done[slot]));
-  uint8_t* hb = c->pinned + static_cast<size_t>(slot) * c->lay.step_bytes;
-  StepSeq* h_seqs = reinterpret_cast<StepSeq*>(hb + c->lay.step_seqs);
-  Patch* h_patches = reinterpret_cast<Patch*>(hb + c->lay.step_patches);
-  Seg* h_segs = reinterpret_cast<Seg*>(hb + c->lay.step_segs);
+  if (c->plan_dirty) {
+    const int st = rebuild_plan(c);
+    if (st != QC_OK) return st;
+  }
 
   // ---- page planning (sequence -> layer -> K_T, V_T) and lengths
-  int n_patches = 0;
   std::vector<Patch> patches;
-  int64_t step_rows = 0;   // K/V rows the step has to read (for the profile)
   for (int i = 0; i < n_seqs; ++i) {
     const int s = seq_ids[i];
     SeqState& st = c->seqs[s];
@@ -653,15 +698,12 @@ int32_t qc_decode_step(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, cons
     }
     st.len_text += 1;
   }
+  const int n_patches = static_cast<int>(patches.size());
   if (c->auto_split) {
     // Larger chunks mean fewer partial results to write and merge; smaller chunks mean more
     // work items to balance over the workers.  Take the largest chunk that still leaves
     // every worker several items per launch.
-    const int n_launches =
-        c->layers_per_launch <= 0
-            ? 1
-            : static_cast<int>((c->block_jobs.size() + c->layers_per_launch - 1) / c->layers_per_launch);
-    const int64_t want = 5LL * c->ctx->n_sms * kAttendWarps * n_launches;
+    const int64_t want = 5LL * c->ctx->n_sms * kAttendWarps * static_cast<int64_t>(c->groups.size());
     int pick = c->min_chunk_pages;
     for (int cp = kMaxChunkPages; cp > c->min_chunk_pages; cp /= 2) {
       int64_t cv = 0, ct = 0;
@@ -677,61 +719,44 @@ int32_t qc_decode_step(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, cons
     }
     c->chunk_pages = pick;
   }
+
+  // ---- step descriptors: as a kernel argument when they are small and no page table entry
+  // changes, otherwise through a pinned slot and one copy
+  const bool inline_step = n_seqs <= kInlineSeqs && n_patches == 0;
+  StepInline inl;
+  StepSeq* h_seqs = inl.seqs;
+  int slot = -1;
+  uint8_t* hb = nullptr;
+  if (!inline_step) {
+    slot = c->stage_next;
+    c->stage_next = (c->stage_next + 1) % kStageSlots;
+    if (c->stage_used[slot]) QC_CUDA(cudaEventSynchronize(c->stage_done[slot]));   // its last copy must have run
+    hb = c->pinned + static_cast<size_t>(slot) * c->lay.step_bytes;
+    h_seqs = reinterpret_cast<StepSeq*>(hb + c->lay.step_seqs);
+    if (n_patches) std::memcpy(hb + c->lay.step_patches, patches.data(), n_patches * sizeof(Patch));
+  }
+  int64_t tot_v = 0, tot_t = 0, step_rows = 0;   // step_rows: K/V rows the step has to read (for the profile)
   for (int i = 0; i < n_seqs; ++i) {
     const int s = seq_ids[i];
     const SeqState& st = c->seqs[s];
     const int ncv = (pages_for(st.len_vis) + c->chunk_pages - 1) / c->chunk_pages;
     const int nct = (pages_for(st.len_text) + c->chunk_pages - 1) / c->chunk_pages;
-    h_seqs[i] = StepSeq{s, st.len_text, st.len_vis, ncv + nct};
+    h_seqs[i] = StepSeq{s, st.len_text, st.len_vis, ncv + nct, static_cast<int32_t>(tot_v),
+                        static_cast<int32_t>(tot_t), ncv, 0};
+    tot_v += static_cast<int64_t>(ncv) * c->items_per_chunk;
+    tot_t += static_cast<int64_t>(nct) * c->items_per_chunk;
+    step_rows += st.len_vis * c->visual_row_reads + st.len_text * c->text_row_reads;
   }
-  n_patches = static_cast<int>(patches.size());
-  if (n_patches) std::memcpy(h_patches, patches.data(), n_patches * sizeof(Patch));
-
-  // ---- segments, launch group by launch group
-  std::vector<LaunchGroup> groups;
-  {
-    const int nb = static_cast<int>(c->block_jobs.size());
-    const int per = c->layers_per_launch <= 0 ? nb : c->layers_per_launch;
-    for (int b = 0; b < nb; b += per) {
-      const int e = std::min(nb, b + per);
-      groups.push_back(LaunchGroup{c->block_jobs[b].first, c->block_jobs[e - 1].second, c->block_layers[b].first,
-                                   c->block_layers[e - 1].second});
-    }
-  }
-  int n_segs = 0, n_items = 0;
-  std::vector<std::pair<int, int>> group_items;
-  std::vector<int> order;
-  for (const LaunchGroup& g : groups) {
-    const int begin = n_items;
-    // items are claimed in list order: heaviest sweeps (most tiles per page, visual before
-    // text) first, so that the work left for the end of the launch comes in small pieces
-    order.resize(g.job_end - g.job_begin);
-    for (int j = g.job_begin; j < g.job_end; ++j) order[j - g.job_begin] = j;
-    std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
-      const Job &ja = c->jobs[a], &jb = c->jobs[b];
-      if (ja.n_cons != jb.n_cons) return ja.n_cons > jb.n_cons;
-      return ja.stream > jb.stream;
-    });
-    for (int j : order) {
-      const Job& jb = c->jobs[j];
-      for (int i = 0; i < n_seqs; ++i) {
-        const StepSeq& sq = h_seqs[i];
-        const int len = jb.stream ? sq.len_vis : sq.len_text;
-        if (len == 0) continue;
-        const int nch = (pages_for(len) + c->chunk_pages - 1) / c->chunk_pages;
-        const int ncv = (pages_for(sq.len_vis) + c->chunk_pages - 1) / c->chunk_pages;
-        h_segs[n_segs++] = Seg{j, i, sq.seq_id, len, n_items, nch, jb.stream ? 0 : ncv, 0};
-        n_items += nch * c->items_per_chunk;
-        step_rows += static_cast<int64_t>(len) * (1 + jb.n_cons);
-      }
-    }
-    group_items.emplace_back(begin, n_items);
-  }
+  const int n_pos = static_cast<int>(c->plan.size());
+  const int64_t n_items64 = c->plan_vis_before[n_pos] * tot_v + c->plan_text_before[n_pos] * tot_t;
+  const int n_items = static_cast<int>(n_items64);   // <= max_items: the item list was sized at allocation
 
   // ---- enqueue
-  QC_CUDA(cudaMemcpyAsync(c->ws + c->lay.step, hb, c->lay.step_bytes, cudaMemcpyHostToDevice, stream));
-  QC_CUDA(cudaEventRecord(c->stage_done[slot], stream));
-  c->stage_used[slot] = true;
+  if (!inline_step) {
+    QC_CUDA(cudaMemcpyAsync(c->ws + c->lay.step, hb, c->lay.step_bytes, cudaMemcpyHostToDevice, stream));
+    QC_CUDA(cudaEventRecord(c->stage_done[slot], stream));
+    c->stage_used[slot] = true;
+  }
 
   Params p = base_params(c);
   p.q = static_cast<const uint16_t*>(q_dev);
@@ -740,9 +765,13 @@ int32_t qc_decode_step(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, cons
   p.out = static_cast<uint16_t*>(out_dev);
   p.lse = lse_out_dev;
   p.n_seqs = n_seqs;
-  p.n_segs = n_segs;
+  p.n_pos = n_pos;
   p.n_items = n_items;
   p.n_patches = n_patches;
+  p.tot_v = static_cast<int32_t>(tot_v);
+  p.tot_t = static_cast<int32_t>(tot_t);
+  p.inline_seqs = inline_step ? 1 : 0;
+  p.fused_append = n_patches == 0 ? 1 : 0;   // the append reads the page table: not beside its patches
 
   cudaEvent_t* ev = nullptr;
   if (c->profile && c->ev_steps < kMaxProfileSteps) {
@@ -756,22 +785,28 @@ int32_t qc_decode_step(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, cons
     ev = &c->ev[4 * c->ev_steps];
     QC_CUDA(cudaEventRecord(ev[0], stream));
   }
-  QC_CUDA(launch_setup(p, stream));
-  QC_CUDA(launch_append(p, stream));
-  for (size_t gi = 0; gi < groups.size(); ++gi) {
-    p.item_begin = group_items[gi].first;
-    p.item_end = group_items[gi].second;
-    p.layer_begin = groups[gi].layer_begin;
-    p.layer_end = groups[gi].layer_end;
+  QC_CUDA(launch_setup(p, inline_step ? &inl : nullptr, stream));
+  c->kernel_launches++;
+  if (!p.fused_append) {
+    QC_CUDA(launch_append(p, stream));
+    c->kernel_launches++;
+  }
+  for (size_t gi = 0; gi < c->groups.size(); ++gi) {
+    const int pb = c->group_pos[gi].first, pe = c->group_pos[gi].second;
+    p.item_begin = static_cast<int32_t>(c->plan_vis_before[pb] * tot_v + c->plan_text_before[pb] * tot_t);
+    p.item_end = static_cast<int32_t>(c->plan_vis_before[pe] * tot_v + c->plan_text_before[pe] * tot_t);
+    p.layer_begin = c->groups[gi].layer_begin;
+    p.layer_end = c->groups[gi].layer_end;
     p.launch_index = static_cast<int32_t>(gi);
     if (ev && gi == 0) QC_CUDA(cudaEventRecord(ev[1], stream));
     if (c->group > 1)
       QC_CUDA(launch_attend_tc(p, c->ctx->n_sms, stream));
     else
       QC_CUDA(launch_attend(p, c->ctx->n_sms, stream));
-    if (ev && gi + 1 == groups.size()) QC_CUDA(cudaEventRecord(ev[2], stream));
+    if (ev && gi + 1 == c->groups.size()) QC_CUDA(cudaEventRecord(ev[2], stream));
     QC_CUDA(launch_merge(p, stream));
     c->attend_launches++;
+    c->kernel_launches += 2;
   }
   if (ev) {
     QC_CUDA(cudaEventRecord(ev[3], stream));
@@ -858,6 +893,7 @@ int32_t qc_get_stats(qc_cache* c, qc_stats* out) {
   out->qcache_bytes = static_cast<int64_t>(N) * c->cfg.max_seqs * c->hq * c->D * 2;
   out->decode_steps = c->decode_steps;
   out->attend_launches = c->attend_launches;
+  out->kernel_launches = c->kernel_launches;
   QC_CUDA(cudaSetDevice(c->ctx->device));
   int32_t err = 0;
   QC_CUDA(cudaMemcpyAsync(&err, c->ws + c->lay.err, sizeof(err), cudaMemcpyDeviceToHost, c->ctx->stream));
@@ -931,6 +967,7 @@ int32_t qc_set_option(qc_cache* c, const char* key, int64_t value) {
   if (k == "layers_per_launch") {
     if (value < 0 || value > c->cfg.n_layers) return QC_ERR_INVALID_ARG;
     c->layers_per_launch = static_cast<int>(value);
+    c->plan_dirty = true;
     return QC_OK;
   }
   if (k == "profile") {
