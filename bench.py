@@ -166,10 +166,10 @@ def cpu_oracle_sample(w, mode: int, first_step: int, budget_s: float = 12.0):
 # GPU arms
 # ------------------------------------------------------------------------------------------
 
-def _gen_inputs(w, first, count, device):
+def _gen_inputs(w, first, count, device, seq_offset=0):
     from paper_2602_01901_b200 import workloads as W
 
-    return [W.decode_qkv_torch(w, s, device) for s in range(first, first + count)]
+    return [W.decode_qkv_torch(w, s, device, seq_offset) for s in range(first, first + count)]
 
 
 def run_gpu(args, w, mode, rank, world, local_rank):
@@ -178,25 +178,16 @@ def run_gpu(args, w, mode, rank, world, local_rank):
     from paper_2602_01901_b200 import binding as qc
     from paper_2602_01901_b200.session import Session
 
-    dist = None
-    if world > 1:
-        import torch.distributed as dist_mod
+    from paper_2602_01901_b200.ranks import RankGroup
 
-        dist = dist_mod
-        torch.cuda.set_device(local_rank)
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    group = RankGroup()          # NCCL when launched by torchrun with WORLD_SIZE > 1
+    seq_offset = rank * w.batch  # every rank serves its own sequences of the global batch
 
     def barrier():
-        if dist is not None:
-            dist.barrier()
+        group.barrier()
         torch.cuda.synchronize()
 
-    def max_over_ranks(x: float) -> float:
-        if dist is None:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=f"cuda:{local_rank}")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+    max_over_ranks = group.max_over_ranks
 
     W_, K = args.warmup, args.steps
     total_steps = W_ + K
@@ -208,8 +199,8 @@ def run_gpu(args, w, mode, rank, world, local_rank):
 
     # ---- arm 1: inputs resident in HBM ---------------------------------------------------
     s = Session.for_workload(w, lazy_mode=mode, device=local_rank, split_tokens=args.split_tokens)
-    s.prefill_workload(w)
-    inputs = _gen_inputs(w, 0, total_steps, dev)
+    s.prefill_workload(w, seq_offset)
+    inputs = _gen_inputs(w, 0, total_steps, dev, seq_offset)
     out = torch.empty(shape_o, dtype=torch.bfloat16, device=dev)
     for i in range(W_):
         s.decode_step(ids, *inputs[i], out)
@@ -233,29 +224,55 @@ def run_gpu(args, w, mode, rank, world, local_rank):
     if not np.isfinite(checksum) or checksum == 0.0:
         raise SystemExit("output is not finite / all zero")
     s.close()
-    del s, inputs
+    del s
+
+    # ---- arm 1b (one GPU only): the same steps on a cache whose layers are all ordinary -------
+    all_full = None
+    if world == 1 and not args.no_all_full:
+        s = Session.for_workload(w, lazy_mode=mode, device=local_rank, split_tokens=args.split_tokens, all_full=True)
+        s.prefill_workload(w, seq_offset)
+        for i in range(W_):
+            s.decode_step(ids, *inputs[i], out)
+        torch.cuda.synchronize()
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        f0.record()
+        for i in range(W_, total_steps):
+            s.decode_step(ids, *inputs[i], out)
+        f1.record()
+        torch.cuda.synchronize()
+        ms_full = f0.elapsed_time(f1)
+        st_full = s.stats()
+        s.close()
+        del s
+        all_full = {"ms_per_step": ms_full / K, "tokens_per_s": w.batch * K / (ms_full / 1e3),
+                    "kv_bytes_stored": st_full.kv_bytes_stored, "speedup_of_lazy": ms_full / ms,
+                    "note": "same inputs and steps, every layer ordinary (Eq. 2 only)"}
+    del inputs
     torch.cuda.empty_cache()
 
     # ---- arm 2: host buffers through qc_decode_step_host -----------------------------------
     Ke = min(K, args.e2e_steps)
     s = Session.for_workload(w, lazy_mode=mode, device=local_rank, split_tokens=args.split_tokens)
-    s.prefill_workload(w)
-    dev_in = _gen_inputs(w, 0, W_ + Ke, dev)
+    s.prefill_workload(w, seq_offset)
+    dev_in = _gen_inputs(w, 0, W_ + Ke, dev, seq_offset)
     for i in range(W_):
         s.decode_step(ids, *dev_in[i], out)
     host_in = [tuple(t.cpu().pin_memory() for t in dev_in[i]) for i in range(W_, W_ + Ke)]
     host_out = torch.empty(shape_o, dtype=torch.bfloat16).pin_memory()
     del dev_in
     barrier()
-    t0 = time.perf_counter()
+    g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    g0.record()
     for i in range(Ke):
         s.decode_step_host(ids, *host_in[i], host_out)     # returns after the copy back has finished
-    torch.cuda.synchronize()
-    e2e_s = max_over_ranks(time.perf_counter() - t0)
+    g1.record()
+    barrier()
+    e2e_s = max_over_ranks(g0.elapsed_time(g1)) / 1e3
     h2d = sum(t.numel() * 2 for t in host_in[0])
     d2h = host_out.numel() * 2
     s.close()
 
+    group.close()
     if rank != 0:
         return None
     peak, peak_kind = _peaks()
@@ -293,6 +310,7 @@ def run_gpu(args, w, mode, rank, world, local_rank):
             "saved_frac_paged": 1 - st.kv_bytes_stored_paged / st.kv_bytes_all_full_paged,
             "qcache_bytes": st.qcache_bytes,
         },
+        "vs_all_full": all_full,
         "step_ms_by_events": prof.step_ms / max(1, prof.steps),
         "paper_context": "paper reports ~35% KV saved and 1.5x-1.6x decode throughput for LLaVA-NeXT-7B on one 80GB A100 (whole model)",
     }
@@ -309,6 +327,7 @@ def main():
     ap.add_argument("--mode", default="vla_qc", choices=sorted(MODES))
     ap.add_argument("--e2e-steps", type=int, default=64)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-all-full", action="store_true", help="skip the all-ordinary-layers comparison run")
     ap.add_argument("--split-tokens", type=int, default=0, help="keys per split-KV work item (0 = library default)")
     ap.add_argument("--layers", type=int, default=0, help="cut the stack to its first N layers (profiling-size case)")
     ap.add_argument("--batch", type=int, default=0, help="override the batch (profiling-size case)")
@@ -354,10 +373,6 @@ def main():
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_oracle_sample(w, mode, args.warmup)
         print(json.dumps(line))
-    if world > 1:
-        import torch.distributed as dist
-
-        dist.destroy_process_group()
 
 
 if __name__ == "__main__":

@@ -41,8 +41,9 @@ class Session:
     def for_workload(cls, w: W.Workload, lazy_mode=qc.QC_MODE_VLA_QC, split_tokens=0, device=0,
                      all_full=False, poison_pool=False, slack_pages=0) -> "Session":
         kind = np.zeros(w.n_layers, np.uint8) if all_full else w.layer_kind()
-        pages_per_stream = (w.max_tokens + 15) // 16 + 1
-        n_pages = w.n_layers * 4 * w.batch * pages_per_stream + slack_pages if w.page_size else 0
+        # room for an all-ordinary cache at the end of decoding: K and V, visual + text streams
+        pages_per_tensor = (w.n_visual_kept + 15) // 16 + (w.n_text_prompt + w.decode_steps + 15) // 16
+        n_pages = w.n_layers * 2 * w.batch * pages_per_tensor + slack_pages if w.page_size else 0
         return cls(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, kind.tolist(), page_size=w.page_size,
                    max_seqs=w.batch, max_tokens_per_seq=w.max_tokens, n_pages=n_pages, lazy_mode=lazy_mode,
                    split_tokens=split_tokens, device=device, poison_pool=poison_pool)
@@ -62,10 +63,11 @@ class Session:
         qc.qc_decode_step_host(self.cache, seq_ids, q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
                                lse.data_ptr() if lse is not None else 0)
 
-    def prefill_workload(self, w: W.Workload):
-        """Prefill every sequence of a synthetic workload, one sequence per call."""
+    def prefill_workload(self, w: W.Workload, seq_offset: int = 0):
+        """Prefill every sequence of a synthetic workload, one sequence per call.  Library
+        sequence s holds the generator's sequence ``seq_offset + s``."""
         for s in range(w.batch):
-            kind, k, v = W.prefill_kv_torch(w, s, self.device)
+            kind, k, v = W.prefill_kv_torch(w, seq_offset + s, self.device)
             self.prefill_append([s], [len(kind)], kind, k, v)
             del k, v
 

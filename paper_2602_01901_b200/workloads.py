@@ -128,6 +128,11 @@ WORKLOADS: Tuple[Workload, ...] = (
     Workload(2, "llava_next_anyres", 32, 32, 32, 128, 16, 8, 35, 2880, 2880, 93, 512, _odd(3, 31)),
     Workload(3, "qwen2vl_gqa", 28, 28, 4, 128, 16, 32, 35, 1024, 1024, 61, 256, _odd(3, 27)),
     Workload(4, "long_video_pruned", 32, 32, 32, 128, 16, 4, 35, 8192, 4096, 221, 2048, _odd(3, 31)),
+    # Beyond the five benchmark shapes: the regime of the paper's efficiency evaluation (7B MHA
+    # stack, input length 2048, batch 32, about 35 % of the KV cache saved): 22 of 32 layers lazy,
+    # in blocks of one ordinary layer followed by three lazy ones.
+    Workload(5, "llava_next_2048_lazy22", 32, 32, 32, 128, 16, 32, 35, 1920, 1920, 93, 256,
+             tuple(l for l in range(2, 32) if (l - 2) % 4 != 0)),
 )
 
 
@@ -301,9 +306,11 @@ def prefill_kv_torch(w: Workload, seq: int, device):
     return kind, k, v
 
 
-def decode_qkv_torch(w: Workload, step: int, device):
-    """Device twin of ``decode_qkv_np`` for the whole batch (bf16 tensors)."""
+def decode_qkv_torch(w: Workload, step: int, device, seq_offset: int = 0):
+    """Device twin of ``decode_qkv_np`` for the whole batch (bf16 tensors).  ``seq_offset``
+    shifts the sequence coordinate: rank r of a multi-GPU run draws sequences r*batch ..."""
     one = lambda tensor, n_heads: draw_block_torch(
-        w.seed, tensor, _all(w.n_layers), _all(w.batch), [step], _all(n_heads), w.head_dim, device
+        w.seed, tensor, _all(w.n_layers), range(seq_offset, seq_offset + w.batch), [step], _all(n_heads), w.head_dim,
+        device
     )[:, :, 0].contiguous()
     return one(T_DECODE_Q, w.n_q_heads), one(T_DECODE_K, w.n_kv_heads), one(T_DECODE_V, w.n_kv_heads)

@@ -267,6 +267,47 @@ def _samples(w, n, rng):
     return out
 
 
+@pytest.mark.parametrize("mode", MODES, ids=MODE_IDS)
+def test_multi_turn_prefill_after_decode(mode):
+    """A conversation with a second image: prompt, a few generated tokens, more prompt tokens
+    (text and visual) appended to the same sequence, more generated tokens."""
+    layer_kind = [0, 1, 1, 0, 1]
+    w = _small_workload(128, 2, layer_kind, 23)
+    n_pages = w.n_layers * 4 * 2 * 24
+    s = Session(w.n_layers, w.n_q_heads, w.n_kv_heads, 128, layer_kind, max_seqs=2, max_tokens_per_seq=384,
+                n_pages=n_pages, lazy_mode=mode, split_tokens=64, poison_pool=True)
+    o = LazyAttentionOracle(w.n_layers, w.n_q_heads, w.n_kv_heads, 128, layer_kind, mode, n_seqs=2)
+    model = pg.PagedCacheModel(layer_kind, mode, 16, n_pages, 2)
+    dev = lambda a: torch.from_numpy(a.astype(np.int16)).view(torch.bfloat16).to(s.device).contiguous()
+    kinds, ks, vs = zip(*[W.prefill_kv_np(w, b) for b in range(2)])
+    out = torch.empty((w.n_layers, 2, w.n_q_heads, 128), dtype=torch.bfloat16, device=s.device)
+    step = 0
+
+    def turn(first, last, n_decode):
+        nonlocal step
+        for b in range(2):
+            kd, k, v = kinds[b][first:last], ks[b][:, first:last], vs[b][:, first:last]
+            s.prefill_append([b], [last - first], kd, dev(k), dev(v))
+            o.prefill_append(b, kd.tolist(), f64(k), f64(v))
+            model.prefill_append([b], [int((kd == 0).sum())], [int((kd == 1).sum())])
+        for _ in range(n_decode):
+            qn, kn, vn = W.decode_qkv_np(w, step, seqs=[0, 1])
+            s.decode_step([0, 1], dev(qn), dev(kn), dev(vn), out)
+            model.decode_step([0, 1])
+            got = bits_of(out)
+            for b in range(2):
+                ref, _ = o.decode_step(b, f64(qn[:, b]), f64(kn[:, b]), f64(vn[:, b]))
+                for l in range(w.n_layers):
+                    assert_close(got[l, b], ref[l], f"turn ending at {last}, step {step}, seq {b}, layer {l}")
+            step += 1
+        _compare_tables(s, model, w.n_layers, [0, 1])
+
+    turn(0, 60, 5)          # 5 text + 55 visual tokens, then 5 generated
+    turn(60, 177, 7)        # the rest of the image and the trailing text arrive later
+    assert s.stats().device_error == 0
+    s.close()
+
+
 FULL_CASES = [
     ("llava15_7b", qc.QC_MODE_VLA_QC, 40),
     ("llava15_7b", qc.QC_MODE_VLA_EQ8, 16),
@@ -274,6 +315,8 @@ FULL_CASES = [
     ("llava_next_anyres", qc.QC_MODE_VLA_QC, 32),
     ("qwen2vl_gqa", qc.QC_MODE_VLA_QC, 40),
     ("long_video_pruned", qc.QC_MODE_VLA_QC, 24),
+    ("llava_next_2048_lazy22", qc.QC_MODE_VLA_QC, 24),     # blocks of one ordinary + three lazy layers
+    ("llava_next_2048_lazy22", qc.QC_MODE_GLA, 16),
 ]
 
 

@@ -126,7 +126,7 @@ def test_vanilla_cache_size_matches_table_3():
 
 
 def test_workload_shapes_follow_the_config_strings():
-    tiny, c2, c3, c4, c5 = W.WORKLOADS
+    tiny, c2, c3, c4, c5 = W.WORKLOADS[:5]
     assert (tiny.n_prompt, tiny.max_tokens) == (672, 688)
     pos, kind = tiny.prompt_layout(0)
     assert kind[64] == 1 and kind[63] == 0 and kind[639] == 1 and kind[640] == 0
