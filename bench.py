@@ -200,6 +200,8 @@ def run_gpu(args, w, mode, rank, world, local_rank):
     # ---- arm 1: inputs resident in HBM ---------------------------------------------------
     s = Session.for_workload(w, lazy_mode=mode, device=local_rank, split_tokens=args.split_tokens)
     s.prefill_workload(w, seq_offset)
+    if args.blocks_per_launch:
+        s.set_option("layers_per_launch", args.blocks_per_launch)
     inputs = _gen_inputs(w, 0, total_steps, dev, seq_offset)
     out = torch.empty(shape_o, dtype=torch.bfloat16, device=dev)
     for i in range(W_):
@@ -329,6 +331,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-all-full", action="store_true", help="skip the all-ordinary-layers comparison run")
     ap.add_argument("--split-tokens", type=int, default=0, help="keys per split-KV work item (0 = library default)")
+    ap.add_argument("--blocks-per-launch", type=int, default=0,
+                    help="0 = one attention launch per step; k = one launch per k lazy blocks, in layer order")
     ap.add_argument("--layers", type=int, default=0, help="cut the stack to its first N layers (profiling-size case)")
     ap.add_argument("--batch", type=int, default=0, help="override the batch (profiling-size case)")
     args = ap.parse_args()

@@ -227,6 +227,8 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
     fence_mbar_init();
   }
   __syncthreads();
+  pdl_launch_dependents();
+  pdl_wait();
 
   WorkerState st;
   worker_init(st, 0);
@@ -291,10 +293,8 @@ cudaError_t launch_attend_tc(const Params& p, int n_sms, cudaStream_t stream) {
   if (n_items <= 0) return cudaSuccess;
   const int grid = min(n_sms, (n_items + kWarps - 1) / kWarps);
   if (p.d == 128)
-    attend_tc_kernel<128><<<grid, kThreads, attend_tc_smem_bytes<128>(), stream>>>(p);
-  else
-    attend_tc_kernel<64><<<grid, kThreads, attend_tc_smem_bytes<64>(), stream>>>(p);
-  return cudaGetLastError();
+    return launch_pdl(attend_tc_kernel<128>, dim3(grid), dim3(kThreads), attend_tc_smem_bytes<128>(), stream, p);
+  return launch_pdl(attend_tc_kernel<64>, dim3(grid), dim3(kThreads), attend_tc_smem_bytes<64>(), stream, p);
 }
 
 }  // namespace qc

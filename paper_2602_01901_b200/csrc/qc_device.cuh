@@ -7,6 +7,8 @@
 
 #include <math.h>
 
+#include <utility>
+
 namespace qc {
 namespace {
 
@@ -65,6 +67,31 @@ __device__ __forceinline__ void tensor_g2s_2d(uint32_t dst_smem, const void* tma
           "r"(dst_smem),
       "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(smem_u32(bar))
       : "memory");
+}
+
+// Programmatic dependent launch: the kernels of a decode step are launched back to back with
+// the programmatic-serialization attribute.  Each one first lets its successor start getting
+// scheduled, does its set-up that touches no global data, and then waits for its predecessor
+// to have completed (and its writes to be visible) before it reads or writes global memory.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// Launch with the programmatic-serialization attribute (plain stream order if the predecessor
+// in the stream is not a kernel).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                              Args&&... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
 
 __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {

@@ -59,6 +59,8 @@ __device__ __forceinline__ void append_rows(const Params& P, const StepSeq& sq, 
 // n_layers blocks do the append.  (The append reads page ids from the table, so it is only
 // fused on steps without patches.)
 __global__ void setup_kernel(const __grid_constant__ Params P, const __grid_constant__ StepInline inl) {
+  pdl_launch_dependents();
+  pdl_wait();
   const StepSeq* seqs = P.inline_seqs ? inl.seqs : P.seqs;
   const int n_expand = P.n_pos * P.n_seqs;
   const int n_house = (max(max(P.n_patches, P.n_layers), P.n_seqs * 8) + blockDim.x - 1) / blockDim.x;
@@ -126,6 +128,8 @@ __global__ void setup_kernel(const __grid_constant__ Params P, const __grid_cons
 // ------------------------------------------------------------------------------------------
 
 __global__ void append_kernel(const __grid_constant__ Params P) {
+  pdl_launch_dependents();
+  pdl_wait();
   append_rows(P, P.seqs[blockIdx.x], blockIdx.x, blockIdx.y);
 }
 
@@ -360,6 +364,8 @@ __global__ void __launch_bounds__(kThreads, 1) attend_kernel(const __grid_consta
     fence_mbar_init();
   }
   __syncthreads();
+  pdl_launch_dependents();
+  pdl_wait();
 
   WorkerState st;
   worker_init(st, 0);
@@ -409,8 +415,10 @@ __global__ void __launch_bounds__(kThreads, 1) attend_kernel(const __grid_consta
 // ------------------------------------------------------------------------------------------
 
 template <int D>
-__global__ void merge_kernel(Params P) {
+__global__ void merge_kernel(const __grid_constant__ Params P) {
   constexpr int VPL = D / 32;
+  pdl_launch_dependents();
+  pdl_wait();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_layers = P.layer_end - P.layer_begin;
   const int idx = blockIdx.x * (blockDim.x >> 5) + warp;
@@ -488,14 +496,12 @@ cudaError_t launch_setup(const Params& p, const StepInline* inl, cudaStream_t st
   const int n_house = (max(max(p.n_patches, p.n_layers), p.n_seqs * 8) + kBlock - 1) / kBlock;
   const int blocks = p.n_pos * p.n_seqs + n_house + (p.fused_append ? p.n_seqs * p.n_layers : 0);
   static const StepInline kNone{};
-  setup_kernel<<<blocks, kBlock, 0, stream>>>(p, inl ? *inl : kNone);
-  return cudaGetLastError();
+  return launch_pdl(setup_kernel, dim3(blocks), dim3(kBlock), 0, stream, p, inl ? *inl : kNone);
 }
 
 cudaError_t launch_append(const Params& p, cudaStream_t stream) {
   dim3 grid(p.n_seqs, p.n_layers);
-  append_kernel<<<grid, 128, 0, stream>>>(p);
-  return cudaGetLastError();
+  return launch_pdl(append_kernel, grid, dim3(128), 0, stream, p);
 }
 
 cudaError_t launch_attend(const Params& p, int n_sms, cudaStream_t stream) {
@@ -503,10 +509,8 @@ cudaError_t launch_attend(const Params& p, int n_sms, cudaStream_t stream) {
   if (n_items <= 0) return cudaSuccess;
   const int grid = min(n_sms, (n_items + kWarps - 1) / kWarps);
   if (p.d == 128)
-    attend_kernel<128><<<grid, kThreads, attend_smem_bytes<128>(), stream>>>(p);
-  else
-    attend_kernel<64><<<grid, kThreads, attend_smem_bytes<64>(), stream>>>(p);
-  return cudaGetLastError();
+    return launch_pdl(attend_kernel<128>, dim3(grid), dim3(kThreads), attend_smem_bytes<128>(), stream, p);
+  return launch_pdl(attend_kernel<64>, dim3(grid), dim3(kThreads), attend_smem_bytes<64>(), stream, p);
 }
 
 cudaError_t launch_merge(const Params& p, cudaStream_t stream) {
@@ -515,10 +519,8 @@ cudaError_t launch_merge(const Params& p, cudaStream_t stream) {
   const int warps_per_block = 8;
   const int blocks = (n + warps_per_block - 1) / warps_per_block;
   if (p.d == 128)
-    merge_kernel<128><<<blocks, warps_per_block * 32, 0, stream>>>(p);
-  else
-    merge_kernel<64><<<blocks, warps_per_block * 32, 0, stream>>>(p);
-  return cudaGetLastError();
+    return launch_pdl(merge_kernel<128>, dim3(blocks), dim3(warps_per_block * 32), 0, stream, p);
+  return launch_pdl(merge_kernel<64>, dim3(blocks), dim3(warps_per_block * 32), 0, stream, p);
 }
 
 cudaError_t launch_prefill_scatter(const Params& p, const int32_t* tok_seq, const int32_t* tok_stream,
