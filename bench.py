@@ -249,6 +249,30 @@ def run_gpu(args, w, mode, rank, world, local_rank):
         all_full = {"ms_per_step": ms_full / K, "tokens_per_s": w.batch * K / (ms_full / 1e3),
                     "kv_bytes_stored": st_full.kv_bytes_stored, "speedup_of_lazy": ms_full / ms,
                     "note": "same inputs and steps, every layer ordinary (Eq. 2 only)"}
+    # ---- arm 1c (one GPU only): the same steps with one attention launch per lazy block, in layer
+    # order: the schedule of a model that computes a layer's q/k/v from the previous layer's output
+    per_block = None
+    if world == 1 and not args.no_per_block and not args.blocks_per_launch:
+        s = Session.for_workload(w, lazy_mode=mode, device=local_rank, split_tokens=args.split_tokens)
+        s.prefill_workload(w, seq_offset)
+        s.set_option("layers_per_launch", 1)
+        for i in range(W_):
+            s.decode_step(ids, *inputs[i], out)
+        torch.cuda.synchronize()
+        launches0 = s.stats().kernel_launches
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        f0.record()
+        for i in range(W_, total_steps):
+            s.decode_step(ids, *inputs[i], out)
+        f1.record()
+        torch.cuda.synchronize()
+        ms_pb = f0.elapsed_time(f1)
+        per_block = {"ms_per_step": ms_pb / K, "tokens_per_s": w.batch * K / (ms_pb / 1e3),
+                     "gpu_launches": int(s.stats().kernel_launches - launches0),
+                     "kv_gb_per_s_whole_step": prof.kv_bytes_read / (ms_pb / 1e3) / 1e9,
+                     "note": "one attention + merge launch per lazy block, blocks in layer order"}
+        s.close()
+        del s
     del inputs
     torch.cuda.empty_cache()
 
@@ -313,6 +337,7 @@ def run_gpu(args, w, mode, rank, world, local_rank):
             "qcache_bytes": st.qcache_bytes,
         },
         "vs_all_full": all_full,
+        "per_block_launches": per_block,
         "step_ms_by_events": prof.step_ms / max(1, prof.steps),
         "paper_context": "paper reports ~35% KV saved and 1.5x-1.6x decode throughput for LLaVA-NeXT-7B on one 80GB A100 (whole model)",
     }
@@ -330,6 +355,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=64)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-all-full", action="store_true", help="skip the all-ordinary-layers comparison run")
+    ap.add_argument("--no-per-block", action="store_true", help="skip the launch-per-lazy-block comparison run")
     ap.add_argument("--split-tokens", type=int, default=0, help="keys per split-KV work item (0 = library default)")
     ap.add_argument("--blocks-per-launch", type=int, default=0,
                     help="0 = one attention launch per step; k = one launch per k lazy blocks, in layer order")

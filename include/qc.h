@@ -82,7 +82,7 @@ typedef struct qc_config {
   int32_t split_tokens;        /* keys per split-KV work item, a multiple of 16 in 16..512.  Every
                                   stream is cut into ceil(len/split_tokens) chunks whose partial
                                   results are merged by log-sum-exp.  0 => chosen per step among
-                                  128, 256 and 512 from the amount of work (workspace sized for 128). */
+                                  64, 128, 256 and 512 from the amount of work (workspace sized for 64). */
   const uint8_t* layer_kind;   /* host, [n_layers], QC_LAYER_*; layer 0 must be FULL; copied */
 } qc_config;
 

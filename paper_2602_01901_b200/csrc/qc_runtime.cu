@@ -223,7 +223,7 @@ int compute_sizes(const qc_config* cfg, Sizes* s) {
   s->hq = cfg->n_q_heads;
   s->hkv = cfg->n_kv_heads;
   s->max_pages = (cfg->max_tokens_per_seq + kPage - 1) / kPage;
-  const int split = cfg->split_tokens ? cfg->split_tokens : 128;
+  const int split = cfg->split_tokens ? cfg->split_tokens : 64;   // auto: the smallest chunk the per-step choice may take
   s->chunk_pages = split / kPage;
   s->max_slots = 2 * ((s->max_pages + s->chunk_pages - 1) / s->chunk_pages);
   s->page_bytes = static_cast<size_t>(s->hkv) * kPage * s->D * 2;
@@ -704,8 +704,10 @@ int32_t qc_decode_step(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, cons
     // work items to balance over the workers.  Take the largest chunk that still leaves
     // every worker several items per launch.
     const int64_t want = 5LL * c->ctx->n_sms * kAttendWarps * static_cast<int64_t>(c->groups.size());
-    int pick = c->min_chunk_pages;
-    for (int cp = kMaxChunkPages; cp > c->min_chunk_pages; cp /= 2) {
+    // (a query group writes one partial row per head and chunk: its chunks stay at 128 keys or more)
+    const int floor_pages = c->group > 1 ? std::max(c->min_chunk_pages, 8) : c->min_chunk_pages;
+    int pick = floor_pages;
+    for (int cp = kMaxChunkPages; cp > floor_pages; cp /= 2) {
       int64_t cv = 0, ct = 0;
       for (int i = 0; i < n_seqs; ++i) {
         const SeqState& st = c->seqs[seq_ids[i]];
