@@ -137,6 +137,23 @@ int32_t qc_prefill_append(qc_cache* cache, int32_t n_seqs, const int32_t* seq_id
                           const int32_t* n_tokens, const uint8_t* kind, const void* k_dev,
                           const void* v_dev);
 
+/* Prefill attention of one sequence's whole prompt, all layers, followed by what
+ * qc_prefill_append does with the same k/v (section "Q Cache", prefilling forms):
+ *   ordinary layer  Eq. 1: causal softmax((Q K^T + M)/sqrt(D)) V over the prompt;
+ *   GLA lazy layer  Eq. 5: Q = Q Cache (the queries of the block's first layer for every prompt
+ *                   token), K = that layer's K, V own;
+ *   VLA lazy layer  Eq. 7 (both VLA modes): query rows and key rows of VISUAL tokens come from
+ *                   the block's first layer, those of text tokens are the layer's own; V own.
+ * Token t of the prompt sees tokens 0..t in the order given (kind[t] tags it text or visual).
+ *   q_dev   bf16 [n_layers][n_tokens][n_q_heads][head_dim]   (the Q Cache of a block is its first
+ *           layer's slice of this tensor; nothing prompt-sized is kept afterwards)
+ *   k_dev, v_dev bf16 [n_layers][n_tokens][n_kv_heads][head_dim]
+ *   out_dev bf16 [n_layers][n_tokens][n_q_heads][head_dim]
+ * The sequence must be new or empty (a prompt that continues a cached sequence returns
+ * QC_ERR_UNSUPPORTED).  Errors of qc_prefill_append apply; on an error nothing is stored or written. */
+int32_t qc_prefill_attend(qc_cache* cache, int32_t seq_id, int32_t n_tokens, const uint8_t* kind,
+                          const void* q_dev, const void* k_dev, const void* v_dev, void* out_dev);
+
 /* One generated (text) token for each listed sequence through all layers (Eq. 2, 6, 8):
  * appends k/v, refreshes the Q Cache from every ordinary layer's q, computes split-KV partial
  * attention and merges the partials by log-sum-exp.

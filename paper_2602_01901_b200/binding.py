@@ -28,7 +28,7 @@ QC_STREAM_K_TEXT, QC_STREAM_K_VISUAL, QC_STREAM_V_TEXT, QC_STREAM_V_VISUAL = 0, 
 QC_KIND_TEXT, QC_KIND_VISUAL = 0, 1
 
 EXPORTS = (
-    "qc_init", "qc_cache_bytes_required", "qc_alloc_cache", "qc_prefill_append", "qc_decode_step",
+    "qc_init", "qc_cache_bytes_required", "qc_alloc_cache", "qc_prefill_append", "qc_prefill_attend", "qc_decode_step",
     "qc_decode_step_host", "qc_free_seq", "qc_free", "qc_get_stats", "qc_debug_page_table",
     "qc_debug_read_qcache", "qc_debug_read_row", "qc_set_option", "qc_get_profile", "qc_status_string",
     "qc_attend_static",
@@ -89,6 +89,7 @@ def load() -> C.CDLL:
         "qc_cache_bytes_required": [C.POINTER(qc_config), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)],
         "qc_alloc_cache": [vp, C.POINTER(qc_config), vp, C.c_size_t, vp, C.c_size_t, C.POINTER(vp)],
         "qc_prefill_append": [vp, i32, pi32, pi32, pu8, vp, vp],
+        "qc_prefill_attend": [vp, i32, i32, pu8, vp, vp, vp, vp],
         "qc_decode_step": [vp, i32, pi32, vp, vp, vp, vp, vp],
         "qc_decode_step_host": [vp, i32, pi32, vp, vp, vp, vp, vp],
         "qc_free_seq": [vp, i32],
@@ -160,6 +161,14 @@ def qc_prefill_append(cache, seq_ids: Sequence[int], n_tokens: Sequence[int], ki
     _check(load().qc_prefill_append(cache, len(seq_ids), _i32_array(seq_ids), _i32_array(n_tokens),
                                     C.cast(kbuf, C.POINTER(C.c_uint8)), C.c_void_p(k_ptr), C.c_void_p(v_ptr)),
            "qc_prefill_append")
+
+
+def qc_prefill_attend(cache, seq_id: int, kind, q_ptr: int, k_ptr: int, v_ptr: int, out_ptr: int) -> None:
+    kind_bytes = bytes(bytearray(int(x) for x in kind)) if not isinstance(kind, (bytes, bytearray)) else bytes(kind)
+    kbuf = (C.c_uint8 * max(1, len(kind_bytes))).from_buffer_copy(kind_bytes or b"\0")
+    _check(load().qc_prefill_attend(cache, seq_id, len(kind_bytes), C.cast(kbuf, C.POINTER(C.c_uint8)),
+                                    C.c_void_p(q_ptr), C.c_void_p(k_ptr), C.c_void_p(v_ptr), C.c_void_p(out_ptr)),
+           "qc_prefill_attend")
 
 
 def qc_decode_step(cache, seq_ids, q_ptr: int, k_ptr: int, v_ptr: int, out_ptr: int, lse_ptr: int = 0) -> None:

@@ -118,6 +118,10 @@ cudaError_t launch_merge(const Params& p, cudaStream_t stream);
 cudaError_t launch_prefill_scatter(const Params& p, const int32_t* tok_seq, const int32_t* tok_stream,
                                    const int32_t* tok_ord, int32_t n_tokens, int32_t tok_stride,
                                    int32_t tok_offset, cudaStream_t stream);
+cudaError_t launch_prefill_attend(const Params& p, const uint8_t* kind_dev, const uint8_t* layer_kind_dev,
+                                  const uint8_t* leader_dev, const void* q, const void* k, const void* v, void* out,
+                                  int32_t n_tokens, int32_t gla, cudaStream_t stream);   // qc_prefill.cu
+cudaError_t configure_prefill_kernels();
 cudaError_t configure_kernels(int* attend_smem_bytes);
 cudaError_t configure_kernels_tc(int* attend_smem_bytes);
 

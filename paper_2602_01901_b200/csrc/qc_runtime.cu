@@ -34,7 +34,7 @@ struct LaunchGroup {
 };
 
 struct Layout {   // byte offsets into the workspace
-  size_t table, layer_flags, jobs, plan, qcache, part_acc, part_ml, items, step, err, counters, stage_q, stage_k, stage_v,
+  size_t table, layer_flags, layer_kind, leader, jobs, plan, qcache, part_acc, part_ml, items, step, err, counters, stage_q, stage_k, stage_v,
       stage_out, stage_lse, tok, total;
   size_t step_seqs, step_patches, step_bytes;   // offsets inside the step block
 };
@@ -252,6 +252,8 @@ int compute_sizes(const qc_config* cfg, Sizes* s) {
   const size_t N = cfg->n_layers, S = cfg->max_seqs;
   L.table = take(N * 4 * S * s->max_pages * sizeof(int32_t));
   L.layer_flags = take(N);
+  L.layer_kind = take(N);
+  L.leader = take(N);
   L.jobs = take(jobs.size() * sizeof(Job));
   L.plan = take(jobs.size() * sizeof(PlanJob));
   L.qcache = take(N * S * s->hq * s->D * 2);
@@ -432,6 +434,7 @@ int32_t qc_init(int32_t device, void* cuda_stream, qc_ctx** out) {
   int smem = 0, smem_tc = 0;
   QC_CUDA(configure_kernels(&smem));
   QC_CUDA(configure_kernels_tc(&smem_tc));
+  QC_CUDA(configure_prefill_kernels());
   if (static_cast<size_t>(std::max(smem, smem_tc)) > prop.sharedMemPerBlockOptin) return QC_ERR_UNSUPPORTED;
   qc_ctx* ctx = new (std::nothrow) qc_ctx();
   if (!ctx) return QC_ERR_INVALID_ARG;
@@ -530,6 +533,11 @@ int32_t qc_alloc_cache(qc_ctx* ctx, const qc_config* cfg, void* pool_dev, size_t
                              cudaMemcpyHostToDevice, stream) == cudaSuccess;
   ok = ok && cudaMemcpyAsync(c->ws + c->lay.layer_flags, c->layer_flags.data(), c->layer_flags.size(),
                              cudaMemcpyHostToDevice, stream) == cudaSuccess;
+  std::vector<uint8_t> leader8(c->leader.begin(), c->leader.end());
+  ok = ok && cudaMemcpyAsync(c->ws + c->lay.layer_kind, c->kind.data(), c->kind.size(), cudaMemcpyHostToDevice,
+                             stream) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(c->ws + c->lay.leader, leader8.data(), leader8.size(), cudaMemcpyHostToDevice,
+                             stream) == cudaSuccess;
   ok = ok && cudaMemcpyAsync(c->ws + c->lay.jobs, c->jobs.data(), c->jobs.size() * sizeof(Job),
                              cudaMemcpyHostToDevice, stream) == cudaSuccess;
   ok = ok && cudaMemsetAsync(c->ws + c->lay.err, 0, 256, stream) == cudaSuccess;
@@ -649,6 +657,32 @@ int32_t qc_prefill_append(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, c
     // the host vectors and the device token arrays are reused by the next batch
     QC_CUDA(cudaStreamSynchronize(stream));
   }
+  return QC_OK;
+}
+
+int32_t qc_prefill_attend(qc_cache* c, int32_t seq_id, int32_t n_tokens, const uint8_t* kind, const void* q_dev,
+                          const void* k_dev, const void* v_dev, void* out_dev) {
+  if (!c || n_tokens < 0 || seq_id < 0 || seq_id >= c->cfg.max_seqs) return QC_ERR_INVALID_ARG;
+  if (n_tokens == 0) return QC_OK;
+  if (!kind || !q_dev || !k_dev || !v_dev || !out_dev) return QC_ERR_INVALID_ARG;
+  const void* ptrs[4] = {q_dev, k_dev, v_dev, out_dev};
+  for (const void* ptr : ptrs)
+    if (reinterpret_cast<uintptr_t>(ptr) & 15) return QC_ERR_INVALID_ARG;
+  // the prompt attends to itself only: a sequence that already holds tokens is not covered
+  if (c->seqs[seq_id].active && (c->seqs[seq_id].len_text || c->seqs[seq_id].len_vis)) return QC_ERR_UNSUPPORTED;
+  if (static_cast<size_t>(n_tokens) > static_cast<size_t>(kPrefillBatchTokens) * 3 * sizeof(int32_t))
+    return QC_ERR_INVALID_ARG;
+  // store K/V first: this validates everything and leaves the cache unchanged on an error
+  int st = qc_prefill_append(c, 1, &seq_id, &n_tokens, kind, k_dev, v_dev);
+  if (st != QC_OK) return st;
+  cudaStream_t stream = c->ctx->stream;
+  uint8_t* kind_dev = c->ws + c->lay.tok;   // free again: qc_prefill_append has waited for its copies
+  QC_CUDA(cudaMemcpyAsync(kind_dev, kind, n_tokens, cudaMemcpyHostToDevice, stream));
+  QC_CUDA(cudaStreamSynchronize(stream));   // `kind` is the caller's host memory
+  const Params p = base_params(c);
+  QC_CUDA(launch_prefill_attend(p, kind_dev, c->ws + c->lay.layer_kind, c->ws + c->lay.leader, q_dev, k_dev, v_dev,
+                                out_dev, n_tokens, c->cfg.lazy_mode == QC_MODE_GLA ? 1 : 0, stream));
+  c->kernel_launches++;
   return QC_OK;
 }
 

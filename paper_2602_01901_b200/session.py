@@ -54,6 +54,12 @@ class Session:
         qc.qc_prefill_append(self.cache, list(seq_ids), list(n_tokens), bytes(bytearray(np.asarray(kind, np.uint8))),
                              k.data_ptr(), v.data_ptr())
 
+    def prefill_attend(self, seq_id: int, kind, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, out: torch.Tensor):
+        for t in (q, k, v, out):
+            assert t.dtype == torch.bfloat16 and t.is_contiguous()
+        qc.qc_prefill_attend(self.cache, seq_id, bytes(bytearray(np.asarray(kind, np.uint8))), q.data_ptr(),
+                             k.data_ptr(), v.data_ptr(), out.data_ptr())
+
     def decode_step(self, seq_ids, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, out: torch.Tensor,
                     lse: Optional[torch.Tensor] = None):
         qc.qc_decode_step(self.cache, seq_ids, q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),

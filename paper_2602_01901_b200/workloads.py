@@ -41,6 +41,7 @@ T_DECODE_Q = 2
 T_DECODE_K = 3
 T_DECODE_V = 4
 T_PRUNE = 5
+T_PREFILL_Q = 6
 
 
 @dataclass(frozen=True)
@@ -281,6 +282,25 @@ def prefill_kv_np(w: Workload, seq: int, layers=None, heads=None):
     k = draw_block_np(w.seed, T_PREFILL_K, layers, [seq], pos, heads, w.head_dim)[:, 0]
     v = draw_block_np(w.seed, T_PREFILL_V, layers, [seq], pos, heads, w.head_dim)[:, 0]
     return kind, k, v
+
+
+def prefill_q_np(w: Workload, seq: int, layers=None, heads=None):
+    """Query bits of one sequence's prompt, [n_layers, T, heads, D] (prefill attention only)."""
+    layers = _all(w.n_layers) if layers is None else layers
+    heads = _all(w.n_q_heads) if heads is None else heads
+    pos, _ = w.prompt_layout(seq)
+    return draw_block_np(w.seed, T_PREFILL_Q, layers, [seq], pos, heads, w.head_dim)[:, 0]
+
+
+def prefill_q_torch(w: Workload, seq: int, device):
+    """Device twin of ``prefill_q_np`` for all layers and heads (bf16 tensor)."""
+    import torch
+
+    pos, _ = w.prompt_layout(seq)
+    q = torch.empty((w.n_layers, len(pos), w.n_q_heads, w.head_dim), dtype=torch.bfloat16, device=device)
+    for l in range(w.n_layers):
+        q[l] = draw_block_torch(w.seed, T_PREFILL_Q, [l], [seq], pos, _all(w.n_q_heads), w.head_dim, device)[0, 0]
+    return q
 
 
 def decode_qkv_np(w: Workload, step: int, seqs=None, layers=None, q_heads=None, kv_heads=None):

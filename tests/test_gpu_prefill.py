@@ -1,0 +1,114 @@
+"""GPU parity of prefill Lazy Attention (qc_prefill_attend) against the fp64 prefill oracle.
+
+Same bars as the decode tests: every element within 2e-2, relative L2 <= 5e-3 per (layer,
+token-block); the cache the call leaves behind must be the one qc_prefill_append builds.
+"""
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import prefill_attention as OP
+from oracle.lazy_attention import LazyAttentionOracle
+from paper_2602_01901_b200 import binding as qc
+from paper_2602_01901_b200 import workloads as W
+from paper_2602_01901_b200.session import Session, bits_of
+
+from parity_util import MAX_ABS, REL_L2, assert_close, f64
+
+pytestmark = pytest.mark.gpu
+
+MODES = [qc.QC_MODE_VLA_QC, qc.QC_MODE_VLA_EQ8, qc.QC_MODE_GLA]
+MODE_IDS = ["vla_qc", "vla_eq8", "gla"]
+
+
+def _dev(a, device):
+    return torch.from_numpy(a.astype(np.int16)).view(torch.bfloat16).to(device).contiguous()
+
+
+CASES = [
+    # (head_dim, group, layer_kind, n_text_before, n_visual, n_text_after)
+    (128, 1, [0, 1, 0, 1, 1], 5, 150, 22),      # 177 tokens: three query tiles, ragged tail
+    (64, 2, [0, 1, 1], 3, 61, 0),               # exactly 64 tokens, ends on a visual token
+    (128, 7, [0, 1], 9, 40, 8),                 # one tile, GQA group of 7
+    (64, 1, [0, 0, 1], 0, 130, 3),              # starts with a visual token
+    (128, 2, [0, 1, 1, 1, 1, 1, 0], 17, 0, 60),  # text only
+]
+
+
+@pytest.mark.parametrize("mode", MODES, ids=MODE_IDS)
+@pytest.mark.parametrize("case", range(len(CASES)))
+def test_prefill_attend_small(mode, case):
+    D, group, layer_kind, nb, nv, na = CASES[case]
+    lazy = tuple(i for i, k in enumerate(layer_kind) if k)
+    w = W.Workload(40 + case, f"prefill{case}", len(layer_kind), 2 * group, 2, D, 16, 2, nb, nv, nv, na, 4, lazy)
+    s = Session.for_workload(w, lazy_mode=mode, poison_pool=True)
+    dec = LazyAttentionOracle(w.n_layers, w.n_q_heads, w.n_kv_heads, D, layer_kind, mode, n_seqs=w.batch)
+    for b in range(w.batch):
+        kind, k, v = W.prefill_kv_np(w, b)
+        q = W.prefill_q_np(w, b)
+        out = torch.full((w.n_layers, len(kind), w.n_q_heads, D), float("nan"), dtype=torch.bfloat16, device=s.device)
+        s.prefill_attend(b, kind, _dev(q, s.device), _dev(k, s.device), _dev(v, s.device), out)
+        ref = OP.prefill_lazy_attention(f64(q), f64(k), f64(v), kind, layer_kind, mode)
+        got = bits_of(out)
+        for l in range(w.n_layers):
+            for t0 in range(0, len(kind), 64):
+                assert_close(got[l, t0:t0 + 64], ref[l, t0:t0 + 64], f"case {case} seq {b} layer {l} tokens {t0}..")
+        dec.prefill_append(b, kind.tolist(), f64(k), f64(v))
+    # the cache is the one qc_prefill_append builds: decoding from it matches the decode oracle
+    o = torch.empty((w.n_layers, w.batch, w.n_q_heads, D), dtype=torch.bfloat16, device=s.device)
+    for step in range(2):
+        qn, kn, vn = W.decode_qkv_np(w, step)
+        s.decode_step(list(range(w.batch)), _dev(qn, s.device), _dev(kn, s.device), _dev(vn, s.device), o)
+        got = bits_of(o)
+        for b in range(w.batch):
+            ref, _ = dec.decode_step(b, f64(qn[:, b]), f64(kn[:, b]), f64(vn[:, b]))
+            for l in range(w.n_layers):
+                assert_close(got[l, b], ref[l], f"decode after prefill: step {step} seq {b} layer {l}")
+    assert s.stats().device_error == 0
+    # a prompt that continues a cached sequence is refused, and nothing changes
+    kind, k, v = W.prefill_kv_np(w, 0)
+    before = s.page_table(0, 0, 0)
+    with pytest.raises(qc.QcError) as e:
+        s.prefill_attend(0, kind, _dev(W.prefill_q_np(w, 0), s.device), _dev(k, s.device), _dev(v, s.device), out)
+    assert e.value.status == qc.QC_ERR_UNSUPPORTED and s.page_table(0, 0, 0) == before
+    s.close()
+
+
+@pytest.mark.parametrize("name,mode", [("llava15_7b", qc.QC_MODE_VLA_QC), ("llava15_7b", qc.QC_MODE_GLA),
+                                       ("qwen2vl_gqa", qc.QC_MODE_VLA_QC)],
+                         ids=["llava15_7b-vla", "llava15_7b-gla", "qwen2vl_gqa-vla"])
+def test_prefill_attend_full_size_sampled(name, mode):
+    """One full-size prompt (all layers, all heads on the GPU); the oracle checks every row of
+    sampled (layer, head) pairs, lazy layers and their leaders included."""
+    w = W.get_workload(name)
+    s = Session.for_workload(w, lazy_mode=mode)
+    seq = 1
+    kind, k, v = W.prefill_kv_torch(w, seq, s.device)
+    q = W.prefill_q_torch(w, seq, s.device)
+    out = torch.empty_like(q)
+    s.prefill_attend(0, kind, q, k, v, out)
+    torch.cuda.synchronize()
+    assert torch.isfinite(out.float()).all()
+    kinds = w.layer_kind().tolist()
+    leaders = OP.leaders_of(kinds)
+    rng = np.random.default_rng(w.seed)
+    lz = list(w.lazy_layers)
+    samples = [(0, 0), (lz[0], 1), (lz[-1], w.n_q_heads - 1), (w.n_layers - 2, w.n_q_heads // 2)]
+    samples += [(int(rng.integers(w.n_layers)), int(rng.integers(w.n_q_heads))) for _ in range(4)]
+    worst = 0.0
+    for layer, head in samples:
+        c = leaders[layer]
+        layers = [layer] if c == layer else [c, layer]
+        kv = head // w.group
+        qn = W.prefill_q_np(w, seq, layers=layers, heads=[head])
+        _, kn, vn = W.prefill_kv_np(w, seq, layers=layers, heads=[kv])
+        sub_kind = [0] if c == layer else [0, 1]
+        ref = OP.prefill_lazy_attention(f64(qn), f64(kn), f64(vn), kind, sub_kind, mode)[-1, :, 0]
+        got = bits_of(out[layer, :, head])
+        for t0 in range(0, len(kind), 128):
+            _, r = assert_close(got[t0:t0 + 128], ref[t0:t0 + 128], f"{name} layer {layer} head {head} tokens {t0}..")
+            worst = max(worst, r)
+    assert s.stats().device_error == 0
+    print(f"{name} mode {mode}: prefill worst rel-L2 {worst:.3e}")
+    s.close()
