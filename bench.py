@@ -344,6 +344,56 @@ def run_gpu(args, w, mode, rank, world, local_rank):
     return line
 
 
+def run_prefill(args, w, mode, local_rank):
+    """Secondary measurement: prefill Lazy Attention (qc_prefill_attend) over the workload's prompts.
+    One JSON line: prompt tokens/s through the call, and the attention kernel against the tensor peak."""
+    import torch
+
+    from paper_2602_01901_b200 import workloads as W
+    from paper_2602_01901_b200.session import Session
+
+    dev = torch.device("cuda", local_rank)
+    s = Session.for_workload(w, lazy_mode=mode, device=local_rank)
+    n_seqs = min(w.batch, max(4, args.warmup + 1))
+    prompts = []
+    for b in range(n_seqs):
+        kind, k, v = W.prefill_kv_torch(w, b, dev)
+        prompts.append((kind, W.prefill_q_torch(w, b, dev), k, v))
+    out = torch.empty_like(prompts[0][1])
+    from paper_2602_01901_b200 import binding as qc
+
+    s.prefill_attend(0, *prompts[0], out)          # warm-up on sequence 0, then release it
+    qc.qc_free_seq(s.cache, 0)
+    s.set_option("profile", 1)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(_physical_gpu_index(local_rank)) as clocks:
+        e0.record()
+        for b in range(n_seqs):
+            s.prefill_attend(b, *prompts[b], out)
+        e1.record()
+        torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    prof = s.profile()
+    st = s.stats()
+    s.close()
+    T = len(prompts[0][0])
+    with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+        peak = float(json.load(f)["bf16_tflops"])
+    achieved = prof.prefill_flops / (prof.prefill_attend_ms / 1e3) / 1e12
+    return {
+        "metric": "prefill_attention_tokens_per_s", "value": n_seqs * T / (ms / 1e3), "unit": UNIT, "n_gpus": 1,
+        "steps": n_seqs, "warmup": 1, "ms_per_step": ms / n_seqs, "higher_is_better": True, "dtype": "bf16",
+        "data": "synthetic", "config": {"workload": w.name, "mode": args.mode, "prompt_tokens": T,
+                                        "n_layers": w.n_layers, "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads},
+        "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                     "frac": achieved / peak, "traffic": None, "kernel": "prefill_attend_kernel",
+                     "avg_launch_ms": prof.prefill_attend_ms / max(1, prof.prefill_calls),
+                     "flops_per_launch": prof.prefill_flops / max(1, prof.prefill_calls), "peak_kind": "of measured"},
+        "clocks": clocks.summary(), "device_error": st.device_error,
+    }
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -356,6 +406,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-all-full", action="store_true", help="skip the all-ordinary-layers comparison run")
     ap.add_argument("--no-per-block", action="store_true", help="skip the launch-per-lazy-block comparison run")
+    ap.add_argument("--phase", default="decode", choices=["decode", "prefill"],
+                    help="decode (the benchmark) or prefill (secondary: qc_prefill_attend over the prompts)")
     ap.add_argument("--split-tokens", type=int, default=0, help="keys per split-KV work item (0 = library default)")
     ap.add_argument("--blocks-per-launch", type=int, default=0,
                     help="0 = one attention launch per step; k = one launch per k lazy blocks, in layer order")
@@ -398,6 +450,10 @@ def main():
         print(json.dumps(line))
         return
 
+    if args.phase == "prefill":
+        if rank == 0:
+            print(json.dumps(run_prefill(args, w, mode, local_rank)))
+        return
     line = run_gpu(args, w, mode, rank, world, local_rank)
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:

@@ -110,6 +110,10 @@ typedef struct qc_profile {
   int64_t kv_bytes_read;      /* algorithmic K/V bytes those steps had to read: every stored
                                  row of the listed sequences once, per step */
   int64_t items;              /* split-KV work items executed */
+  int64_t prefill_calls;      /* qc_prefill_attend calls covered */
+  double prefill_attend_ms;   /* summed duration of the prefill attention kernel */
+  double prefill_flops;       /* its arithmetic: 4 * head_dim flops per (query, visible key) pair,
+                                 every layer and query head */
 } qc_profile;
 
 /* Create a context on `device` that launches on `cuda_stream` (a cudaStream_t; NULL is the

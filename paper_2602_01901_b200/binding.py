@@ -59,6 +59,7 @@ class qc_profile(C.Structure):
     _fields_ = [
         ("steps", C.c_int64), ("attend_ms", C.c_double), ("step_ms", C.c_double),
         ("kv_bytes_read", C.c_int64), ("items", C.c_int64),
+        ("prefill_calls", C.c_int64), ("prefill_attend_ms", C.c_double), ("prefill_flops", C.c_double),
     ]
 
 

@@ -97,6 +97,9 @@ struct qc_cache {
   std::vector<cudaEvent_t> ev;         // 4 per step: step begin, attend begin, attend end, step end
   int ev_steps = 0;
   int64_t prof_bytes = 0, prof_items = 0;
+  std::vector<cudaEvent_t> ev_prefill; // 2 per profiled qc_prefill_attend call
+  int ev_prefill_calls = 0;
+  double prof_prefill_flops = 0.0;
 
   int64_t decode_steps = 0, attend_launches = 0, kernel_launches = 0;
 };
@@ -560,6 +563,7 @@ int32_t qc_free(qc_ctx* ctx, qc_cache* cache) {
     for (int i = 0; i < kStageSlots; ++i)
       if (cache->stage_done[i]) cudaEventDestroy(cache->stage_done[i]);
     for (cudaEvent_t e : cache->ev) cudaEventDestroy(e);
+    for (cudaEvent_t e : cache->ev_prefill) cudaEventDestroy(e);
     if (cache->pinned) cudaFreeHost(cache->pinned);
     delete cache;
   }
@@ -680,8 +684,26 @@ int32_t qc_prefill_attend(qc_cache* c, int32_t seq_id, int32_t n_tokens, const u
   QC_CUDA(cudaMemcpyAsync(kind_dev, kind, n_tokens, cudaMemcpyHostToDevice, stream));
   QC_CUDA(cudaStreamSynchronize(stream));   // `kind` is the caller's host memory
   const Params p = base_params(c);
+  cudaEvent_t* ev = nullptr;
+  if (c->profile && c->ev_prefill_calls < kMaxProfileSteps) {
+    if (static_cast<int>(c->ev_prefill.size()) < 2 * (c->ev_prefill_calls + 1)) {
+      for (int i = 0; i < 2; ++i) {
+        cudaEvent_t e;
+        QC_CUDA(cudaEventCreate(&e));
+        c->ev_prefill.push_back(e);
+      }
+    }
+    ev = &c->ev_prefill[2 * c->ev_prefill_calls];
+    QC_CUDA(cudaEventRecord(ev[0], stream));
+  }
   QC_CUDA(launch_prefill_attend(p, kind_dev, c->ws + c->lay.layer_kind, c->ws + c->lay.leader, q_dev, k_dev, v_dev,
                                 out_dev, n_tokens, c->cfg.lazy_mode == QC_MODE_GLA ? 1 : 0, stream));
+  if (ev) {
+    QC_CUDA(cudaEventRecord(ev[1], stream));
+    c->ev_prefill_calls++;
+    const double pairs = 0.5 * n_tokens * (n_tokens + 1.0);
+    c->prof_prefill_flops += 4.0 * c->D * pairs * c->hq * c->cfg.n_layers;
+  }
   c->kernel_launches++;
   return QC_OK;
 }
@@ -1025,6 +1047,15 @@ int32_t qc_get_profile(qc_cache* c, qc_profile* out) {
     out->attend_ms += a;
     out->step_ms += t;
   }
+  for (int i = 0; i < c->ev_prefill_calls; ++i) {
+    float a = 0.f;
+    QC_CUDA(cudaEventElapsedTime(&a, c->ev_prefill[2 * i], c->ev_prefill[2 * i + 1]));
+    out->prefill_attend_ms += a;
+  }
+  out->prefill_calls = c->ev_prefill_calls;
+  out->prefill_flops = c->prof_prefill_flops;
+  c->ev_prefill_calls = 0;
+  c->prof_prefill_flops = 0.0;
   out->steps = c->ev_steps;
   out->kv_bytes_read = c->prof_bytes;
   out->items = c->prof_items;
