@@ -223,6 +223,285 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_attend_kernel(const P
   }
 }
 
+// ------------------------------------------------------------------------------------------
+// The same computation on the fifth-generation tensor cores (tcgen05), head_dim 128.
+//
+// One CTA = 128 query rows of one (layer, query head), 128 threads, one thread per row.  Key /
+// value tiles of 64 tokens are staged (with the per-row source-layer selection) into the
+// canonical 128-byte-swizzled shared-memory layout, [two 64-column halves][rows][128 bytes].
+// One elected thread issues
+//     S[128 x 64]   = Q[128 x 128] . K^T      8 x tcgen05.mma (M 128, N 64, K 16), accumulator in TMEM
+//     O[128 x 128] += P[128 x 64]  . V        4 x tcgen05.mma (M 128, N 128, K 16), V read MN-major
+// and commits to an mbarrier.  A thread reads its row of S from TMEM (one TMEM lane per row: no
+// cross-thread reduction), does the online softmax, and writes the bf16 weights as the next
+// A operand into shared memory.  The running maximum is only moved when it grows by more than
+// 2^8 (the weights then stay below 2^8, harmless in fp32/bf16), so the accumulator in TMEM is
+// rescaled rarely (TMEM load, scale, store).  Two CTAs per SM (2 x 192 TMEM columns in use,
+// 2 x 256 allocated) overlap one CTA's softmax with the other's products.
+// Every mbarrier wait is bounded; on expiry the CTA records the error, frees its TMEM and leaves.
+
+constexpr int kTM = 128;        // query rows per CTA
+constexpr int kTN = 64;         // keys per tile
+constexpr int kTD = 128;        // head dim
+constexpr uint32_t kTmemCols = 256;
+constexpr uint32_t kColS = 0, kColO = 128;
+constexpr float kRescaleThreshold = 8.f;   // log2 units
+
+__device__ __forceinline__ uint32_t tc5_off(int row, int chunk, int rows) {   // chunk: 16-byte chunk of the 256-byte row
+  return (chunk >> 3) * (rows * 128) + row * 128 + (((chunk & 7) ^ (row & 7)) << 4);
+}
+__device__ __forceinline__ uint64_t umma_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  // start address, leading / stride byte offsets (all >> 4), descriptor version 1, 128-byte swizzle
+  return static_cast<uint64_t>((saddr >> 4) & 0x3fff) | (static_cast<uint64_t>((lbo_bytes >> 4) & 0x3fff) << 16) |
+         (static_cast<uint64_t>((sbo_bytes >> 4) & 0x3fff) << 32) | (1ull << 46) | (2ull << 61);
+}
+__device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      :: "r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tc5_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc5_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      :: "r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+         "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]),
+         "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
+         "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+
+// Stage `rows` rows starting at row0 of one head into the swizzled two-half layout.
+__device__ __forceinline__ void stage_tc5(uint32_t smem, const uint16_t* base, int own, int lead, bool lazy, bool gla,
+                                          const uint8_t* kind, int row0, int rows, int T, int heads, int head) {
+  constexpr int CH = kTD / 8;
+  for (int e = threadIdx.x; e < rows * CH; e += kTM) {
+    const int r = e / CH, c = e - r * CH;
+    const int t = row0 + r;
+    const uint32_t dst = smem + tc5_off(r, c, rows);
+    if (t < T) {
+      const int layer = (lazy && (gla || kind[t])) ? lead : own;
+      cp_async16(dst, base + ((static_cast<size_t>(layer) * T + t) * heads + head) * kTD + c * 8);
+    } else {
+      asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(dst), "r"(0u) : "memory");
+    }
+  }
+}
+
+// Bounded wait whose verdict is the same for every thread of the CTA (so that nobody is left
+// alone at a later barrier).
+__device__ __forceinline__ bool bounded_wait(uint64_t* bar, uint32_t parity) {
+  constexpr uint32_t kLimit = 1u << 18;
+  uint32_t done = mbar_try_wait(bar, parity);
+  for (uint32_t spin = 0; !done && spin < kLimit; ++spin) done = mbar_try_wait(bar, parity);
+  return __syncthreads_and(done != 0) != 0;
+}
+
+__global__ void __launch_bounds__(kTM, 2) prefill_attend_tcgen05_kernel(const PrefillArgs A, int32_t* err) {
+  extern __shared__ uint8_t smem_dyn[];
+  __shared__ __align__(8) uint64_t bar_s, bar_o;
+  __shared__ uint32_t tmem_base_slot;
+
+  const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+  const uint32_t sQ = base;                         // [2][128][128 B]  32 KiB
+  const uint32_t sK = sQ + 2 * kTM * 128;           // two buffers of [2][64][128 B] 16 KiB
+  const uint32_t sV = sK + 2 * (2 * kTN * 128);     // two buffers
+  const uint32_t sP = sV + 2 * (2 * kTN * 128);     // [128][128 B]     16 KiB
+  constexpr uint32_t kKV = 2 * kTN * 128;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n_qtiles = (A.T + kTM - 1) / kTM;
+  const int qt = n_qtiles - 1 - blockIdx.x;         // long rows first
+  const int head = blockIdx.y, layer = blockIdx.z;
+  const int kvh = head / A.group;
+  const bool lazy = A.layer_kind[layer] != 0;
+  const int lead = A.leader[layer];
+  const bool gla = A.gla != 0;
+  const int m0 = qt * kTM;
+  const int row = m0 + threadIdx.x;                 // this thread's query row
+  const int n_ktiles = min((A.T + kTN - 1) / kTN, (m0 + kTM + kTN - 1) / kTN);
+
+  if (threadIdx.x == 0) {
+    mbar_init(&bar_s, 1);
+    mbar_init(&bar_o, 1);
+    fence_mbar_init();
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
+                 "r"(kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  stage_tc5(sQ, A.q, layer, lead, lazy, gla, A.kind, m0, kTM, A.T, A.hq, head);
+  stage_tc5(sK, A.k, layer, lead, lazy, gla, A.kind, 0, kTN, A.T, A.hkv, kvh);
+  stage_tc5(sV, A.v, layer, layer, false, false, A.kind, 0, kTN, A.T, A.hkv, kvh);
+  cp_async_commit();
+  cp_async_wait<0>();
+  fence_proxy_async();
+  tc5_fence_before();
+  __syncthreads();
+  tc5_fence_after();
+  const uint32_t tmem = tmem_base_slot;
+  const uint32_t t_row = tmem + (static_cast<uint32_t>(warp * 32) << 16);   // this warp's 32 TMEM lanes
+
+  // instruction descriptors: fp32 accumulate, bf16 operands, M 128; S: N 64, both K-major; PV: N 128, B MN-major
+  constexpr uint32_t kIdescS = (1u << 4) | (1u << 7) | (1u << 10) | ((kTN >> 3) << 17) | ((kTM >> 4) << 24);
+  constexpr uint32_t kIdescO = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((kTD >> 3) << 17) | ((kTM >> 4) << 24);
+
+  float m_ref = -INFINITY, l_sum = 0.f;
+  uint32_t ph_s = 0, ph_o = 0;
+  bool ok = true;
+
+  for (int kt = 0; kt < n_ktiles && ok; ++kt) {
+    const int buf = kt & 1;
+    const uint32_t kb = sK + buf * kKV, vb = sV + buf * kKV;
+    // ---- S = Q K^T
+    if (threadIdx.x == 0) {
+#pragma unroll
+      for (int kk = 0; kk < kTD / 16; ++kk) {
+        const uint64_t ad = umma_desc(sQ + (kk >> 2) * (kTM * 128) + (kk & 3) * 32, 16, 1024);
+        const uint64_t bd = umma_desc(kb + (kk >> 2) * (kTN * 128) + (kk & 3) * 32, 16, 1024);
+        umma_f16(tmem + kColS, ad, bd, kIdescS, kk > 0);
+      }
+      umma_commit(&bar_s);
+    }
+    ok = bounded_wait(&bar_s, ph_s);
+    ph_s ^= 1u;
+    if (!ok) break;
+    tc5_fence_after();
+    // ---- this row's 64 scores
+    float p[kTN];
+    {
+      uint32_t r[32];
+      tmem_ld32(t_row + kColS, r);
+#pragma unroll
+      for (int j = 0; j < 32; ++j) p[j] = __uint_as_float(r[j]);
+      tmem_ld32(t_row + kColS + 32, r);
+#pragma unroll
+      for (int j = 0; j < 32; ++j) p[32 + j] = __uint_as_float(r[j]);
+    }
+    const int n0 = kt * kTN;
+    float m_tile = -INFINITY;
+#pragma unroll
+    for (int j = 0; j < kTN; ++j) {
+      const int key = n0 + j;
+      p[j] = (key <= row && key < A.T) ? p[j] * A.scale_log2 : -INFINITY;
+      m_tile = fmaxf(m_tile, p[j]);
+    }
+    float corr = 1.f;
+    if (m_tile > m_ref + kRescaleThreshold || m_ref == -INFINITY) {
+      if (m_tile != -INFINITY) {
+        corr = exp2f(m_ref - m_tile);     // 0 on the first tile
+        m_ref = m_tile;
+      }
+    }
+    const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
+    float psum = 0.f;
+#pragma unroll
+    for (int j = 0; j < kTN; ++j) {
+      p[j] = exp2f(p[j] - m_use);
+      psum += p[j];
+    }
+    l_sum = l_sum * corr + psum;
+    // ---- the previous value product must be done before P, O or the other K/V buffer change
+    if (kt > 0) {
+      ok = bounded_wait(&bar_o, ph_o);
+      ph_o ^= 1u;
+      if (!ok) break;
+      tc5_fence_after();
+    }
+    if (kt + 1 < n_ktiles) {
+      stage_tc5(sK + (buf ^ 1) * kKV, A.k, layer, lead, lazy, gla, A.kind, (kt + 1) * kTN, kTN, A.T, A.hkv, kvh);
+      stage_tc5(sV + (buf ^ 1) * kKV, A.v, layer, layer, false, false, A.kind, (kt + 1) * kTN, kTN, A.T, A.hkv, kvh);
+      cp_async_commit();
+    }
+    if (kt > 0 && __any_sync(0xffffffffu, corr != 1.f)) {   // rare: move the accumulator to the new reference
+#pragma unroll
+      for (int c = 0; c < kTD / 32; ++c) {
+        uint32_t r[32];
+        tmem_ld32(t_row + kColO + 32 * c, r);
+#pragma unroll
+        for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * corr);
+        tmem_st32(t_row + kColO + 32 * c, r);
+      }
+      asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+    }
+    // ---- weights as the A operand: row threadIdx.x, 64 keys = one 128-byte swizzled line
+#pragma unroll
+    for (int c = 0; c < kTN / 8; ++c) {
+      const uint32_t w0 = pack_bf16x2(p[8 * c + 0], p[8 * c + 1]), w1 = pack_bf16x2(p[8 * c + 2], p[8 * c + 3]);
+      const uint32_t w2 = pack_bf16x2(p[8 * c + 4], p[8 * c + 5]), w3 = pack_bf16x2(p[8 * c + 6], p[8 * c + 7]);
+      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sP + tc5_off(threadIdx.x, c, kTM)), "r"(w0), "r"(w1),
+                   "r"(w2), "r"(w3)
+                   : "memory");
+    }
+    cp_async_wait<0>();
+    fence_proxy_async();     // generic-proxy writes (weights, staged tiles) before the tensor core reads them
+    tc5_fence_before();
+    __syncthreads();
+    // ---- O += P V
+    if (threadIdx.x == 0) {
+      tc5_fence_after();
+#pragma unroll
+      for (int ks = 0; ks < kTN / 16; ++ks) {
+        const uint64_t ad = umma_desc(sP + ks * 32, 16, 1024);
+        const uint64_t bd = umma_desc(vb + ks * (16 * 128), kTN * 128, 1024);
+        umma_f16(tmem + kColO, ad, bd, kIdescO, (kt > 0 || ks > 0) ? 1u : 0u);
+      }
+      umma_commit(&bar_o);
+    }
+  }
+  if (ok) ok = bounded_wait(&bar_o, ph_o);
+  if (ok) {
+    tc5_fence_after();
+    const float inv = 1.f / l_sum;
+    uint16_t* dst = A.out + ((static_cast<size_t>(layer) * A.T + row) * A.hq + head) * kTD;
+#pragma unroll
+    for (int c = 0; c < kTD / 32; ++c) {
+      uint32_t r[32];
+      tmem_ld32(t_row + kColO + 32 * c, r);   // every lane takes part in the load; only rows of the prompt store
+      if (row < A.T) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          uint4 o;
+          o.x = pack_bf16x2(__uint_as_float(r[8 * j + 0]) * inv, __uint_as_float(r[8 * j + 1]) * inv);
+          o.y = pack_bf16x2(__uint_as_float(r[8 * j + 2]) * inv, __uint_as_float(r[8 * j + 3]) * inv);
+          o.z = pack_bf16x2(__uint_as_float(r[8 * j + 4]) * inv, __uint_as_float(r[8 * j + 5]) * inv);
+          o.w = pack_bf16x2(__uint_as_float(r[8 * j + 6]) * inv, __uint_as_float(r[8 * j + 7]) * inv);
+          *reinterpret_cast<uint4*>(dst + 32 * c + 8 * j) = o;
+        }
+      }
+    }
+  } else if (threadIdx.x == 0) {
+    atomicMax(err, kErrTimeout);
+  }
+  cp_async_wait<0>();
+  tc5_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+  }
+}
+
+constexpr int prefill_tcgen05_smem_bytes() { return 1024 + 2 * kTM * 128 + 4 * (2 * kTN * 128) + kTM * 128; }
+
 template <int D>
 constexpr int prefill_smem_bytes() {
   return 5 * kBN * D * 2;
@@ -234,13 +513,16 @@ cudaError_t configure_prefill_kernels() {
   cudaError_t e = cudaFuncSetAttribute(prefill_attend_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        prefill_smem_bytes<128>());
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(prefill_attend_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              prefill_smem_bytes<64>());
+  e = cudaFuncSetAttribute(prefill_attend_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           prefill_smem_bytes<64>());
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(prefill_attend_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              prefill_tcgen05_smem_bytes());
 }
 
 cudaError_t launch_prefill_attend(const Params& p, const uint8_t* kind_dev, const uint8_t* layer_kind_dev,
                                   const uint8_t* leader_dev, const void* q, const void* k, const void* v, void* out,
-                                  int32_t T, int32_t gla, cudaStream_t stream) {
+                                  int32_t T, int32_t gla, int32_t use_tcgen05, cudaStream_t stream) {
   if (T <= 0) return cudaSuccess;
   PrefillArgs a{};
   a.q = static_cast<const uint16_t*>(q);
@@ -257,6 +539,11 @@ cudaError_t launch_prefill_attend(const Params& p, const uint8_t* kind_dev, cons
   a.n_layers = p.n_layers;
   a.gla = gla;
   a.scale_log2 = p.scale_log2;
+  if (p.d == kTD && use_tcgen05) {
+    const dim3 grid5((T + kTM - 1) / kTM, p.hq, p.n_layers);
+    prefill_attend_tcgen05_kernel<<<grid5, kTM, prefill_tcgen05_smem_bytes(), stream>>>(a, p.err);
+    return cudaGetLastError();
+  }
   const dim3 grid((T + kBM - 1) / kBM, p.hq, p.n_layers);
   if (p.d == 128)
     prefill_attend_kernel<128><<<grid, kPrefillThreads, prefill_smem_bytes<128>(), stream>>>(a);

@@ -69,6 +69,7 @@ struct qc_cache {
   std::vector<LaunchGroup> groups;
   std::vector<std::pair<int, int>> group_pos;           // plan positions [begin, end) of each launch
   bool plan_dirty = true;
+  bool prefill_tcgen05 = true;    // head_dim 128: tcgen05 kernel; otherwise (or when switched off) mma.sync kernel
   int64_t n_pool_pages = 0;
   int layers_per_launch = 0;
   float scale = 0.f;
@@ -697,7 +698,7 @@ int32_t qc_prefill_attend(qc_cache* c, int32_t seq_id, int32_t n_tokens, const u
     QC_CUDA(cudaEventRecord(ev[0], stream));
   }
   QC_CUDA(launch_prefill_attend(p, kind_dev, c->ws + c->lay.layer_kind, c->ws + c->lay.leader, q_dev, k_dev, v_dev,
-                                out_dev, n_tokens, c->cfg.lazy_mode == QC_MODE_GLA ? 1 : 0, stream));
+                                out_dev, n_tokens, c->cfg.lazy_mode == QC_MODE_GLA ? 1 : 0, c->prefill_tcgen05 ? 1 : 0, stream));
   if (ev) {
     QC_CUDA(cudaEventRecord(ev[1], stream));
     c->ev_prefill_calls++;
@@ -1026,6 +1027,10 @@ int32_t qc_set_option(qc_cache* c, const char* key, int64_t value) {
     if (value < 0 || value > c->cfg.n_layers) return QC_ERR_INVALID_ARG;
     c->layers_per_launch = static_cast<int>(value);
     c->plan_dirty = true;
+    return QC_OK;
+  }
+  if (k == "prefill_tcgen05") {
+    c->prefill_tcgen05 = value != 0;
     return QC_OK;
   }
   if (k == "profile") {
