@@ -354,6 +354,7 @@ def run_prefill(args, w, mode, local_rank):
 
     dev = torch.device("cuda", local_rank)
     s = Session.for_workload(w, lazy_mode=mode, device=local_rank)
+    s.set_option("prefill_tcgen05", 1 if args.prefill_kernel == "tcgen05" else 0)
     n_seqs = min(w.batch, max(4, args.warmup + 1))
     prompts = []
     for b in range(n_seqs):
@@ -387,7 +388,9 @@ def run_prefill(args, w, mode, local_rank):
         "data": "synthetic", "config": {"workload": w.name, "mode": args.mode, "prompt_tokens": T,
                                         "n_layers": w.n_layers, "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads},
         "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                     "frac": achieved / peak, "traffic": None, "kernel": "prefill_attend_kernel",
+                     "frac": achieved / peak, "traffic": None,
+                     "kernel": "prefill_attend_tcgen05_kernel" if (args.prefill_kernel == "tcgen05" and w.head_dim == 128)
+                     else "prefill_attend_kernel",
                      "avg_launch_ms": prof.prefill_attend_ms / max(1, prof.prefill_calls),
                      "flops_per_launch": prof.prefill_flops / max(1, prof.prefill_calls), "peak_kind": "of measured"},
         "clocks": clocks.summary(), "device_error": st.device_error,
@@ -408,6 +411,8 @@ def main():
     ap.add_argument("--no-per-block", action="store_true", help="skip the launch-per-lazy-block comparison run")
     ap.add_argument("--phase", default="decode", choices=["decode", "prefill"],
                     help="decode (the benchmark) or prefill (secondary: qc_prefill_attend over the prompts)")
+    ap.add_argument("--prefill-kernel", default="tcgen05", choices=["tcgen05", "mma"],
+                    help="prefill phase, head_dim 128: tcgen05 kernel (default) or the mma.sync kernel")
     ap.add_argument("--split-tokens", type=int, default=0, help="keys per split-KV work item (0 = library default)")
     ap.add_argument("--blocks-per-launch", type=int, default=0,
                     help="0 = one attention launch per step; k = one launch per k lazy blocks, in layer order")

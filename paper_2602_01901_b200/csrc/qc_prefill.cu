@@ -52,15 +52,23 @@ struct PrefillArgs {
 template <int D>
 __device__ __forceinline__ void stage_tile(uint32_t smem, const uint16_t* base, int own, int lead, bool lazy, bool gla,
                                            const uint8_t* kind, int row0, int T, int heads, int head) {
-  constexpr int CH = D / 8;
-  for (int e = threadIdx.x; e < kBN * CH; e += kPrefillThreads) {
-    const int r = e / CH, c = e - r * CH;
-    const int t = row0 + r;
+  constexpr int CH = D / 8;                         // 16-byte chunks per row
+  constexpr int RPP = kPrefillThreads / CH;         // rows covered by one pass of the CTA
+  constexpr int NP = kBN / RPP;
+  const int c = threadIdx.x % CH, r0 = threadIdx.x / CH;
+  // the source layer of each of this thread's rows first (independent loads), then the copies
+  int layer_of[NP];
+#pragma unroll
+  for (int i = 0; i < NP; ++i) {
+    const int t = row0 + r0 + i * RPP;
+    layer_of[i] = (lazy && (gla || (t < T && kind[t]))) ? lead : own;
+  }
+#pragma unroll
+  for (int i = 0; i < NP; ++i) {
+    const int r = r0 + i * RPP, t = row0 + r;
     const uint32_t dst = smem + tile_off<D>(r, c);
     if (t < T) {
-      const int layer = (lazy && (gla || kind[t])) ? lead : own;
-      const uint16_t* src = base + ((static_cast<size_t>(layer) * T + t) * heads + head) * D + c * 8;
-      cp_async16(dst, src);
+      cp_async16(dst, base + ((static_cast<size_t>(layer_of[i]) * T + t) * heads + head) * D + c * 8);
     } else {
       asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(dst), "r"(0u) : "memory");
     }
@@ -288,17 +296,26 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
       : "memory");
 }
 
-// Stage `rows` rows starting at row0 of one head into the swizzled two-half layout.
+// Stage ROWS rows starting at row0 of one head into the swizzled two-half layout.
+template <int ROWS>
 __device__ __forceinline__ void stage_tc5(uint32_t smem, const uint16_t* base, int own, int lead, bool lazy, bool gla,
-                                          const uint8_t* kind, int row0, int rows, int T, int heads, int head) {
+                                          const uint8_t* kind, int row0, int T, int heads, int head) {
   constexpr int CH = kTD / 8;
-  for (int e = threadIdx.x; e < rows * CH; e += kTM) {
-    const int r = e / CH, c = e - r * CH;
-    const int t = row0 + r;
-    const uint32_t dst = smem + tc5_off(r, c, rows);
+  constexpr int RPP = kTM / CH;      // 8 rows per pass
+  constexpr int NP = ROWS / RPP;
+  const int c = threadIdx.x % CH, r0 = threadIdx.x / CH;
+  int layer_of[NP];
+#pragma unroll
+  for (int i = 0; i < NP; ++i) {
+    const int t = row0 + r0 + i * RPP;
+    layer_of[i] = (lazy && (gla || (t < T && kind[t]))) ? lead : own;
+  }
+#pragma unroll
+  for (int i = 0; i < NP; ++i) {
+    const int r = r0 + i * RPP, t = row0 + r;
+    const uint32_t dst = smem + tc5_off(r, c, ROWS);
     if (t < T) {
-      const int layer = (lazy && (gla || kind[t])) ? lead : own;
-      cp_async16(dst, base + ((static_cast<size_t>(layer) * T + t) * heads + head) * kTD + c * 8);
+      cp_async16(dst, base + ((static_cast<size_t>(layer_of[i]) * T + t) * heads + head) * kTD + c * 8);
     } else {
       asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(dst), "r"(0u) : "memory");
     }
@@ -315,16 +332,23 @@ __device__ __forceinline__ bool bounded_wait(uint64_t* bar, uint32_t parity) {
 }
 
 __global__ void __launch_bounds__(kTM, 2) prefill_attend_tcgen05_kernel(const PrefillArgs A, int32_t* err) {
-  extern __shared__ uint8_t smem_dyn[];
-  __shared__ __align__(8) uint64_t bar_s, bar_o;
-  __shared__ uint32_t tmem_base_slot;
-
-  const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+  // No static shared memory: the dynamic window then starts on the 1024-byte boundary that the
+  // swizzled tiles need, and two CTAs fit an SM (2 x 112 KiB of tiles).  Checked below.
+  extern __shared__ __align__(1024) uint8_t smem_dyn[];
+  const uint32_t base = smem_u32(smem_dyn);
   const uint32_t sQ = base;                         // [2][128][128 B]  32 KiB
   const uint32_t sK = sQ + 2 * kTM * 128;           // two buffers of [2][64][128 B] 16 KiB
   const uint32_t sV = sK + 2 * (2 * kTN * 128);     // two buffers
   const uint32_t sP = sV + 2 * (2 * kTN * 128);     // [128][128 B]     16 KiB
   constexpr uint32_t kKV = 2 * kTN * 128;
+  constexpr uint32_t kTiles = 2 * kTM * 128 + 4 * kKV + kTM * 128;
+  uint64_t& bar_s = *reinterpret_cast<uint64_t*>(smem_dyn + kTiles);
+  uint64_t& bar_o = *reinterpret_cast<uint64_t*>(smem_dyn + kTiles + 8);
+  uint32_t& tmem_base_slot = *reinterpret_cast<uint32_t*>(smem_dyn + kTiles + 16);
+  if (base & 1023u) {   // cannot happen with the layout above; never run the tensor core on a misplaced tile
+    if (threadIdx.x == 0) atomicMax(err, kErrBadPage);
+    return;
+  }
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_qtiles = (A.T + kTM - 1) / kTM;
@@ -349,9 +373,9 @@ __global__ void __launch_bounds__(kTM, 2) prefill_attend_tcgen05_kernel(const Pr
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  stage_tc5(sQ, A.q, layer, lead, lazy, gla, A.kind, m0, kTM, A.T, A.hq, head);
-  stage_tc5(sK, A.k, layer, lead, lazy, gla, A.kind, 0, kTN, A.T, A.hkv, kvh);
-  stage_tc5(sV, A.v, layer, layer, false, false, A.kind, 0, kTN, A.T, A.hkv, kvh);
+  stage_tc5<kTM>(sQ, A.q, layer, lead, lazy, gla, A.kind, m0, A.T, A.hq, head);
+  stage_tc5<kTN>(sK, A.k, layer, lead, lazy, gla, A.kind, 0, A.T, A.hkv, kvh);
+  stage_tc5<kTN>(sV, A.v, layer, layer, false, false, A.kind, 0, A.T, A.hkv, kvh);
   cp_async_commit();
   cp_async_wait<0>();
   fence_proxy_async();
@@ -428,8 +452,8 @@ __global__ void __launch_bounds__(kTM, 2) prefill_attend_tcgen05_kernel(const Pr
       tc5_fence_after();
     }
     if (kt + 1 < n_ktiles) {
-      stage_tc5(sK + (buf ^ 1) * kKV, A.k, layer, lead, lazy, gla, A.kind, (kt + 1) * kTN, kTN, A.T, A.hkv, kvh);
-      stage_tc5(sV + (buf ^ 1) * kKV, A.v, layer, layer, false, false, A.kind, (kt + 1) * kTN, kTN, A.T, A.hkv, kvh);
+      stage_tc5<kTN>(sK + (buf ^ 1) * kKV, A.k, layer, lead, lazy, gla, A.kind, (kt + 1) * kTN, A.T, A.hkv, kvh);
+      stage_tc5<kTN>(sV + (buf ^ 1) * kKV, A.v, layer, layer, false, false, A.kind, (kt + 1) * kTN, A.T, A.hkv, kvh);
       cp_async_commit();
     }
     if (kt > 0 && __any_sync(0xffffffffu, corr != 1.f)) {   // rare: move the accumulator to the new reference
@@ -500,7 +524,7 @@ __global__ void __launch_bounds__(kTM, 2) prefill_attend_tcgen05_kernel(const Pr
   }
 }
 
-constexpr int prefill_tcgen05_smem_bytes() { return 1024 + 2 * kTM * 128 + 4 * (2 * kTN * 128) + kTM * 128; }
+constexpr int prefill_tcgen05_smem_bytes() { return 2 * kTM * 128 + 4 * (2 * kTN * 128) + kTM * 128 + 64; }
 
 template <int D>
 constexpr int prefill_smem_bytes() {
@@ -516,8 +540,11 @@ cudaError_t configure_prefill_kernels() {
   e = cudaFuncSetAttribute(prefill_attend_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            prefill_smem_bytes<64>());
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(prefill_attend_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              prefill_tcgen05_smem_bytes());
+  e = cudaFuncSetAttribute(prefill_attend_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           prefill_tcgen05_smem_bytes());
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(prefill_attend_tcgen05_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                              cudaSharedmemCarveoutMaxShared);
 }
 
 cudaError_t launch_prefill_attend(const Params& p, const uint8_t* kind_dev, const uint8_t* layer_kind_dev,
