@@ -252,7 +252,7 @@ constexpr int kTM = 128;        // query rows per CTA
 constexpr int kTN = 64;         // keys per tile
 constexpr int kTD = 128;        // head dim
 constexpr uint32_t kTmemCols = 256;
-constexpr uint32_t kColS = 0, kColO = 128;
+constexpr uint32_t kColS = 0, kColO = 128;   // scores: two buffers of 64 columns; accumulator: 128 columns
 constexpr float kRescaleThreshold = 8.f;   // log2 units
 
 __device__ __forceinline__ uint32_t tc5_off(int row, int chunk, int rows) {   // chunk: 16-byte chunk of the 256-byte row
@@ -342,9 +342,9 @@ __global__ void __launch_bounds__(kTM, 2) prefill_attend_tcgen05_kernel(const Pr
   const uint32_t sP = sV + 2 * (2 * kTN * 128);     // [128][128 B]     16 KiB
   constexpr uint32_t kKV = 2 * kTN * 128;
   constexpr uint32_t kTiles = 2 * kTM * 128 + 4 * kKV + kTM * 128;
-  uint64_t& bar_s = *reinterpret_cast<uint64_t*>(smem_dyn + kTiles);
-  uint64_t& bar_o = *reinterpret_cast<uint64_t*>(smem_dyn + kTiles + 8);
-  uint32_t& tmem_base_slot = *reinterpret_cast<uint32_t*>(smem_dyn + kTiles + 16);
+  uint64_t* bar_s = reinterpret_cast<uint64_t*>(smem_dyn + kTiles);          // two: one per score buffer
+  uint64_t& bar_o = *reinterpret_cast<uint64_t*>(smem_dyn + kTiles + 16);
+  uint32_t& tmem_base_slot = *reinterpret_cast<uint32_t*>(smem_dyn + kTiles + 24);
   if (base & 1023u) {   // cannot happen with the layout above; never run the tensor core on a misplaced tile
     if (threadIdx.x == 0) atomicMax(err, kErrBadPage);
     return;
@@ -363,7 +363,8 @@ __global__ void __launch_bounds__(kTM, 2) prefill_attend_tcgen05_kernel(const Pr
   const int n_ktiles = min((A.T + kTN - 1) / kTN, (m0 + kTM + kTN - 1) / kTN);
 
   if (threadIdx.x == 0) {
-    mbar_init(&bar_s, 1);
+    mbar_init(&bar_s[0], 1);
+    mbar_init(&bar_s[1], 1);
     mbar_init(&bar_o, 1);
     fence_mbar_init();
   }
@@ -376,6 +377,7 @@ __global__ void __launch_bounds__(kTM, 2) prefill_attend_tcgen05_kernel(const Pr
   stage_tc5<kTM>(sQ, A.q, layer, lead, lazy, gla, A.kind, m0, A.T, A.hq, head);
   stage_tc5<kTN>(sK, A.k, layer, lead, lazy, gla, A.kind, 0, A.T, A.hkv, kvh);
   stage_tc5<kTN>(sV, A.v, layer, layer, false, false, A.kind, 0, A.T, A.hkv, kvh);
+  if (n_ktiles > 1) stage_tc5<kTN>(sK + kKV, A.k, layer, lead, lazy, gla, A.kind, kTN, A.T, A.hkv, kvh);
   cp_async_commit();
   cp_async_wait<0>();
   fence_proxy_async();
@@ -389,35 +391,46 @@ __global__ void __launch_bounds__(kTM, 2) prefill_attend_tcgen05_kernel(const Pr
   constexpr uint32_t kIdescS = (1u << 4) | (1u << 7) | (1u << 10) | ((kTN >> 3) << 17) | ((kTM >> 4) << 24);
   constexpr uint32_t kIdescO = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((kTD >> 3) << 17) | ((kTM >> 4) << 24);
 
-  float m_ref = -INFINITY, l_sum = 0.f;
-  uint32_t ph_s = 0, ph_o = 0;
-  bool ok = true;
+  // S = Q K^T of key tile kt into score buffer kt & 1 (two buffers of 64 TMEM columns)
+  auto issue_scores = [&](int kt) {
+    const uint32_t kb = sK + (kt & 1) * kKV;
+#pragma unroll
+    for (int kk = 0; kk < kTD / 16; ++kk) {
+      const uint64_t ad = umma_desc(sQ + (kk >> 2) * (kTM * 128) + (kk & 3) * 32, 16, 1024);
+      const uint64_t bd = umma_desc(kb + (kk >> 2) * (kTN * 128) + (kk & 3) * 32, 16, 1024);
+      umma_f16(tmem + kColS + (kt & 1) * kTN, ad, bd, kIdescS, kk > 0);
+    }
+    umma_commit(&bar_s[kt & 1]);
+  };
 
+  float m_ref = -INFINITY, l_sum = 0.f;
+  uint32_t ph_s[2] = {0, 0}, ph_o = 0;
+  bool ok = true;
+  if (threadIdx.x == 0) issue_scores(0);
+
+  // Software pipeline: while the threads work on the scores of tile kt, the tensor core already
+  // computes the scores of tile kt + 1 and the value product of tile kt - 1.
   for (int kt = 0; kt < n_ktiles && ok; ++kt) {
     const int buf = kt & 1;
-    const uint32_t kb = sK + buf * kKV, vb = sV + buf * kKV;
-    // ---- S = Q K^T
-    if (threadIdx.x == 0) {
-#pragma unroll
-      for (int kk = 0; kk < kTD / 16; ++kk) {
-        const uint64_t ad = umma_desc(sQ + (kk >> 2) * (kTM * 128) + (kk & 3) * 32, 16, 1024);
-        const uint64_t bd = umma_desc(kb + (kk >> 2) * (kTN * 128) + (kk & 3) * 32, 16, 1024);
-        umma_f16(tmem + kColS, ad, bd, kIdescS, kk > 0);
-      }
-      umma_commit(&bar_s);
-    }
-    ok = bounded_wait(&bar_s, ph_s);
-    ph_s ^= 1u;
+    const uint32_t vb = sV + buf * kKV;
+    ok = bounded_wait(&bar_s[buf], ph_s[buf]);
+    ph_s[buf] ^= 1u;
     if (!ok) break;
     tc5_fence_after();
+    // the next tile's scores go to the other buffer (its last reader finished before the barrier
+    // at the end of the previous iteration; its K tile was staged and fenced there too)
+    if (threadIdx.x == 0 && kt + 1 < n_ktiles) issue_scores(kt + 1);
+    // K buffer `buf` is free now: fetch the key tile after next
+    if (kt + 2 < n_ktiles)
+      stage_tc5<kTN>(sK + buf * kKV, A.k, layer, lead, lazy, gla, A.kind, (kt + 2) * kTN, A.T, A.hkv, kvh);
     // ---- this row's 64 scores
     float p[kTN];
     {
       uint32_t r[32];
-      tmem_ld32(t_row + kColS, r);
+      tmem_ld32(t_row + kColS + buf * kTN, r);
 #pragma unroll
       for (int j = 0; j < 32; ++j) p[j] = __uint_as_float(r[j]);
-      tmem_ld32(t_row + kColS + 32, r);
+      tmem_ld32(t_row + kColS + buf * kTN + 32, r);
 #pragma unroll
       for (int j = 0; j < 32; ++j) p[32 + j] = __uint_as_float(r[j]);
     }
@@ -444,18 +457,16 @@ __global__ void __launch_bounds__(kTM, 2) prefill_attend_tcgen05_kernel(const Pr
       psum += p[j];
     }
     l_sum = l_sum * corr + psum;
-    // ---- the previous value product must be done before P, O or the other K/V buffer change
+    // ---- the previous value product must be done before P, O or the other V buffer change
     if (kt > 0) {
       ok = bounded_wait(&bar_o, ph_o);
       ph_o ^= 1u;
       if (!ok) break;
       tc5_fence_after();
     }
-    if (kt + 1 < n_ktiles) {
-      stage_tc5<kTN>(sK + (buf ^ 1) * kKV, A.k, layer, lead, lazy, gla, A.kind, (kt + 1) * kTN, A.T, A.hkv, kvh);
+    if (kt + 1 < n_ktiles)
       stage_tc5<kTN>(sV + (buf ^ 1) * kKV, A.v, layer, layer, false, false, A.kind, (kt + 1) * kTN, A.T, A.hkv, kvh);
-      cp_async_commit();
-    }
+    cp_async_commit();
     if (kt > 0 && __any_sync(0xffffffffu, corr != 1.f)) {   // rare: move the accumulator to the new reference
 #pragma unroll
       for (int c = 0; c < kTD / 32; ++c) {
