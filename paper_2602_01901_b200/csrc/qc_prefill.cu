@@ -285,6 +285,22 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
       : "r"(taddr));
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
+__device__ __forceinline__ void tmem_ld32_nowait(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+}
+// 2^x, single MUFU instruction (2^-inf = 0)
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
@@ -301,23 +317,27 @@ template <int ROWS>
 __device__ __forceinline__ void stage_tc5(uint32_t smem, const uint16_t* base, int own, int lead, bool lazy, bool gla,
                                           const uint8_t* kind, int row0, int T, int heads, int head) {
   constexpr int CH = kTD / 8;
-  constexpr int RPP = kTM / CH;      // 8 rows per pass
+  constexpr int RPP = kTM / CH;      // 8 rows per pass: (row & 7) is the same in every pass of a thread
   constexpr int NP = ROWS / RPP;
   const int c = threadIdx.x % CH, r0 = threadIdx.x / CH;
-  int layer_of[NP];
+  const size_t row_elems = static_cast<size_t>(heads) * kTD;
+  const uint16_t* src = base + (static_cast<size_t>(own) * T + row0 + r0) * row_elems + head * kTD + c * 8;
+  const ptrdiff_t to_lead = (static_cast<ptrdiff_t>(lead) - own) * static_cast<ptrdiff_t>(T) * row_elems;
+  const uint32_t dst = smem + tc5_off(r0, c, ROWS);
+  const bool by_kind = lazy && !gla;
+  bool use_lead[NP];
 #pragma unroll
   for (int i = 0; i < NP; ++i) {
     const int t = row0 + r0 + i * RPP;
-    layer_of[i] = (lazy && (gla || (t < T && kind[t]))) ? lead : own;
+    use_lead[i] = lazy && (gla || (by_kind && t < T && kind[t]));
   }
 #pragma unroll
   for (int i = 0; i < NP; ++i) {
-    const int r = r0 + i * RPP, t = row0 + r;
-    const uint32_t dst = smem + tc5_off(r, c, ROWS);
+    const int t = row0 + r0 + i * RPP;
     if (t < T) {
-      cp_async16(dst, base + ((static_cast<size_t>(layer_of[i]) * T + t) * heads + head) * kTD + c * 8);
+      cp_async16(dst + i * (RPP * 128), src + i * RPP * row_elems + (use_lead[i] ? to_lead : 0));
     } else {
-      asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(dst), "r"(0u) : "memory");
+      asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(dst + i * (RPP * 128)), "r"(0u) : "memory");
     }
   }
 }
@@ -413,6 +433,10 @@ __global__ void __launch_bounds__(kTM, 2) prefill_attend_tcgen05_kernel(const Pr
   for (int kt = 0; kt < n_ktiles && ok; ++kt) {
     const int buf = kt & 1;
     const uint32_t vb = sV + buf * kKV;
+    // Copy groups, oldest first: ..., K(kt+1), V(kt) | this iteration adds K(kt+2), then V(kt+1).
+    // Here K(kt+1) must have landed (it feeds the score product issued below): one group may pend.
+    cp_async_wait<1>();
+    fence_proxy_async();
     ok = bounded_wait(&bar_s[buf], ph_s[buf]);
     ph_s[buf] ^= 1u;
     if (!ok) break;
@@ -423,25 +447,29 @@ __global__ void __launch_bounds__(kTM, 2) prefill_attend_tcgen05_kernel(const Pr
     // K buffer `buf` is free now: fetch the key tile after next
     if (kt + 2 < n_ktiles)
       stage_tc5<kTN>(sK + buf * kKV, A.k, layer, lead, lazy, gla, A.kind, (kt + 2) * kTN, A.T, A.hkv, kvh);
-    // ---- this row's 64 scores
+    cp_async_commit();
+    // ---- this row's 64 scores (raw dot products; the scale is folded into the exponent)
     float p[kTN];
     {
-      uint32_t r[32];
-      tmem_ld32(t_row + kColS + buf * kTN, r);
+      uint32_t r0[32], r1[32];
+      tmem_ld32_nowait(t_row + kColS + buf * kTN, r0);
+      tmem_ld32_nowait(t_row + kColS + buf * kTN + 32, r1);
+      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-      for (int j = 0; j < 32; ++j) p[j] = __uint_as_float(r[j]);
-      tmem_ld32(t_row + kColS + buf * kTN + 32, r);
-#pragma unroll
-      for (int j = 0; j < 32; ++j) p[32 + j] = __uint_as_float(r[j]);
+      for (int j = 0; j < 32; ++j) p[j] = __uint_as_float(r0[j]), p[32 + j] = __uint_as_float(r1[j]);
     }
     const int n0 = kt * kTN;
-    float m_tile = -INFINITY;
+    if (n0 + kTN - 1 > m0 || n0 + kTN > A.T) {   // only tiles on the diagonal or at the end of the prompt need the mask
 #pragma unroll
-    for (int j = 0; j < kTN; ++j) {
-      const int key = n0 + j;
-      p[j] = (key <= row && key < A.T) ? p[j] * A.scale_log2 : -INFINITY;
-      m_tile = fmaxf(m_tile, p[j]);
+      for (int j = 0; j < kTN; ++j) {
+        const int key = n0 + j;
+        if (!(key <= row && key < A.T)) p[j] = -INFINITY;
+      }
     }
+    float m_raw = p[0];
+#pragma unroll
+    for (int j = 1; j < kTN; ++j) m_raw = fmaxf(m_raw, p[j]);
+    const float m_tile = m_raw * A.scale_log2;   // the scale is positive
     float corr = 1.f;
     if (m_tile > m_ref + kRescaleThreshold || m_ref == -INFINITY) {
       if (m_tile != -INFINITY) {
@@ -449,11 +477,11 @@ __global__ void __launch_bounds__(kTM, 2) prefill_attend_tcgen05_kernel(const Pr
         m_ref = m_tile;
       }
     }
-    const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
+    const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
     float psum = 0.f;
 #pragma unroll
     for (int j = 0; j < kTN; ++j) {
-      p[j] = exp2f(p[j] - m_use);
+      p[j] = ex2_approx(fmaf(p[j], A.scale_log2, neg_m));
       psum += p[j];
     }
     l_sum = l_sum * corr + psum;
@@ -487,7 +515,7 @@ __global__ void __launch_bounds__(kTM, 2) prefill_attend_tcgen05_kernel(const Pr
                    "r"(w2), "r"(w3)
                    : "memory");
     }
-    cp_async_wait<0>();
+    cp_async_wait<2>();      // V(kt) has landed; the two groups of this iteration may still be in flight
     fence_proxy_async();     // generic-proxy writes (weights, staged tiles) before the tensor core reads them
     tc5_fence_before();
     __syncthreads();
