@@ -342,16 +342,29 @@ __device__ __forceinline__ void stage_tc5(uint32_t smem, const uint16_t* base, i
   }
 }
 
-// Bounded wait whose verdict is the same for every thread of the CTA (so that nobody is left
-// alone at a later barrier).
+// Bounded wait on an mbarrier phase.
 __device__ __forceinline__ bool bounded_wait(uint64_t* bar, uint32_t parity) {
   constexpr uint32_t kLimit = 1u << 18;
   uint32_t done = mbar_try_wait(bar, parity);
   for (uint32_t spin = 0; !done && spin < kLimit; ++spin) done = mbar_try_wait(bar, parity);
-  return __syncthreads_and(done != 0) != 0;
+  return done != 0;
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
-__global__ void __launch_bounds__(kTM, 2) prefill_attend_tcgen05_kernel(const PrefillArgs A, int32_t* err) {
+constexpr int kTc5Threads = kTM + 32;   // 128 softmax threads (one per query row) + one warp that issues the products
+
+// Warp roles.  Warps 0-3: one thread per query row -- stage the K/V tiles (cp.async), read the
+// row's scores from TMEM, online softmax, write the bf16 weights.  Warp 4, one lane: issues every
+// tcgen05.mma (issue can block while the tensor core is busy, so it must not sit on the softmax
+// path).  Hand-offs are mbarriers only:
+//   bar_s[b]  tensor core -> softmax   score buffer b holds S(kt)            (tcgen05.commit)
+//   bar_p     softmax -> issuer        weights P(kt) written, S(kt) read, K(kt+2) and V(kt) staged (128 arrivals)
+//   bar_o     tensor core -> softmax   value product of tile kt done: P, O and a V buffer may change
+// Order of products on the tensor core: S(0) S(1) | PV(0) S(2) | PV(1) S(3) | ...  While the threads
+// work on tile kt, the tensor core runs PV(kt-1) and S(kt+1).
+__global__ void __launch_bounds__(kTc5Threads, 2) prefill_attend_tcgen05_kernel(const PrefillArgs A, int32_t* err) {
   // No static shared memory: the dynamic window then starts on the 1024-byte boundary that the
   // swizzled tiles need, and two CTAs fit an SM (2 x 112 KiB of tiles).  Checked below.
   extern __shared__ __align__(1024) uint8_t smem_dyn[];
@@ -364,13 +377,16 @@ __global__ void __launch_bounds__(kTM, 2) prefill_attend_tcgen05_kernel(const Pr
   constexpr uint32_t kTiles = 2 * kTM * 128 + 4 * kKV + kTM * 128;
   uint64_t* bar_s = reinterpret_cast<uint64_t*>(smem_dyn + kTiles);          // two: one per score buffer
   uint64_t& bar_o = *reinterpret_cast<uint64_t*>(smem_dyn + kTiles + 16);
-  uint32_t& tmem_base_slot = *reinterpret_cast<uint32_t*>(smem_dyn + kTiles + 24);
+  uint64_t& bar_p = *reinterpret_cast<uint64_t*>(smem_dyn + kTiles + 24);
+  uint32_t& tmem_base_slot = *reinterpret_cast<uint32_t*>(smem_dyn + kTiles + 32);
+  volatile int32_t& failed = *reinterpret_cast<volatile int32_t*>(smem_dyn + kTiles + 36);
   if (base & 1023u) {   // cannot happen with the layout above; never run the tensor core on a misplaced tile
     if (threadIdx.x == 0) atomicMax(err, kErrBadPage);
     return;
   }
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const bool softmax_thread = threadIdx.x < kTM;
   const int n_qtiles = (A.T + kTM - 1) / kTM;
   const int qt = n_qtiles - 1 - blockIdx.x;         // long rows first
   const int head = blockIdx.y, layer = blockIdx.z;
@@ -379,186 +395,198 @@ __global__ void __launch_bounds__(kTM, 2) prefill_attend_tcgen05_kernel(const Pr
   const int lead = A.leader[layer];
   const bool gla = A.gla != 0;
   const int m0 = qt * kTM;
-  const int row = m0 + threadIdx.x;                 // this thread's query row
+  const int row = m0 + threadIdx.x;                 // a softmax thread's query row
   const int n_ktiles = min((A.T + kTN - 1) / kTN, (m0 + kTM + kTN - 1) / kTN);
 
   if (threadIdx.x == 0) {
     mbar_init(&bar_s[0], 1);
     mbar_init(&bar_s[1], 1);
     mbar_init(&bar_o, 1);
+    mbar_init(&bar_p, kTM);
     fence_mbar_init();
+    failed = 0;
   }
-  if (warp == 0) {
+  if (warp == 4) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
                  "r"(kTmemCols)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  stage_tc5<kTM>(sQ, A.q, layer, lead, lazy, gla, A.kind, m0, A.T, A.hq, head);
-  stage_tc5<kTN>(sK, A.k, layer, lead, lazy, gla, A.kind, 0, A.T, A.hkv, kvh);
-  stage_tc5<kTN>(sV, A.v, layer, layer, false, false, A.kind, 0, A.T, A.hkv, kvh);
-  if (n_ktiles > 1) stage_tc5<kTN>(sK + kKV, A.k, layer, lead, lazy, gla, A.kind, kTN, A.T, A.hkv, kvh);
-  cp_async_commit();
-  cp_async_wait<0>();
-  fence_proxy_async();
+  if (softmax_thread) {
+    stage_tc5<kTM>(sQ, A.q, layer, lead, lazy, gla, A.kind, m0, A.T, A.hq, head);
+    stage_tc5<kTN>(sK, A.k, layer, lead, lazy, gla, A.kind, 0, A.T, A.hkv, kvh);
+    stage_tc5<kTN>(sV, A.v, layer, layer, false, false, A.kind, 0, A.T, A.hkv, kvh);
+    if (n_ktiles > 1) stage_tc5<kTN>(sK + kKV, A.k, layer, lead, lazy, gla, A.kind, kTN, A.T, A.hkv, kvh);
+    cp_async_commit();
+    cp_async_wait<0>();
+    fence_proxy_async();
+  }
   tc5_fence_before();
   __syncthreads();
   tc5_fence_after();
   const uint32_t tmem = tmem_base_slot;
-  const uint32_t t_row = tmem + (static_cast<uint32_t>(warp * 32) << 16);   // this warp's 32 TMEM lanes
 
   // instruction descriptors: fp32 accumulate, bf16 operands, M 128; S: N 64, both K-major; PV: N 128, B MN-major
   constexpr uint32_t kIdescS = (1u << 4) | (1u << 7) | (1u << 10) | ((kTN >> 3) << 17) | ((kTM >> 4) << 24);
   constexpr uint32_t kIdescO = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((kTD >> 3) << 17) | ((kTM >> 4) << 24);
 
-  // S = Q K^T of key tile kt into score buffer kt & 1 (two buffers of 64 TMEM columns)
-  auto issue_scores = [&](int kt) {
-    const uint32_t kb = sK + (kt & 1) * kKV;
+  if (warp == 4) {
+    // ------------------------------------------------------------------ product issuer
+    if (lane == 0) {
+      // S = Q K^T of key tile kt into score buffer kt & 1 (two buffers of 64 TMEM columns)
+      auto issue_scores = [&](int kt) {
+        const uint32_t kb = sK + (kt & 1) * kKV;
 #pragma unroll
-    for (int kk = 0; kk < kTD / 16; ++kk) {
-      const uint64_t ad = umma_desc(sQ + (kk >> 2) * (kTM * 128) + (kk & 3) * 32, 16, 1024);
-      const uint64_t bd = umma_desc(kb + (kk >> 2) * (kTN * 128) + (kk & 3) * 32, 16, 1024);
-      umma_f16(tmem + kColS + (kt & 1) * kTN, ad, bd, kIdescS, kk > 0);
-    }
-    umma_commit(&bar_s[kt & 1]);
-  };
-
-  float m_ref = -INFINITY, l_sum = 0.f;
-  uint32_t ph_s[2] = {0, 0}, ph_o = 0;
-  bool ok = true;
-  if (threadIdx.x == 0) issue_scores(0);
-
-  // Software pipeline: while the threads work on the scores of tile kt, the tensor core already
-  // computes the scores of tile kt + 1 and the value product of tile kt - 1.
-  for (int kt = 0; kt < n_ktiles && ok; ++kt) {
-    const int buf = kt & 1;
-    const uint32_t vb = sV + buf * kKV;
-    // Copy groups, oldest first: ..., K(kt+1), V(kt) | this iteration adds K(kt+2), then V(kt+1).
-    // Here K(kt+1) must have landed (it feeds the score product issued below): one group may pend.
-    cp_async_wait<1>();
-    fence_proxy_async();
-    ok = bounded_wait(&bar_s[buf], ph_s[buf]);
-    ph_s[buf] ^= 1u;
-    if (!ok) break;
-    tc5_fence_after();
-    // the next tile's scores go to the other buffer (its last reader finished before the barrier
-    // at the end of the previous iteration; its K tile was staged and fenced there too)
-    if (threadIdx.x == 0 && kt + 1 < n_ktiles) issue_scores(kt + 1);
-    // K buffer `buf` is free now: fetch the key tile after next
-    if (kt + 2 < n_ktiles)
-      stage_tc5<kTN>(sK + buf * kKV, A.k, layer, lead, lazy, gla, A.kind, (kt + 2) * kTN, A.T, A.hkv, kvh);
-    cp_async_commit();
-    // ---- this row's 64 scores (raw dot products; the scale is folded into the exponent)
-    float p[kTN];
-    {
-      uint32_t r0[32], r1[32];
-      tmem_ld32_nowait(t_row + kColS + buf * kTN, r0);
-      tmem_ld32_nowait(t_row + kColS + buf * kTN + 32, r1);
-      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        for (int kk = 0; kk < kTD / 16; ++kk) {
+          const uint64_t ad = umma_desc(sQ + (kk >> 2) * (kTM * 128) + (kk & 3) * 32, 16, 1024);
+          const uint64_t bd = umma_desc(kb + (kk >> 2) * (kTN * 128) + (kk & 3) * 32, 16, 1024);
+          umma_f16(tmem + kColS + (kt & 1) * kTN, ad, bd, kIdescS, kk > 0);
+        }
+        umma_commit(&bar_s[kt & 1]);
+      };
+      issue_scores(0);
+      if (n_ktiles > 1) issue_scores(1);
+      uint32_t ph_p = 0;
+      for (int kt = 0; kt < n_ktiles; ++kt) {
+        if (!bounded_wait(&bar_p, ph_p) || failed) {
+          failed = 1;
+          break;
+        }
+        ph_p ^= 1u;
+        tc5_fence_after();
+        const uint32_t vb = sV + (kt & 1) * kKV;
 #pragma unroll
-      for (int j = 0; j < 32; ++j) p[j] = __uint_as_float(r0[j]), p[32 + j] = __uint_as_float(r1[j]);
+        for (int ks = 0; ks < kTN / 16; ++ks) {   // O += P V
+          const uint64_t ad = umma_desc(sP + ks * 32, 16, 1024);
+          const uint64_t bd = umma_desc(vb + ks * (16 * 128), kTN * 128, 1024);
+          umma_f16(tmem + kColO, ad, bd, kIdescO, (kt > 0 || ks > 0) ? 1u : 0u);
+        }
+        umma_commit(&bar_o);
+        if (kt + 2 < n_ktiles) issue_scores(kt + 2);
+      }
     }
-    const int n0 = kt * kTN;
-    if (n0 + kTN - 1 > m0 || n0 + kTN > A.T) {   // only tiles on the diagonal or at the end of the prompt need the mask
+    __syncwarp();
+  } else {
+    // ------------------------------------------------------------------ softmax threads
+    const uint32_t t_row = tmem + (static_cast<uint32_t>(warp * 32) << 16);   // this warp's 32 TMEM lanes
+    float m_ref = -INFINITY, l_sum = 0.f;
+    uint32_t ph_s[2] = {0, 0}, ph_o = 0;
+    bool ok = true;
+    for (int kt = 0; kt < n_ktiles; ++kt) {
+      const int buf = kt & 1;
+      ok = bounded_wait(&bar_s[buf], ph_s[buf]) && !failed;
+      ph_s[buf] ^= 1u;
+      if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+      tc5_fence_after();
+      // K buffer `buf` is free now (S(kt) is done): fetch the key tile after next
+      if (kt + 2 < n_ktiles)
+        stage_tc5<kTN>(sK + buf * kKV, A.k, layer, lead, lazy, gla, A.kind, (kt + 2) * kTN, A.T, A.hkv, kvh);
+      cp_async_commit();
+      // ---- this row's 64 scores (raw dot products; the scale is folded into the exponent)
+      float p[kTN];
+      {
+        uint32_t r0[32], r1[32];
+        tmem_ld32_nowait(t_row + kColS + buf * kTN, r0);
+        tmem_ld32_nowait(t_row + kColS + buf * kTN + 32, r1);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+        for (int j = 0; j < 32; ++j) p[j] = __uint_as_float(r0[j]), p[32 + j] = __uint_as_float(r1[j]);
+      }
+      const int n0 = kt * kTN;
+      if (n0 + kTN - 1 > m0 || n0 + kTN > A.T) {   // only tiles on the diagonal or at the end of the prompt need the mask
+#pragma unroll
+        for (int j = 0; j < kTN; ++j) {
+          const int key = n0 + j;
+          if (!(key <= row && key < A.T)) p[j] = -INFINITY;
+        }
+      }
+      float mx[4] = {p[0], p[1], p[2], p[3]};
+#pragma unroll
+      for (int j = 4; j < kTN; ++j) mx[j & 3] = fmaxf(mx[j & 3], p[j]);
+      const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * A.scale_log2;   // the scale is positive
+      float corr = 1.f;
+      if (m_tile > m_ref + kRescaleThreshold || m_ref == -INFINITY) {
+        if (m_tile != -INFINITY) {
+          corr = exp2f(m_ref - m_tile);     // 0 on the first tile
+          m_ref = m_tile;
+        }
+      }
+      const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
+      float ps[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int j = 0; j < kTN; ++j) {
-        const int key = n0 + j;
-        if (!(key <= row && key < A.T)) p[j] = -INFINITY;
+        p[j] = ex2_approx(fmaf(p[j], A.scale_log2, neg_m));
+        ps[j & 3] += p[j];
       }
-    }
-    float m_raw = p[0];
-#pragma unroll
-    for (int j = 1; j < kTN; ++j) m_raw = fmaxf(m_raw, p[j]);
-    const float m_tile = m_raw * A.scale_log2;   // the scale is positive
-    float corr = 1.f;
-    if (m_tile > m_ref + kRescaleThreshold || m_ref == -INFINITY) {
-      if (m_tile != -INFINITY) {
-        corr = exp2f(m_ref - m_tile);     // 0 on the first tile
-        m_ref = m_tile;
+      l_sum = l_sum * corr + ((ps[0] + ps[1]) + (ps[2] + ps[3]));
+      // ---- the previous value product must be done before P, O or the other V buffer change
+      if (kt > 0) {
+        ok = bounded_wait(&bar_o, ph_o) && !failed;
+        ph_o ^= 1u;
+        if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+        tc5_fence_after();
       }
-    }
-    const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
-    float psum = 0.f;
+      if (kt + 1 < n_ktiles)
+        stage_tc5<kTN>(sV + (buf ^ 1) * kKV, A.v, layer, layer, false, false, A.kind, (kt + 1) * kTN, A.T, A.hkv, kvh);
+      cp_async_commit();
+      if (kt > 0 && __any_sync(0xffffffffu, corr != 1.f)) {   // rare: move the accumulator to the new reference
 #pragma unroll
-    for (int j = 0; j < kTN; ++j) {
-      p[j] = ex2_approx(fmaf(p[j], A.scale_log2, neg_m));
-      psum += p[j];
+        for (int c = 0; c < kTD / 32; ++c) {
+          uint32_t r[32];
+          tmem_ld32(t_row + kColO + 32 * c, r);
+#pragma unroll
+          for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * corr);
+          tmem_st32(t_row + kColO + 32 * c, r);
+        }
+        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+      }
+      // ---- weights as the A operand: row threadIdx.x, 64 keys = one 128-byte swizzled line
+#pragma unroll
+      for (int c = 0; c < kTN / 8; ++c) {
+        const uint32_t w0 = pack_bf16x2(p[8 * c + 0], p[8 * c + 1]), w1 = pack_bf16x2(p[8 * c + 2], p[8 * c + 3]);
+        const uint32_t w2 = pack_bf16x2(p[8 * c + 4], p[8 * c + 5]), w3 = pack_bf16x2(p[8 * c + 6], p[8 * c + 7]);
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sP + tc5_off(threadIdx.x, c, kTM)), "r"(w0),
+                     "r"(w1), "r"(w2), "r"(w3)
+                     : "memory");
+      }
+      // Copy groups, oldest first: ..., V(kt) | K(kt+2), V(kt+1).  All but the newest must have landed:
+      // V(kt) feeds the value product issued next, K(kt+2) the score product issued right after it.
+      cp_async_wait<1>();
+      fence_proxy_async();     // generic-proxy writes (weights, staged tiles) before the tensor core reads them
+      tc5_fence_before();
+      mbar_arrive(&bar_p);
     }
-    l_sum = l_sum * corr + psum;
-    // ---- the previous value product must be done before P, O or the other V buffer change
-    if (kt > 0) {
-      ok = bounded_wait(&bar_o, ph_o);
-      ph_o ^= 1u;
-      if (!ok) break;
+    if (ok) ok = bounded_wait(&bar_o, ph_o) && !failed;
+    ok = __all_sync(0xffffffffu, ok);
+    if (ok) {
       tc5_fence_after();
-    }
-    if (kt + 1 < n_ktiles)
-      stage_tc5<kTN>(sV + (buf ^ 1) * kKV, A.v, layer, layer, false, false, A.kind, (kt + 1) * kTN, A.T, A.hkv, kvh);
-    cp_async_commit();
-    if (kt > 0 && __any_sync(0xffffffffu, corr != 1.f)) {   // rare: move the accumulator to the new reference
+      const float inv = 1.f / l_sum;
+      uint16_t* dst = A.out + ((static_cast<size_t>(layer) * A.T + row) * A.hq + head) * kTD;
 #pragma unroll
       for (int c = 0; c < kTD / 32; ++c) {
         uint32_t r[32];
-        tmem_ld32(t_row + kColO + 32 * c, r);
+        tmem_ld32(t_row + kColO + 32 * c, r);   // every lane takes part in the load; only rows of the prompt store
+        if (row < A.T) {
 #pragma unroll
-        for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * corr);
-        tmem_st32(t_row + kColO + 32 * c, r);
-      }
-      asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-    }
-    // ---- weights as the A operand: row threadIdx.x, 64 keys = one 128-byte swizzled line
-#pragma unroll
-    for (int c = 0; c < kTN / 8; ++c) {
-      const uint32_t w0 = pack_bf16x2(p[8 * c + 0], p[8 * c + 1]), w1 = pack_bf16x2(p[8 * c + 2], p[8 * c + 3]);
-      const uint32_t w2 = pack_bf16x2(p[8 * c + 4], p[8 * c + 5]), w3 = pack_bf16x2(p[8 * c + 6], p[8 * c + 7]);
-      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sP + tc5_off(threadIdx.x, c, kTM)), "r"(w0), "r"(w1),
-                   "r"(w2), "r"(w3)
-                   : "memory");
-    }
-    cp_async_wait<2>();      // V(kt) has landed; the two groups of this iteration may still be in flight
-    fence_proxy_async();     // generic-proxy writes (weights, staged tiles) before the tensor core reads them
-    tc5_fence_before();
-    __syncthreads();
-    // ---- O += P V
-    if (threadIdx.x == 0) {
-      tc5_fence_after();
-#pragma unroll
-      for (int ks = 0; ks < kTN / 16; ++ks) {
-        const uint64_t ad = umma_desc(sP + ks * 32, 16, 1024);
-        const uint64_t bd = umma_desc(vb + ks * (16 * 128), kTN * 128, 1024);
-        umma_f16(tmem + kColO, ad, bd, kIdescO, (kt > 0 || ks > 0) ? 1u : 0u);
-      }
-      umma_commit(&bar_o);
-    }
-  }
-  if (ok) ok = bounded_wait(&bar_o, ph_o);
-  if (ok) {
-    tc5_fence_after();
-    const float inv = 1.f / l_sum;
-    uint16_t* dst = A.out + ((static_cast<size_t>(layer) * A.T + row) * A.hq + head) * kTD;
-#pragma unroll
-    for (int c = 0; c < kTD / 32; ++c) {
-      uint32_t r[32];
-      tmem_ld32(t_row + kColO + 32 * c, r);   // every lane takes part in the load; only rows of the prompt store
-      if (row < A.T) {
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          uint4 o;
-          o.x = pack_bf16x2(__uint_as_float(r[8 * j + 0]) * inv, __uint_as_float(r[8 * j + 1]) * inv);
-          o.y = pack_bf16x2(__uint_as_float(r[8 * j + 2]) * inv, __uint_as_float(r[8 * j + 3]) * inv);
-          o.z = pack_bf16x2(__uint_as_float(r[8 * j + 4]) * inv, __uint_as_float(r[8 * j + 5]) * inv);
-          o.w = pack_bf16x2(__uint_as_float(r[8 * j + 6]) * inv, __uint_as_float(r[8 * j + 7]) * inv);
-          *reinterpret_cast<uint4*>(dst + 32 * c + 8 * j) = o;
+          for (int j = 0; j < 4; ++j) {
+            uint4 o;
+            o.x = pack_bf16x2(__uint_as_float(r[8 * j + 0]) * inv, __uint_as_float(r[8 * j + 1]) * inv);
+            o.y = pack_bf16x2(__uint_as_float(r[8 * j + 2]) * inv, __uint_as_float(r[8 * j + 3]) * inv);
+            o.z = pack_bf16x2(__uint_as_float(r[8 * j + 4]) * inv, __uint_as_float(r[8 * j + 5]) * inv);
+            o.w = pack_bf16x2(__uint_as_float(r[8 * j + 6]) * inv, __uint_as_float(r[8 * j + 7]) * inv);
+            *reinterpret_cast<uint4*>(dst + 32 * c + 8 * j) = o;
+          }
         }
       }
+    } else {
+      failed = 1;
+      if (lane == 0) atomicMax(err, kErrTimeout);
     }
-  } else if (threadIdx.x == 0) {
-    atomicMax(err, kErrTimeout);
+    cp_async_wait<0>();
   }
-  cp_async_wait<0>();
   tc5_fence_before();
   __syncthreads();
-  if (warp == 0) {
+  if (warp == 4) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
   }
 }
@@ -607,7 +635,7 @@ cudaError_t launch_prefill_attend(const Params& p, const uint8_t* kind_dev, cons
   a.scale_log2 = p.scale_log2;
   if (p.d == kTD && use_tcgen05) {
     const dim3 grid5((T + kTM - 1) / kTM, p.hq, p.n_layers);
-    prefill_attend_tcgen05_kernel<<<grid5, kTM, prefill_tcgen05_smem_bytes(), stream>>>(a, p.err);
+    prefill_attend_tcgen05_kernel<<<grid5, kTc5Threads, prefill_tcgen05_smem_bytes(), stream>>>(a, p.err);
     return cudaGetLastError();
   }
   const dim3 grid((T + kBM - 1) / kBM, p.hq, p.n_layers);
