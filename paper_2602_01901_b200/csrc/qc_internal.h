@@ -120,7 +120,8 @@ cudaError_t launch_prefill_scatter(const Params& p, const int32_t* tok_seq, cons
                                    int32_t tok_offset, cudaStream_t stream);
 cudaError_t launch_prefill_attend(const Params& p, const uint8_t* kind_dev, const uint8_t* layer_kind_dev,
                                   const uint8_t* leader_dev, const void* q, const void* k, const void* v, void* out,
-                                  int32_t n_tokens, int32_t gla, int32_t use_tcgen05, cudaStream_t stream);   // qc_prefill.cu
+                                  int32_t n_tokens, int32_t gla, const CUtensorMap* tmap_k, const CUtensorMap* tmap_v,
+                                  const uint8_t* tile_code_dev, cudaStream_t stream);   // qc_prefill.cu; maps null = mma.sync kernel
 cudaError_t configure_prefill_kernels();
 cudaError_t configure_kernels(int* attend_smem_bytes);
 cudaError_t configure_kernels_tc(int* attend_smem_bytes);

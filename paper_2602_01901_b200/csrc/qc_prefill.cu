@@ -36,6 +36,8 @@ __device__ __forceinline__ uint32_t tile_off(int row, int chunk) {
 }
 
 struct PrefillArgs {
+  CUtensorMap tmap_k, tmap_v;  // k / v as 3-D tensors {D, hkv, n_layers * T}, box {64, 1, 64}, 128-byte swizzle (tcgen05 kernel)
+  const uint8_t* tile_code;    // [ceil(T / 64)] device: 0 = the 64-token tile is all text, 1 = all visual, 2 = mixed
   const uint16_t* q;     // [n_layers][T][hq][D]
   const uint16_t* k;     // [n_layers][T][hkv][D]
   const uint16_t* v;     // [n_layers][T][hkv][D]
@@ -353,18 +355,32 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
+__device__ __forceinline__ void tensor_g2s_3d(uint32_t dst_smem, const void* tmap, int32_t x, int32_t y, int32_t z,
+                                              uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::
+          "r"(dst_smem),
+      "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(z), "r"(smem_u32(bar))
+      : "memory");
+}
+
 constexpr int kTc5Threads = kTM + 32;   // 128 softmax threads (one per query row) + one warp that issues the products
 
-// Warp roles.  Warps 0-3: one thread per query row -- stage the K/V tiles (cp.async), read the
-// row's scores from TMEM, online softmax, write the bf16 weights.  Warp 4, one lane: issues every
+// Warp roles.  Warps 0-3: one thread per query row -- read the row's scores from TMEM, online
+// softmax, write the bf16 weights.  Warp 4: fetches the K/V tiles and, one lane, issues every
 // tcgen05.mma (issue can block while the tensor core is busy, so it must not sit on the softmax
-// path).  Hand-offs are mbarriers only:
-//   bar_s[b]  tensor core -> softmax   score buffer b holds S(kt)            (tcgen05.commit)
-//   bar_p     softmax -> issuer        weights P(kt) written, S(kt) read, K(kt+2) and V(kt) staged (128 arrivals)
-//   bar_o     tensor core -> softmax   value product of tile kt done: P, O and a V buffer may change
+// path).  A K/V tile whose 64 rows all come from one layer -- every tile of an ordinary or GLA
+// layer, and the all-text / all-visual tiles of a VLA lazy layer -- is fetched by two tensor-map
+// copies; only a tile that mixes text and visual rows of a VLA lazy layer is gathered row by row
+// with 16-byte copies by the 32 lanes.  Hand-offs are mbarriers only:
+//   bar_k[b], bar_v[b]  copies -> issuer   K / V tile landed in buffer b
+//   bar_s[b]  tensor core -> softmax, issuer   score buffer b holds S(kt): K buffer b is free
+//   bar_p     softmax -> issuer        weights P(kt) written, S(kt) read, PV(kt-1) seen complete (128 arrivals)
+//   bar_o     tensor core -> softmax   value product of tile kt done: P and O may change
 // Order of products on the tensor core: S(0) S(1) | PV(0) S(2) | PV(1) S(3) | ...  While the threads
 // work on tile kt, the tensor core runs PV(kt-1) and S(kt+1).
-__global__ void __launch_bounds__(kTc5Threads, 2) prefill_attend_tcgen05_kernel(const PrefillArgs A, int32_t* err) {
+__global__ void __launch_bounds__(kTc5Threads, 2)
+    prefill_attend_tcgen05_kernel(const __grid_constant__ PrefillArgs A, int32_t* err) {
   // No static shared memory: the dynamic window then starts on the 1024-byte boundary that the
   // swizzled tiles need, and two CTAs fit an SM (2 x 112 KiB of tiles).  Checked below.
   extern __shared__ __align__(1024) uint8_t smem_dyn[];
@@ -378,8 +394,10 @@ __global__ void __launch_bounds__(kTc5Threads, 2) prefill_attend_tcgen05_kernel(
   uint64_t* bar_s = reinterpret_cast<uint64_t*>(smem_dyn + kTiles);          // two: one per score buffer
   uint64_t& bar_o = *reinterpret_cast<uint64_t*>(smem_dyn + kTiles + 16);
   uint64_t& bar_p = *reinterpret_cast<uint64_t*>(smem_dyn + kTiles + 24);
-  uint32_t& tmem_base_slot = *reinterpret_cast<uint32_t*>(smem_dyn + kTiles + 32);
-  volatile int32_t& failed = *reinterpret_cast<volatile int32_t*>(smem_dyn + kTiles + 36);
+  uint64_t* bar_k = reinterpret_cast<uint64_t*>(smem_dyn + kTiles + 32);          // two
+  uint64_t* bar_v = reinterpret_cast<uint64_t*>(smem_dyn + kTiles + 48);          // two
+  uint32_t& tmem_base_slot = *reinterpret_cast<uint32_t*>(smem_dyn + kTiles + 64);
+  volatile int32_t& failed = *reinterpret_cast<volatile int32_t*>(smem_dyn + kTiles + 68);
   if (base & 1023u) {   // cannot happen with the layout above; never run the tensor core on a misplaced tile
     if (threadIdx.x == 0) atomicMax(err, kErrBadPage);
     return;
@@ -403,6 +421,10 @@ __global__ void __launch_bounds__(kTc5Threads, 2) prefill_attend_tcgen05_kernel(
     mbar_init(&bar_s[1], 1);
     mbar_init(&bar_o, 1);
     mbar_init(&bar_p, kTM);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&bar_k[b], 1);
+      mbar_init(&bar_v[b], 1);
+    }
     fence_mbar_init();
     failed = 0;
   }
@@ -414,9 +436,6 @@ __global__ void __launch_bounds__(kTc5Threads, 2) prefill_attend_tcgen05_kernel(
   }
   if (softmax_thread) {
     stage_tc5<kTM>(sQ, A.q, layer, lead, lazy, gla, A.kind, m0, A.T, A.hq, head);
-    stage_tc5<kTN>(sK, A.k, layer, lead, lazy, gla, A.kind, 0, A.T, A.hkv, kvh);
-    stage_tc5<kTN>(sV, A.v, layer, layer, false, false, A.kind, 0, A.T, A.hkv, kvh);
-    if (n_ktiles > 1) stage_tc5<kTN>(sK + kKV, A.k, layer, lead, lazy, gla, A.kind, kTN, A.T, A.hkv, kvh);
     cp_async_commit();
     cp_async_wait<0>();
     fence_proxy_async();
@@ -431,30 +450,87 @@ __global__ void __launch_bounds__(kTc5Threads, 2) prefill_attend_tcgen05_kernel(
   constexpr uint32_t kIdescO = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((kTD >> 3) << 17) | ((kTM >> 4) << 24);
 
   if (warp == 4) {
-    // ------------------------------------------------------------------ product issuer
-    if (lane == 0) {
-      // S = Q K^T of key tile kt into score buffer kt & 1 (two buffers of 64 TMEM columns)
-      auto issue_scores = [&](int kt) {
-        const uint32_t kb = sK + (kt & 1) * kKV;
+    // ------------------------------------------------------------------ tile fetch + product issuer
+    // Fetch key tile (is_k) or value tile kt into `dst`; completion is one phase of `bar`.
+    auto fetch_tile = [&](bool is_k, int kt, uint32_t dst, uint64_t* bar) {
+      int src = layer;
+      bool mixed = false;
+      if (is_k && lazy) {
+        if (gla) {
+          src = lead;
+        } else {
+          const int code = A.tile_code[kt];
+          mixed = code == 2;
+          src = code == 1 ? lead : layer;
+        }
+      }
+      if (!mixed) {
+        if (lane == 0) {
+          const void* tm = is_k ? static_cast<const void*>(&A.tmap_k) : static_cast<const void*>(&A.tmap_v);
+          mbar_expect_tx(bar, kKV);
+          tensor_g2s_3d(dst, tm, 0, kvh, src * A.T + kt * kTN, bar);
+          tensor_g2s_3d(dst + kTN * 128, tm, 64, kvh, src * A.T + kt * kTN, bar);
+        }
+      } else {   // rows of two layers: gather with 16-byte copies (64 rows x 16 chunks over 32 lanes)
+        for (int e = lane; e < kTN * (kTD / 8); e += 32) {
+          const int r = e >> 4, c = e & 15, t = kt * kTN + r;
+          const uint32_t d = dst + tc5_off(r, c, kTN);
+          if (t < A.T) {
+            const int l = A.kind[t] ? lead : layer;
+            cp_async16(d, A.k + ((static_cast<size_t>(l) * A.T + t) * A.hkv + kvh) * kTD + c * 8);
+          } else {
+            asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(d), "r"(0u) : "memory");
+          }
+        }
+        cp_async_commit();
+        cp_async_wait<0>();
+        fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar);
+      }
+    };
+    // S = Q K^T of key tile kt into score buffer kt & 1 (two buffers of 64 TMEM columns)
+    auto issue_scores = [&](int kt) {
+      const uint32_t kb = sK + (kt & 1) * kKV;
 #pragma unroll
-        for (int kk = 0; kk < kTD / 16; ++kk) {
-          const uint64_t ad = umma_desc(sQ + (kk >> 2) * (kTM * 128) + (kk & 3) * 32, 16, 1024);
-          const uint64_t bd = umma_desc(kb + (kk >> 2) * (kTN * 128) + (kk & 3) * 32, 16, 1024);
-          umma_f16(tmem + kColS + (kt & 1) * kTN, ad, bd, kIdescS, kk > 0);
-        }
-        umma_commit(&bar_s[kt & 1]);
-      };
-      issue_scores(0);
-      if (n_ktiles > 1) issue_scores(1);
-      uint32_t ph_p = 0;
-      for (int kt = 0; kt < n_ktiles; ++kt) {
-        if (!bounded_wait(&bar_p, ph_p) || failed) {
-          failed = 1;
-          break;
-        }
-        ph_p ^= 1u;
+      for (int kk = 0; kk < kTD / 16; ++kk) {
+        const uint64_t ad = umma_desc(sQ + (kk >> 2) * (kTM * 128) + (kk & 3) * 32, 16, 1024);
+        const uint64_t bd = umma_desc(kb + (kk >> 2) * (kTN * 128) + (kk & 3) * 32, 16, 1024);
+        umma_f16(tmem + kColS + (kt & 1) * kTN, ad, bd, kIdescS, kk > 0);
+      }
+      umma_commit(&bar_s[kt & 1]);
+    };
+    uint32_t ph_k[2] = {0, 0}, ph_v[2] = {0, 0}, ph_sw[2] = {0, 0}, ph_p = 0;
+    bool ok = true;
+    auto wait_on = [&](uint64_t* bar, uint32_t& phase) {   // warp-uniform bounded wait
+      if (ok) ok = __all_sync(0xffffffffu, bounded_wait(bar, phase) && !failed);
+      phase ^= 1u;
+    };
+    fetch_tile(true, 0, sK, &bar_k[0]);
+    fetch_tile(false, 0, sV, &bar_v[0]);
+    if (n_ktiles > 1) fetch_tile(true, 1, sK + kKV, &bar_k[1]);
+    for (int kt = 0; kt < 2 && kt < n_ktiles; ++kt) {
+      wait_on(&bar_k[kt], ph_k[kt]);
+      if (ok && lane == 0) {
         tc5_fence_after();
-        const uint32_t vb = sV + (kt & 1) * kKV;
+        issue_scores(kt);
+      }
+    }
+    // once S(0) is complete its K buffer can take tile 2
+    if (n_ktiles > 2) {
+      wait_on(&bar_s[0], ph_sw[0]);
+      if (ok) fetch_tile(true, 2, sK, &bar_k[0]);
+    }
+    for (int kt = 0; kt < n_ktiles && ok; ++kt) {
+      const int buf = kt & 1;
+      wait_on(&bar_p, ph_p);                      // P(kt) ready; the threads have seen PV(kt-1) complete
+      if (!ok) break;
+      if (kt + 1 < n_ktiles) fetch_tile(false, kt + 1, sV + (buf ^ 1) * kKV, &bar_v[buf ^ 1]);
+      wait_on(&bar_v[buf], ph_v[buf]);            // V(kt) landed
+      if (!ok) break;
+      if (lane == 0) {
+        tc5_fence_after();
+        const uint32_t vb = sV + buf * kKV;
 #pragma unroll
         for (int ks = 0; ks < kTN / 16; ++ks) {   // O += P V
           const uint64_t ad = umma_desc(sP + ks * 32, 16, 1024);
@@ -462,9 +538,22 @@ __global__ void __launch_bounds__(kTc5Threads, 2) prefill_attend_tcgen05_kernel(
           umma_f16(tmem + kColO, ad, bd, kIdescO, (kt > 0 || ks > 0) ? 1u : 0u);
         }
         umma_commit(&bar_o);
-        if (kt + 2 < n_ktiles) issue_scores(kt + 2);
+      }
+      if (kt + 2 < n_ktiles) {
+        wait_on(&bar_k[buf], ph_k[buf]);          // K(kt+2) landed (fetched one iteration ago)
+        if (!ok) break;
+        if (lane == 0) {
+          tc5_fence_after();
+          issue_scores(kt + 2);
+        }
+      }
+      if (kt + 3 < n_ktiles) {                    // S(kt+1) complete: its K buffer takes tile kt+3
+        wait_on(&bar_s[buf ^ 1], ph_sw[buf ^ 1]);
+        if (!ok) break;
+        fetch_tile(true, kt + 3, sK + (buf ^ 1) * kKV, &bar_k[buf ^ 1]);
       }
     }
+    if (!ok) failed = 1;
     __syncwarp();
   } else {
     // ------------------------------------------------------------------ softmax threads
@@ -478,10 +567,6 @@ __global__ void __launch_bounds__(kTc5Threads, 2) prefill_attend_tcgen05_kernel(
       ph_s[buf] ^= 1u;
       if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
       tc5_fence_after();
-      // K buffer `buf` is free now (S(kt) is done): fetch the key tile after next
-      if (kt + 2 < n_ktiles)
-        stage_tc5<kTN>(sK + buf * kKV, A.k, layer, lead, lazy, gla, A.kind, (kt + 2) * kTN, A.T, A.hkv, kvh);
-      cp_async_commit();
       // ---- this row's 64 scores (raw dot products; the scale is folded into the exponent)
       float p[kTN];
       {
@@ -526,9 +611,6 @@ __global__ void __launch_bounds__(kTc5Threads, 2) prefill_attend_tcgen05_kernel(
         if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
         tc5_fence_after();
       }
-      if (kt + 1 < n_ktiles)
-        stage_tc5<kTN>(sV + (buf ^ 1) * kKV, A.v, layer, layer, false, false, A.kind, (kt + 1) * kTN, A.T, A.hkv, kvh);
-      cp_async_commit();
       if (kt > 0 && __any_sync(0xffffffffu, corr != 1.f)) {   // rare: move the accumulator to the new reference
 #pragma unroll
         for (int c = 0; c < kTD / 32; ++c) {
@@ -549,10 +631,7 @@ __global__ void __launch_bounds__(kTc5Threads, 2) prefill_attend_tcgen05_kernel(
                      "r"(w1), "r"(w2), "r"(w3)
                      : "memory");
       }
-      // Copy groups, oldest first: ..., V(kt) | K(kt+2), V(kt+1).  All but the newest must have landed:
-      // V(kt) feeds the value product issued next, K(kt+2) the score product issued right after it.
-      cp_async_wait<1>();
-      fence_proxy_async();     // generic-proxy writes (weights, staged tiles) before the tensor core reads them
+      fence_proxy_async();     // generic-proxy writes (the weights) before the tensor core reads them
       tc5_fence_before();
       mbar_arrive(&bar_p);
     }
@@ -582,7 +661,6 @@ __global__ void __launch_bounds__(kTc5Threads, 2) prefill_attend_tcgen05_kernel(
       failed = 1;
       if (lane == 0) atomicMax(err, kErrTimeout);
     }
-    cp_async_wait<0>();
   }
   tc5_fence_before();
   __syncthreads();
@@ -616,7 +694,8 @@ cudaError_t configure_prefill_kernels() {
 
 cudaError_t launch_prefill_attend(const Params& p, const uint8_t* kind_dev, const uint8_t* layer_kind_dev,
                                   const uint8_t* leader_dev, const void* q, const void* k, const void* v, void* out,
-                                  int32_t T, int32_t gla, int32_t use_tcgen05, cudaStream_t stream) {
+                                  int32_t T, int32_t gla, const CUtensorMap* tmap_k, const CUtensorMap* tmap_v,
+                                  const uint8_t* tile_code_dev, cudaStream_t stream) {
   if (T <= 0) return cudaSuccess;
   PrefillArgs a{};
   a.q = static_cast<const uint16_t*>(q);
@@ -633,7 +712,10 @@ cudaError_t launch_prefill_attend(const Params& p, const uint8_t* kind_dev, cons
   a.n_layers = p.n_layers;
   a.gla = gla;
   a.scale_log2 = p.scale_log2;
-  if (p.d == kTD && use_tcgen05) {
+  if (p.d == kTD && tmap_k && tmap_v) {
+    a.tmap_k = *tmap_k;
+    a.tmap_v = *tmap_v;
+    a.tile_code = tile_code_dev;
     const dim3 grid5((T + kTM - 1) / kTM, p.hq, p.n_layers);
     prefill_attend_tcgen05_kernel<<<grid5, kTc5Threads, prefill_tcgen05_smem_bytes(), stream>>>(a, p.err);
     return cudaGetLastError();

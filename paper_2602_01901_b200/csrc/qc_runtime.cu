@@ -337,22 +337,45 @@ inline int pages_for(int tokens) { return (tokens + kPage - 1) / kPage; }
 // 16 consecutive rows.  Box = 16 rows x 64 elements (128 bytes) with the 128-byte swizzle, so
 // a D = 128 tile is fetched as two column halves.  The driver entry point is looked up at run
 // time; nothing links against the driver library.
-int make_pool_tensor_map(qc_cache* c) {
-  typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                               const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                               CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                             const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                             CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeFn tensor_map_encoder() {
   void* fn = nullptr;
   cudaDriverEntryPointQueryResult qres;
   if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
       qres != cudaDriverEntryPointSuccess)
-    return QC_ERR_CUDA;
+    return nullptr;
+  return reinterpret_cast<EncodeFn>(fn);
+}
+
+// A prompt tensor [n_layers][T][heads][128] bf16 as a 3-D tensor {128, heads, n_layers * T}: a
+// box is 64 tokens x one head x 64 elements (128 bytes) with the 128-byte swizzle.  Rows past
+// the end of the tensor read as zero.
+int make_prompt_tensor_map(CUtensorMap* out, const void* base, int n_layers, int T, int heads) {
+  EncodeFn enc = tensor_map_encoder();
+  if (!enc) return QC_ERR_CUDA;
+  const cuuint64_t dims[3] = {128, static_cast<cuuint64_t>(heads), static_cast<cuuint64_t>(n_layers) * T};
+  const cuuint64_t strides[2] = {128 * 2, static_cast<cuuint64_t>(heads) * 128 * 2};
+  const cuuint32_t box[3] = {64, 1, 64};
+  const cuuint32_t elem_strides[3] = {1, 1, 1};
+  const CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box,
+                         elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                         CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? QC_OK : QC_ERR_CUDA;
+}
+
+int make_pool_tensor_map(qc_cache* c) {
+  EncodeFn enc = tensor_map_encoder();
+  if (!enc) return QC_ERR_CUDA;
   const cuuint64_t rows = static_cast<cuuint64_t>(c->n_pool_pages) * c->hkv * kPage;
   if (rows > 0x7fffffffULL) return QC_ERR_INVALID_ARG;   // tile coordinates are 32-bit
   const cuuint64_t dims[2] = {static_cast<cuuint64_t>(c->D), rows};
   const cuuint64_t strides[1] = {static_cast<cuuint64_t>(c->D) * 2};
   const cuuint32_t box[2] = {64, kPage};
   const cuuint32_t elem_strides[2] = {1, 1};
-  const CUresult r = reinterpret_cast<EncodeFn>(fn)(
+  const CUresult r = enc(
       &c->tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, c->pool, dims, strides, box, elem_strides,
       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -682,8 +705,25 @@ int32_t qc_prefill_attend(qc_cache* c, int32_t seq_id, int32_t n_tokens, const u
   if (st != QC_OK) return st;
   cudaStream_t stream = c->ctx->stream;
   uint8_t* kind_dev = c->ws + c->lay.tok;   // free again: qc_prefill_append has waited for its copies
+  // per 64-token tile: all text, all visual or mixed (the tcgen05 kernel fetches unmixed tiles whole)
+  const int n_tiles = (n_tokens + 63) / 64;
+  std::vector<uint8_t> codes(n_tiles);
+  for (int i = 0; i < n_tiles; ++i) {
+    int nv = 0, n = std::min(64, n_tokens - 64 * i);
+    for (int t = 0; t < n; ++t) nv += kind[64 * i + t] == QC_KIND_VISUAL;
+    codes[i] = nv == 0 ? 0 : (nv == n ? 1 : 2);
+  }
+  uint8_t* codes_dev = kind_dev + align_up(n_tokens, 256);
   QC_CUDA(cudaMemcpyAsync(kind_dev, kind, n_tokens, cudaMemcpyHostToDevice, stream));
+  QC_CUDA(cudaMemcpyAsync(codes_dev, codes.data(), n_tiles, cudaMemcpyHostToDevice, stream));
   QC_CUDA(cudaStreamSynchronize(stream));   // `kind` is the caller's host memory
+  CUtensorMap tmap_k, tmap_v;
+  const bool tc5 = c->prefill_tcgen05 && c->D == 128;
+  if (tc5) {
+    if (make_prompt_tensor_map(&tmap_k, k_dev, c->cfg.n_layers, n_tokens, c->hkv) != QC_OK ||
+        make_prompt_tensor_map(&tmap_v, v_dev, c->cfg.n_layers, n_tokens, c->hkv) != QC_OK)
+      return QC_ERR_CUDA;
+  }
   const Params p = base_params(c);
   cudaEvent_t* ev = nullptr;
   if (c->profile && c->ev_prefill_calls < kMaxProfileSteps) {
@@ -698,7 +738,8 @@ int32_t qc_prefill_attend(qc_cache* c, int32_t seq_id, int32_t n_tokens, const u
     QC_CUDA(cudaEventRecord(ev[0], stream));
   }
   QC_CUDA(launch_prefill_attend(p, kind_dev, c->ws + c->lay.layer_kind, c->ws + c->lay.leader, q_dev, k_dev, v_dev,
-                                out_dev, n_tokens, c->cfg.lazy_mode == QC_MODE_GLA ? 1 : 0, c->prefill_tcgen05 ? 1 : 0, stream));
+                                out_dev, n_tokens, c->cfg.lazy_mode == QC_MODE_GLA ? 1 : 0, tc5 ? &tmap_k : nullptr,
+                                tc5 ? &tmap_v : nullptr, codes_dev, stream));
   if (ev) {
     QC_CUDA(cudaEventRecord(ev[1], stream));
     c->ev_prefill_calls++;
