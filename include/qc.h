@@ -158,6 +158,27 @@ int32_t qc_prefill_append(qc_cache* cache, int32_t n_seqs, const int32_t* seq_id
 int32_t qc_prefill_attend(qc_cache* cache, int32_t seq_id, int32_t n_tokens, const uint8_t* kind,
                           const void* q_dev, const void* k_dev, const void* v_dev, void* out_dev);
 
+/* Calibration by-product (section "Lazy Attention", Eq. 3).  For a cache whose layers are ALL
+ * ordinary (the analysis runs on the unmodified stack; otherwise QC_ERR_STATE) and one query
+ * token per listed sequence -- normally the prompt's last token, whose K/V are already cached --
+ * computes per layer the attention distribution of that query over every cached token, averaged
+ * over the query heads, and the Jensen-Shannon divergence (natural log, 0..ln 2) between the
+ * distributions of adjacent layers, averaged over the listed sequences:
+ *   similarity_host[l] = mean_i JS(a_i^l, a_i^{l+1}),  l = 0 .. n_layers - 2   (host, written on return)
+ *   q_dev     bf16 [n_layers][n_seqs][n_q_heads][head_dim]
+ *   rows_dev  fp32 [n_layers][n_seqs][max_len], caller-owned scratch and by-product: the
+ *             distributions, text tokens first then visual tokens, zero past a sequence's length
+ * max_len >= every listed sequence's token count and <= 12288 (else QC_ERR_UNSUPPORTED).  The
+ * cache is not changed.  Synchronises the stream. */
+int32_t qc_layer_similarity(qc_cache* cache, int32_t n_seqs, const int32_t* seq_ids, const void* q_dev,
+                            float* rows_dev, int32_t max_len, float* similarity_host);
+
+/* Eq. 4 (host only): layer l+1 joins the lazy block of layer l when similarity[l] < eps
+ * (0 < eps <= 1) and, if max_block > 0, the block has fewer than max_block layers.  Writes
+ * layer_kind[n_layers] for qc_config: the first layer of every block stays ordinary. */
+int32_t qc_lazy_blocks(const float* similarity, int32_t n_layers, float eps, int32_t max_block,
+                       uint8_t* layer_kind);
+
 /* One generated (text) token for each listed sequence through all layers (Eq. 2, 6, 8):
  * appends k/v, refreshes the Q Cache from every ordinary layer's q, computes split-KV partial
  * attention and merges the partials by log-sum-exp.

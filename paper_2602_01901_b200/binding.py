@@ -29,7 +29,7 @@ QC_KIND_TEXT, QC_KIND_VISUAL = 0, 1
 
 EXPORTS = (
     "qc_init", "qc_cache_bytes_required", "qc_alloc_cache", "qc_prefill_append", "qc_prefill_attend", "qc_decode_step",
-    "qc_decode_step_host", "qc_free_seq", "qc_free", "qc_get_stats", "qc_debug_page_table",
+    "qc_decode_step_host", "qc_layer_similarity", "qc_lazy_blocks", "qc_free_seq", "qc_free", "qc_get_stats", "qc_debug_page_table",
     "qc_debug_read_qcache", "qc_debug_read_row", "qc_set_option", "qc_get_profile", "qc_status_string",
     "qc_attend_static",
 )
@@ -92,6 +92,8 @@ def load() -> C.CDLL:
         "qc_prefill_append": [vp, i32, pi32, pi32, pu8, vp, vp],
         "qc_prefill_attend": [vp, i32, i32, pu8, vp, vp, vp, vp],
         "qc_decode_step": [vp, i32, pi32, vp, vp, vp, vp, vp],
+        "qc_layer_similarity": [vp, i32, pi32, vp, vp, i32, C.POINTER(C.c_float)],
+        "qc_lazy_blocks": [C.POINTER(C.c_float), i32, C.c_float, i32, pu8],
         "qc_decode_step_host": [vp, i32, pi32, vp, vp, vp, vp, vp],
         "qc_free_seq": [vp, i32],
         "qc_free": [vp, vp],
@@ -170,6 +172,21 @@ def qc_prefill_attend(cache, seq_id: int, kind, q_ptr: int, k_ptr: int, v_ptr: i
     _check(load().qc_prefill_attend(cache, seq_id, len(kind_bytes), C.cast(kbuf, C.POINTER(C.c_uint8)),
                                     C.c_void_p(q_ptr), C.c_void_p(k_ptr), C.c_void_p(v_ptr), C.c_void_p(out_ptr)),
            "qc_prefill_attend")
+
+
+def qc_layer_similarity(cache, seq_ids: Sequence[int], q_ptr: int, rows_ptr: int, max_len: int, n_layers: int):
+    sim = (C.c_float * max(1, n_layers - 1))()
+    _check(load().qc_layer_similarity(cache, len(seq_ids), _i32_array(seq_ids), C.c_void_p(q_ptr), C.c_void_p(rows_ptr),
+                                      max_len, sim), "qc_layer_similarity")
+    return [float(x) for x in sim[: n_layers - 1]]
+
+
+def qc_lazy_blocks(similarity: Sequence[float], eps: float, max_block: int = 0):
+    n_layers = len(similarity) + 1
+    sim = (C.c_float * max(1, len(similarity)))(*similarity)
+    kind = (C.c_uint8 * n_layers)()
+    _check(load().qc_lazy_blocks(sim, n_layers, eps, max_block, kind), "qc_lazy_blocks")
+    return list(kind)
 
 
 def qc_decode_step(cache, seq_ids, q_ptr: int, k_ptr: int, v_ptr: int, out_ptr: int, lse_ptr: int = 0) -> None:

@@ -10,7 +10,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libqcache.so")
-SOURCES = ["qc_runtime.cu", "qc_kernels.cu", "qc_attend_tc.cu", "qc_prefill.cu", "qc_static.cu"]
+SOURCES = ["qc_runtime.cu", "qc_kernels.cu", "qc_attend_tc.cu", "qc_prefill.cu", "qc_calib.cu", "qc_static.cu"]
 HEADERS = ["qc_internal.h", "qc_device.cuh", os.path.join("..", "..", "include", "qc.h")]
 
 

@@ -123,6 +123,9 @@ cudaError_t launch_prefill_attend(const Params& p, const uint8_t* kind_dev, cons
                                   int32_t n_tokens, int32_t gla, const CUtensorMap* tmap_k, const CUtensorMap* tmap_v,
                                   const uint8_t* tile_code_dev, cudaStream_t stream);   // qc_prefill.cu; maps null = mma.sync kernel
 cudaError_t configure_prefill_kernels();
+cudaError_t launch_calibration(const Params& p, const int32_t* seq_ids_dev, const int32_t* len_text_dev,
+                               const int32_t* len_vis_dev, float* rows_dev, int32_t max_len, float* js_dev,
+                               cudaStream_t stream);   // qc_calib.cu
 cudaError_t configure_kernels(int* attend_smem_bytes);
 cudaError_t configure_kernels_tc(int* attend_smem_bytes);
 

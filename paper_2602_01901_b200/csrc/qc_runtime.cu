@@ -750,6 +750,65 @@ int32_t qc_prefill_attend(qc_cache* c, int32_t seq_id, int32_t n_tokens, const u
   return QC_OK;
 }
 
+int32_t qc_layer_similarity(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, const void* q_dev, float* rows_dev,
+                            int32_t max_len, float* similarity_host) {
+  if (!c || n_seqs < 1 || n_seqs > c->cfg.max_seqs || !seq_ids || !q_dev || !rows_dev || !similarity_host)
+    return QC_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(q_dev) & 15) || (reinterpret_cast<uintptr_t>(rows_dev) & 15)) return QC_ERR_INVALID_ARG;
+  if (max_len < 1 || max_len > 12288) return QC_ERR_UNSUPPORTED;   // one head's logits live in shared memory
+  const int N = c->cfg.n_layers;
+  for (int l = 0; l < N; ++l)
+    if (c->kind[l] != QC_LAYER_FULL) return QC_ERR_STATE;          // the analysis runs on the unmodified stack
+  std::vector<int32_t> host(3 * static_cast<size_t>(n_seqs));
+  for (int i = 0; i < n_seqs; ++i) {
+    const int s = seq_ids[i];
+    if (s < 0 || s >= c->cfg.max_seqs) return QC_ERR_INVALID_ARG;
+    const SeqState& st = c->seqs[s];
+    if (!st.active || st.len_text + st.len_vis == 0) return QC_ERR_STATE;
+    if (st.len_text + st.len_vis > max_len) return QC_ERR_INVALID_ARG;
+    host[i] = s;
+    host[n_seqs + i] = st.len_text;
+    host[2 * n_seqs + i] = st.len_vis;
+  }
+  QC_CUDA(cudaSetDevice(c->ctx->device));
+  cudaStream_t stream = c->ctx->stream;
+  int32_t* ids_dev = reinterpret_cast<int32_t*>(c->ws + c->lay.tok);
+  float* js_dev = reinterpret_cast<float*>(c->ws + c->lay.stage_lse);   // (n_layers - 1) * n_seqs floats fit
+  QC_CUDA(cudaMemcpyAsync(ids_dev, host.data(), host.size() * sizeof(int32_t), cudaMemcpyHostToDevice, stream));
+  Params p = base_params(c);
+  p.q = static_cast<const uint16_t*>(q_dev);
+  p.n_seqs = n_seqs;
+  QC_CUDA(launch_calibration(p, ids_dev, ids_dev + n_seqs, ids_dev + 2 * n_seqs, rows_dev, max_len, js_dev, stream));
+  c->kernel_launches += N > 1 ? 2 : 1;
+  std::vector<float> js(static_cast<size_t>(std::max(0, N - 1)) * n_seqs);
+  if (!js.empty())
+    QC_CUDA(cudaMemcpyAsync(js.data(), js_dev, js.size() * sizeof(float), cudaMemcpyDeviceToHost, stream));
+  QC_CUDA(cudaStreamSynchronize(stream));
+  for (int l = 0; l + 1 < N; ++l) {
+    double acc = 0.0;
+    for (int i = 0; i < n_seqs; ++i) acc += js[static_cast<size_t>(l) * n_seqs + i];
+    similarity_host[l] = static_cast<float>(acc / n_seqs);
+  }
+  return QC_OK;
+}
+
+int32_t qc_lazy_blocks(const float* similarity, int32_t n_layers, float eps, int32_t max_block, uint8_t* layer_kind) {
+  if (n_layers < 1 || !layer_kind || (n_layers > 1 && !similarity) || !(eps > 0.f) || eps > 1.f)
+    return QC_ERR_INVALID_ARG;
+  layer_kind[0] = QC_LAYER_FULL;
+  int size = 1;
+  for (int l = 1; l < n_layers; ++l) {
+    if (similarity[l - 1] < eps && (max_block <= 0 || size < max_block)) {
+      layer_kind[l] = QC_LAYER_LAZY;
+      ++size;
+    } else {
+      layer_kind[l] = QC_LAYER_FULL;
+      size = 1;
+    }
+  }
+  return QC_OK;
+}
+
 int32_t qc_decode_step(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, const void* q_dev, const void* k_dev,
                        const void* v_dev, void* out_dev, float* lse_out_dev) {
   if (!c || n_seqs < 0 || (n_seqs > 0 && !seq_ids)) return QC_ERR_INVALID_ARG;

@@ -65,3 +65,16 @@ def test_no_device_means_an_error_status_not_a_fallback(lib):
 
     with pytest.raises(RuntimeError):
         Session(2, 2, 2, 128, [0, 1])
+
+
+def test_lazy_blocks_on_the_host_match_the_oracle(lib):
+    from oracle import calibration as OC
+
+    S = [0.30, 0.01, 0.02, 0.40, 0.03, 0.03, 0.03, 0.50]
+    for eps, max_block in ((0.05, 0), (0.05, 2), (0.005, 0), (1.0, 0), (0.2, 3)):
+        assert qc.qc_lazy_blocks(S, eps, max_block) == OC.lazy_blocks(S, eps, max_block)
+    assert qc.qc_lazy_blocks([], 0.5) == [0]
+    with pytest.raises(qc.QcError):
+        qc.qc_lazy_blocks(S, 0.0)
+    with pytest.raises(qc.QcError):
+        qc.qc_lazy_blocks(S, 1.5)
