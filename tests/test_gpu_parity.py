@@ -308,6 +308,35 @@ def test_multi_turn_prefill_after_decode(mode):
     s.close()
 
 
+def test_many_short_sequences_and_a_partial_batch():
+    """More sequences than travel as a kernel argument (descriptor copy path), ragged lengths, and
+    steps that list only some of the active sequences."""
+    layer_kind = [0, 1, 0]
+    n_seqs, D = 70, 64
+    w = W.Workload(24, "many", 3, 4, 2, D, 16, n_seqs, 2, 30, 30, 5, 6, (1,))
+    s = Session(3, 4, 2, D, layer_kind, max_seqs=n_seqs, max_tokens_per_seq=64, n_pages=3 * 4 * n_seqs * 4,
+                lazy_mode=qc.QC_MODE_VLA_QC, poison_pool=True)
+    o = LazyAttentionOracle(3, 4, 2, D, layer_kind, qc.QC_MODE_VLA_QC, n_seqs=n_seqs)
+    dev = lambda a: torch.from_numpy(a.astype(np.int16)).view(torch.bfloat16).to(s.device).contiguous()
+    for b in range(n_seqs):
+        kind, k, v = W.prefill_kv_np(w, b)
+        T = 8 + (b * 7) % 29                     # 8..36 tokens: ragged, some without a full page
+        s.prefill_append([b], [T], kind[:T], dev(k[:, :T]), dev(v[:, :T]))
+        o.prefill_append(b, kind[:T].tolist(), f64(k[:, :T]), f64(v[:, :T]))
+    for step, ids in enumerate([list(range(n_seqs)), list(range(0, n_seqs, 3)), list(range(n_seqs))[::-1],
+                                [5, 69, 17]]):
+        qn, kn, vn = W.decode_qkv_np(w, step, seqs=ids)
+        out = torch.empty((3, len(ids), 4, D), dtype=torch.bfloat16, device=s.device)
+        s.decode_step(ids, dev(qn), dev(kn), dev(vn), out)
+        got = bits_of(out)
+        for i, b in enumerate(ids):
+            ref, _ = o.decode_step(b, f64(qn[:, i]), f64(kn[:, i]), f64(vn[:, i]))
+            for l in range(3):
+                assert_close(got[l, i], ref[l], f"step {step} seq {b} layer {l}")
+    assert s.stats().device_error == 0
+    s.close()
+
+
 FULL_CASES = [
     ("llava15_7b", qc.QC_MODE_VLA_QC, 40),
     ("llava15_7b", qc.QC_MODE_VLA_EQ8, 16),
