@@ -191,9 +191,11 @@ int32_t qc_lazy_blocks(const float* similarity, int32_t n_layers, float eps, int
 int32_t qc_decode_step(qc_cache* cache, int32_t n_seqs, const int32_t* seq_ids, const void* q_dev,
                        const void* k_dev, const void* v_dev, void* out_dev, float* lse_out_dev);
 
-/* Same step with HOST buffers of the same layouts: copies q, k, v to staging in the
- * workspace, runs the step, copies out (and lse if not NULL) back and waits for the stream.
- * Pinned host buffers make the copies asynchronous; pageable ones also work. */
+/* Same step with HOST buffers of the same layouts.  The step runs as up to four launch groups of
+ * consecutive lazy blocks; on two internal copy streams the inputs of a group are copied to
+ * staging in the workspace while the previous group computes, and its outputs are copied back
+ * while the next one computes.  Returns when everything has been copied back.  Pinned host
+ * buffers make the copies asynchronous; pageable ones also work (without the overlap). */
 int32_t qc_decode_step_host(qc_cache* cache, int32_t n_seqs, const int32_t* seq_ids,
                             const void* q_host, const void* k_host, const void* v_host,
                             void* out_host, float* lse_out_host);

@@ -130,7 +130,7 @@ __global__ void setup_kernel(const __grid_constant__ Params P, const __grid_cons
 __global__ void append_kernel(const __grid_constant__ Params P) {
   pdl_launch_dependents();
   pdl_wait();
-  append_rows(P, P.seqs[blockIdx.x], blockIdx.x, blockIdx.y);
+  append_rows(P, P.seqs[blockIdx.x], blockIdx.x, P.layer_begin + blockIdx.y);   // layers of one launch group
 }
 
 // ------------------------------------------------------------------------------------------
@@ -500,7 +500,7 @@ cudaError_t launch_setup(const Params& p, const StepInline* inl, cudaStream_t st
 }
 
 cudaError_t launch_append(const Params& p, cudaStream_t stream) {
-  dim3 grid(p.n_seqs, p.n_layers);
+  dim3 grid(p.n_seqs, p.layer_end - p.layer_begin);
   return launch_pdl(append_kernel, grid, dim3(128), 0, stream, p);
 }
 

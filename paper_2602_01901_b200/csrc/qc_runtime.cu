@@ -69,6 +69,10 @@ struct qc_cache {
   std::vector<LaunchGroup> groups;
   std::vector<std::pair<int, int>> group_pos;           // plan positions [begin, end) of each launch
   bool plan_dirty = true;
+  int plan_per = 0;               // blocks per launch the plan was built for (0 = all in one)
+  // host-buffer entry point: copies of one launch group overlap the kernels of the others
+  cudaStream_t copy_in = nullptr, copy_out = nullptr;
+  std::vector<cudaEvent_t> ev_in, ev_done;
   bool prefill_tcgen05 = true;    // head_dim 128: tcgen05 kernel; otherwise (or when switched off) mma.sync kernel
   int64_t n_pool_pages = 0;
   int layers_per_launch = 0;
@@ -385,14 +389,14 @@ int make_pool_tensor_map(qc_cache* c) {
 // Launch groups and the item-list order of the jobs.  Within a launch the heaviest sweeps (most
 // tiles per page, visual before text) come first: items are claimed in list order, so the work
 // left for the end of the launch comes in small pieces.
-int rebuild_plan(qc_cache* c) {
+int rebuild_plan(qc_cache* c, int per_launch) {
   c->groups.clear();
   c->group_pos.clear();
   c->plan.clear();
   c->plan_vis_before.assign(1, 0);
   c->plan_text_before.assign(1, 0);
   const int nb = static_cast<int>(c->block_jobs.size());
-  const int per = c->layers_per_launch <= 0 ? nb : c->layers_per_launch;
+  const int per = per_launch <= 0 ? nb : per_launch;
   std::vector<int> order;
   for (int b = 0; b < nb; b += per) {
     const int e = std::min(nb, b + per);
@@ -419,6 +423,7 @@ int rebuild_plan(qc_cache* c) {
                           cudaMemcpyHostToDevice, c->ctx->stream));
   QC_CUDA(cudaStreamSynchronize(c->ctx->stream));   // the host vector may be rebuilt later
   c->plan_dirty = false;
+  c->plan_per = per_launch;
   return QC_OK;
 }
 
@@ -587,6 +592,10 @@ int32_t qc_free(qc_ctx* ctx, qc_cache* cache) {
     for (int i = 0; i < kStageSlots; ++i)
       if (cache->stage_done[i]) cudaEventDestroy(cache->stage_done[i]);
     for (cudaEvent_t e : cache->ev) cudaEventDestroy(e);
+    for (cudaEvent_t e : cache->ev_in) cudaEventDestroy(e);
+    for (cudaEvent_t e : cache->ev_done) cudaEventDestroy(e);
+    if (cache->copy_in) cudaStreamDestroy(cache->copy_in);
+    if (cache->copy_out) cudaStreamDestroy(cache->copy_out);
     for (cudaEvent_t e : cache->ev_prefill) cudaEventDestroy(e);
     if (cache->pinned) cudaFreeHost(cache->pinned);
     delete cache;
@@ -809,8 +818,20 @@ int32_t qc_lazy_blocks(const float* similarity, int32_t n_layers, float eps, int
   return QC_OK;
 }
 
-int32_t qc_decode_step(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, const void* q_dev, const void* k_dev,
-                       const void* v_dev, void* out_dev, float* lse_out_dev) {
+}  // extern "C"
+
+namespace {
+
+// Events of the host-buffer entry point: launch group g waits for in[g] (its inputs have been
+// copied) and records done[g] (its outputs may be copied back).
+struct HostPipe {
+  int per_launch;
+  cudaEvent_t* in;
+  cudaEvent_t* done;
+};
+
+int decode_step_core(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, const void* q_dev, const void* k_dev,
+                     const void* v_dev, void* out_dev, float* lse_out_dev, const HostPipe* pipe) {
   if (!c || n_seqs < 0 || (n_seqs > 0 && !seq_ids)) return QC_ERR_INVALID_ARG;
   if (n_seqs == 0) return QC_OK;
   if (!q_dev || !k_dev || !v_dev || !out_dev) return QC_ERR_INVALID_ARG;
@@ -836,8 +857,9 @@ int32_t qc_decode_step(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, cons
   QC_CUDA(cudaSetDevice(c->ctx->device));
   cudaStream_t stream = c->ctx->stream;
 
-  if (c->plan_dirty) {
-    const int st = rebuild_plan(c);
+  const int want_per = pipe ? pipe->per_launch : c->layers_per_launch;
+  if (c->plan_dirty || c->plan_per != want_per) {
+    const int st = rebuild_plan(c, want_per);
     if (st != QC_OK) return st;
   }
 
@@ -930,7 +952,9 @@ int32_t qc_decode_step(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, cons
   p.tot_v = static_cast<int32_t>(tot_v);
   p.tot_t = static_cast<int32_t>(tot_t);
   p.inline_seqs = inline_step ? 1 : 0;
-  p.fused_append = n_patches == 0 ? 1 : 0;   // the append reads the page table: not beside its patches
+  // the append reads the page table (not beside its patches) and every layer's k/v (not before
+  // the host pipe has copied them)
+  p.fused_append = (n_patches == 0 && !pipe) ? 1 : 0;
 
   cudaEvent_t* ev = nullptr;
   if (c->profile && c->ev_steps < kMaxProfileSteps) {
@@ -946,7 +970,9 @@ int32_t qc_decode_step(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, cons
   }
   QC_CUDA(launch_setup(p, inline_step ? &inl : nullptr, stream));
   c->kernel_launches++;
-  if (!p.fused_append) {
+  if (!p.fused_append && !pipe) {
+    p.layer_begin = 0;
+    p.layer_end = N;
     QC_CUDA(launch_append(p, stream));
     c->kernel_launches++;
   }
@@ -957,6 +983,11 @@ int32_t qc_decode_step(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, cons
     p.layer_begin = c->groups[gi].layer_begin;
     p.layer_end = c->groups[gi].layer_end;
     p.launch_index = static_cast<int32_t>(gi);
+    if (pipe) {
+      QC_CUDA(cudaStreamWaitEvent(stream, pipe->in[gi], 0));
+      QC_CUDA(launch_append(p, stream));   // this group's layers only
+      c->kernel_launches++;
+    }
     if (ev && gi == 0) QC_CUDA(cudaEventRecord(ev[1], stream));
     if (c->group > 1)
       QC_CUDA(launch_attend_tc(p, c->ctx->n_sms, stream));
@@ -964,6 +995,7 @@ int32_t qc_decode_step(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, cons
       QC_CUDA(launch_attend(p, c->ctx->n_sms, stream));
     if (ev && gi + 1 == c->groups.size()) QC_CUDA(cudaEventRecord(ev[2], stream));
     QC_CUDA(launch_merge(p, stream));
+    if (pipe) QC_CUDA(cudaEventRecord(pipe->done[gi], stream));
     c->attend_launches++;
     c->kernel_launches += 2;
   }
@@ -977,6 +1009,15 @@ int32_t qc_decode_step(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, cons
   return QC_OK;
 }
 
+}  // namespace
+
+extern "C" {
+
+int32_t qc_decode_step(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, const void* q_dev, const void* k_dev,
+                       const void* v_dev, void* out_dev, float* lse_out_dev) {
+  return decode_step_core(c, n_seqs, seq_ids, q_dev, k_dev, v_dev, out_dev, lse_out_dev, nullptr);
+}
+
 int32_t qc_decode_step_host(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, const void* q_host,
                             const void* k_host, const void* v_host, void* out_host, float* lse_out_host) {
   if (!c || n_seqs < 0) return QC_ERR_INVALID_ARG;
@@ -984,24 +1025,62 @@ int32_t qc_decode_step_host(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids,
   if (!q_host || !k_host || !v_host || !out_host || n_seqs > c->cfg.max_seqs) return QC_ERR_INVALID_ARG;
   QC_CUDA(cudaSetDevice(c->ctx->device));
   cudaStream_t stream = c->ctx->stream;
-  const size_t N = c->cfg.n_layers;
-  const size_t qb = N * n_seqs * c->hq * c->D * 2, kb = N * n_seqs * c->hkv * c->D * 2;
+  // The step runs as up to four launch groups of consecutive lazy blocks: while one group
+  // computes, the inputs of the next are copied in and the outputs of the previous copied out.
+  const int nb = static_cast<int>(c->block_jobs.size());
+  const int per = (nb + 3) / 4;
+  if (c->plan_dirty || c->plan_per != per) {
+    const int st = rebuild_plan(c, per);
+    if (st != QC_OK) return st;
+  }
+  const size_t G = c->groups.size();
+  if (!c->copy_in) {
+    QC_CUDA(cudaStreamCreateWithFlags(&c->copy_in, cudaStreamNonBlocking));
+    QC_CUDA(cudaStreamCreateWithFlags(&c->copy_out, cudaStreamNonBlocking));
+  }
+  while (c->ev_in.size() < G) {
+    cudaEvent_t a, b;
+    QC_CUDA(cudaEventCreateWithFlags(&a, cudaEventDisableTiming));
+    QC_CUDA(cudaEventCreateWithFlags(&b, cudaEventDisableTiming));
+    c->ev_in.push_back(a);
+    c->ev_done.push_back(b);
+  }
+  const size_t q_layer = static_cast<size_t>(n_seqs) * c->hq * c->D * 2;    // bytes of one layer's q (and out)
+  const size_t kv_layer = static_cast<size_t>(n_seqs) * c->hkv * c->D * 2;
+  const size_t lse_layer = static_cast<size_t>(n_seqs) * c->hq * sizeof(float);
   uint8_t* dq = c->ws + c->lay.stage_q;
   uint8_t* dk = c->ws + c->lay.stage_k;
   uint8_t* dv = c->ws + c->lay.stage_v;
   uint8_t* dout = c->ws + c->lay.stage_out;
-  float* dlse = reinterpret_cast<float*>(c->ws + c->lay.stage_lse);
-  QC_CUDA(cudaMemcpyAsync(dq, q_host, qb, cudaMemcpyHostToDevice, stream));
-  QC_CUDA(cudaMemcpyAsync(dk, k_host, kb, cudaMemcpyHostToDevice, stream));
-  QC_CUDA(cudaMemcpyAsync(dv, v_host, kb, cudaMemcpyHostToDevice, stream));
-  int st = qc_decode_step(c, n_seqs, seq_ids, dq, dk, dv, dout, lse_out_host ? dlse : nullptr);
+  uint8_t* dlse = c->ws + c->lay.stage_lse;
+  const uint8_t* hq = static_cast<const uint8_t*>(q_host);
+  const uint8_t* hk = static_cast<const uint8_t*>(k_host);
+  const uint8_t* hv = static_cast<const uint8_t*>(v_host);
+  for (size_t g = 0; g < G; ++g) {
+    const size_t lb = c->groups[g].layer_begin, nl = c->groups[g].layer_end - lb;
+    QC_CUDA(cudaMemcpyAsync(dq + lb * q_layer, hq + lb * q_layer, nl * q_layer, cudaMemcpyHostToDevice, c->copy_in));
+    QC_CUDA(cudaMemcpyAsync(dk + lb * kv_layer, hk + lb * kv_layer, nl * kv_layer, cudaMemcpyHostToDevice, c->copy_in));
+    QC_CUDA(cudaMemcpyAsync(dv + lb * kv_layer, hv + lb * kv_layer, nl * kv_layer, cudaMemcpyHostToDevice, c->copy_in));
+    QC_CUDA(cudaEventRecord(c->ev_in[g], c->copy_in));
+  }
+  const HostPipe pipe{per, c->ev_in.data(), c->ev_done.data()};
+  const int st = decode_step_core(c, n_seqs, seq_ids, dq, dk, dv, dout,
+                                  lse_out_host ? reinterpret_cast<float*>(dlse) : nullptr, &pipe);
   if (st != QC_OK) {
+    cudaStreamSynchronize(c->copy_in);
     cudaStreamSynchronize(stream);
     return st;
   }
-  QC_CUDA(cudaMemcpyAsync(out_host, dout, qb, cudaMemcpyDeviceToHost, stream));
-  if (lse_out_host)
-    QC_CUDA(cudaMemcpyAsync(lse_out_host, dlse, N * n_seqs * c->hq * sizeof(float), cudaMemcpyDeviceToHost, stream));
+  for (size_t g = 0; g < G; ++g) {
+    const size_t lb = c->groups[g].layer_begin, nl = c->groups[g].layer_end - lb;
+    QC_CUDA(cudaStreamWaitEvent(c->copy_out, c->ev_done[g], 0));
+    QC_CUDA(cudaMemcpyAsync(static_cast<uint8_t*>(out_host) + lb * q_layer, dout + lb * q_layer, nl * q_layer,
+                            cudaMemcpyDeviceToHost, c->copy_out));
+    if (lse_out_host)
+      QC_CUDA(cudaMemcpyAsync(reinterpret_cast<uint8_t*>(lse_out_host) + lb * lse_layer, dlse + lb * lse_layer,
+                              nl * lse_layer, cudaMemcpyDeviceToHost, c->copy_out));
+  }
+  QC_CUDA(cudaStreamSynchronize(c->copy_out));
   QC_CUDA(cudaStreamSynchronize(stream));
   return QC_OK;
 }
