@@ -180,7 +180,7 @@ def run_gpu(args, w, mode, rank, world, local_rank):
 
     from paper_2602_01901_b200.ranks import RankGroup
 
-    group = RankGroup()          # NCCL when launched by torchrun with WORLD_SIZE > 1
+    group = RankGroup(backend=args.dist_backend)   # NCCL when launched by torchrun with WORLD_SIZE > 1
     seq_offset = rank * w.batch  # every rank serves its own sequences of the global batch
 
     def barrier():
@@ -409,6 +409,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-all-full", action="store_true", help="skip the all-ordinary-layers comparison run")
     ap.add_argument("--no-per-block", action="store_true", help="skip the launch-per-lazy-block comparison run")
+    ap.add_argument("--dist-backend", default=None, help="torch.distributed backend (default: nccl on GPUs)")
+    ap.add_argument("--force-device", type=int, default=-1,
+                    help="use this CUDA device on every rank (to exercise the multi-rank plumbing on one GPU)")
     ap.add_argument("--phase", default="decode", choices=["decode", "prefill"],
                     help="decode (the benchmark) or prefill (secondary: qc_prefill_attend over the prompts)")
     ap.add_argument("--prefill-kernel", default="tcgen05", choices=["tcgen05", "mma"],
@@ -437,6 +440,8 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.force_device >= 0:     # several ranks on one GPU: a plumbing check, not a measurement
+        local_rank = args.force_device
 
     if args.impl == "reference":
         if rank != 0:
