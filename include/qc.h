@@ -153,8 +153,11 @@ int32_t qc_prefill_append(qc_cache* cache, int32_t n_seqs, const int32_t* seq_id
  *           layer's slice of this tensor; nothing prompt-sized is kept afterwards)
  *   k_dev, v_dev bf16 [n_layers][n_tokens][n_kv_heads][head_dim]
  *   out_dev bf16 [n_layers][n_tokens][n_q_heads][head_dim]
- * The sequence must be new or empty (a prompt that continues a cached sequence returns
- * QC_ERR_UNSUPPORTED).  Errors of qc_prefill_append apply; on an error nothing is stored or written. */
+ * If the sequence already holds tokens (an earlier prompt chunk, generated tokens: a later turn of
+ * a conversation), they precede the new ones: every new token also sees all of them, read from
+ * the cache with the cache's own sharing (a lazy layer's visual keys -- in GLA all its keys -- are
+ * its leader's), which is what Eq. 5 / Eq. 7 select for those tokens.
+ * Errors of qc_prefill_append apply; on an error nothing is stored or written. */
 int32_t qc_prefill_attend(qc_cache* cache, int32_t seq_id, int32_t n_tokens, const uint8_t* kind,
                           const void* q_dev, const void* k_dev, const void* v_dev, void* out_dev);
 

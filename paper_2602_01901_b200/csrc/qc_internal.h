@@ -121,7 +121,8 @@ cudaError_t launch_prefill_scatter(const Params& p, const int32_t* tok_seq, cons
 cudaError_t launch_prefill_attend(const Params& p, const uint8_t* kind_dev, const uint8_t* layer_kind_dev,
                                   const uint8_t* leader_dev, const void* q, const void* k, const void* v, void* out,
                                   int32_t n_tokens, int32_t gla, const CUtensorMap* tmap_k, const CUtensorMap* tmap_v,
-                                  const uint8_t* tile_code_dev, cudaStream_t stream);   // qc_prefill.cu; maps null = mma.sync kernel
+                                  const uint8_t* tile_code_dev, int32_t seq_id, int32_t n0_text, int32_t n0_vis,
+                                  cudaStream_t stream);   // qc_prefill.cu; maps null or a non-empty sequence = mma.sync kernel
 cudaError_t configure_prefill_kernels();
 cudaError_t launch_calibration(const Params& p, const int32_t* seq_ids_dev, const int32_t* len_text_dev,
                                const int32_t* len_vis_dev, float* rows_dev, int32_t max_len, float* js_dev,

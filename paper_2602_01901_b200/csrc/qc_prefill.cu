@@ -47,6 +47,12 @@ struct PrefillArgs {
   const uint8_t* leader;       // [n_layers] device
   int32_t T, hq, hkv, group, n_layers, gla;
   float scale_log2;
+  // tokens the sequence already held before this prompt chunk (mma.sync kernel only): they are
+  // read from the paged cache, text stream then visual stream, and are visible to every new token
+  const uint16_t* pool;
+  const int32_t* table;        // [n_layers][4][max_seqs][max_pages]
+  const uint8_t* layer_flags;  // kLayerOwnsTextK: the layer's text K is its own
+  int32_t max_seqs, max_pages, seq_id, n0_text, n0_vis;
 };
 
 // Stage rows [row0, row0 + 64) of one head of a [n_layers][T][heads][D] tensor; row t comes
@@ -77,6 +83,34 @@ __device__ __forceinline__ void stage_tile(uint32_t smem, const uint16_t* base, 
   }
 }
 
+// Stage 64 cached tokens [ord0, ord0 + 64) of one stream of (src_layer, sequence) from the paged
+// pool; tokens at or past n_valid are zero-filled (their pool rows may hold anything).
+template <int D>
+__device__ __forceinline__ void stage_cached(uint32_t smem, const PrefillArgs& A, int src_layer, int stream, int ord0,
+                                             int n_valid, int head) {
+  constexpr int CH = D / 8;
+  constexpr int RPP = kPrefillThreads / CH;
+  constexpr int NP = kBN / RPP;
+  const int c = threadIdx.x % CH, r0 = threadIdx.x / CH;
+  const size_t trow = ((static_cast<size_t>(src_layer) * 4 + stream) * A.max_seqs + A.seq_id) * A.max_pages;
+  int pid[NP];
+#pragma unroll
+  for (int i = 0; i < NP; ++i) {
+    const int ord = ord0 + r0 + i * RPP;
+    pid[i] = ord < n_valid ? A.table[trow + ord / kPage] : -1;
+  }
+#pragma unroll
+  for (int i = 0; i < NP; ++i) {
+    const int r = r0 + i * RPP, ord = ord0 + r;
+    const uint32_t dst = smem + tile_off<D>(r, c);
+    if (pid[i] >= 0) {
+      cp_async16(dst, A.pool + ((static_cast<size_t>(pid[i]) * A.hkv + head) * kPage + ord % kPage) * D + c * 8);
+    } else {
+      asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(dst), "r"(0u) : "memory");
+    }
+  }
+}
+
 template <int D>
 __global__ void __launch_bounds__(kPrefillThreads) prefill_attend_kernel(const PrefillArgs A) {
   constexpr int KS = D / 16;   // k-steps of the score product
@@ -97,12 +131,31 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_attend_kernel(const P
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t4 = lane & 3;
   const int m0 = qt * kBM;
-  const int n_ktiles = qt + 1;                       // causal: key tiles 0 .. qt
+  // Key tiles, in order: the cached text tokens, the cached visual tokens (all visible, read from
+  // the pool: a lazy layer's visual K -- and in GLA its text K -- are its leader's pages, which is
+  // Eq. 5 / Eq. 7's selection for tokens already cached), then the new tokens 0 .. qt (causal).
+  const int ct_text = (A.n0_text + kBN - 1) / kBN, ct_vis = (A.n0_vis + kBN - 1) / kBN;
+  const int n_cached_tiles = ct_text + ct_vis;
+  const int n_ktiles = n_cached_tiles + qt + 1;
+  const int k_text_layer = (A.n0_text && !(A.layer_flags[layer] & kLayerOwnsTextK)) ? lead : layer;
+  const int k_vis_layer = lazy ? lead : layer;
+  auto stage_kv = [&](int i, uint32_t kdst, uint32_t vdst) {
+    if (i < ct_text) {
+      stage_cached<D>(kdst, A, k_text_layer, 0, i * kBN, A.n0_text, kvh);
+      stage_cached<D>(vdst, A, layer, 2, i * kBN, A.n0_text, kvh);
+    } else if (i < n_cached_tiles) {
+      stage_cached<D>(kdst, A, k_vis_layer, 1, (i - ct_text) * kBN, A.n0_vis, kvh);
+      stage_cached<D>(vdst, A, layer, 3, (i - ct_text) * kBN, A.n0_vis, kvh);
+    } else {
+      const int t0 = (i - n_cached_tiles) * kBN;
+      stage_tile<D>(kdst, A.k, layer, lead, lazy, gla, A.kind, t0, A.T, A.hkv, kvh);
+      stage_tile<D>(vdst, A.v, layer, layer, false, false, A.kind, t0, A.T, A.hkv, kvh);
+    }
+  };
 
   // stage Q and the first K/V tiles
   stage_tile<D>(sQ, A.q, layer, lead, lazy, gla, A.kind, m0, A.T, A.hq, head);
-  stage_tile<D>(sK, A.k, layer, lead, lazy, gla, A.kind, 0, A.T, A.hkv, kvh);
-  stage_tile<D>(sV, A.v, layer, layer, false, false, A.kind, 0, A.T, A.hkv, kvh);
+  stage_kv(0, sK, sV);
   cp_async_commit();
   cp_async_wait<0>();
   __syncthreads();
@@ -124,13 +177,16 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_attend_kernel(const P
   for (int kt = 0; kt < n_ktiles; ++kt) {
     const int buf = kt & 1;
     if (kt + 1 < n_ktiles) {   // prefetch the next tiles into the other buffer
-      stage_tile<D>(sK + (buf ^ 1) * kTileBytes, A.k, layer, lead, lazy, gla, A.kind, (kt + 1) * kBN, A.T, A.hkv, kvh);
-      stage_tile<D>(sV + (buf ^ 1) * kTileBytes, A.v, layer, layer, false, false, A.kind, (kt + 1) * kBN, A.T, A.hkv,
-                    kvh);
+      stage_kv(kt + 1, sK + (buf ^ 1) * kTileBytes, sV + (buf ^ 1) * kTileBytes);
       cp_async_commit();
     }
     const uint32_t kb = sK + buf * kTileBytes, vb = sV + buf * kTileBytes;
-    const int n0 = kt * kBN;
+    // visibility of the tile's keys: a cached tile shows its first n_show tokens to every row; a
+    // tile of new tokens starts at prompt position n0 and is causal
+    const bool cached_tile = kt < n_cached_tiles;
+    const int n_show = !cached_tile ? 0
+                       : (kt < ct_text ? min(kBN, A.n0_text - kt * kBN) : min(kBN, A.n0_vis - (kt - ct_text) * kBN));
+    const int n0 = (kt - n_cached_tiles) * kBN;
 
     // ---- S = Q K^T for 16 rows x 64 keys
     float s[kBN / 8][4];
@@ -154,9 +210,10 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_attend_kernel(const P
     for (int j = 0; j < kBN / 8; ++j) {
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        const int key = n0 + j * 8 + 2 * t4 + (e & 1);
+        const int col = j * 8 + 2 * t4 + (e & 1), key = n0 + col;
         const int qrow = qrow0 + ((e >> 1) << 3);
-        const float x = (key <= qrow && key < A.T) ? s[j][e] * A.scale_log2 : -INFINITY;
+        const bool visible = cached_tile ? col < n_show : (key <= qrow && key < A.T);
+        const float x = visible ? s[j][e] * A.scale_log2 : -INFINITY;
         s[j][e] = x;
         tmax[e >> 1] = fmaxf(tmax[e >> 1], x);
       }
@@ -695,7 +752,8 @@ cudaError_t configure_prefill_kernels() {
 cudaError_t launch_prefill_attend(const Params& p, const uint8_t* kind_dev, const uint8_t* layer_kind_dev,
                                   const uint8_t* leader_dev, const void* q, const void* k, const void* v, void* out,
                                   int32_t T, int32_t gla, const CUtensorMap* tmap_k, const CUtensorMap* tmap_v,
-                                  const uint8_t* tile_code_dev, cudaStream_t stream) {
+                                  const uint8_t* tile_code_dev, int32_t seq_id, int32_t n0_text, int32_t n0_vis,
+                                  cudaStream_t stream) {
   if (T <= 0) return cudaSuccess;
   PrefillArgs a{};
   a.q = static_cast<const uint16_t*>(q);
@@ -712,7 +770,15 @@ cudaError_t launch_prefill_attend(const Params& p, const uint8_t* kind_dev, cons
   a.n_layers = p.n_layers;
   a.gla = gla;
   a.scale_log2 = p.scale_log2;
-  if (p.d == kTD && tmap_k && tmap_v) {
+  a.pool = p.pool;
+  a.table = p.table;
+  a.layer_flags = p.layer_flags;
+  a.max_seqs = p.max_seqs;
+  a.max_pages = p.max_pages;
+  a.seq_id = seq_id;
+  a.n0_text = n0_text;
+  a.n0_vis = n0_vis;
+  if (p.d == kTD && tmap_k && tmap_v && n0_text + n0_vis == 0) {
     a.tmap_k = *tmap_k;
     a.tmap_v = *tmap_v;
     a.tile_code = tile_code_dev;

@@ -705,8 +705,9 @@ int32_t qc_prefill_attend(qc_cache* c, int32_t seq_id, int32_t n_tokens, const u
   const void* ptrs[4] = {q_dev, k_dev, v_dev, out_dev};
   for (const void* ptr : ptrs)
     if (reinterpret_cast<uintptr_t>(ptr) & 15) return QC_ERR_INVALID_ARG;
-  // the prompt attends to itself only: a sequence that already holds tokens is not covered
-  if (c->seqs[seq_id].active && (c->seqs[seq_id].len_text || c->seqs[seq_id].len_vis)) return QC_ERR_UNSUPPORTED;
+  // tokens the sequence holds already (an earlier prompt chunk, generated tokens) precede the new ones
+  const int n0_text = c->seqs[seq_id].active ? c->seqs[seq_id].len_text : 0;
+  const int n0_vis = c->seqs[seq_id].active ? c->seqs[seq_id].len_vis : 0;
   if (static_cast<size_t>(n_tokens) > static_cast<size_t>(kPrefillBatchTokens) * 3 * sizeof(int32_t))
     return QC_ERR_INVALID_ARG;
   // store K/V first: this validates everything and leaves the cache unchanged on an error
@@ -727,7 +728,7 @@ int32_t qc_prefill_attend(qc_cache* c, int32_t seq_id, int32_t n_tokens, const u
   QC_CUDA(cudaMemcpyAsync(codes_dev, codes.data(), n_tiles, cudaMemcpyHostToDevice, stream));
   QC_CUDA(cudaStreamSynchronize(stream));   // `kind` is the caller's host memory
   CUtensorMap tmap_k, tmap_v;
-  const bool tc5 = c->prefill_tcgen05 && c->D == 128;
+  const bool tc5 = c->prefill_tcgen05 && c->D == 128 && n0_text + n0_vis == 0;
   if (tc5) {
     if (make_prompt_tensor_map(&tmap_k, k_dev, c->cfg.n_layers, n_tokens, c->hkv) != QC_OK ||
         make_prompt_tensor_map(&tmap_v, v_dev, c->cfg.n_layers, n_tokens, c->hkv) != QC_OK)
@@ -748,11 +749,11 @@ int32_t qc_prefill_attend(qc_cache* c, int32_t seq_id, int32_t n_tokens, const u
   }
   QC_CUDA(launch_prefill_attend(p, kind_dev, c->ws + c->lay.layer_kind, c->ws + c->lay.leader, q_dev, k_dev, v_dev,
                                 out_dev, n_tokens, c->cfg.lazy_mode == QC_MODE_GLA ? 1 : 0, tc5 ? &tmap_k : nullptr,
-                                tc5 ? &tmap_v : nullptr, codes_dev, stream));
+                                tc5 ? &tmap_v : nullptr, codes_dev, seq_id, n0_text, n0_vis, stream));
   if (ev) {
     QC_CUDA(cudaEventRecord(ev[1], stream));
     c->ev_prefill_calls++;
-    const double pairs = 0.5 * n_tokens * (n_tokens + 1.0);
+    const double pairs = 0.5 * n_tokens * (n_tokens + 1.0) + static_cast<double>(n_tokens) * (n0_text + n0_vis);
     c->prof_prefill_flops += 4.0 * c->D * pairs * c->hq * c->cfg.n_layers;
   }
   c->kernel_launches++;

@@ -66,12 +66,6 @@ def test_prefill_attend_small(mode, case):
             for l in range(w.n_layers):
                 assert_close(got[l, b], ref[l], f"decode after prefill: step {step} seq {b} layer {l}")
     assert s.stats().device_error == 0
-    # a prompt that continues a cached sequence is refused, and nothing changes
-    kind, k, v = W.prefill_kv_np(w, 0)
-    before = s.page_table(0, 0, 0)
-    with pytest.raises(qc.QcError) as e:
-        s.prefill_attend(0, kind, _dev(W.prefill_q_np(w, 0), s.device), _dev(k, s.device), _dev(v, s.device), out)
-    assert e.value.status == qc.QC_ERR_UNSUPPORTED and s.page_table(0, 0, 0) == before
     s.close()
 
 
@@ -111,4 +105,44 @@ def test_prefill_attend_full_size_sampled(name, mode):
             worst = max(worst, r)
     assert s.stats().device_error == 0
     print(f"{name} mode {mode}: prefill worst rel-L2 {worst:.3e}")
+    s.close()
+
+
+@pytest.mark.parametrize("mode", MODES, ids=MODE_IDS)
+@pytest.mark.parametrize("head_dim,group", [(128, 1), (64, 2), (128, 7)])
+def test_prefill_attend_continues_a_cached_sequence(mode, head_dim, group):
+    """A later turn: prompt chunk, a few generated tokens, then a second chunk (text and a new
+    image).  The second chunk's rows must equal the oracle's rows for one prefill over the whole
+    token sequence (chunk 1, generated tokens, chunk 2)."""
+    layer_kind = [0, 1, 1, 0, 1]
+    lazy = tuple(i for i, k in enumerate(layer_kind) if k)
+    w = W.Workload(60 + group, f"turns{group}", len(layer_kind), 2 * group, 2, head_dim, 16, 1, 7, 90, 90, 80, 5, lazy)
+    s = Session(w.n_layers, w.n_q_heads, w.n_kv_heads, head_dim, layer_kind, max_seqs=1, max_tokens_per_seq=256,
+                n_pages=w.n_layers * 4 * 20, lazy_mode=mode, poison_pool=True)
+    kind, k, v = W.prefill_kv_np(w, 0)
+    q = W.prefill_q_np(w, 0)
+    T1 = 70                       # 7 text + 63 visual: the image is cut in the middle
+    dev = s.device
+    out1 = torch.empty((w.n_layers, T1, w.n_q_heads, head_dim), dtype=torch.bfloat16, device=dev)
+    s.prefill_attend(0, kind[:T1], _dev(q[:, :T1], dev), _dev(k[:, :T1], dev), _dev(v[:, :T1], dev), out1)
+    gen_q, gen_k, gen_v = [], [], []
+    o = torch.empty((w.n_layers, 1, w.n_q_heads, head_dim), dtype=torch.bfloat16, device=dev)
+    for step in range(3):
+        qn, kn, vn = W.decode_qkv_np(w, step)
+        s.decode_step([0], _dev(qn, dev), _dev(kn, dev), _dev(vn, dev), o)
+        gen_q.append(qn[:, 0]), gen_k.append(kn[:, 0]), gen_v.append(vn[:, 0])
+    T2 = len(kind) - T1
+    out2 = torch.full((w.n_layers, T2, w.n_q_heads, head_dim), float("nan"), dtype=torch.bfloat16, device=dev)
+    s.prefill_attend(0, kind[T1:], _dev(q[:, T1:], dev), _dev(k[:, T1:], dev), _dev(v[:, T1:], dev), out2)
+    # the oracle sees one sequence: chunk 1, the generated (text) tokens, chunk 2
+    cat = lambda a, g, b: np.concatenate([a, np.stack(g, axis=1), b], axis=1)
+    q_all, k_all, v_all = cat(q[:, :T1], gen_q, q[:, T1:]), cat(k[:, :T1], gen_k, k[:, T1:]), cat(v[:, :T1], gen_v, v[:, T1:])
+    kind_all = np.concatenate([kind[:T1], np.zeros(3, np.uint8), kind[T1:]])
+    ref = OP.prefill_lazy_attention(f64(q_all), f64(k_all), f64(v_all), kind_all, layer_kind, mode)
+    got1, got2 = bits_of(out1), bits_of(out2)
+    for l in range(w.n_layers):
+        assert_close(got1[l], ref[l, :T1], f"first chunk layer {l}")
+        for t0 in range(0, T2, 64):
+            assert_close(got2[l, t0:t0 + 64], ref[l, T1 + 3 + t0: T1 + 3 + t0 + 64], f"second chunk layer {l} tokens {t0}..")
+    assert s.stats().device_error == 0
     s.close()
