@@ -421,21 +421,22 @@ __device__ __forceinline__ void tensor_g2s_3d(uint32_t dst_smem, const void* tma
       : "memory");
 }
 
-constexpr int kTc5Threads = kTM + 32;   // 128 softmax threads (one per query row) + one warp that issues the products
+constexpr int kTc5Threads = kTM + 64;   // 128 softmax threads (one per query row) + a score warp + a value warp
 
 // Warp roles.  Warps 0-3: one thread per query row -- read the row's scores from TMEM, online
-// softmax, write the bf16 weights.  Warp 4: fetches the K/V tiles and, one lane, issues every
-// tcgen05.mma (issue can block while the tensor core is busy, so it must not sit on the softmax
-// path).  A K/V tile whose 64 rows all come from one layer -- every tile of an ordinary or GLA
-// layer, and the all-text / all-visual tiles of a VLA lazy layer -- is fetched by two tensor-map
-// copies; only a tile that mixes text and visual rows of a VLA lazy layer is gathered row by row
-// with 16-byte copies by the 32 lanes.  Hand-offs are mbarriers only:
-//   bar_k[b], bar_v[b]  copies -> issuer   K / V tile landed in buffer b
-//   bar_s[b]  tensor core -> softmax, issuer   score buffer b holds S(kt): K buffer b is free
-//   bar_p     softmax -> issuer        weights P(kt) written, S(kt) read, PV(kt-1) seen complete (128 arrivals)
-//   bar_o     tensor core -> softmax   value product of tile kt done: P and O may change
-// Order of products on the tensor core: S(0) S(1) | PV(0) S(2) | PV(1) S(3) | ...  While the threads
-// work on tile kt, the tensor core runs PV(kt-1) and S(kt+1).
+// softmax, write the bf16 weights.  Warp 4 (score warp) fetches the K tiles and issues S = Q K^T;
+// warp 5 (value warp) fetches the V tiles and issues O += P V.  Issuing a product or a copy and
+// polling an mbarrier each cost a few hundred cycles of one lane, so the two streams run in
+// separate warps and off the softmax path; all shared-memory descriptors are built once.
+// A K/V tile whose 64 rows all come from one layer -- every tile of an ordinary or GLA layer, and
+// the all-text / all-visual tiles of a VLA lazy layer -- is fetched by two tensor-map copies; only
+// a tile that mixes text and visual rows of a VLA lazy layer is gathered row by row with 16-byte
+// copies by the 32 lanes.  Hand-offs are mbarriers only:
+//   bar_k[b], bar_v[b]  copies -> score / value warp    K / V tile landed in buffer b
+//   bar_s[b]      tensor core -> softmax, score warp    score buffer b holds S(kt); K buffer b is free
+//   bar_sfree[b]  softmax -> score warp    the 128 threads have read score buffer b
+//   bar_p         softmax -> value warp    weights P(kt) written; the threads have seen PV(kt-1) complete
+//   bar_o         tensor core -> softmax   value product of tile kt done: P and O may change
 __global__ void __launch_bounds__(kTc5Threads, 2)
     prefill_attend_tcgen05_kernel(const __grid_constant__ PrefillArgs A, int32_t* err) {
   // No static shared memory: the dynamic window then starts on the 1024-byte boundary that the
@@ -453,8 +454,9 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
   uint64_t& bar_p = *reinterpret_cast<uint64_t*>(smem_dyn + kTiles + 24);
   uint64_t* bar_k = reinterpret_cast<uint64_t*>(smem_dyn + kTiles + 32);          // two
   uint64_t* bar_v = reinterpret_cast<uint64_t*>(smem_dyn + kTiles + 48);          // two
-  uint32_t& tmem_base_slot = *reinterpret_cast<uint32_t*>(smem_dyn + kTiles + 64);
-  volatile int32_t& failed = *reinterpret_cast<volatile int32_t*>(smem_dyn + kTiles + 68);
+  uint64_t* bar_sfree = reinterpret_cast<uint64_t*>(smem_dyn + kTiles + 64);      // two
+  uint32_t& tmem_base_slot = *reinterpret_cast<uint32_t*>(smem_dyn + kTiles + 80);
+  volatile int32_t& failed = *reinterpret_cast<volatile int32_t*>(smem_dyn + kTiles + 84);
   if (base & 1023u) {   // cannot happen with the layout above; never run the tensor core on a misplaced tile
     if (threadIdx.x == 0) atomicMax(err, kErrBadPage);
     return;
@@ -481,11 +483,12 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
     for (int b = 0; b < 2; ++b) {
       mbar_init(&bar_k[b], 1);
       mbar_init(&bar_v[b], 1);
+      mbar_init(&bar_sfree[b], kTM);
     }
     fence_mbar_init();
     failed = 0;
   }
-  if (warp == 4) {
+  if (warp == 4) {   // the score warp owns the TMEM allocation
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
                  "r"(kTmemCols)
                  : "memory");
@@ -506,8 +509,8 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
   constexpr uint32_t kIdescS = (1u << 4) | (1u << 7) | (1u << 10) | ((kTN >> 3) << 17) | ((kTM >> 4) << 24);
   constexpr uint32_t kIdescO = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((kTD >> 3) << 17) | ((kTM >> 4) << 24);
 
-  if (warp == 4) {
-    // ------------------------------------------------------------------ tile fetch + product issuer
+  if (warp >= 4) {
+    // ------------------------------------------------------------------ tile fetch + product issue
     // Fetch key tile (is_k) or value tile kt into `dst`; completion is one phase of `bar`.
     auto fetch_tile = [&](bool is_k, int kt, uint32_t dst, uint64_t* bar) {
       int src = layer;
@@ -546,68 +549,74 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
         if (lane == 0) mbar_arrive(bar);
       }
     };
-    // S = Q K^T of key tile kt into score buffer kt & 1 (two buffers of 64 TMEM columns)
-    auto issue_scores = [&](int kt) {
-      const uint32_t kb = sK + (kt & 1) * kKV;
-#pragma unroll
-      for (int kk = 0; kk < kTD / 16; ++kk) {
-        const uint64_t ad = umma_desc(sQ + (kk >> 2) * (kTM * 128) + (kk & 3) * 32, 16, 1024);
-        const uint64_t bd = umma_desc(kb + (kk >> 2) * (kTN * 128) + (kk & 3) * 32, 16, 1024);
-        umma_f16(tmem + kColS + (kt & 1) * kTN, ad, bd, kIdescS, kk > 0);
-      }
-      umma_commit(&bar_s[kt & 1]);
-    };
-    uint32_t ph_k[2] = {0, 0}, ph_v[2] = {0, 0}, ph_sw[2] = {0, 0}, ph_p = 0;
     bool ok = true;
     auto wait_on = [&](uint64_t* bar, uint32_t& phase) {   // warp-uniform bounded wait
       if (ok) ok = __all_sync(0xffffffffu, bounded_wait(bar, phase) && !failed);
       phase ^= 1u;
     };
-    fetch_tile(true, 0, sK, &bar_k[0]);
-    fetch_tile(false, 0, sV, &bar_v[0]);
-    if (n_ktiles > 1) fetch_tile(true, 1, sK + kKV, &bar_k[1]);
-    for (int kt = 0; kt < 2 && kt < n_ktiles; ++kt) {
-      wait_on(&bar_k[kt], ph_k[kt]);
-      if (ok && lane == 0) {
-        tc5_fence_after();
-        issue_scores(kt);
-      }
-    }
-    // once S(0) is complete its K buffer can take tile 2
-    if (n_ktiles > 2) {
-      wait_on(&bar_s[0], ph_sw[0]);
-      if (ok) fetch_tile(true, 2, sK, &bar_k[0]);
-    }
-    for (int kt = 0; kt < n_ktiles && ok; ++kt) {
-      const int buf = kt & 1;
-      wait_on(&bar_p, ph_p);                      // P(kt) ready; the threads have seen PV(kt-1) complete
-      if (!ok) break;
-      if (kt + 1 < n_ktiles) fetch_tile(false, kt + 1, sV + (buf ^ 1) * kKV, &bar_v[buf ^ 1]);
-      wait_on(&bar_v[buf], ph_v[buf]);            // V(kt) landed
-      if (!ok) break;
-      if (lane == 0) {
-        tc5_fence_after();
-        const uint32_t vb = sV + buf * kKV;
+    if (warp == 4) {
+      // ---------------- score warp: K tiles and S(kt) = Q K(kt)^T into score buffer kt & 1
+      uint64_t qd[kTD / 16], kd[2][kTD / 16];
 #pragma unroll
-        for (int ks = 0; ks < kTN / 16; ++ks) {   // O += P V
-          const uint64_t ad = umma_desc(sP + ks * 32, 16, 1024);
-          const uint64_t bd = umma_desc(vb + ks * (16 * 128), kTN * 128, 1024);
-          umma_f16(tmem + kColO, ad, bd, kIdescO, (kt > 0 || ks > 0) ? 1u : 0u);
-        }
-        umma_commit(&bar_o);
+      for (int kk = 0; kk < kTD / 16; ++kk) {
+        qd[kk] = umma_desc(sQ + (kk >> 2) * (kTM * 128) + (kk & 3) * 32, 16, 1024);
+        kd[0][kk] = umma_desc(sK + (kk >> 2) * (kTN * 128) + (kk & 3) * 32, 16, 1024);
+        kd[1][kk] = umma_desc(sK + kKV + (kk >> 2) * (kTN * 128) + (kk & 3) * 32, 16, 1024);
       }
-      if (kt + 2 < n_ktiles) {
-        wait_on(&bar_k[buf], ph_k[buf]);          // K(kt+2) landed (fetched one iteration ago)
+      uint32_t ph_k[2] = {0, 0}, ph_s[2] = {0, 0}, ph_f[2] = {0, 0};
+      fetch_tile(true, 0, sK, &bar_k[0]);
+      if (n_ktiles > 1) fetch_tile(true, 1, sK + kKV, &bar_k[1]);
+      for (int kt = 0; kt < n_ktiles && ok; ++kt) {
+        const int buf = kt & 1;
+        if (kt >= 2) wait_on(&bar_sfree[buf], ph_f[buf]);   // the threads have read S(kt-2)
+        wait_on(&bar_k[buf], ph_k[buf]);                    // K(kt) landed
         if (!ok) break;
         if (lane == 0) {
           tc5_fence_after();
-          issue_scores(kt + 2);
+          if (buf == 0) {
+#pragma unroll
+            for (int kk = 0; kk < kTD / 16; ++kk) umma_f16(tmem + kColS, qd[kk], kd[0][kk], kIdescS, kk > 0);
+          } else {
+#pragma unroll
+            for (int kk = 0; kk < kTD / 16; ++kk) umma_f16(tmem + kColS + kTN, qd[kk], kd[1][kk], kIdescS, kk > 0);
+          }
+          umma_commit(&bar_s[buf]);
+        }
+        if (kt >= 1 && kt + 1 < n_ktiles) {                 // S(kt-1) complete: its K buffer takes tile kt+1
+          wait_on(&bar_s[buf ^ 1], ph_s[buf ^ 1]);
+          if (!ok) break;
+          fetch_tile(true, kt + 1, sK + (buf ^ 1) * kKV, &bar_k[buf ^ 1]);
         }
       }
-      if (kt + 3 < n_ktiles) {                    // S(kt+1) complete: its K buffer takes tile kt+3
-        wait_on(&bar_s[buf ^ 1], ph_sw[buf ^ 1]);
+    } else {
+      // ---------------- value warp: V tiles and O += P(kt) V(kt)
+      uint64_t pd[kTN / 16], vd[2][kTN / 16];
+#pragma unroll
+      for (int ks = 0; ks < kTN / 16; ++ks) {
+        pd[ks] = umma_desc(sP + ks * 32, 16, 1024);
+        vd[0][ks] = umma_desc(sV + ks * (16 * 128), kTN * 128, 1024);
+        vd[1][ks] = umma_desc(sV + kKV + ks * (16 * 128), kTN * 128, 1024);
+      }
+      uint32_t ph_v[2] = {0, 0}, ph_p = 0;
+      fetch_tile(false, 0, sV, &bar_v[0]);
+      for (int kt = 0; kt < n_ktiles && ok; ++kt) {
+        const int buf = kt & 1;
+        wait_on(&bar_p, ph_p);                      // P(kt) ready; the threads have seen PV(kt-1) complete
         if (!ok) break;
-        fetch_tile(true, kt + 3, sK + (buf ^ 1) * kKV, &bar_k[buf ^ 1]);
+        if (kt + 1 < n_ktiles) fetch_tile(false, kt + 1, sV + (buf ^ 1) * kKV, &bar_v[buf ^ 1]);
+        wait_on(&bar_v[buf], ph_v[buf]);            // V(kt) landed
+        if (!ok) break;
+        if (lane == 0) {
+          tc5_fence_after();
+          if (buf == 0) {
+#pragma unroll
+            for (int ks = 0; ks < kTN / 16; ++ks) umma_f16(tmem + kColO, pd[ks], vd[0][ks], kIdescO, (kt > 0 || ks > 0) ? 1u : 0u);
+          } else {
+#pragma unroll
+            for (int ks = 0; ks < kTN / 16; ++ks) umma_f16(tmem + kColO, pd[ks], vd[1][ks], kIdescO, 1u);
+          }
+          umma_commit(&bar_o);
+        }
       }
     }
     if (!ok) failed = 1;
@@ -634,6 +643,8 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
 #pragma unroll
         for (int j = 0; j < 32; ++j) p[j] = __uint_as_float(r0[j]), p[32 + j] = __uint_as_float(r1[j]);
       }
+      tc5_fence_before();
+      mbar_arrive(&bar_sfree[buf]);   // score buffer `buf` may be overwritten by S(kt+2)
       const int n0 = kt * kTN;
       if (n0 + kTN - 1 > m0 || n0 + kTN > A.T) {   // only tiles on the diagonal or at the end of the prompt need the mask
 #pragma unroll
@@ -726,7 +737,7 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
   }
 }
 
-constexpr int prefill_tcgen05_smem_bytes() { return 2 * kTM * 128 + 4 * (2 * kTN * 128) + kTM * 128 + 64; }
+constexpr int prefill_tcgen05_smem_bytes() { return 2 * kTM * 128 + 4 * (2 * kTN * 128) + kTM * 128 + 128; }
 
 template <int D>
 constexpr int prefill_smem_bytes() {
