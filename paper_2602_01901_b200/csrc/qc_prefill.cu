@@ -328,6 +328,14 @@ __device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t adesc, uint64
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       :: "r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
+// same product with the A operand in tensor memory (128 lanes = rows, 16-bit elements packed two per column)
+__device__ __forceinline__ void umma_f16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc,
+                                            uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      :: "r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
@@ -434,9 +442,13 @@ constexpr int kTc5Threads = kTM + 64;   // 128 softmax threads (one per query ro
 // copies by the 32 lanes.  Hand-offs are mbarriers only:
 //   bar_k[b], bar_v[b]  copies -> score / value warp    K / V tile landed in buffer b
 //   bar_s[b]      tensor core -> softmax, score warp    score buffer b holds S(kt); K buffer b is free
-//   bar_sfree[b]  softmax -> score warp    the 128 threads have read score buffer b
-//   bar_p         softmax -> value warp    weights P(kt) written; the threads have seen PV(kt-1) complete
-//   bar_o         tensor core -> softmax   value product of tile kt done: P and O may change
+//   bar_p         softmax -> value warp    weights P(kt) written
+//   bar_o[b]      tensor core -> score warp, value warp, softmax   PV(kt) done (kt & 1 == b): score buffer b, V
+//                 buffer b and the accumulator may change
+// The bf16 weights P(kt) overwrite the first 32 columns of score buffer kt & 1 in tensor memory and
+// are the A operand of the value product from there: no shared-memory round trip, and since there
+// are two score buffers the softmax of tile kt+1 never waits for PV(kt) (only a rescale of the
+// accumulator does).
 __global__ void __launch_bounds__(kTc5Threads, 2)
     prefill_attend_tcgen05_kernel(const __grid_constant__ PrefillArgs A, int32_t* err) {
   // No static shared memory: the dynamic window then starts on the 1024-byte boundary that the
@@ -446,15 +458,13 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
   const uint32_t sQ = base;                         // [2][128][128 B]  32 KiB
   const uint32_t sK = sQ + 2 * kTM * 128;           // two buffers of [2][64][128 B] 16 KiB
   const uint32_t sV = sK + 2 * (2 * kTN * 128);     // two buffers
-  const uint32_t sP = sV + 2 * (2 * kTN * 128);     // [128][128 B]     16 KiB
   constexpr uint32_t kKV = 2 * kTN * 128;
-  constexpr uint32_t kTiles = 2 * kTM * 128 + 4 * kKV + kTM * 128;
+  constexpr uint32_t kTiles = 2 * kTM * 128 + 4 * kKV;
   uint64_t* bar_s = reinterpret_cast<uint64_t*>(smem_dyn + kTiles);          // two: one per score buffer
-  uint64_t& bar_o = *reinterpret_cast<uint64_t*>(smem_dyn + kTiles + 16);
   uint64_t& bar_p = *reinterpret_cast<uint64_t*>(smem_dyn + kTiles + 24);
   uint64_t* bar_k = reinterpret_cast<uint64_t*>(smem_dyn + kTiles + 32);          // two
   uint64_t* bar_v = reinterpret_cast<uint64_t*>(smem_dyn + kTiles + 48);          // two
-  uint64_t* bar_sfree = reinterpret_cast<uint64_t*>(smem_dyn + kTiles + 64);      // two
+  uint64_t* bar_o = reinterpret_cast<uint64_t*>(smem_dyn + kTiles + 64);          // two: PV(kt) -> bar_o[kt & 1]
   uint32_t& tmem_base_slot = *reinterpret_cast<uint32_t*>(smem_dyn + kTiles + 80);
   volatile int32_t& failed = *reinterpret_cast<volatile int32_t*>(smem_dyn + kTiles + 84);
   if (base & 1023u) {   // cannot happen with the layout above; never run the tensor core on a misplaced tile
@@ -478,12 +488,11 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
   if (threadIdx.x == 0) {
     mbar_init(&bar_s[0], 1);
     mbar_init(&bar_s[1], 1);
-    mbar_init(&bar_o, 1);
     mbar_init(&bar_p, kTM);
     for (int b = 0; b < 2; ++b) {
       mbar_init(&bar_k[b], 1);
       mbar_init(&bar_v[b], 1);
-      mbar_init(&bar_sfree[b], kTM);
+      mbar_init(&bar_o[b], 1);
     }
     fence_mbar_init();
     failed = 0;
@@ -568,7 +577,7 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
       if (n_ktiles > 1) fetch_tile(true, 1, sK + kKV, &bar_k[1]);
       for (int kt = 0; kt < n_ktiles && ok; ++kt) {
         const int buf = kt & 1;
-        if (kt >= 2) wait_on(&bar_sfree[buf], ph_f[buf]);   // the threads have read S(kt-2)
+        if (kt >= 2) wait_on(&bar_o[buf], ph_f[buf]);       // PV(kt-2) has consumed the weights held in this buffer
         wait_on(&bar_k[buf], ph_k[buf]);                    // K(kt) landed
         if (!ok) break;
         if (lane == 0) {
@@ -590,32 +599,35 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
       }
     } else {
       // ---------------- value warp: V tiles and O += P(kt) V(kt)
-      uint64_t pd[kTN / 16], vd[2][kTN / 16];
+      uint64_t vd[2][kTN / 16];
 #pragma unroll
       for (int ks = 0; ks < kTN / 16; ++ks) {
-        pd[ks] = umma_desc(sP + ks * 32, 16, 1024);
         vd[0][ks] = umma_desc(sV + ks * (16 * 128), kTN * 128, 1024);
         vd[1][ks] = umma_desc(sV + kKV + ks * (16 * 128), kTN * 128, 1024);
       }
-      uint32_t ph_v[2] = {0, 0}, ph_p = 0;
+      uint32_t ph_v[2] = {0, 0}, ph_p = 0, ph_o[2] = {0, 0};
       fetch_tile(false, 0, sV, &bar_v[0]);
       for (int kt = 0; kt < n_ktiles && ok; ++kt) {
         const int buf = kt & 1;
-        wait_on(&bar_p, ph_p);                      // P(kt) ready; the threads have seen PV(kt-1) complete
-        if (!ok) break;
+        if (kt >= 1 && kt + 1 < n_ktiles) {         // PV(kt-1) done: its V buffer takes tile kt+1
+          wait_on(&bar_o[buf ^ 1], ph_o[buf ^ 1]);
+          if (!ok) break;
+        }
         if (kt + 1 < n_ktiles) fetch_tile(false, kt + 1, sV + (buf ^ 1) * kKV, &bar_v[buf ^ 1]);
+        wait_on(&bar_p, ph_p);                      // P(kt) is in tensor memory
         wait_on(&bar_v[buf], ph_v[buf]);            // V(kt) landed
         if (!ok) break;
         if (lane == 0) {
           tc5_fence_after();
+          const uint32_t pa = tmem + kColS + buf * kTN;   // 16 keys of bf16 weights = 8 columns per k-step
           if (buf == 0) {
 #pragma unroll
-            for (int ks = 0; ks < kTN / 16; ++ks) umma_f16(tmem + kColO, pd[ks], vd[0][ks], kIdescO, (kt > 0 || ks > 0) ? 1u : 0u);
+            for (int ks = 0; ks < kTN / 16; ++ks) umma_f16_ts(tmem + kColO, pa + 8 * ks, vd[0][ks], kIdescO, (kt > 0 || ks > 0) ? 1u : 0u);
           } else {
 #pragma unroll
-            for (int ks = 0; ks < kTN / 16; ++ks) umma_f16(tmem + kColO, pd[ks], vd[1][ks], kIdescO, 1u);
+            for (int ks = 0; ks < kTN / 16; ++ks) umma_f16_ts(tmem + kColO, pa + 8 * ks, vd[1][ks], kIdescO, 1u);
           }
-          umma_commit(&bar_o);
+          umma_commit(&bar_o[buf]);
         }
       }
     }
@@ -625,7 +637,7 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
     // ------------------------------------------------------------------ softmax threads
     const uint32_t t_row = tmem + (static_cast<uint32_t>(warp * 32) << 16);   // this warp's 32 TMEM lanes
     float m_ref = -INFINITY, l_sum = 0.f;
-    uint32_t ph_s[2] = {0, 0}, ph_o = 0;
+    uint32_t ph_s[2] = {0, 0};
     bool ok = true;
     for (int kt = 0; kt < n_ktiles; ++kt) {
       const int buf = kt & 1;
@@ -643,8 +655,6 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
 #pragma unroll
         for (int j = 0; j < 32; ++j) p[j] = __uint_as_float(r0[j]), p[32 + j] = __uint_as_float(r1[j]);
       }
-      tc5_fence_before();
-      mbar_arrive(&bar_sfree[buf]);   // score buffer `buf` may be overwritten by S(kt+2)
       const int n0 = kt * kTN;
       if (n0 + kTN - 1 > m0 || n0 + kTN > A.T) {   // only tiles on the diagonal or at the end of the prompt need the mask
 #pragma unroll
@@ -672,14 +682,11 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
         ps[j & 3] += p[j];
       }
       l_sum = l_sum * corr + ((ps[0] + ps[1]) + (ps[2] + ps[3]));
-      // ---- the previous value product must be done before P, O or the other V buffer change
-      if (kt > 0) {
-        ok = bounded_wait(&bar_o, ph_o) && !failed;
-        ph_o ^= 1u;
+      if (kt > 0 && __any_sync(0xffffffffu, corr != 1.f)) {   // rare: move the accumulator to the new reference
+        // PV(kt-1) -- and with it every earlier value product -- must be done: phase (kt-1)/2 of its barrier
+        ok = bounded_wait(&bar_o[(kt - 1) & 1], ((kt - 1) >> 1) & 1) && !failed;
         if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
         tc5_fence_after();
-      }
-      if (kt > 0 && __any_sync(0xffffffffu, corr != 1.f)) {   // rare: move the accumulator to the new reference
 #pragma unroll
         for (int c = 0; c < kTD / 32; ++c) {
           uint32_t r[32];
@@ -690,20 +697,18 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
         }
         asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
       }
-      // ---- weights as the A operand: row threadIdx.x, 64 keys = one 128-byte swizzled line
+      // ---- weights as the A operand, in place of the scores just read: 64 bf16 = 32 columns of this row's lane
+      {
+        uint32_t w[32];
 #pragma unroll
-      for (int c = 0; c < kTN / 8; ++c) {
-        const uint32_t w0 = pack_bf16x2(p[8 * c + 0], p[8 * c + 1]), w1 = pack_bf16x2(p[8 * c + 2], p[8 * c + 3]);
-        const uint32_t w2 = pack_bf16x2(p[8 * c + 4], p[8 * c + 5]), w3 = pack_bf16x2(p[8 * c + 6], p[8 * c + 7]);
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sP + tc5_off(threadIdx.x, c, kTM)), "r"(w0),
-                     "r"(w1), "r"(w2), "r"(w3)
-                     : "memory");
+        for (int j = 0; j < 32; ++j) w[j] = pack_bf16x2(p[2 * j], p[2 * j + 1]);
+        tmem_st32(t_row + kColS + buf * kTN, w);
+        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
       }
-      fence_proxy_async();     // generic-proxy writes (the weights) before the tensor core reads them
       tc5_fence_before();
       mbar_arrive(&bar_p);
     }
-    if (ok) ok = bounded_wait(&bar_o, ph_o) && !failed;
+    if (ok) ok = bounded_wait(&bar_o[(n_ktiles - 1) & 1], ((n_ktiles - 1) >> 1) & 1) && !failed;   // the last value product
     ok = __all_sync(0xffffffffu, ok);
     if (ok) {
       tc5_fence_after();
@@ -737,7 +742,7 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
   }
 }
 
-constexpr int prefill_tcgen05_smem_bytes() { return 2 * kTM * 128 + 4 * (2 * kTN * 128) + kTM * 128 + 128; }
+constexpr int prefill_tcgen05_smem_bytes() { return 2 * kTM * 128 + 4 * (2 * kTN * 128) + 128; }
 
 template <int D>
 constexpr int prefill_smem_bytes() {
