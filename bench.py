@@ -34,7 +34,7 @@ MODES = {"vla_qc": 0, "vla_eq8": 1, "gla": 2}
 # from the ncu captures of small cases summarised in profiles/attend_kernels_small_cases_ncu_full.md.
 # Traffic grows in proportion to the K/V bytes swept (every tile is fetched once; partial results are
 # written once per chunk), so a full launch's traffic is this ratio times its algorithmic bytes.
-NCU_TRAFFIC_RATIO = {"attend_kernel": 1.055, "attend_tc_kernel": 1.078}
+NCU_TRAFFIC_RATIO = {"attend_kernel": 1.069, "attend_tc_kernel": 1.077}
 
 
 def _peaks():
