@@ -429,8 +429,13 @@ __global__ void merge_kernel(const __grid_constant__ Params P) {
   const int n_slots = P.seqs[si].n_slots;
   const size_t base = (static_cast<size_t>(layer) * P.max_seqs + si) * P.max_slots;
 
+  // Lane s holds the (max, sum) pair of slot s; the accumulator rows do not depend on them, so
+  // their loads are issued four at a time without waiting for the pairs.
   float mmax = -INFINITY;
-  for (int s = lane; s < n_slots; s += 32) mmax = fmaxf(mmax, P.part_ml[(base + s) * P.hq + head].x);
+  float2 my_ml = make_float2(-INFINITY, 0.f);
+  if (lane < n_slots) my_ml = P.part_ml[(base + lane) * P.hq + head];
+  mmax = my_ml.x;
+  for (int s = lane + 32; s < n_slots; s += 32) mmax = fmaxf(mmax, P.part_ml[(base + s) * P.hq + head].x);
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xffffffffu, mmax, o));
 
@@ -438,22 +443,36 @@ __global__ void merge_kernel(const __grid_constant__ Params P) {
   float acc[VPL];
 #pragma unroll
   for (int e = 0; e < VPL; ++e) acc[e] = 0.f;
-  for (int s = 0; s < n_slots; ++s) {
-    const size_t row = (base + s) * P.hq + head;
-    const float2 ml = P.part_ml[row];
-    const float w = exp2f(ml.x - mmax);
-    lsum = fmaf(ml.y, w, lsum);
-    const float* src = P.part_acc + row * D + lane * VPL;
-    if (VPL == 4) {
-      const float4 a = *reinterpret_cast<const float4*>(src);
-      acc[0] = fmaf(a.x, w, acc[0]);
-      acc[1] = fmaf(a.y, w, acc[1]);
-      acc[2 % VPL] = fmaf(a.z, w, acc[2 % VPL]);
-      acc[3 % VPL] = fmaf(a.w, w, acc[3 % VPL]);
-    } else {
-      const float2 a = *reinterpret_cast<const float2*>(src);
-      acc[0] = fmaf(a.x, w, acc[0]);
-      acc[1] = fmaf(a.y, w, acc[1]);
+  for (int s0 = 0; s0 < n_slots; s0 += 4) {
+    float v[4][VPL];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int s = min(s0 + u, n_slots - 1);
+      const float* src = P.part_acc + ((base + s) * P.hq + head) * D + lane * VPL;
+      if (VPL == 4) {
+        const float4 a = *reinterpret_cast<const float4*>(src);
+        v[u][0] = a.x, v[u][1] = a.y, v[u][2 % VPL] = a.z, v[u][3 % VPL] = a.w;
+      } else {
+        const float2 a = *reinterpret_cast<const float2*>(src);
+        v[u][0] = a.x, v[u][1] = a.y;
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int s = s0 + u;
+      float2 ml;
+      if (s < 32) {
+        ml.x = __shfl_sync(0xffffffffu, my_ml.x, s & 31);
+        ml.y = __shfl_sync(0xffffffffu, my_ml.y, s & 31);
+      } else {
+        ml = P.part_ml[(base + min(s, n_slots - 1)) * P.hq + head];
+      }
+      if (s < n_slots) {
+        const float w = exp2f(ml.x - mmax);
+        lsum = fmaf(ml.y, w, lsum);
+#pragma unroll
+        for (int e = 0; e < VPL; ++e) acc[e] = fmaf(v[u][e], w, acc[e]);
+      }
     }
   }
   const float inv = 1.f / lsum;
