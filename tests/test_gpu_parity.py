@@ -1,7 +1,7 @@
 """GPU parity: the CUDA library through its C ABI against the fp64 oracle, same seeded inputs.
 
-Bars (written here, from the task's stated tolerances): every output element within 2e-2 of
-the oracle and relative L2 error <= 5e-3 (bf16 storage, fp32 accumulation); page tables,
+Bars: every output element within 2e-2 of the oracle and relative L2 error <= 5e-3
+(bf16 storage, fp32 accumulation); page tables,
 stream lengths, owner layers and Q Cache contents bit-exact.
 """
 
