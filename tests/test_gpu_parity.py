@@ -337,6 +337,40 @@ def test_many_short_sequences_and_a_partial_batch():
     s.close()
 
 
+def test_empty_calls_and_the_length_limit():
+    """Empty lists are accepted and do nothing; a sequence can grow exactly to max_tokens_per_seq."""
+    layer_kind = [0, 1]
+    w = W.Workload(25, "edge", 2, 2, 2, 64, 16, 1, 3, 9, 9, 2, 4, (1,))
+    s = Session(2, 2, 2, 64, layer_kind, max_seqs=2, max_tokens_per_seq=8, n_pages=2 * 4 * 2 * 2, poison_pool=True)
+    o = LazyAttentionOracle(2, 2, 2, 64, layer_kind, qc.QC_MODE_VLA_QC, n_seqs=1)
+    dev = lambda a: torch.from_numpy(a.astype(np.int16)).view(torch.bfloat16).to(s.device).contiguous()
+    kind, k, v = W.prefill_kv_np(w, 0)                  # 3 text, 9 visual, 2 text
+    out = torch.zeros((2, 1, 2, 64), dtype=torch.bfloat16, device=s.device)
+    lib = qc.load()
+    assert lib.qc_decode_step(s.cache, 0, None, None, None, None, None, None) == qc.QC_OK
+    assert lib.qc_prefill_append(s.cache, 0, None, None, None, None, None) == qc.QC_OK
+    s.prefill_append([0], [0], [], dev(k[:, :1]), dev(v[:, :1]))        # a listed sequence with no tokens
+    assert s.page_table(0, 0, 0)[1] == 0
+    with pytest.raises(qc.QcError) as e:                                  # 9 visual tokens exceed the bound of 8
+        s.prefill_append([0], [14], kind, dev(k), dev(v))
+    assert e.value.status == qc.QC_ERR_INVALID_ARG and s.page_table(0, 1, 0)[1] == 0
+    keep = np.r_[0:3, 3:11, 12:14]                                        # 5 text + 8 visual
+    s.prefill_append([0], [len(keep)], kind[keep], dev(k[:, keep]), dev(v[:, keep]))
+    o.prefill_append(0, kind[keep].tolist(), f64(k[:, keep]), f64(v[:, keep]))
+    for step in range(3):                                                 # text length 5 -> 8: the limit
+        qn, kn, vn = W.decode_qkv_np(w, step)
+        s.decode_step([0], dev(qn), dev(kn), dev(vn), out)
+        ref, _ = o.decode_step(0, f64(qn[:, 0]), f64(kn[:, 0]), f64(vn[:, 0]))
+        got = bits_of(out)
+        for l in range(2):
+            assert_close(got[l, 0], ref[l], f"step {step} layer {l}")
+    with pytest.raises(qc.QcError) as e:                                  # one token too many
+        s.decode_step([0], dev(qn), dev(kn), dev(vn), out)
+    assert e.value.status == qc.QC_ERR_INVALID_ARG and s.page_table(0, 0, 0)[1] == 8
+    assert s.stats().device_error == 0
+    s.close()
+
+
 FULL_CASES = [
     ("llava15_7b", qc.QC_MODE_VLA_QC, 40),
     ("llava15_7b", qc.QC_MODE_VLA_EQ8, 16),
