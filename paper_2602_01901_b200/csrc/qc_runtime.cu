@@ -1028,8 +1028,10 @@ int32_t qc_decode_step_host(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids,
   cudaStream_t stream = c->ctx->stream;
   // The step runs as up to four launch groups of consecutive lazy blocks: while one group
   // computes, the inputs of the next are copied in and the outputs of the previous copied out.
+  // (a small step is not worth cutting up: one group)
   const int nb = static_cast<int>(c->block_jobs.size());
-  const int per = (nb + 3) / 4;
+  const size_t in_bytes = static_cast<size_t>(c->cfg.n_layers) * n_seqs * (c->hq + 2 * c->hkv) * c->D * 2;
+  const int per = in_bytes < (1u << 20) ? nb : (nb + 3) / 4;
   if (c->plan_dirty || c->plan_per != per) {
     const int st = rebuild_plan(c, per);
     if (st != QC_OK) return st;
