@@ -1,14 +1,17 @@
 // CUDA kernels of the Lazy Attention decode path (sm_100a).
 //
-//   setup_kernel    applies this step's page-table patches and expands (job, sequence)
-//                   segments into split-KV work items
+//   setup_kernel    expands the step's (plan position, sequence) pairs into split-KV work items,
+//                   applies page-table patches, resets the work counters and -- on steps without
+//                   patches -- also does the append
 //   append_kernel   writes the new token's k / v rows into the text streams and every
-//                   ordinary layer's q into the Q Cache
-//   attend_kernel   persistent split-KV partial attention: each warp is an independent
-//                   worker that streams K/V page tiles through its own shared-memory ring
-//                   with bulk asynchronous copies and keeps an online softmax in registers
+//                   ordinary layer's q into the Q Cache (a launch of its own on steps with patches
+//                   and per launch group of the host-buffer entry point)
+//   attend_kernel   persistent split-KV partial attention, one query head per work item (MHA):
+//                   each warp is an independent worker that claims items from a counter, streams
+//                   K/V page tiles through its own shared-memory ring with bulk asynchronous
+//                   copies and keeps an online softmax in registers
+//                   (the grouped-query variant on tensor cores is in qc_attend_tc.cu)
 //   merge_kernel    log-sum-exp merge of the partials, bf16 output
-// (the grouped-query variant of the attention kernel is in qc_attend_tc.cu)
 //   prefill_scatter_kernel  stores prompt K/V rows into their pages
 //
 // Attention arithmetic: scores are kept in the log2 domain (q is pre-multiplied by
