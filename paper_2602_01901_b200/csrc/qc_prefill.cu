@@ -324,20 +324,23 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t saddr, uint32_t lbo_bytes
 }
 __device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      "{\n\t.reg .pred p, e;\n\tsetp.ne.b32 p, %4, 0;\n\telect.sync _|e, 0xffffffff;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       :: "r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
 // same product with the A operand in tensor memory (128 lanes = rows, 16-bit elements packed two per column)
 __device__ __forceinline__ void umma_f16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc,
                                             uint32_t accumulate) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      "{\n\t.reg .pred p, e;\n\tsetp.ne.b32 p, %4, 0;\n\telect.sync _|e, 0xffffffff;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
       :: "r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+  asm volatile(
+      "{\n\t.reg .pred e;\n\telect.sync _|e, 0xffffffff;\n\t"
+      "@e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}" ::"r"(smem_u32(bar))
+      : "memory");
 }
 __device__ __forceinline__ void tc5_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc5_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -415,6 +418,18 @@ __device__ __forceinline__ bool bounded_wait(uint64_t* bar, uint32_t parity) {
   uint32_t done = mbar_try_wait(bar, parity);
   for (uint32_t spin = 0; !done && spin < kLimit; ++spin) done = mbar_try_wait(bar, parity);
   return done != 0;
+}
+// one non-blocking look at an mbarrier phase
+__device__ __forceinline__ uint32_t mbar_test_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t done;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(done)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return done;
 }
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
@@ -564,60 +579,43 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
       phase ^= 1u;
     };
     if (warp == 4) {
-      // ---------------- score warp: K tiles and S(kt) = Q K(kt)^T into score buffer kt & 1
-      uint64_t qd[kTD / 16], kd[2][kTD / 16];
+      // ---------------- issue warp: S(kt) = Q K(kt)^T into score buffer kt & 1, O += P(kt) V(kt)
+      uint64_t qd[kTD / 16], kd[2][kTD / 16], vd[2][kTN / 16];
 #pragma unroll
       for (int kk = 0; kk < kTD / 16; ++kk) {
         qd[kk] = umma_desc(sQ + (kk >> 2) * (kTM * 128) + (kk & 3) * 32, 16, 1024);
         kd[0][kk] = umma_desc(sK + (kk >> 2) * (kTN * 128) + (kk & 3) * 32, 16, 1024);
         kd[1][kk] = umma_desc(sK + kKV + (kk >> 2) * (kTN * 128) + (kk & 3) * 32, 16, 1024);
       }
-      uint32_t ph_k[2] = {0, 0}, ph_s[2] = {0, 0}, ph_f[2] = {0, 0};
-      fetch_tile(true, 0, sK, &bar_k[0]);
-      if (n_ktiles > 1) fetch_tile(true, 1, sK + kKV, &bar_k[1]);
-      for (int kt = 0; kt < n_ktiles && ok; ++kt) {
-        const int buf = kt & 1;
-        if (kt >= 2) wait_on(&bar_o[buf], ph_f[buf]);       // PV(kt-2) has consumed the weights held in this buffer
-        wait_on(&bar_k[buf], ph_k[buf]);                    // K(kt) landed
-        if (!ok) break;
-        if (lane == 0) {
-          tc5_fence_after();
-          if (buf == 0) {
-#pragma unroll
-            for (int kk = 0; kk < kTD / 16; ++kk) umma_f16(tmem + kColS, qd[kk], kd[0][kk], kIdescS, kk > 0);
-          } else {
-#pragma unroll
-            for (int kk = 0; kk < kTD / 16; ++kk) umma_f16(tmem + kColS + kTN, qd[kk], kd[1][kk], kIdescS, kk > 0);
-          }
-          umma_commit(&bar_s[buf]);
-        }
-        if (kt >= 1 && kt + 1 < n_ktiles) {                 // S(kt-1) complete: its K buffer takes tile kt+1
-          wait_on(&bar_s[buf ^ 1], ph_s[buf ^ 1]);
-          if (!ok) break;
-          fetch_tile(true, kt + 1, sK + (buf ^ 1) * kKV, &bar_k[buf ^ 1]);
-        }
-      }
-    } else {
-      // ---------------- value warp: V tiles and O += P(kt) V(kt)
-      uint64_t vd[2][kTN / 16];
 #pragma unroll
       for (int ks = 0; ks < kTN / 16; ++ks) {
         vd[0][ks] = umma_desc(sV + ks * (16 * 128), kTN * 128, 1024);
         vd[1][ks] = umma_desc(sV + kKV + ks * (16 * 128), kTN * 128, 1024);
       }
-      uint32_t ph_v[2] = {0, 0}, ph_p = 0, ph_o[2] = {0, 0};
-      fetch_tile(false, 0, sV, &bar_v[0]);
+      uint32_t ph_k[2] = {0, 0}, ph_v[2] = {0, 0}, ph_p = 0;
+      auto issue_scores = [&](int buf) {   // whole warp; one elected lane issues
+        if (buf == 0) {
+#pragma unroll
+          for (int kk = 0; kk < kTD / 16; ++kk) umma_f16(tmem + kColS, qd[kk], kd[0][kk], kIdescS, kk > 0);
+        } else {
+#pragma unroll
+          for (int kk = 0; kk < kTD / 16; ++kk) umma_f16(tmem + kColS + kTN, qd[kk], kd[1][kk], kIdescS, kk > 0);
+        }
+        umma_commit(&bar_s[buf]);
+      };
+      for (int kt = 0; kt < 2 && kt < n_ktiles && ok; ++kt) {   // the first two score tiles have nothing to wait for but K
+        wait_on(&bar_k[kt], ph_k[kt]);
+        if (ok) {
+          tc5_fence_after();
+          issue_scores(kt);
+        }
+      }
       for (int kt = 0; kt < n_ktiles && ok; ++kt) {
         const int buf = kt & 1;
-        if (kt >= 1 && kt + 1 < n_ktiles) {         // PV(kt-1) done: its V buffer takes tile kt+1
-          wait_on(&bar_o[buf ^ 1], ph_o[buf ^ 1]);
-          if (!ok) break;
-        }
-        if (kt + 1 < n_ktiles) fetch_tile(false, kt + 1, sV + (buf ^ 1) * kKV, &bar_v[buf ^ 1]);
         wait_on(&bar_p, ph_p);                      // P(kt) is in tensor memory
         wait_on(&bar_v[buf], ph_v[buf]);            // V(kt) landed
         if (!ok) break;
-        if (lane == 0) {
+        {
           tc5_fence_after();
           const uint32_t pa = tmem + kColS + buf * kTN;   // 16 keys of bf16 weights = 8 columns per k-step
           if (buf == 0) {
@@ -628,6 +626,50 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
             for (int ks = 0; ks < kTN / 16; ++ks) umma_f16_ts(tmem + kColO, pa + 8 * ks, vd[1][ks], kIdescO, 1u);
           }
           umma_commit(&bar_o[buf]);
+        }
+        if (kt + 2 < n_ktiles) {
+          wait_on(&bar_k[buf], ph_k[buf]);          // K(kt+2) landed
+          if (!ok) break;
+          // S(kt+2) overwrites the buffer that holds P(kt): products issued by one thread run in issue
+          // order, so it starts after PV(kt) has read the weights
+          issue_scores(buf);
+        }
+      }
+    } else {
+      // ---------------- load warp: K(kt) once S(kt-2) is complete, V(kt) once PV(kt-2) is complete.
+      // The two streams advance independently (the products complete in the order S, S, PV, S, PV, ...),
+      // so the warp polls both barriers without blocking on either.
+      uint32_t ph_s[2] = {0, 0}, ph_o[2] = {0, 0};
+      for (int kt = 0; kt < 2 && kt < n_ktiles; ++kt) {
+        fetch_tile(true, kt, sK + kt * kKV, &bar_k[kt]);
+        fetch_tile(false, kt, sV + kt * kKV, &bar_v[kt]);
+      }
+      int k_next = 2, v_next = 2;
+      uint32_t idle = 0;
+      while ((k_next < n_ktiles || v_next < n_ktiles) && ok) {
+        bool progress = false;
+        if (k_next < n_ktiles) {
+          const int b = k_next & 1;
+          if (__all_sync(0xffffffffu, mbar_test_wait(&bar_s[b], ph_s[b]))) {
+            ph_s[b] ^= 1u;
+            fetch_tile(true, k_next, sK + b * kKV, &bar_k[b]);
+            ++k_next;
+            progress = true;
+          }
+        }
+        if (v_next < n_ktiles) {
+          const int b = v_next & 1;
+          if (__all_sync(0xffffffffu, mbar_test_wait(&bar_o[b], ph_o[b]))) {
+            ph_o[b] ^= 1u;
+            fetch_tile(false, v_next, sV + b * kKV, &bar_v[b]);
+            ++v_next;
+            progress = true;
+          }
+        }
+        if (progress) {
+          idle = 0;
+        } else if (++idle > (1u << 20) || ((idle & 1023u) == 0 && failed)) {
+          ok = false;
         }
       }
     }
