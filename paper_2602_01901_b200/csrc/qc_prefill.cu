@@ -336,6 +336,49 @@ __device__ __forceinline__ void umma_f16_ts(uint32_t tmem_d, uint32_t tmem_a, ui
       "@e tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
       :: "r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
+// S = Q K^T for one tile: eight products (k-steps of 16 along the head dimension) issued by one
+// elected lane from warp-uniform code.  adesc/bdesc address k-step 0; a k-step advances the start
+// address by 32 bytes inside a 128-byte swizzle row, and the second 64 elements of the head
+// dimension sit one half-tile further (a_half / b_half bytes).
+template <uint32_t A_HALF, uint32_t B_HALF>
+__device__ __forceinline__ void umma_scores(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc) {
+  asm volatile(
+      "{\n\t.reg .pred e, pz, po;\n\t.reg .b64 da, db;\n\t"
+      "elect.sync _|e, 0xffffffff;\n\tsetp.ne.b32 pz, 0, 0;\n\tsetp.eq.b32 po, 0, 0;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, pz;\n\t"
+      "add.u64 da, %1, 2;\n\tadd.u64 db, %2, 2;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, po;\n\t"
+      "add.u64 da, %1, 4;\n\tadd.u64 db, %2, 4;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, po;\n\t"
+      "add.u64 da, %1, 6;\n\tadd.u64 db, %2, 6;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, po;\n\t"
+      "add.u64 da, %1, %4;\n\tadd.u64 db, %2, %5;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, po;\n\t"
+      "add.u64 da, %1, %4 + 2;\n\tadd.u64 db, %2, %5 + 2;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, po;\n\t"
+      "add.u64 da, %1, %4 + 4;\n\tadd.u64 db, %2, %5 + 4;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, po;\n\t"
+      "add.u64 da, %1, %4 + 6;\n\tadd.u64 db, %2, %5 + 6;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, po;\n\t}"
+      :: "r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "n"(A_HALF >> 4), "n"(B_HALF >> 4) : "memory");
+}
+// O (+)= P V for one tile of 64 keys: four products (k-steps of 16 keys).  The weights are read from
+// tensor memory (8 columns per k-step), the V rows MN-major from shared memory (16 rows = 2048 bytes
+// per k-step).  `accumulate` = 0 starts a new accumulator.
+__device__ __forceinline__ void umma_values(uint32_t tmem_d, uint32_t tmem_p, uint64_t bdesc, uint32_t idesc,
+                                            uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred e, pa, po;\n\t.reg .b64 db;\n\t.reg .b32 ta;\n\t"
+      "elect.sync _|e, 0xffffffff;\n\tsetp.ne.b32 pa, %4, 0;\n\tsetp.eq.b32 po, 0, 0;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, pa;\n\t"
+      "add.u32 ta, %1, 8;\n\tadd.u64 db, %2, 128;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], [ta], db, %3, po;\n\t"
+      "add.u32 ta, %1, 16;\n\tadd.u64 db, %2, 256;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], [ta], db, %3, po;\n\t"
+      "add.u32 ta, %1, 24;\n\tadd.u64 db, %2, 384;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], [ta], db, %3, po;\n\t}"
+      :: "r"(tmem_d), "r"(tmem_p), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
   asm volatile(
       "{\n\t.reg .pred e;\n\telect.sync _|e, 0xffffffff;\n\t"
@@ -580,27 +623,12 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
     };
     if (warp == 4) {
       // ---------------- issue warp: S(kt) = Q K(kt)^T into score buffer kt & 1, O += P(kt) V(kt)
-      uint64_t qd[kTD / 16], kd[2][kTD / 16], vd[2][kTN / 16];
-#pragma unroll
-      for (int kk = 0; kk < kTD / 16; ++kk) {
-        qd[kk] = umma_desc(sQ + (kk >> 2) * (kTM * 128) + (kk & 3) * 32, 16, 1024);
-        kd[0][kk] = umma_desc(sK + (kk >> 2) * (kTN * 128) + (kk & 3) * 32, 16, 1024);
-        kd[1][kk] = umma_desc(sK + kKV + (kk >> 2) * (kTN * 128) + (kk & 3) * 32, 16, 1024);
-      }
-#pragma unroll
-      for (int ks = 0; ks < kTN / 16; ++ks) {
-        vd[0][ks] = umma_desc(sV + ks * (16 * 128), kTN * 128, 1024);
-        vd[1][ks] = umma_desc(sV + kKV + ks * (16 * 128), kTN * 128, 1024);
-      }
+      const uint64_t qd = umma_desc(sQ, 16, 1024);
+      const uint64_t kd0 = umma_desc(sK, 16, 1024), kd1 = umma_desc(sK + kKV, 16, 1024);
+      const uint64_t vd0 = umma_desc(sV, kTN * 128, 1024), vd1 = umma_desc(sV + kKV, kTN * 128, 1024);
       uint32_t ph_k[2] = {0, 0}, ph_v[2] = {0, 0}, ph_p = 0;
       auto issue_scores = [&](int buf) {   // whole warp; one elected lane issues
-        if (buf == 0) {
-#pragma unroll
-          for (int kk = 0; kk < kTD / 16; ++kk) umma_f16(tmem + kColS, qd[kk], kd[0][kk], kIdescS, kk > 0);
-        } else {
-#pragma unroll
-          for (int kk = 0; kk < kTD / 16; ++kk) umma_f16(tmem + kColS + kTN, qd[kk], kd[1][kk], kIdescS, kk > 0);
-        }
+        umma_scores<kTM * 128, kTN * 128>(tmem + kColS + buf * kTN, qd, buf ? kd1 : kd0, kIdescS);
         umma_commit(&bar_s[buf]);
       };
       for (int kt = 0; kt < 2 && kt < n_ktiles && ok; ++kt) {   // the first two score tiles have nothing to wait for but K
@@ -617,14 +645,7 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
         if (!ok) break;
         {
           tc5_fence_after();
-          const uint32_t pa = tmem + kColS + buf * kTN;   // 16 keys of bf16 weights = 8 columns per k-step
-          if (buf == 0) {
-#pragma unroll
-            for (int ks = 0; ks < kTN / 16; ++ks) umma_f16_ts(tmem + kColO, pa + 8 * ks, vd[0][ks], kIdescO, (kt > 0 || ks > 0) ? 1u : 0u);
-          } else {
-#pragma unroll
-            for (int ks = 0; ks < kTN / 16; ++ks) umma_f16_ts(tmem + kColO, pa + 8 * ks, vd[1][ks], kIdescO, 1u);
-          }
+          umma_values(tmem + kColO, tmem + kColS + buf * kTN, buf ? vd1 : vd0, kIdescO, kt > 0 ? 1u : 0u);
           umma_commit(&bar_o[buf]);
         }
         if (kt + 2 < n_ktiles) {
