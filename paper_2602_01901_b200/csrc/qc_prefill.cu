@@ -293,18 +293,19 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_attend_kernel(const P
 // ------------------------------------------------------------------------------------------
 // The same computation on the fifth-generation tensor cores (tcgen05), head_dim 128.
 //
-// One CTA = 128 query rows of one (layer, query head), 128 threads, one thread per row.  Key /
-// value tiles of 64 tokens are staged (with the per-row source-layer selection) into the
-// canonical 128-byte-swizzled shared-memory layout, [two 64-column halves][rows][128 bytes].
-// One elected thread issues
+// One CTA = 128 query rows of one (layer, query head): 128 softmax threads, one per row, plus an
+// issue warp and a load warp.  Key / value tiles of 64 tokens are staged (with the per-row
+// source-layer selection) into the canonical 128-byte-swizzled shared-memory layout,
+// [two 64-column halves][rows][128 bytes].  One elected lane issues
 //     S[128 x 64]   = Q[128 x 128] . K^T      8 x tcgen05.mma (M 128, N 64, K 16), accumulator in TMEM
-//     O[128 x 128] += P[128 x 64]  . V        4 x tcgen05.mma (M 128, N 128, K 16), V read MN-major
+//     O[128 x 128] += P[128 x 64]  . V        4 x tcgen05.mma (M 128, N 128, K 16), P read from TMEM,
+//                                             V read MN-major from shared memory
 // and commits to an mbarrier.  A thread reads its row of S from TMEM (one TMEM lane per row: no
-// cross-thread reduction), does the online softmax, and writes the bf16 weights as the next
-// A operand into shared memory.  The running maximum is only moved when it grows by more than
+// cross-thread reduction), does the online softmax, and writes the bf16 weights back into TMEM as
+// the next A operand.  The running maximum is only moved when it grows by more than
 // 2^8 (the weights then stay below 2^8, harmless in fp32/bf16), so the accumulator in TMEM is
-// rescaled rarely (TMEM load, scale, store).  Two CTAs per SM (2 x 192 TMEM columns in use,
-// 2 x 256 allocated) overlap one CTA's softmax with the other's products.
+// rescaled rarely (TMEM load, scale, store).  Two CTAs per SM (2 x 256 TMEM columns) overlap one
+// CTA's softmax with the other's products.
 // Every mbarrier wait is bounded; on expiry the CTA records the error, frees its TMEM and leaves.
 
 constexpr int kTM = 128;        // query rows per CTA
@@ -487,26 +488,28 @@ __device__ __forceinline__ void tensor_g2s_3d(uint32_t dst_smem, const void* tma
       : "memory");
 }
 
-constexpr int kTc5Threads = kTM + 64;   // 128 softmax threads (one per query row) + a score warp + a value warp
+constexpr int kTc5Threads = kTM + 64;   // 128 softmax threads (one per query row) + an issue warp + a load warp
 
 // Warp roles.  Warps 0-3: one thread per query row -- read the row's scores from TMEM, online
-// softmax, write the bf16 weights.  Warp 4 (score warp) fetches the K tiles and issues S = Q K^T;
-// warp 5 (value warp) fetches the V tiles and issues O += P V.  Issuing a product or a copy and
-// polling an mbarrier each cost a few hundred cycles of one lane, so the two streams run in
-// separate warps and off the softmax path; all shared-memory descriptors are built once.
+// softmax, write the bf16 weights.  Warp 4 (issue warp) issues every product: S(0), S(1), then per
+// tile PV(kt) followed by S(kt+2).  Warp 5 (load warp) fetches the K and V tiles.  A product costs
+// the issuing lane some tens of cycles and a look at an mbarrier about as much, so both streams
+// stay off the softmax path; the issue warp runs warp-uniform code and elects the issuing lane
+// inside the asm block, which lets the descriptors live in uniform registers.
 // A K/V tile whose 64 rows all come from one layer -- every tile of an ordinary or GLA layer, and
 // the all-text / all-visual tiles of a VLA lazy layer -- is fetched by two tensor-map copies; only
 // a tile that mixes text and visual rows of a VLA lazy layer is gathered row by row with 16-byte
 // copies by the 32 lanes.  Hand-offs are mbarriers only:
-//   bar_k[b], bar_v[b]  copies -> score / value warp    K / V tile landed in buffer b
-//   bar_s[b]      tensor core -> softmax, score warp    score buffer b holds S(kt); K buffer b is free
-//   bar_p         softmax -> value warp    weights P(kt) written
-//   bar_o[b]      tensor core -> score warp, value warp, softmax   PV(kt) done (kt & 1 == b): score buffer b, V
-//                 buffer b and the accumulator may change
+//   bar_k[b], bar_v[b]  copies -> issue warp        K / V tile landed in buffer b
+//   bar_s[b]      tensor core -> softmax, load warp     score buffer b holds S(kt); K buffer b is free
+//   bar_p         softmax -> issue warp                 weights P(kt) written
+//   bar_o[b]      tensor core -> load warp, softmax     PV(kt) done (kt & 1 == b): V buffer b is free and
+//                 the accumulator may be rescaled
 // The bf16 weights P(kt) overwrite the first 32 columns of score buffer kt & 1 in tensor memory and
-// are the A operand of the value product from there: no shared-memory round trip, and since there
-// are two score buffers the softmax of tile kt+1 never waits for PV(kt) (only a rescale of the
-// accumulator does).
+// are the A operand of the value product from there: no shared-memory round trip.  S(kt+2) goes
+// into the same buffer; it is issued by the same lane right after PV(kt), and products of one
+// thread execute in issue order, so it cannot overtake the read of the weights.  With two score
+// buffers the softmax of tile kt+1 overlaps PV(kt) and S(kt+2).
 __global__ void __launch_bounds__(kTc5Threads, 2)
     prefill_attend_tcgen05_kernel(const __grid_constant__ PrefillArgs A, int32_t* err) {
   // No static shared memory: the dynamic window then starts on the 1024-byte boundary that the
