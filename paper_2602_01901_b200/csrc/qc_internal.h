@@ -118,9 +118,16 @@ cudaError_t launch_merge(const Params& p, cudaStream_t stream);
 cudaError_t launch_prefill_scatter(const Params& p, const int32_t* tok_seq, const int32_t* tok_stream,
                                    const int32_t* tok_ord, int32_t n_tokens, int32_t tok_stride,
                                    int32_t tok_offset, cudaStream_t stream);
+// Tensor maps of one prompt for the tcgen05 prefill kernel: q, k, v as 3-D tensors
+// {128, heads, n_layers * T} read in boxes of 64 tokens x one head x 64 elements, and the output
+// as a 4-D tensor {128, hq, T, n_layers} written in boxes of 128 tokens x one head x 64 elements
+// (the token dimension of its own so that a store is clipped at the end of the prompt).
+struct PrefillMaps {
+  CUtensorMap q, k, v, out;
+};
 cudaError_t launch_prefill_attend(const Params& p, const uint8_t* kind_dev, const uint8_t* layer_kind_dev,
                                   const uint8_t* leader_dev, const void* q, const void* k, const void* v, void* out,
-                                  int32_t n_tokens, int32_t gla, const CUtensorMap* tmap_k, const CUtensorMap* tmap_v,
+                                  int32_t n_tokens, int32_t gla, const PrefillMaps* maps,
                                   const uint8_t* tile_code_dev, int32_t seq_id, int32_t n0_text, int32_t n0_vis,
                                   cudaStream_t stream);   // qc_prefill.cu; maps null or a non-empty sequence = mma.sync kernel
 cudaError_t configure_prefill_kernels();

@@ -36,7 +36,9 @@ __device__ __forceinline__ uint32_t tile_off(int row, int chunk) {
 }
 
 struct PrefillArgs {
-  CUtensorMap tmap_k, tmap_v;  // k / v as 3-D tensors {D, hkv, n_layers * T}, box {64, 1, 64}, 128-byte swizzle (tcgen05 kernel)
+  // tcgen05 kernel: q / k / v as 3-D tensors {D, heads, n_layers * T}, box {64, 1, 64}; the output as a
+  // 4-D tensor {D, hq, T, n_layers}, box {64, 1, 128, 1}; 128-byte swizzle
+  CUtensorMap tmap_q, tmap_k, tmap_v, tmap_o;
   const uint8_t* tile_code;    // [ceil(T / 64)] device: 0 = the 64-token tile is all text, 1 = all visual, 2 = mixed
   const uint16_t* q;     // [n_layers][T][hq][D]
   const uint16_t* k;     // [n_layers][T][hkv][D]
@@ -426,36 +428,6 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
       : "memory");
 }
 
-// Stage ROWS rows starting at row0 of one head into the swizzled two-half layout.
-template <int ROWS>
-__device__ __forceinline__ void stage_tc5(uint32_t smem, const uint16_t* base, int own, int lead, bool lazy, bool gla,
-                                          const uint8_t* kind, int row0, int T, int heads, int head) {
-  constexpr int CH = kTD / 8;
-  constexpr int RPP = kTM / CH;      // 8 rows per pass: (row & 7) is the same in every pass of a thread
-  constexpr int NP = ROWS / RPP;
-  const int c = threadIdx.x % CH, r0 = threadIdx.x / CH;
-  const size_t row_elems = static_cast<size_t>(heads) * kTD;
-  const uint16_t* src = base + (static_cast<size_t>(own) * T + row0 + r0) * row_elems + head * kTD + c * 8;
-  const ptrdiff_t to_lead = (static_cast<ptrdiff_t>(lead) - own) * static_cast<ptrdiff_t>(T) * row_elems;
-  const uint32_t dst = smem + tc5_off(r0, c, ROWS);
-  const bool by_kind = lazy && !gla;
-  bool use_lead[NP];
-#pragma unroll
-  for (int i = 0; i < NP; ++i) {
-    const int t = row0 + r0 + i * RPP;
-    use_lead[i] = lazy && (gla || (by_kind && t < T && kind[t]));
-  }
-#pragma unroll
-  for (int i = 0; i < NP; ++i) {
-    const int t = row0 + r0 + i * RPP;
-    if (t < T) {
-      cp_async16(dst + i * (RPP * 128), src + i * RPP * row_elems + (use_lead[i] ? to_lead : 0));
-    } else {
-      asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(dst + i * (RPP * 128)), "r"(0u) : "memory");
-    }
-  }
-}
-
 // Bounded wait on an mbarrier phase.
 __device__ __forceinline__ bool bounded_wait(uint64_t* bar, uint32_t parity) {
   constexpr uint32_t kLimit = 1u << 18;
@@ -486,6 +458,13 @@ __device__ __forceinline__ void tensor_g2s_3d(uint32_t dst_smem, const void* tma
           "r"(dst_smem),
       "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(z), "r"(smem_u32(bar))
       : "memory");
+}
+
+__device__ __forceinline__ void tensor_s2g_4d(const void* tmap, uint32_t src_smem, int32_t x, int32_t y, int32_t z, int32_t w) {
+  asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4, %5}], [%1];" ::
+                   "l"(reinterpret_cast<uint64_t>(tmap)),
+               "r"(src_smem), "r"(x), "r"(y), "r"(z), "r"(w)
+               : "memory");
 }
 
 constexpr int kTc5Threads = kTM + 64;   // 128 softmax threads (one per query row) + an issue warp + a load warp
@@ -528,6 +507,7 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
   uint64_t* bar_o = reinterpret_cast<uint64_t*>(smem_dyn + kTiles + 64);          // two: PV(kt) -> bar_o[kt & 1]
   uint32_t& tmem_base_slot = *reinterpret_cast<uint32_t*>(smem_dyn + kTiles + 80);
   volatile int32_t& failed = *reinterpret_cast<volatile int32_t*>(smem_dyn + kTiles + 84);
+  uint64_t& bar_q = *reinterpret_cast<uint64_t*>(smem_dyn + kTiles + 88);   // the two 64-row halves of the Q tile
   if (base & 1023u) {   // cannot happen with the layout above; never run the tensor core on a misplaced tile
     if (threadIdx.x == 0) atomicMax(err, kErrBadPage);
     return;
@@ -550,6 +530,7 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
     mbar_init(&bar_s[0], 1);
     mbar_init(&bar_s[1], 1);
     mbar_init(&bar_p, kTM);
+    mbar_init(&bar_q, 2);
     for (int b = 0; b < 2; ++b) {
       mbar_init(&bar_k[b], 1);
       mbar_init(&bar_v[b], 1);
@@ -564,12 +545,6 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  if (softmax_thread) {
-    stage_tc5<kTM>(sQ, A.q, layer, lead, lazy, gla, A.kind, m0, A.T, A.hq, head);
-    cp_async_commit();
-    cp_async_wait<0>();
-    fence_proxy_async();
-  }
   tc5_fence_before();
   __syncthreads();
   tc5_fence_after();
@@ -582,10 +557,12 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
   if (warp >= 4) {
     // ------------------------------------------------------------------ tile fetch + product issue
     // Fetch key tile (is_k) or value tile kt into `dst`; completion is one phase of `bar`.
-    auto fetch_tile = [&](bool is_k, int kt, uint32_t dst, uint64_t* bar) {
+    // `which`: 0 = 64 query rows (tile index kt counts 64-row tiles), 1 = key tile, 2 = value tile.
+    // The 64 rows go to `dst` and `dst + half` (the two 64-column halves).
+    auto fetch_tile = [&](int which, int kt, uint32_t dst, uint32_t half, uint64_t* bar) {
       int src = layer;
       bool mixed = false;
-      if (is_k && lazy) {
+      if (which != 2 && lazy && kt * kTN < A.T) {   // queries and keys of a lazy layer: the leader's for visual rows
         if (gla) {
           src = lead;
         } else {
@@ -596,18 +573,22 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
       }
       if (!mixed) {
         if (lane == 0) {
-          const void* tm = is_k ? static_cast<const void*>(&A.tmap_k) : static_cast<const void*>(&A.tmap_v);
+          const void* tm = which == 0 ? static_cast<const void*>(&A.tmap_q)
+                                      : (which == 1 ? static_cast<const void*>(&A.tmap_k) : static_cast<const void*>(&A.tmap_v));
+          const int h = which == 0 ? head : kvh;
           mbar_expect_tx(bar, kKV);
-          tensor_g2s_3d(dst, tm, 0, kvh, src * A.T + kt * kTN, bar);
-          tensor_g2s_3d(dst + kTN * 128, tm, 64, kvh, src * A.T + kt * kTN, bar);
+          tensor_g2s_3d(dst, tm, 0, h, src * A.T + kt * kTN, bar);
+          tensor_g2s_3d(dst + half, tm, 64, h, src * A.T + kt * kTN, bar);
         }
       } else {   // rows of two layers: gather with 16-byte copies (64 rows x 16 chunks over 32 lanes)
+        const uint16_t* from = which == 0 ? A.q : A.k;
+        const int heads = which == 0 ? A.hq : A.hkv, h = which == 0 ? head : kvh;
         for (int e = lane; e < kTN * (kTD / 8); e += 32) {
           const int r = e >> 4, c = e & 15, t = kt * kTN + r;
-          const uint32_t d = dst + tc5_off(r, c, kTN);
+          const uint32_t d = dst + (c >> 3) * half + r * 128 + (((c & 7) ^ (r & 7)) << 4);
           if (t < A.T) {
             const int l = A.kind[t] ? lead : layer;
-            cp_async16(d, A.k + ((static_cast<size_t>(l) * A.T + t) * A.hkv + kvh) * kTD + c * 8);
+            cp_async16(d, from + ((static_cast<size_t>(l) * A.T + t) * heads + h) * kTD + c * 8);
           } else {
             asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(d), "r"(0u) : "memory");
           }
@@ -634,6 +615,10 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
         umma_scores<kTM * 128, kTN * 128>(tmem + kColS + buf * kTN, qd, buf ? kd1 : kd0, kIdescS);
         umma_commit(&bar_s[buf]);
       };
+      {
+        uint32_t ph_q = 0;
+        wait_on(&bar_q, ph_q);
+      }
       for (int kt = 0; kt < 2 && kt < n_ktiles && ok; ++kt) {   // the first two score tiles have nothing to wait for but K
         wait_on(&bar_k[kt], ph_k[kt]);
         if (ok) {
@@ -664,9 +649,13 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
       // The two streams advance independently (the products complete in the order S, S, PV, S, PV, ...),
       // so the warp polls both barriers without blocking on either.
       uint32_t ph_s[2] = {0, 0}, ph_o[2] = {0, 0};
-      for (int kt = 0; kt < 2 && kt < n_ktiles; ++kt) {
-        fetch_tile(true, kt, sK + kt * kKV, &bar_k[kt]);
-        fetch_tile(false, kt, sV + kt * kKV, &bar_v[kt]);
+      fetch_tile(0, 2 * qt, sQ, kTM * 128, &bar_q);
+      fetch_tile(1, 0, sK, kTN * 128, &bar_k[0]);
+      fetch_tile(0, 2 * qt + 1, sQ + kTN * 128, kTM * 128, &bar_q);
+      fetch_tile(2, 0, sV, kTN * 128, &bar_v[0]);
+      if (n_ktiles > 1) {
+        fetch_tile(1, 1, sK + kKV, kTN * 128, &bar_k[1]);
+        fetch_tile(2, 1, sV + kKV, kTN * 128, &bar_v[1]);
       }
       int k_next = 2, v_next = 2;
       uint32_t idle = 0;
@@ -676,7 +665,7 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
           const int b = k_next & 1;
           if (__all_sync(0xffffffffu, mbar_test_wait(&bar_s[b], ph_s[b]))) {
             ph_s[b] ^= 1u;
-            fetch_tile(true, k_next, sK + b * kKV, &bar_k[b]);
+            fetch_tile(1, k_next, sK + b * kKV, kTN * 128, &bar_k[b]);
             ++k_next;
             progress = true;
           }
@@ -685,7 +674,7 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
           const int b = v_next & 1;
           if (__all_sync(0xffffffffu, mbar_test_wait(&bar_o[b], ph_o[b]))) {
             ph_o[b] ^= 1u;
-            fetch_tile(false, v_next, sV + b * kKV, &bar_v[b]);
+            fetch_tile(2, v_next, sV + b * kKV, kTN * 128, &bar_v[b]);
             ++v_next;
             progress = true;
           }
@@ -777,28 +766,39 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
     if (ok) ok = bounded_wait(&bar_o[(n_ktiles - 1) & 1], ((n_ktiles - 1) >> 1) & 1) && !failed;   // the last value product
     ok = __all_sync(0xffffffffu, ok);
     if (ok) {
+      // every product has completed: the Q tile's shared memory is free and takes the output tile in
+      // the same swizzled layout, from where two tensor-map stores write it (clipped at token T)
       tc5_fence_after();
       const float inv = 1.f / l_sum;
-      uint16_t* dst = A.out + ((static_cast<size_t>(layer) * A.T + row) * A.hq + head) * kTD;
+      const uint32_t orow = sQ + threadIdx.x * 128;
+      const uint32_t sw = threadIdx.x & 7;
 #pragma unroll
       for (int c = 0; c < kTD / 32; ++c) {
         uint32_t r[32];
-        tmem_ld32(t_row + kColO + 32 * c, r);   // every lane takes part in the load; only rows of the prompt store
-        if (row < A.T) {
+        tmem_ld32(t_row + kColO + 32 * c, r);
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            uint4 o;
-            o.x = pack_bf16x2(__uint_as_float(r[8 * j + 0]) * inv, __uint_as_float(r[8 * j + 1]) * inv);
-            o.y = pack_bf16x2(__uint_as_float(r[8 * j + 2]) * inv, __uint_as_float(r[8 * j + 3]) * inv);
-            o.z = pack_bf16x2(__uint_as_float(r[8 * j + 4]) * inv, __uint_as_float(r[8 * j + 5]) * inv);
-            o.w = pack_bf16x2(__uint_as_float(r[8 * j + 6]) * inv, __uint_as_float(r[8 * j + 7]) * inv);
-            *reinterpret_cast<uint4*>(dst + 32 * c + 8 * j) = o;
-          }
+        for (int j = 0; j < 4; ++j) {
+          const int chunk = 4 * c + j;   // 16-byte chunk of the 256-byte row
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(orow + (chunk >> 3) * (kTM * 128) + (((chunk & 7) ^ sw) << 4)),
+                       "r"(pack_bf16x2(__uint_as_float(r[8 * j + 0]) * inv, __uint_as_float(r[8 * j + 1]) * inv)),
+                       "r"(pack_bf16x2(__uint_as_float(r[8 * j + 2]) * inv, __uint_as_float(r[8 * j + 3]) * inv)),
+                       "r"(pack_bf16x2(__uint_as_float(r[8 * j + 4]) * inv, __uint_as_float(r[8 * j + 5]) * inv)),
+                       "r"(pack_bf16x2(__uint_as_float(r[8 * j + 6]) * inv, __uint_as_float(r[8 * j + 7]) * inv))
+                       : "memory");
         }
+      }
+      fence_proxy_async();
+      asm volatile("bar.sync 1, %0;" ::"n"(kTM) : "memory");   // the 128 softmax threads
+      if (threadIdx.x == 0) {
+        tensor_s2g_4d(&A.tmap_o, sQ, 0, head, m0, layer);
+        tensor_s2g_4d(&A.tmap_o, sQ + kTM * 128, 64, head, m0, layer);
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // shared memory is released at exit
       }
     } else {
       failed = 1;
       if (lane == 0) atomicMax(err, kErrTimeout);
+      asm volatile("bar.arrive 1, %0;" ::"n"(kTM) : "memory");   // do not hold the other softmax warps
     }
   }
   tc5_fence_before();
@@ -833,7 +833,7 @@ cudaError_t configure_prefill_kernels() {
 
 cudaError_t launch_prefill_attend(const Params& p, const uint8_t* kind_dev, const uint8_t* layer_kind_dev,
                                   const uint8_t* leader_dev, const void* q, const void* k, const void* v, void* out,
-                                  int32_t T, int32_t gla, const CUtensorMap* tmap_k, const CUtensorMap* tmap_v,
+                                  int32_t T, int32_t gla, const PrefillMaps* maps,
                                   const uint8_t* tile_code_dev, int32_t seq_id, int32_t n0_text, int32_t n0_vis,
                                   cudaStream_t stream) {
   if (T <= 0) return cudaSuccess;
@@ -860,9 +860,11 @@ cudaError_t launch_prefill_attend(const Params& p, const uint8_t* kind_dev, cons
   a.seq_id = seq_id;
   a.n0_text = n0_text;
   a.n0_vis = n0_vis;
-  if (p.d == kTD && tmap_k && tmap_v && n0_text + n0_vis == 0) {
-    a.tmap_k = *tmap_k;
-    a.tmap_v = *tmap_v;
+  if (p.d == kTD && maps && n0_text + n0_vis == 0) {
+    a.tmap_q = maps->q;
+    a.tmap_k = maps->k;
+    a.tmap_v = maps->v;
+    a.tmap_o = maps->out;
     a.tile_code = tile_code_dev;
     const dim3 grid5((T + kTM - 1) / kTM, p.hq, p.n_layers);
     prefill_attend_tcgen05_kernel<<<grid5, kTc5Threads, prefill_tcgen05_smem_bytes(), stream>>>(a, p.err);

@@ -370,6 +370,23 @@ int make_prompt_tensor_map(CUtensorMap* out, const void* base, int n_layers, int
   return r == CUDA_SUCCESS ? QC_OK : QC_ERR_CUDA;
 }
 
+// The prefill output [n_layers][T][hq][128] bf16 as a 4-D tensor {128, hq, T, n_layers}: a box is
+// 128 tokens x one head x 64 elements; rows of a box past token T are not written.
+int make_output_tensor_map(CUtensorMap* out, void* base, int n_layers, int T, int heads) {
+  EncodeFn enc = tensor_map_encoder();
+  if (!enc) return QC_ERR_CUDA;
+  const cuuint64_t dims[4] = {128, static_cast<cuuint64_t>(heads), static_cast<cuuint64_t>(T),
+                              static_cast<cuuint64_t>(n_layers)};
+  const cuuint64_t strides[3] = {128 * 2, static_cast<cuuint64_t>(heads) * 128 * 2,
+                                 static_cast<cuuint64_t>(T) * heads * 128 * 2};
+  const cuuint32_t box[4] = {64, 1, 128, 1};
+  const cuuint32_t elem_strides[4] = {1, 1, 1, 1};
+  const CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, base, dims, strides, box, elem_strides,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                         CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? QC_OK : QC_ERR_CUDA;
+}
+
 int make_pool_tensor_map(qc_cache* c) {
   EncodeFn enc = tensor_map_encoder();
   if (!enc) return QC_ERR_CUDA;
@@ -727,11 +744,13 @@ int32_t qc_prefill_attend(qc_cache* c, int32_t seq_id, int32_t n_tokens, const u
   QC_CUDA(cudaMemcpyAsync(kind_dev, kind, n_tokens, cudaMemcpyHostToDevice, stream));
   QC_CUDA(cudaMemcpyAsync(codes_dev, codes.data(), n_tiles, cudaMemcpyHostToDevice, stream));
   QC_CUDA(cudaStreamSynchronize(stream));   // `kind` is the caller's host memory
-  CUtensorMap tmap_k, tmap_v;
+  PrefillMaps maps;
   const bool tc5 = c->prefill_tcgen05 && c->D == 128 && n0_text + n0_vis == 0;
   if (tc5) {
-    if (make_prompt_tensor_map(&tmap_k, k_dev, c->cfg.n_layers, n_tokens, c->hkv) != QC_OK ||
-        make_prompt_tensor_map(&tmap_v, v_dev, c->cfg.n_layers, n_tokens, c->hkv) != QC_OK)
+    if (make_prompt_tensor_map(&maps.q, q_dev, c->cfg.n_layers, n_tokens, c->hq) != QC_OK ||
+        make_prompt_tensor_map(&maps.k, k_dev, c->cfg.n_layers, n_tokens, c->hkv) != QC_OK ||
+        make_prompt_tensor_map(&maps.v, v_dev, c->cfg.n_layers, n_tokens, c->hkv) != QC_OK ||
+        make_output_tensor_map(&maps.out, out_dev, c->cfg.n_layers, n_tokens, c->hq) != QC_OK)
       return QC_ERR_CUDA;
   }
   const Params p = base_params(c);
@@ -748,8 +767,8 @@ int32_t qc_prefill_attend(qc_cache* c, int32_t seq_id, int32_t n_tokens, const u
     QC_CUDA(cudaEventRecord(ev[0], stream));
   }
   QC_CUDA(launch_prefill_attend(p, kind_dev, c->ws + c->lay.layer_kind, c->ws + c->lay.leader, q_dev, k_dev, v_dev,
-                                out_dev, n_tokens, c->cfg.lazy_mode == QC_MODE_GLA ? 1 : 0, tc5 ? &tmap_k : nullptr,
-                                tc5 ? &tmap_v : nullptr, codes_dev, seq_id, n0_text, n0_vis, stream));
+                                out_dev, n_tokens, c->cfg.lazy_mode == QC_MODE_GLA ? 1 : 0, tc5 ? &maps : nullptr,
+                                codes_dev, seq_id, n0_text, n0_vis, stream));
   if (ev) {
     QC_CUDA(cudaEventRecord(ev[1], stream));
     c->ev_prefill_calls++;
