@@ -317,27 +317,10 @@ constexpr uint32_t kTmemCols = 256;
 constexpr uint32_t kColS = 0, kColO = 128;   // scores: two buffers of 64 columns; accumulator: 128 columns
 constexpr float kRescaleThreshold = 8.f;   // log2 units
 
-__device__ __forceinline__ uint32_t tc5_off(int row, int chunk, int rows) {   // chunk: 16-byte chunk of the 256-byte row
-  return (chunk >> 3) * (rows * 128) + row * 128 + (((chunk & 7) ^ (row & 7)) << 4);
-}
 __device__ __forceinline__ uint64_t umma_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
   // start address, leading / stride byte offsets (all >> 4), descriptor version 1, 128-byte swizzle
   return static_cast<uint64_t>((saddr >> 4) & 0x3fff) | (static_cast<uint64_t>((lbo_bytes >> 4) & 0x3fff) << 16) |
          (static_cast<uint64_t>((sbo_bytes >> 4) & 0x3fff) << 32) | (1ull << 46) | (2ull << 61);
-}
-__device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p, e;\n\tsetp.ne.b32 p, %4, 0;\n\telect.sync _|e, 0xffffffff;\n\t"
-      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      :: "r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
-}
-// same product with the A operand in tensor memory (128 lanes = rows, 16-bit elements packed two per column)
-__device__ __forceinline__ void umma_f16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc,
-                                            uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p, e;\n\tsetp.ne.b32 p, %4, 0;\n\telect.sync _|e, 0xffffffff;\n\t"
-      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-      :: "r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
 // S = Q K^T for one tile: eight products (k-steps of 16 along the head dimension) issued by one
 // elected lane from warp-uniform code.  adesc/bdesc address k-step 0; a k-step advances the start
@@ -514,7 +497,6 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
   }
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const bool softmax_thread = threadIdx.x < kTM;
   const int n_qtiles = (A.T + kTM - 1) / kTM;
   const int qt = n_qtiles - 1 - blockIdx.x;         // long rows first
   const int head = blockIdx.y, layer = blockIdx.z;
