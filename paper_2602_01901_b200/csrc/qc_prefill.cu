@@ -465,13 +465,13 @@ constexpr int kTc5Threads = kTM + 64;   // 128 softmax threads (one per query ro
 //   bar_k[b], bar_v[b]  copies -> issue warp        K / V tile landed in buffer b
 //   bar_s[b]      tensor core -> softmax, load warp     score buffer b holds S(kt); K buffer b is free
 //   bar_p         softmax -> issue warp                 weights P(kt) written
-//   bar_o[b]      tensor core -> load warp, softmax     PV(kt) done (kt & 1 == b): V buffer b is free and
-//                 the accumulator may be rescaled
+//   bar_o[b]      tensor core -> load warp, issue warp, softmax     PV(kt) done (kt & 1 == b): V buffer b and
+//                 score buffer b are free and the accumulator may be rescaled
 // The bf16 weights P(kt) overwrite the first 32 columns of score buffer kt & 1 in tensor memory and
 // are the A operand of the value product from there: no shared-memory round trip.  S(kt+2) goes
-// into the same buffer; it is issued by the same lane right after PV(kt), and products of one
-// thread execute in issue order, so it cannot overtake the read of the weights.  With two score
-// buffers the softmax of tile kt+1 overlaps PV(kt) and S(kt+2).
+// into the same buffer, so the issue warp waits for PV(kt) to complete before it issues S(kt+2)
+// (an earlier version relied on issue order alone and produced a corrupted tile now and then).
+// With two score buffers the softmax of tile kt+1 overlaps PV(kt) and S(kt+2).
 __global__ void __launch_bounds__(kTc5Threads, 2)
     prefill_attend_tcgen05_kernel(const __grid_constant__ PrefillArgs A, int32_t* err) {
   // No static shared memory: the dynamic window then starts on the 1024-byte boundary that the
@@ -584,7 +584,8 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
     };
     bool ok = true;
     auto wait_on = [&](uint64_t* bar, uint32_t& phase) {   // warp-uniform bounded wait
-      if (ok) ok = __all_sync(0xffffffffu, bounded_wait(bar, phase) && !failed);
+      if (ok && !__all_sync(0xffffffffu, mbar_try_wait(bar, phase)))   // usually complete at the first look
+        ok = __all_sync(0xffffffffu, bounded_wait(bar, phase) && !failed);
       phase ^= 1u;
     };
     if (warp == 4) {
@@ -592,7 +593,7 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
       const uint64_t qd = umma_desc(sQ, 16, 1024);
       const uint64_t kd0 = umma_desc(sK, 16, 1024), kd1 = umma_desc(sK + kKV, 16, 1024);
       const uint64_t vd0 = umma_desc(sV, kTN * 128, 1024), vd1 = umma_desc(sV + kKV, kTN * 128, 1024);
-      uint32_t ph_k[2] = {0, 0}, ph_v[2] = {0, 0}, ph_p = 0;
+      uint32_t ph_k[2] = {0, 0}, ph_v[2] = {0, 0}, ph_o[2] = {0, 0}, ph_p = 0;
       auto issue_scores = [&](int buf) {   // whole warp; one elected lane issues
         umma_scores<kTM * 128, kTN * 128>(tmem + kColS + buf * kTN, qd, buf ? kd1 : kd0, kIdescS);
         umma_commit(&bar_s[buf]);
@@ -619,10 +620,12 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
           umma_commit(&bar_o[buf]);
         }
         if (kt + 2 < n_ktiles) {
+          // S(kt+2) overwrites the buffer that holds P(kt).  Products with different accumulators are
+          // not documented to run in issue order, so wait until PV(kt) has completed.
+          wait_on(&bar_o[buf], ph_o[buf]);
           wait_on(&bar_k[buf], ph_k[buf]);          // K(kt+2) landed
           if (!ok) break;
-          // S(kt+2) overwrites the buffer that holds P(kt): products issued by one thread run in issue
-          // order, so it starts after PV(kt) has read the weights
+          tc5_fence_after();
           issue_scores(buf);
         }
       }
@@ -678,9 +681,11 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
     bool ok = true;
     for (int kt = 0; kt < n_ktiles; ++kt) {
       const int buf = kt & 1;
-      ok = bounded_wait(&bar_s[buf], ph_s[buf]) && !failed;
+      if (!__all_sync(0xffffffffu, mbar_try_wait(&bar_s[buf], ph_s[buf]))) {
+        ok = bounded_wait(&bar_s[buf], ph_s[buf]) && !failed;
+        if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+      }
       ph_s[buf] ^= 1u;
-      if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
       tc5_fence_after();
       // ---- this row's 64 scores (raw dot products; the scale is folded into the exponent)
       float p[kTN];
