@@ -541,6 +541,19 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
     // Fetch key tile (is_k) or value tile kt into `dst`; completion is one phase of `bar`.
     // `which`: 0 = 64 query rows (tile index kt counts 64-row tiles), 1 = key tile, 2 = value tile.
     // The 64 rows go to `dst` and `dst + half` (the two 64-column halves).
+    // The tile codes of a VLA lazy layer, read once: lane i holds tiles i, i + 32, i + 64.
+    uint32_t codes[3] = {0u, 0u, 0u};
+    if (warp == 5 && lazy && !gla) {
+      const int n_tiles = (A.T + kTN - 1) / kTN;
+#pragma unroll
+      for (int i = 0; i < 3; ++i)
+        if (lane + 32 * i < n_tiles) codes[i] = A.tile_code[lane + 32 * i];
+    }
+    auto code_of = [&](int kt) -> int {   // whole warp
+      if (kt >= 96) return A.tile_code[kt];
+      const uint32_t c = kt < 32 ? codes[0] : (kt < 64 ? codes[1] : codes[2]);
+      return static_cast<int>(__shfl_sync(0xffffffffu, c, kt & 31));
+    };
     auto fetch_tile = [&](int which, int kt, uint32_t dst, uint32_t half, uint64_t* bar) {
       int src = layer;
       bool mixed = false;
@@ -548,7 +561,7 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
         if (gla) {
           src = lead;
         } else {
-          const int code = A.tile_code[kt];
+          const int code = code_of(kt);
           mixed = code == 2;
           src = code == 1 ? lead : layer;
         }
