@@ -464,7 +464,9 @@ constexpr int kTc5Threads = kTM + 64;   // 128 softmax threads (one per query ro
 // copies by the 32 lanes.  Hand-offs are mbarriers only:
 //   bar_k[b], bar_v[b]  copies -> issue warp        K / V tile landed in buffer b
 //   bar_s[b]      tensor core -> softmax, load warp     score buffer b holds S(kt); K buffer b is free
-//   bar_p         softmax -> issue warp                 weights P(kt) written
+//   bar_p[b]      softmax -> issue warp                 weights P(kt) written (one barrier per score buffer: P(kt+2)
+//                 needs S(kt+2), which is issued after the issue warp has seen P(kt), so a barrier is never
+//                 more than one completion ahead of its waiter -- a parity wait could not tell otherwise)
 //   bar_o[b]      tensor core -> load warp, issue warp, softmax     PV(kt) done (kt & 1 == b): V buffer b and
 //                 score buffer b are free and the accumulator may be rescaled
 // The bf16 weights P(kt) overwrite the first 32 columns of score buffer kt & 1 in tensor memory and
@@ -484,7 +486,7 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
   constexpr uint32_t kKV = 2 * kTN * 128;
   constexpr uint32_t kTiles = 2 * kTM * 128 + 4 * kKV;
   uint64_t* bar_s = reinterpret_cast<uint64_t*>(smem_dyn + kTiles);          // two: one per score buffer
-  uint64_t& bar_p = *reinterpret_cast<uint64_t*>(smem_dyn + kTiles + 24);
+  uint64_t* bar_p = reinterpret_cast<uint64_t*>(smem_dyn + kTiles + 16);          // two
   uint64_t* bar_k = reinterpret_cast<uint64_t*>(smem_dyn + kTiles + 32);          // two
   uint64_t* bar_v = reinterpret_cast<uint64_t*>(smem_dyn + kTiles + 48);          // two
   uint64_t* bar_o = reinterpret_cast<uint64_t*>(smem_dyn + kTiles + 64);          // two: PV(kt) -> bar_o[kt & 1]
@@ -511,12 +513,12 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
   if (threadIdx.x == 0) {
     mbar_init(&bar_s[0], 1);
     mbar_init(&bar_s[1], 1);
-    mbar_init(&bar_p, kTM);
     mbar_init(&bar_q, 2);
     for (int b = 0; b < 2; ++b) {
       mbar_init(&bar_k[b], 1);
       mbar_init(&bar_v[b], 1);
       mbar_init(&bar_o[b], 1);
+      mbar_init(&bar_p[b], kTM);
     }
     fence_mbar_init();
     failed = 0;
@@ -606,7 +608,7 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
       const uint64_t qd = umma_desc(sQ, 16, 1024);
       const uint64_t kd0 = umma_desc(sK, 16, 1024), kd1 = umma_desc(sK + kKV, 16, 1024);
       const uint64_t vd0 = umma_desc(sV, kTN * 128, 1024), vd1 = umma_desc(sV + kKV, kTN * 128, 1024);
-      uint32_t ph_k[2] = {0, 0}, ph_v[2] = {0, 0}, ph_o[2] = {0, 0}, ph_p = 0;
+      uint32_t ph_k[2] = {0, 0}, ph_v[2] = {0, 0}, ph_o[2] = {0, 0}, ph_p[2] = {0, 0};
       auto issue_scores = [&](int buf) {   // whole warp; one elected lane issues
         umma_scores<kTM * 128, kTN * 128>(tmem + kColS + buf * kTN, qd, buf ? kd1 : kd0, kIdescS);
         umma_commit(&bar_s[buf]);
@@ -624,7 +626,7 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
       }
       for (int kt = 0; kt < n_ktiles && ok; ++kt) {
         const int buf = kt & 1;
-        wait_on(&bar_p, ph_p);                      // P(kt) is in tensor memory
+        wait_on(&bar_p[buf], ph_p[buf]);            // P(kt) is in tensor memory
         wait_on(&bar_v[buf], ph_v[buf]);            // V(kt) landed
         if (!ok) break;
         {
@@ -761,7 +763,7 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
         asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
       }
       tc5_fence_before();
-      mbar_arrive(&bar_p);
+      mbar_arrive(&bar_p[buf]);
     }
     if (ok) ok = bounded_wait(&bar_o[(n_ktiles - 1) & 1], ((n_ktiles - 1) >> 1) & 1) && !failed;   // the last value product
     ok = __all_sync(0xffffffffu, ok);
