@@ -233,7 +233,16 @@ int32_t qc_debug_read_row(qc_cache* cache, int32_t layer, int32_t stream, int32_
 /* Tuning knobs (all optional).  key: "split_tokens" (as in qc_config, never below the value
  * the cache was created with; 0 = per-step choice), "layers_per_launch"
  * (0 = one attention launch for the whole step; k>0 = one launch per k consecutive lazy
- * blocks, in layer order), "profile" (1 = record CUDA events per step). */
+ * blocks, in layer order), "per_layer_logit_cache" (1 = one attention + merge launch per layer,
+ * in layer order: the schedule of a model in which a layer's q/k/v only exist after the previous
+ * layer has run.  A leader with followers then also stores its scaled scores -- of the visual keys
+ * in VLA_QC, of all keys in GLA -- in a logit cache inside the workspace, 4 bytes per key and
+ * query head, and a follower weights its own V rows with them instead of reading the leader's K
+ * again; by Eq. 6 / the Q Cache rule the follower's scores are the leader's, so the result is the
+ * one of the fused schedule.  VLA_EQ8 followers score with their own query and re-read the
+ * leader's visual K.  0 = back to one launch per step.  qc_decode_step only),
+ * "prefill_tcgen05" (0 = use the mma.sync prefill kernel), "profile" (1 = record CUDA events per
+ * step). */
 int32_t qc_set_option(qc_cache* cache, const char* key, int64_t value);
 
 /* Sum the recorded kernel times since the last call (synchronises), then reset them. */

@@ -46,7 +46,9 @@ __device__ __forceinline__ uint32_t swz(int row, int chunk) {
 
 // One item: NQ query groups score the K tiles, NV value streams are accumulated.
 // NQ == 1: every consumer shares the weights; NQ == NV: consumer x has its own queries.
-template <int D, int NQ, int NV>
+// MODE 1 (one query group, one consumer) also stores the scaled scores in the logit cache; MODE 2
+// takes them from there instead of reading K tiles (the ring then carries V tiles only).
+template <int D, int NQ, int NV, int MODE = 0>
 __device__ __forceinline__ void process_item_tc(WorkerState& st, const TcCtx* ctx, uint32_t ring, uint64_t* full,
                                                 const Params& P, int lane) {
   constexpr int KS = D / 16;    // k-steps of the score product = m-tiles of the value product
@@ -88,32 +90,68 @@ __device__ __forceinline__ void process_item_tc(WorkerState& st, const TcCtx* ct
   const int k_row = lrow + ((lmat & 1) << 3), k_chunk = lmat >> 1;    // K: matrices (keys lo/hi) x (chunk +0/+1)
   const int v_row = lrow + ((lmat >> 1) << 3), v_chunk = lmat & 1;    // V: matrices (chunk +0/+1) x (keys lo/hi)
 
+  // Logit cache rows of heads 2t and 2t + 1 at this item's first key (lane (g, t) holds the scores
+  // of keys g and g + 8 for those two heads).
+  float* lg0 = nullptr;
+  float* lg1 = nullptr;
+  float lg_next[4] = {0.f, 0.f, 0.f, 0.f};
+  const bool h0 = 2 * t < n_heads, h1 = 2 * t + 1 < n_heads;
+  if (MODE != 0) {
+    lg0 = logit_row(P, it.stream, it.seq_id, it.head + (h0 ? 2 * t : 0)) + it.first_page * kPage;
+    lg1 = logit_row(P, it.stream, it.seq_id, it.head + (h1 ? 2 * t + 1 : 0)) + it.first_page * kPage;
+    if (MODE == 2) {
+      lg_next[0] = lg0[g], lg_next[1] = lg1[g], lg_next[2] = lg0[g + 8], lg_next[3] = lg1[g + 8];
+    }
+  }
+
   for (int pg = 0; pg < n_pages && !st.dead; ++pg) {
     const int nvalid = (pg == n_pages - 1) ? n_valid_last : kPage;
     uint32_t pb[NQ][2];
     // ---- K tile: scores of 16 keys for 8 heads
     {
-      const uint32_t tile = wait_tile<D>(st, ring, full, P, lane);
-      if (st.dead) break;
       float s[NQ][4];
+      if (MODE == 2) {
+        // the scaled scores of this page from the logit cache; the next page's are requested now
 #pragma unroll
-      for (int x = 0; x < NQ; ++x) s[x][0] = s[x][1] = s[x][2] = s[x][3] = 0.f;
+        for (int i = 0; i < 4; ++i) s[0][i] = lg_next[i];
+        if (pg + 1 < n_pages) {
+          const int o = (pg + 1) * kPage + g;
+          lg_next[0] = lg0[o], lg_next[1] = lg1[o], lg_next[2] = lg0[o + 8], lg_next[3] = lg1[o + 8];
+        }
+      } else {
+        const uint32_t tile = wait_tile<D>(st, ring, full, P, lane);
+        if (st.dead) break;
 #pragma unroll
-      for (int kk = 0; kk < KS; ++kk) {
-        uint32_t a[4];
-        ldmatrix_x4(a, tile + swz<D>(k_row, 2 * kk + k_chunk));
+        for (int x = 0; x < NQ; ++x) s[x][0] = s[x][1] = s[x][2] = s[x][3] = 0.f;
 #pragma unroll
-        for (int x = 0; x < NQ; ++x) mma_bf16_16816(s[x], a, qb[x][kk]);
+        for (int kk = 0; kk < KS; ++kk) {
+          uint32_t a[4];
+          ldmatrix_x4(a, tile + swz<D>(k_row, 2 * kk + k_chunk));
+#pragma unroll
+          for (int x = 0; x < NQ; ++x) mma_bf16_16816(s[x], a, qb[x][kk]);
+        }
+        release_tile<kRingTc>(st);
+        fill_ring<D, kRingTc, true>(st, ctx_of, ring, full, P, lane);
+#pragma unroll
+        for (int x = 0; x < NQ; ++x) {
+#pragma unroll
+          for (int i = 0; i < 4; ++i) s[x][i] *= P.scale_log2;
+        }
       }
-      release_tile<kRingTc>(st);
-      fill_ring<D, kRingTc, true>(st, ctx_of, ring, full, P, lane);
       const bool ok_lo = g < nvalid, ok_hi = g + 8 < nvalid;
+      if (MODE == 1) {
+        const int o = pg * kPage + g;
+        if (ok_lo && h0) lg0[o] = s[0][0];
+        if (ok_lo && h1) lg1[o] = s[0][1];
+        if (ok_hi && h0) lg0[o + 8] = s[0][2];
+        if (ok_hi && h1) lg1[o + 8] = s[0][3];
+      }
 #pragma unroll
       for (int x = 0; x < NQ; ++x) {
-        const float s0 = ok_lo ? s[x][0] * P.scale_log2 : -INFINITY;   // key g,     head 2t
-        const float s1 = ok_lo ? s[x][1] * P.scale_log2 : -INFINITY;   // key g,     head 2t + 1
-        const float s2 = ok_hi ? s[x][2] * P.scale_log2 : -INFINITY;   // key g + 8, head 2t
-        const float s3 = ok_hi ? s[x][3] * P.scale_log2 : -INFINITY;   // key g + 8, head 2t + 1
+        const float s0 = ok_lo ? s[x][0] : -INFINITY;   // key g,     head 2t
+        const float s1 = ok_lo ? s[x][1] : -INFINITY;   // key g,     head 2t + 1
+        const float s2 = ok_hi ? s[x][2] : -INFINITY;   // key g + 8, head 2t
+        const float s3 = ok_hi ? s[x][3] : -INFINITY;   // key g + 8, head 2t + 1
         float t0 = fmaxf(s0, s2), t1 = fmaxf(s1, s3);
 #pragma unroll
         for (int off = 4; off < 32; off <<= 1) {
@@ -250,7 +288,9 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
     const bool shared = it.flags & kFlagShared;
     // claim the item after next now; the answer is needed only when this item is done
     const int issued = (next >= 0) ? claim_issue(P, lane) : 0;
-    if (nc == 1) process_item_tc<D, 1, 1>(st, ctx, ring, full, P, lane);
+    if (nc == 1 && (it.flags & kFlagReadLogits)) process_item_tc<D, 1, 1, 2>(st, ctx, ring, full, P, lane);
+    else if (nc == 1 && (it.flags & kFlagWriteLogits)) process_item_tc<D, 1, 1, 1>(st, ctx, ring, full, P, lane);
+    else if (nc == 1) process_item_tc<D, 1, 1>(st, ctx, ring, full, P, lane);
     else if (shared && nc == 2) process_item_tc<D, 1, 2>(st, ctx, ring, full, P, lane);
     else if (shared && nc == 3) process_item_tc<D, 1, 3>(st, ctx, ring, full, P, lane);
     else if (shared) process_item_tc<D, 1, 4>(st, ctx, ring, full, P, lane);

@@ -194,6 +194,7 @@ __device__ __forceinline__ bool issue_one(WorkerState& st, CtxFn ctx, uint32_t r
   if (st.dead || st.iss_k >= st.n_my || st.iss_k > st.cons_k + 1) return false;
   const ItemPages& c = ctx(st.iss_k);
   const int n_cons = c.item.n_cons;
+  if (st.iss_which == 0 && (c.item.flags & kFlagReadLogits)) st.iss_which = 1;   // scores come from the logit cache
   int pid = c.pages[st.iss_which][st.iss_page];
   if (static_cast<uint32_t>(pid) >= static_cast<uint64_t>(P.n_pool_pages)) {   // never read outside the pool
     if (lane == 0) atomicMax(P.err, kErrBadPage);
@@ -302,6 +303,13 @@ __device__ __forceinline__ int claim_issue(const Params& P, int lane) {
   if (lane == 0) idx = atomicAdd(P.work_counter + P.launch_index, 1);
   return idx;
 }
+// Where the scaled scores of (stream, sequence, head) start in the logit cache; key j of the stream
+// is element j.
+__device__ __forceinline__ float* logit_row(const Params& P, int stream, int seq_id, int head) {
+  return P.logits + ((static_cast<size_t>(stream) * P.max_seqs + seq_id) * P.hq + head) *
+                        (static_cast<size_t>(P.max_pages) * kPage);
+}
+
 // Turns the value returned by claim_issue into an item index, or -1 when the list is used up.
 __device__ __forceinline__ int claim_take(const Params& P, int issued) {
   const int idx = __shfl_sync(0xffffffffu, issued, 0);

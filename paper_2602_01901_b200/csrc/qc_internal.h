@@ -15,6 +15,8 @@ constexpr int kAttendWarps = 12;   // independent workers (warps) per attention 
 
 // flags of Job / Item
 constexpr uint8_t kFlagShared = 1;      // one query scores for every consumer (same weights)
+constexpr uint8_t kFlagWriteLogits = 2; // the sweep also stores its scaled scores in the logit cache
+constexpr uint8_t kFlagReadLogits = 4;  // the sweep takes its scores from the logit cache: no K tile is read
 constexpr int kFlagCachedShift = 4;     // bit (4 + x): consumer x's query is read from the Q Cache
 
 // layer flags
@@ -81,6 +83,7 @@ struct Params {
   uint16_t* qcache;        // bf16 [n_layers][max_seqs][hq][d]
   float* part_acc;         // [n_layers][max_seqs][max_slots][hq][d]
   float2* part_ml;         // [n_layers][max_seqs][max_slots][hq]  (max, sum) in the log2 domain
+  float* logits;           // [2 streams][max_seqs][hq][max_pages * 16] scaled scores (log2 domain) of a block's leader
   Item* items;
   const PlanJob* plan;
   const Job* jobs;

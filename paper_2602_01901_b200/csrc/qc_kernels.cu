@@ -197,7 +197,9 @@ __device__ __forceinline__ void load_ctx(WarpCtx<D>& c, const Params& P, int ite
 
 // One item: NQ queries score the K tiles, NV value streams are accumulated.
 // NQ == 1: every consumer shares the weights; NQ == NV: consumer x has its own query.
-template <int D, int NQ, int NV>
+// MODE 1 (one query, one consumer) also stores the scaled scores in the logit cache; MODE 2 takes
+// them from there instead of reading K tiles (the ring then carries V tiles only).
+template <int D, int NQ, int NV, int MODE = 0>
 __device__ __forceinline__ void process_item(WorkerState& st, const WarpCtx<D>* ctx, uint32_t ring, uint64_t* full,
                                              const Params& P, int lane) {
   auto ctx_of = [ctx](int k) -> const ItemPages& { return ctx[k & 1].ip; };
@@ -232,12 +234,29 @@ __device__ __forceinline__ void process_item(WorkerState& st, const WarpCtx<D>* 
 
   const int n_pages = c.ip.item.n_pages;
   const int n_valid_last = c.ip.item.n_valid_last;
+  float* lg = nullptr;      // this item's first key in the logit cache
+  float lg_next[4] = {0.f, 0.f, 0.f, 0.f};
+  if (MODE != 0) {
+    lg = logit_row(P, c.ip.item.stream, c.ip.item.seq_id, c.ip.item.head) + c.ip.item.first_page * kPage;
+    if (MODE == 2) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) lg_next[i] = lg[4 * i + kg];
+    }
+  }
 
   for (int pg = 0; pg < n_pages && !st.dead; ++pg) {
     const int nvalid = (pg == n_pages - 1) ? n_valid_last : kPage;
     float p[NQ][4];
-    // ---- K tile: scores of 16 keys
-    {
+    if (MODE == 2) {
+      // ---- scores of 16 keys from the logit cache; the next page's are requested now
+#pragma unroll
+      for (int i = 0; i < 4; ++i) p[0][i] = lg_next[i];
+      if (pg + 1 < n_pages) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) lg_next[i] = lg[(pg + 1) * kPage + 4 * i + kg];
+      }
+    } else {
+      // ---- K tile: scores of 16 keys
       const uint8_t* tile = static_cast<const uint8_t*>(__cvta_shared_to_generic(wait_tile<D>(st, ring, full, P, lane)));
       if (st.dead) break;
 #pragma unroll
@@ -266,9 +285,12 @@ __device__ __forceinline__ void process_item(WorkerState& st, const WarpCtx<D>* 
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         float s = p[x][i];
-        s += __shfl_xor_sync(0xffffffffu, s, 1);
-        s += __shfl_xor_sync(0xffffffffu, s, 2);
-        s += __shfl_xor_sync(0xffffffffu, s, 4);
+        if (MODE != 2) {
+          s += __shfl_xor_sync(0xffffffffu, s, 1);
+          s += __shfl_xor_sync(0xffffffffu, s, 2);
+          s += __shfl_xor_sync(0xffffffffu, s, 4);
+        }
+        if (MODE == 1 && c8 == 0 && 4 * i + kg < nvalid) lg[pg * kPage + 4 * i + kg] = s;
         p[x][i] = (4 * i + kg < nvalid) ? s : -INFINITY;
       }
       float tmax = fmaxf(fmaxf(p[x][0], p[x][1]), fmaxf(p[x][2], p[x][3]));
@@ -390,7 +412,9 @@ __global__ void __launch_bounds__(kThreads, 1) attend_kernel(const __grid_consta
     const bool shared = it.flags & kFlagShared;
     // claim the item after next now; the answer is needed only when this item is done
     const int issued = (next >= 0) ? claim_issue(P, lane) : 0;
-    if (nc == 1) process_item<D, 1, 1>(st, ctx, ring, full, P, lane);
+    if (nc == 1 && (it.flags & kFlagReadLogits)) process_item<D, 1, 1, 2>(st, ctx, ring, full, P, lane);
+    else if (nc == 1 && (it.flags & kFlagWriteLogits)) process_item<D, 1, 1, 1>(st, ctx, ring, full, P, lane);
+    else if (nc == 1) process_item<D, 1, 1>(st, ctx, ring, full, P, lane);
     else if (shared && nc == 2) process_item<D, 1, 2>(st, ctx, ring, full, P, lane);
     else if (shared && nc == 3) process_item<D, 1, 3>(st, ctx, ring, full, P, lane);
     else if (shared) process_item<D, 1, 4>(st, ctx, ring, full, P, lane);

@@ -34,7 +34,7 @@ struct LaunchGroup {
 };
 
 struct Layout {   // byte offsets into the workspace
-  size_t table, layer_flags, layer_kind, leader, jobs, plan, qcache, part_acc, part_ml, items, step, err, counters, stage_q, stage_k, stage_v,
+  size_t table, layer_flags, layer_kind, leader, jobs, plan, qcache, part_acc, part_ml, logits, items, step, err, counters, stage_q, stage_k, stage_v,
       stage_out, stage_lse, tok, total;
   size_t step_seqs, step_patches, step_bytes;   // offsets inside the step block
 };
@@ -89,6 +89,8 @@ struct qc_cache {
   std::vector<Job> jobs;
   std::vector<std::pair<int, int>> block_jobs;   // per lazy block: [job_begin, job_end)
   std::vector<std::pair<int, int>> block_layers; // per lazy block: [layer_begin, layer_end)
+  std::vector<Job> layer_jobs;                    // per-layer schedule (logit cache)
+  std::vector<std::pair<int, int>> layer_job_range;   // per layer: [job_begin, job_end) in layer_jobs
   int text_streams_per_seq = 0;        // pages a sequence needs when its text crosses a page
 
   // pinned staging ring for step descriptors
@@ -217,6 +219,45 @@ void build_jobs(const qc_config* cfg, std::vector<Job>& jobs, std::vector<std::p
   }
 }
 
+// Jobs of the per-layer schedule, layer by layer: every sweep feeds one layer.  A leader with
+// followers stores the scaled scores that its followers share (VLA_QC: of the visual keys; GLA: of
+// all keys) in the logit cache; such a follower sweeps its own V pages with those scores and reads
+// no K at all.  VLA_EQ8 followers score the leader's visual keys with their own query.
+void build_layer_jobs(const qc_config* cfg, std::vector<Job>& jobs, std::vector<std::pair<int, int>>& layer_jobs) {
+  const int N = cfg->n_layers;
+  int leader = 0;
+  for (int l = 0; l < N; ++l) {
+    const bool lazy = cfg->layer_kind[l] == QC_LAYER_LAZY;
+    if (!lazy) leader = l;
+    const bool has_followers = !lazy && l + 1 < N && cfg->layer_kind[l + 1] == QC_LAYER_LAZY;
+    const int job0 = static_cast<int>(jobs.size());
+    for (int stream = 1; stream >= 0; --stream) {
+      const bool shared_scores =
+          cfg->lazy_mode == QC_MODE_GLA || (cfg->lazy_mode == QC_MODE_VLA_QC && stream == 1);
+      Job j{};
+      j.stream = static_cast<uint8_t>(stream);
+      j.n_cons = 1;
+      j.flags = kFlagShared;
+      j.v_layer[0] = static_cast<uint8_t>(l);
+      j.q_layer[0] = static_cast<uint8_t>(l);
+      j.k_layer = static_cast<uint8_t>(l);
+      if (lazy) {
+        if (shared_scores) {
+          j.k_layer = static_cast<uint8_t>(leader);   // (lengths and chunking follow the leader's stream)
+          j.q_layer[0] = static_cast<uint8_t>(leader);
+          j.flags |= kFlagReadLogits;
+        } else if (stream == 1) {
+          j.k_layer = static_cast<uint8_t>(leader);   // Eq. 8: own query on the leader's visual keys
+        }
+      } else if (has_followers && shared_scores) {
+        j.flags |= kFlagWriteLogits;
+      }
+      jobs.push_back(j);
+    }
+    layer_jobs.emplace_back(job0, static_cast<int>(jobs.size()));
+  }
+}
+
 struct Sizes {
   int D, hq, hkv, max_pages, chunk_pages, max_slots;
   int64_t n_pool_pages;
@@ -245,8 +286,12 @@ int compute_sizes(const qc_config* cfg, Sizes* s) {
   std::vector<Job> jobs;
   std::vector<std::pair<int, int>> bj, bl;
   build_jobs(cfg, jobs, bj, bl);
+  std::vector<Job> layer_jobs;
+  std::vector<std::pair<int, int>> lj;
+  build_layer_jobs(cfg, layer_jobs, lj);
+  const size_t n_jobs = std::max(jobs.size(), layer_jobs.size());   // either schedule fits
   const size_t chunks_per_stream = (s->max_pages + s->chunk_pages - 1) / s->chunk_pages;
-  s->max_segs = jobs.size() * cfg->max_seqs;
+  s->max_segs = n_jobs * cfg->max_seqs;
   s->max_items = s->max_segs * chunks_per_stream * s->hq;
   s->max_patches = static_cast<size_t>(cfg->n_layers) * 2 * cfg->max_seqs;
 
@@ -262,11 +307,12 @@ int compute_sizes(const qc_config* cfg, Sizes* s) {
   L.layer_flags = take(N);
   L.layer_kind = take(N);
   L.leader = take(N);
-  L.jobs = take(jobs.size() * sizeof(Job));
-  L.plan = take(jobs.size() * sizeof(PlanJob));
+  L.jobs = take(n_jobs * sizeof(Job));
+  L.plan = take(n_jobs * sizeof(PlanJob));
   L.qcache = take(N * S * s->hq * s->D * 2);
   L.part_acc = take(N * S * s->max_slots * s->hq * s->D * sizeof(float));
   L.part_ml = take(N * S * s->max_slots * s->hq * sizeof(float2));
+  L.logits = take(2 * S * s->hq * static_cast<size_t>(s->max_pages) * kPage * sizeof(float));
   L.items = take(s->max_items * sizeof(Item));
   // step block: header-free arrays at fixed offsets
   L.step_seqs = 0;
@@ -298,6 +344,7 @@ Params base_params(const qc_cache* c) {
   p.qcache = reinterpret_cast<uint16_t*>(c->ws + c->lay.qcache);
   p.part_acc = reinterpret_cast<float*>(c->ws + c->lay.part_acc);
   p.part_ml = reinterpret_cast<float2*>(c->ws + c->lay.part_ml);
+  p.logits = reinterpret_cast<float*>(c->ws + c->lay.logits);
   p.items = reinterpret_cast<Item*>(c->ws + c->lay.items);
   p.plan = reinterpret_cast<const PlanJob*>(c->ws + c->lay.plan);
   p.jobs = reinterpret_cast<const Job*>(c->ws + c->lay.jobs);
@@ -412,27 +459,39 @@ int rebuild_plan(qc_cache* c, int per_launch) {
   c->plan.clear();
   c->plan_vis_before.assign(1, 0);
   c->plan_text_before.assign(1, 0);
-  const int nb = static_cast<int>(c->block_jobs.size());
-  const int per = per_launch <= 0 ? nb : per_launch;
+  // per_launch < 0: the per-layer schedule (one launch per layer, logit cache); otherwise launches
+  // of `per_launch` lazy blocks (0 = all blocks in one launch)
+  const bool per_layer = per_launch < 0;
+  const std::vector<Job>& jobs = per_layer ? c->layer_jobs : c->jobs;
+  const int nb = static_cast<int>(per_layer ? c->layer_job_range.size() : c->block_jobs.size());
+  const int per = per_layer ? 1 : (per_launch == 0 ? nb : per_launch);
+  c->n_visual_jobs = c->n_text_jobs = 0;
+  c->visual_row_reads = c->text_row_reads = 0;
+  for (const Job& j : jobs) {
+    (j.stream ? c->n_visual_jobs : c->n_text_jobs)++;
+    (j.stream ? c->visual_row_reads : c->text_row_reads) += ((j.flags & kFlagReadLogits) ? 0 : 1) + j.n_cons;
+  }
   std::vector<int> order;
   for (int b = 0; b < nb; b += per) {
     const int e = std::min(nb, b + per);
-    const LaunchGroup g{c->block_jobs[b].first, c->block_jobs[e - 1].second, c->block_layers[b].first,
-                        c->block_layers[e - 1].second};
+    const LaunchGroup g = per_layer
+                              ? LaunchGroup{c->layer_job_range[b].first, c->layer_job_range[b].second, b, b + 1}
+                              : LaunchGroup{c->block_jobs[b].first, c->block_jobs[e - 1].second,
+                                            c->block_layers[b].first, c->block_layers[e - 1].second};
     c->groups.push_back(g);
     order.resize(g.job_end - g.job_begin);
     for (int j = g.job_begin; j < g.job_end; ++j) order[j - g.job_begin] = j;
     std::stable_sort(order.begin(), order.end(), [&](int x, int y) {
-      const Job &jx = c->jobs[x], &jy = c->jobs[y];
+      const Job &jx = jobs[x], &jy = jobs[y];
       if (jx.n_cons != jy.n_cons) return jx.n_cons > jy.n_cons;
       return jx.stream > jy.stream;
     });
     const int begin = static_cast<int>(c->plan.size());
     for (int j : order) {
       const int vb = c->plan_vis_before.back(), tb = c->plan_text_before.back();
-      c->plan.push_back(PlanJob{c->jobs[j], vb, tb, 0, 0});
-      c->plan_vis_before.push_back(vb + (c->jobs[j].stream ? 1 : 0));
-      c->plan_text_before.push_back(tb + (c->jobs[j].stream ? 0 : 1));
+      c->plan.push_back(PlanJob{jobs[j], vb, tb, 0, 0});
+      c->plan_vis_before.push_back(vb + (jobs[j].stream ? 1 : 0));
+      c->plan_text_before.push_back(tb + (jobs[j].stream ? 0 : 1));
     }
     c->group_pos.emplace_back(begin, static_cast<int>(c->plan.size()));
   }
@@ -554,10 +613,7 @@ int32_t qc_alloc_cache(qc_ctx* ctx, const qc_config* cfg, void* pool_dev, size_t
     c->text_streams_per_seq += 1 + (owns(c, l, QC_STREAM_K_TEXT) ? 1 : 0);
   }
   build_jobs(&c->cfg, c->jobs, c->block_jobs, c->block_layers);
-  for (const Job& j : c->jobs) {
-    (j.stream ? c->n_visual_jobs : c->n_text_jobs)++;
-    (j.stream ? c->visual_row_reads : c->text_row_reads) += 1 + j.n_cons;
-  }
+  build_layer_jobs(&c->cfg, c->layer_jobs, c->layer_job_range);
   c->seqs.resize(cfg->max_seqs);
   c->table.assign(static_cast<size_t>(cfg->n_layers) * 4 * cfg->max_seqs * c->max_pages, -1);
   if (c->paged) {
@@ -1227,6 +1283,11 @@ int32_t qc_set_option(qc_cache* c, const char* key, int64_t value) {
   if (k == "layers_per_launch") {
     if (value < 0 || value > c->cfg.n_layers) return QC_ERR_INVALID_ARG;
     c->layers_per_launch = static_cast<int>(value);
+    c->plan_dirty = true;
+    return QC_OK;
+  }
+  if (k == "per_layer_logit_cache") {   // one launch per layer; followers take shared scores from the logit cache
+    c->layers_per_launch = value ? -1 : 0;
     c->plan_dirty = true;
     return QC_OK;
   }

@@ -74,6 +74,10 @@ def test_tiny_every_step(mode):
     s.close()
 
 
+def _dev(a, device):
+    return torch.from_numpy(a.astype(np.int16)).view(torch.bfloat16).to(device).contiguous()
+
+
 # ------------------------------------------------------------------------------------------
 # small paged case: ragged batch, GQA, several lazy-block shapes, split sizes, D in {64, 128}
 # ------------------------------------------------------------------------------------------
@@ -189,6 +193,53 @@ def test_launch_grouping_and_host_entry_give_identical_bits():
         s.close()
     assert np.array_equal(results[0], results[1])
     assert np.array_equal(results[0], results[2])
+
+
+@pytest.mark.parametrize("mode", MODES, ids=MODE_IDS)
+@pytest.mark.parametrize("case", [0, 1, 4, 5, 6])
+def test_per_layer_schedule_with_logit_cache(mode, case):
+    """One launch per layer, in layer order; a leader stores the scores its followers share and
+    the followers read them instead of the leader's K.  By Eq. 6 (GLA) and the Q Cache rule (VLA_QC)
+    those scores ARE the follower's, so the outputs must equal the fused schedule's bit for bit at
+    the same split, and the oracle's within tolerance.  Ragged batch: a sequence without visual
+    tokens, different lengths, pages that fill up during the steps."""
+    head_dim, group, layer_kind, split = SMALL[case]
+    w = _small_workload(head_dim, group, layer_kind, 40 + case)
+    trunc = [w.n_prompt, 9, 70]
+    seq_ids = [2, 0, 3]
+    o = LazyAttentionOracle(w.n_layers, w.n_q_heads, w.n_kv_heads, head_dim, layer_kind, mode, n_seqs=3)
+    sessions = []
+    for per_layer in (False, True):
+        s = Session(w.n_layers, w.n_q_heads, w.n_kv_heads, head_dim, layer_kind, max_seqs=4, max_tokens_per_seq=256,
+                    n_pages=w.n_layers * 4 * 3 * 17, lazy_mode=mode, split_tokens=split, poison_pool=True)
+        if per_layer:
+            s.set_option("per_layer_logit_cache", 1)
+        sessions.append(s)
+    for b, sid in enumerate(seq_ids):
+        kind, k, v = W.prefill_kv_np(w, b)
+        T = trunc[b]
+        kind, k, v = kind[:T].copy(), k[:, :T], v[:, :T]
+        if b == 1:
+            kind[:] = 0
+        for s in sessions:
+            s.prefill_append([sid], [T], kind, _dev(k, s.device), _dev(v, s.device))
+        o.prefill_append(b, kind.tolist(), f64(k), f64(v))
+    outs = [torch.empty((w.n_layers, 3, w.n_q_heads, head_dim), dtype=torch.bfloat16, device=s.device) for s in sessions]
+    lses = [torch.empty((w.n_layers, 3, w.n_q_heads), dtype=torch.float32, device=s.device) for s in sessions]
+    for step in range(w.decode_steps):
+        qn, kn, vn = W.decode_qkv_np(w, step)
+        for s, out, lse in zip(sessions, outs, lses):
+            s.decode_step(seq_ids, _dev(qn, s.device), _dev(kn, s.device), _dev(vn, s.device), out, lse)
+        assert torch.equal(outs[0].view(torch.int16), outs[1].view(torch.int16)), f"step {step}: schedules differ"
+        assert torch.equal(lses[0], lses[1]), f"step {step}: log-sum-exp differs"
+        got = bits_of(outs[1])
+        for b in range(3):
+            ref, _ = o.decode_step(b, f64(qn[:, b]), f64(kn[:, b]), f64(vn[:, b]))
+            for l in range(w.n_layers):
+                assert_close(got[l, b], ref[l], f"per-layer schedule: case {case} step {step} seq {b} layer {l}")
+    for s in sessions:
+        assert s.stats().device_error == 0
+        s.close()
 
 
 def test_split_size_changes_only_rounding():
