@@ -249,30 +249,41 @@ def run_gpu(args, w, mode, rank, world, local_rank):
         all_full = {"ms_per_step": ms_full / K, "tokens_per_s": w.batch * K / (ms_full / 1e3),
                     "kv_bytes_stored": st_full.kv_bytes_stored, "speedup_of_lazy": ms_full / ms,
                     "note": "same inputs and steps, every layer ordinary (Eq. 2 only)"}
-    # ---- arm 1c (one GPU only): the same steps with one attention launch per lazy block, in layer
-    # order: the schedule of a model that computes a layer's q/k/v from the previous layer's output
-    per_block = None
-    if world == 1 and not args.no_per_block and not args.blocks_per_launch:
-        s = Session.for_workload(w, lazy_mode=mode, device=local_rank, split_tokens=args.split_tokens)
-        s.prefill_workload(w, seq_offset)
-        s.set_option("layers_per_launch", 1)
+    # ---- arms 1c, 1d (one GPU only): the same steps under the two schedules that issue layers in order.
+    # per_block: one attention + merge launch per lazy block (needs a block's q/k/v at once).
+    # per_layer: one launch pair per layer, followers reading the leader's scores from the logit
+    # cache: the schedule of a model in which a layer's q/k/v only exist after the previous layer.
+    def ordered_arm(option, value, note):
+        s2 = Session.for_workload(w, lazy_mode=mode, device=local_rank, split_tokens=args.split_tokens)
+        s2.prefill_workload(w, seq_offset)
+        s2.set_option(option, value)
         for i in range(W_):
-            s.decode_step(ids, *inputs[i], out)
+            s2.decode_step(ids, *inputs[i], out)
+        s2.set_option("profile", 1)
         torch.cuda.synchronize()
-        launches0 = s.stats().kernel_launches
+        launches0 = s2.stats().kernel_launches
         f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         f0.record()
         for i in range(W_, total_steps):
-            s.decode_step(ids, *inputs[i], out)
+            s2.decode_step(ids, *inputs[i], out)
         f1.record()
         torch.cuda.synchronize()
-        ms_pb = f0.elapsed_time(f1)
-        per_block = {"ms_per_step": ms_pb / K, "tokens_per_s": w.batch * K / (ms_pb / 1e3),
-                     "gpu_launches": int(s.stats().kernel_launches - launches0),
-                     "kv_gb_per_s_whole_step": prof.kv_bytes_read / (ms_pb / 1e3) / 1e9,
-                     "note": "one attention + merge launch per lazy block, blocks in layer order"}
-        s.close()
-        del s
+        ms2 = f0.elapsed_time(f1)
+        prof2 = s2.profile()
+        res = {"ms_per_step": ms2 / K, "tokens_per_s": w.batch * K / (ms2 / 1e3),
+               "gpu_launches": int(s2.stats().kernel_launches - launches0),
+               "kv_gb_per_s_whole_step": prof2.kv_bytes_read / (ms2 / 1e3) / 1e9,
+               "kv_bytes_read_per_step": prof2.kv_bytes_read / max(1, prof2.steps), "note": note}
+        s2.close()
+        return res
+
+    per_block = per_layer = None
+    if world == 1 and not args.no_per_block and not args.blocks_per_launch:
+        per_block = ordered_arm("layers_per_launch", 1,
+                                "one attention + merge launch per lazy block, blocks in layer order")
+        per_layer = ordered_arm("per_layer_logit_cache", 1,
+                                "one attention + merge launch per layer, layers in order; followers take the "
+                                "leader's scores from the logit cache instead of reading its K")
     del inputs
     torch.cuda.empty_cache()
 
@@ -338,6 +349,7 @@ def run_gpu(args, w, mode, rank, world, local_rank):
         },
         "vs_all_full": all_full,
         "per_block_launches": per_block,
+        "per_layer_launches": per_layer,
         "step_ms_by_events": prof.step_ms / max(1, prof.steps),
         "paper_context": "paper reports ~35% KV saved and 1.5x-1.6x decode throughput for LLaVA-NeXT-7B on one 80GB A100 (whole model)",
     }

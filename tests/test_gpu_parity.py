@@ -431,17 +431,25 @@ FULL_CASES = [
     ("long_video_pruned", qc.QC_MODE_VLA_QC, 24),
     ("llava_next_2048_lazy22", qc.QC_MODE_VLA_QC, 24),     # blocks of one ordinary + three lazy layers
     ("llava_next_2048_lazy22", qc.QC_MODE_GLA, 16),
+    # the per-layer schedule with the logit cache (the configuration bench.py times as per_layer_launches)
+    ("llava15_7b", qc.QC_MODE_VLA_QC, 16, "per_layer"),
+    ("qwen2vl_gqa", qc.QC_MODE_VLA_QC, 16, "per_layer"),
+    ("llava_next_2048_lazy22", qc.QC_MODE_GLA, 16, "per_layer"),
 ]
 
 
-@pytest.mark.parametrize("name,mode,n_samples", FULL_CASES, ids=[f"{c[0]}-{MODE_IDS[c[1]]}" for c in FULL_CASES])
-def test_full_size_sampled(name, mode, n_samples):
+@pytest.mark.parametrize("case", FULL_CASES, ids=["-".join([c[0], MODE_IDS[c[1]]] + list(c[3:])) for c in FULL_CASES])
+def test_full_size_sampled(case):
+    name, mode, n_samples = case[:3]
+    per_layer = len(case) > 3
     w = W.get_workload(name)
     rng = np.random.default_rng(w.seed)
     samples = _samples(w, n_samples, rng)
     oracles = [SampledOracle(w, mode, *t) for t in samples]
     schedule = set(step_schedule(w.decode_steps))
     s = Session.for_workload(w, lazy_mode=mode)
+    if per_layer:
+        s.set_option("per_layer_logit_cache", 1)
     s.prefill_workload(w)
     model = pg.PagedCacheModel(w.layer_kind().tolist(), mode, 16, s.cfg.n_pages, w.batch)
     for b in range(w.batch):
