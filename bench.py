@@ -34,7 +34,7 @@ MODES = {"vla_qc": 0, "vla_eq8": 1, "gla": 2}
 # from the ncu captures of small cases summarised in profiles/attend_kernels_small_cases_ncu_full.md.
 # Traffic grows in proportion to the K/V bytes swept (every tile is fetched once; partial results are
 # written once per chunk), so a full launch's traffic is this ratio times its algorithmic bytes.
-NCU_TRAFFIC_RATIO = {"attend_kernel": 1.069, "attend_tc_kernel": 1.077}
+NCU_TRAFFIC_RATIO = {"attend_kernel": 1.069, "attend_tc_kernel": 1.070}
 
 
 def _peaks():
@@ -202,6 +202,8 @@ def run_gpu(args, w, mode, rank, world, local_rank):
     s.prefill_workload(w, seq_offset)
     if args.blocks_per_launch:
         s.set_option("layers_per_launch", args.blocks_per_launch)
+    if args.per_layer:
+        s.set_option("per_layer_logit_cache", 1)
     inputs = _gen_inputs(w, 0, total_steps, dev, seq_offset)
     out = torch.empty(shape_o, dtype=torch.bfloat16, device=dev)
     for i in range(W_):
@@ -278,7 +280,7 @@ def run_gpu(args, w, mode, rank, world, local_rank):
         return res
 
     per_block = per_layer = None
-    if world == 1 and not args.no_per_block and not args.blocks_per_launch:
+    if world == 1 and not args.no_per_block and not args.blocks_per_launch and not args.per_layer:
         per_block = ordered_arm("layers_per_launch", 1,
                                 "one attention + merge launch per lazy block, blocks in layer order")
         per_layer = ordered_arm("per_layer_logit_cache", 1,
@@ -420,7 +422,10 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=64)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-all-full", action="store_true", help="skip the all-ordinary-layers comparison run")
-    ap.add_argument("--no-per-block", action="store_true", help="skip the launch-per-lazy-block comparison run")
+    ap.add_argument("--no-per-block", action="store_true",
+                    help="skip the comparison runs with one launch per lazy block / per layer")
+    ap.add_argument("--per-layer", action="store_true",
+                    help="run the main arm under the per-layer schedule with the logit cache (for profiling it)")
     ap.add_argument("--dist-backend", default=None, help="torch.distributed backend (default: nccl on GPUs)")
     ap.add_argument("--force-device", type=int, default=-1,
                     help="use this CUDA device on every rank (to exercise the multi-rank plumbing on one GPU)")
