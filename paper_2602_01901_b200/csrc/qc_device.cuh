@@ -153,7 +153,8 @@ __device__ __forceinline__ size_t table_row(const Params& P, int layer, int stre
 //
 // A warp owns RING tile slots in shared memory and one mbarrier per slot.  Lane 0 issues the
 // copies of the K tile and the V tiles of each page of the warp's current item (and of the
-// next one, so the ring never drains at an item boundary); all lanes wait on a slot's
+// next one, so the ring never drains at an item boundary; an item that takes its scores from
+// the logit cache has no K tiles); all lanes wait on a slot's
 // barrier before reading it.  Every wait is bounded: when it runs out the worker records the
 // error, stops fetching, lets the copies in flight land (again bounded) and leaves.
 

@@ -9,7 +9,9 @@
 //   attend_kernel   persistent split-KV partial attention, one query head per work item (MHA):
 //                   each warp is an independent worker that claims items from a counter, streams
 //                   K/V page tiles through its own shared-memory ring with bulk asynchronous
-//                   copies and keeps an online softmax in registers
+//                   copies and keeps an online softmax in registers; under the per-layer
+//                   schedule a leader's sweep also stores its scaled scores in the logit cache
+//                   and a follower's sweep reads them there instead of any K tile
 //                   (the grouped-query variant on tensor cores is in qc_attend_tc.cu)
 //   merge_kernel    log-sum-exp merge of the partials, bf16 output
 //   prefill_scatter_kernel  stores prompt K/V rows into their pages
