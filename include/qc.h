@@ -105,7 +105,10 @@ typedef struct qc_stats {
 /* Per-step kernel timing (CUDA events on the library's stream), for roofline accounting. */
 typedef struct qc_profile {
   int64_t steps;              /* decode steps covered */
-  double attend_ms;           /* summed duration of the attention (split-KV partial) kernel */
+  double attend_ms;           /* summed duration of the attention (split-KV partial) kernel; when a
+                                 step runs as several launches, from the start of its first
+                                 attention launch to the end of its last (merges between them
+                                 included) */
   double step_ms;             /* summed duration of whole steps (setup+append+attend+merge) */
   int64_t kv_bytes_read;      /* algorithmic K/V bytes those steps had to read: every stored
                                  row of the listed sequences once, per step */
@@ -121,7 +124,8 @@ typedef struct qc_profile {
 int32_t qc_init(int32_t device, void* cuda_stream, qc_ctx** out);
 
 /* Bytes the caller must provide for a cache of this configuration.  pool_bytes covers the
- * K/V pages, workspace_bytes the page tables, Q Cache, split-KV partials, plans and staging. */
+ * K/V pages, workspace_bytes the page tables, Q Cache, split-KV partials, logit cache, plans and
+ * staging. */
 int32_t qc_cache_bytes_required(const qc_config* cfg, size_t* pool_bytes, size_t* workspace_bytes);
 
 /* Build a cache over caller-owned device memory (both 256-byte aligned).  Page layout: one
