@@ -171,16 +171,18 @@ def _compare_tables(s, model, n_layers, seq_ids):
 def test_launch_grouping_and_host_entry_give_identical_bits():
     w = _small_workload(128, 1, [0, 1, 0, 0, 1, 1], 20)
     results = []
-    for variant in ("one_launch", "per_block", "host_buffers"):
+    for variant in ("one_launch", "per_block", "host_buffers", "per_layer", "per_layer_set_then_host_buffers"):
         s = Session.for_workload(w, lazy_mode=qc.QC_MODE_VLA_QC, split_tokens=64)
         s.prefill_workload(w)
         if variant == "per_block":
             s.set_option("layers_per_launch", 1)
+        if variant.startswith("per_layer"):
+            s.set_option("per_layer_logit_cache", 1)   # (the host-buffer entry point keeps its own launch groups)
         out, lse = _outputs(w, s.device)
         outs = []
         for step in range(6):
             q, k, v = W.decode_qkv_torch(w, step, s.device)
-            if variant == "host_buffers":
+            if variant.endswith("host_buffers"):
                 hq, hk, hv = q.cpu().pin_memory(), k.cpu().pin_memory(), v.cpu().pin_memory()
                 ho = torch.empty(out.shape, dtype=torch.bfloat16).pin_memory()
                 s.decode_step_host(list(range(w.batch)), hq, hk, hv, ho)
@@ -191,8 +193,8 @@ def test_launch_grouping_and_host_entry_give_identical_bits():
         assert s.stats().device_error == 0
         results.append(np.stack(outs))
         s.close()
-    assert np.array_equal(results[0], results[1])
-    assert np.array_equal(results[0], results[2])
+    for other in results[1:]:
+        assert np.array_equal(results[0], other)
 
 
 @pytest.mark.parametrize("mode", MODES, ids=MODE_IDS)
