@@ -958,7 +958,11 @@ int decode_step_core(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, const 
     // Larger chunks mean fewer partial results to write and merge; smaller chunks mean more
     // work items to balance over the workers.  Take the largest chunk that still leaves
     // every worker several items per launch.
-    const int64_t want = 5LL * c->ctx->n_sms * kAttendWarps * static_cast<int64_t>(c->groups.size());
+    // (one launch per layer: a launch is short, so its partial rows and their merge weigh more than
+    // the balance of its tail -- one and a half items per worker measured best, against five)
+    const int64_t twice_per_worker = c->plan_per < 0 ? 3 : 10;
+    const int64_t want =
+        twice_per_worker * c->ctx->n_sms * kAttendWarps * static_cast<int64_t>(c->groups.size()) / 2;
     // (a query group writes one partial row per head and chunk: its chunks stay at 128 keys or more)
     const int floor_pages = c->group > 1 ? std::max(c->min_chunk_pages, 8) : c->min_chunk_pages;
     int pick = floor_pages;
