@@ -377,7 +377,25 @@ def run_prefill(args, w, mode, local_rank):
     out = torch.empty_like(prompts[0][1])
     from paper_2602_01901_b200 import binding as qc
 
-    s.prefill_attend(0, *prompts[0], out)          # warm-up on sequence 0, then release it
+    n_chunks = max(1, args.prefill_chunks)
+    T = len(prompts[0][0])
+    cuts = [T * i // n_chunks for i in range(n_chunks + 1)]
+
+    chunks = None
+    if n_chunks > 1:   # a chunk's tensors must be dense: materialise them before the timed region
+        chunks = []
+        for kind, q, k, v in prompts:
+            chunks.append([(kind[a:e], q[:, a:e].contiguous(), k[:, a:e].contiguous(), v[:, a:e].contiguous(),
+                            torch.empty_like(q[:, a:e].contiguous())) for a, e in zip(cuts[:-1], cuts[1:])])
+
+    def prefill(b):   # the prompt in one call, or as consecutive chunks (later ones see the cached tokens)
+        if n_chunks == 1:
+            s.prefill_attend(b, *prompts[b], out)
+            return
+        for kind_c, q_c, k_c, v_c, out_c in chunks[b]:
+            s.prefill_attend(b, kind_c, q_c, k_c, v_c, out_c)
+
+    prefill(0)          # warm-up on sequence 0, then release it
     qc.qc_free_seq(s.cache, 0)
     s.set_option("profile", 1)
     torch.cuda.synchronize()
@@ -385,21 +403,20 @@ def run_prefill(args, w, mode, local_rank):
     with ClockSampler(_physical_gpu_index(local_rank)) as clocks:
         e0.record()
         for b in range(n_seqs):
-            s.prefill_attend(b, *prompts[b], out)
+            prefill(b)
         e1.record()
         torch.cuda.synchronize()
     ms = e0.elapsed_time(e1)
     prof = s.profile()
     st = s.stats()
     s.close()
-    T = len(prompts[0][0])
     with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
         peak = float(json.load(f)["bf16_tflops"])
     achieved = prof.prefill_flops / (prof.prefill_attend_ms / 1e3) / 1e12
     return {
         "metric": "prefill_attention_tokens_per_s", "value": n_seqs * T / (ms / 1e3), "unit": UNIT, "n_gpus": 1,
         "steps": n_seqs, "warmup": 1, "ms_per_step": ms / n_seqs, "higher_is_better": True, "dtype": "bf16",
-        "data": "synthetic", "config": {"workload": w.name, "mode": args.mode, "prompt_tokens": T,
+        "data": "synthetic", "config": {"workload": w.name, "mode": args.mode, "prompt_tokens": T, "prompt_chunks": n_chunks,
                                         "n_layers": w.n_layers, "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads},
         "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                      "frac": achieved / peak, "traffic": None,
@@ -431,6 +448,8 @@ def main():
                     help="use this CUDA device on every rank (to exercise the multi-rank plumbing on one GPU)")
     ap.add_argument("--phase", default="decode", choices=["decode", "prefill"],
                     help="decode (the benchmark) or prefill (secondary: qc_prefill_attend over the prompts)")
+    ap.add_argument("--prefill-chunks", type=int, default=1,
+                    help="prefill phase: give each prompt as this many consecutive calls (chunked prefill)")
     ap.add_argument("--prefill-kernel", default="tcgen05", choices=["tcgen05", "mma"],
                     help="prefill phase, head_dim 128: tcgen05 kernel (default) or the mma.sync kernel")
     ap.add_argument("--split-tokens", type=int, default=0, help="keys per split-KV work item (0 = library default)")

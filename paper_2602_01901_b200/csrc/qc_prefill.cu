@@ -39,6 +39,8 @@ struct PrefillArgs {
   // tcgen05 kernel: q / k / v as 3-D tensors {D, heads, n_layers * T}, box {64, 1, 64}; the output as a
   // 4-D tensor {D, hq, T, n_layers}, box {64, 1, 128, 1}; 128-byte swizzle
   CUtensorMap tmap_q, tmap_k, tmap_v, tmap_o;
+  CUtensorMap tmap_pool;   // the paged pool as a 2-D tensor [pages * hkv * 16 rows][D], box 16 rows x 64 elements
+  int64_t n_pool_pages;    // bound for page ids read from the table
   const uint8_t* tile_code;    // [ceil(T / 64)] device: 0 = the 64-token tile is all text, 1 = all visual, 2 = mixed
   const uint16_t* q;     // [n_layers][T][hq][D]
   const uint16_t* k;     // [n_layers][T][hkv][D]
@@ -49,8 +51,8 @@ struct PrefillArgs {
   const uint8_t* leader;       // [n_layers] device
   int32_t T, hq, hkv, group, n_layers, gla;
   float scale_log2;
-  // tokens the sequence already held before this prompt chunk (mma.sync kernel only): they are
-  // read from the paged cache, text stream then visual stream, and are visible to every new token
+  // tokens the sequence already held before this prompt chunk: they are read from the paged cache,
+  // text stream then visual stream, and are visible to every new token
   const uint16_t* pool;
   const int32_t* table;        // [n_layers][4][max_seqs][max_pages]
   const uint8_t* layer_flags;  // kLayerOwnsTextK: the layer's text K is its own
@@ -508,7 +510,12 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
   const bool gla = A.gla != 0;
   const int m0 = qt * kTM;
   const int row = m0 + threadIdx.x;                 // a softmax thread's query row
-  const int n_ktiles = min((A.T + kTN - 1) / kTN, (m0 + kTM + kTN - 1) / kTN);
+  // Key tiles, in order: the cached text tokens, the cached visual tokens (all visible, read from
+  // the pool: a lazy layer's visual K -- and in GLA its text K -- are its leader's pages, which is
+  // Eq. 5 / Eq. 7's selection for tokens already cached), then the new tokens (causal).
+  const int ct_text = (A.n0_text + kTN - 1) / kTN, ct_vis = (A.n0_vis + kTN - 1) / kTN;
+  const int n_cached = ct_text + ct_vis;
+  const int n_ktiles = n_cached + min((A.T + kTN - 1) / kTN, (m0 + kTM + kTN - 1) / kTN);
 
   if (threadIdx.x == 0) {
     mbar_init(&bar_s[0], 1);
@@ -556,7 +563,96 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
       const uint32_t c = kt < 32 ? codes[0] : (kt < 64 ? codes[1] : codes[2]);
       return static_cast<int>(__shfl_sync(0xffffffffu, c, kt & 31));
     };
+    const int k_text_layer = (A.n0_text && !(A.layer_flags[layer] & kLayerOwnsTextK)) ? lead : layer;
+    // Where cached tile kt of the key (which = 1) or value (which = 2) sequence lives: source layer,
+    // stream, first token and the stream's length.
+    auto cached_tile = [&](int which, int kt, int& src, int& stream, int& ord0, int& n_valid) {
+      if (kt < ct_text) {
+        src = which == 1 ? k_text_layer : layer, stream = which == 1 ? 0 : 2, ord0 = kt * kTN, n_valid = A.n0_text;
+      } else {
+        src = which == 1 ? (lazy ? lead : layer) : layer, stream = which == 1 ? 1 : 3;
+        ord0 = (kt - ct_text) * kTN, n_valid = A.n0_vis;
+      }
+    };
+    // Lanes 0..3 read the page ids of a cached tile's four pages (0 where the page holds no token).
+    auto load_page_ids = [&](int which, int kt) -> int {
+      int src, stream, ord0, n_valid, pid = 0;
+      cached_tile(which, kt, src, stream, ord0, n_valid);
+      if (lane < 4 && ord0 + 16 * lane < n_valid) {
+        const size_t trow = ((static_cast<size_t>(src) * 4 + stream) * A.max_seqs + A.seq_id) * A.max_pages;
+        pid = A.table[trow + ord0 / 16 + lane];
+      }
+      return pid;
+    };
+    // Fetch cached tile kt: 64 tokens of one stream of (source layer, this sequence) from the paged
+    // pool, as four pages.  A page that is full arrives by two tensor-map copies; the rows of a
+    // page that is not (the stream's last page, or pages past its end) are gathered or zeroed by
+    // the lanes, since their pool rows may hold anything and a zero weight does not cancel a NaN.
+    int ahead_tile[2] = {-1, -1}, ahead_pid[2] = {0, 0};   // page ids requested one tile ahead, per which
+    auto fetch_cached = [&](int which, int kt, uint32_t dst, uint32_t half, uint64_t* bar) {
+      int src, stream, ord0, n_valid;
+      cached_tile(which, kt, src, stream, ord0, n_valid);
+      int pid = ahead_tile[which - 1] == kt ? ahead_pid[which - 1] : load_page_ids(which, kt);
+      if (kt + 1 < n_cached) {   // the next tile's ids travel while this tile is fetched and consumed
+        ahead_tile[which - 1] = kt + 1;
+        ahead_pid[which - 1] = load_page_ids(which, kt + 1);
+      }
+      if (static_cast<uint32_t>(pid) >= static_cast<uint64_t>(A.n_pool_pages)) {   // never read outside the pool
+        atomicMax(err, kErrBadPage);
+        pid = 0;
+      }
+      int n_full = 0;
+      bool gathered = false;
+#pragma unroll
+      for (int pg = 0; pg < 4; ++pg) {
+        const int p_id = __shfl_sync(0xffffffffu, pid, pg);
+        const int n_tok = min(16, max(0, n_valid - (ord0 + 16 * pg)));
+        if (n_tok == 16) {
+          ++n_full;
+          continue;
+        }
+        gathered = true;
+        for (int e = lane; e < 16 * (kTD / 8); e += 32) {
+          const int r = 16 * pg + (e >> 4), c = e & 15;
+          const uint32_t d = dst + (c >> 3) * half + r * 128 + (((c & 7) ^ (r & 7)) << 4);
+          if ((e >> 4) < n_tok) {
+            cp_async16(d, A.pool + ((static_cast<size_t>(p_id) * A.hkv + kvh) * 16 + (e >> 4)) * kTD + c * 8);
+          } else {
+            asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(d), "r"(0u) : "memory");
+          }
+        }
+      }
+      if (gathered) {
+        cp_async_commit();
+        cp_async_wait<0>();
+        fence_proxy_async();
+        __syncwarp();
+      }
+      if (n_full == 0) {
+        if (lane == 0) mbar_arrive(bar);
+        return;
+      }
+      if (lane == 0) mbar_expect_tx(bar, n_full * 4096);
+#pragma unroll
+      for (int pg = 0; pg < 4; ++pg) {
+        const int p_id = __shfl_sync(0xffffffffu, pid, pg);
+        if (n_valid - (ord0 + 16 * pg) >= 16 && lane == 0) {
+          const int32_t row = (p_id * A.hkv + kvh) * 16;
+          tensor_g2s_2d(dst + pg * 2048, &A.tmap_pool, 0, row, bar);
+          tensor_g2s_2d(dst + half + pg * 2048, &A.tmap_pool, 64, row, bar);
+        }
+      }
+    };
+    // `which`: 0 = 64 query rows (kt counts 64-row tiles of the prompt), 1 = key tile kt, 2 = value
+    // tile kt of the CTA's tile sequence (cached tiles first).
     auto fetch_tile = [&](int which, int kt, uint32_t dst, uint32_t half, uint64_t* bar) {
+      if (which != 0) {
+        if (kt < n_cached) {
+          fetch_cached(which, kt, dst, half, bar);
+          return;
+        }
+        kt -= n_cached;   // a tile of new tokens
+      }
       int src = layer;
       bool mixed = false;
       if (which != 2 && lazy && kt * kTN < A.T) {   // queries and keys of a lazy layer: the leader's for visual rows
@@ -712,8 +808,16 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
 #pragma unroll
         for (int j = 0; j < 32; ++j) p[j] = __uint_as_float(r0[j]), p[32 + j] = __uint_as_float(r1[j]);
       }
-      const int n0 = kt * kTN;
-      if (n0 + kTN - 1 > m0 || n0 + kTN > A.T) {   // only tiles on the diagonal or at the end of the prompt need the mask
+      if (kt < n_cached) {   // cached tokens: all visible; only a stream's last tile is short
+        const int n_show = kt < ct_text ? A.n0_text - kt * kTN : A.n0_vis - (kt - ct_text) * kTN;
+        if (n_show < kTN) {
+#pragma unroll
+          for (int j = 0; j < kTN; ++j)
+            if (j >= n_show) p[j] = -INFINITY;
+        }
+      }
+      const int n0 = (kt - n_cached) * kTN;
+      if (kt >= n_cached && (n0 + kTN - 1 > m0 || n0 + kTN > A.T)) {   // only tiles on the diagonal or at the end of the prompt need the mask
 #pragma unroll
         for (int j = 0; j < kTN; ++j) {
           const int key = n0 + j;
@@ -862,7 +966,9 @@ cudaError_t launch_prefill_attend(const Params& p, const uint8_t* kind_dev, cons
   a.seq_id = seq_id;
   a.n0_text = n0_text;
   a.n0_vis = n0_vis;
-  if (p.d == kTD && maps && n0_text + n0_vis == 0) {
+  if (p.d == kTD && maps) {
+    a.tmap_pool = p.tmap;
+    a.n_pool_pages = p.n_pool_pages;
     a.tmap_q = maps->q;
     a.tmap_k = maps->k;
     a.tmap_v = maps->v;

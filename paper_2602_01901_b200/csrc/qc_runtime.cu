@@ -74,6 +74,7 @@ struct qc_cache {
   cudaStream_t copy_in = nullptr, copy_out = nullptr;
   std::vector<cudaEvent_t> ev_in, ev_done;
   bool prefill_tcgen05 = true;    // head_dim 128: tcgen05 kernel; otherwise (or when switched off) mma.sync kernel
+  bool pool_map_ok = false;       // c->tmap was encoded
   int64_t n_pool_pages = 0;
   int layers_per_launch = 0;
   float scale = 0.f;
@@ -624,7 +625,10 @@ int32_t qc_alloc_cache(qc_ctx* ctx, const qc_config* cfg, void* pool_dev, size_t
     for (size_t i = 0; i < c->table.size(); ++i) c->table[i] = static_cast<int32_t>(i);
   }
 
-  if (c->group > 1 && make_pool_tensor_map(c) != QC_OK) {
+  // the pool's tensor map: needed by the query-group decode kernel; the prefill kernel uses it for
+  // cached tiles when it exists
+  c->pool_map_ok = make_pool_tensor_map(c) == QC_OK;
+  if (c->group > 1 && !c->pool_map_ok) {
     delete c;
     return QC_ERR_CUDA;
   }
@@ -801,7 +805,7 @@ int32_t qc_prefill_attend(qc_cache* c, int32_t seq_id, int32_t n_tokens, const u
   QC_CUDA(cudaMemcpyAsync(codes_dev, codes.data(), n_tiles, cudaMemcpyHostToDevice, stream));
   QC_CUDA(cudaStreamSynchronize(stream));   // `kind` is the caller's host memory
   PrefillMaps maps;
-  const bool tc5 = c->prefill_tcgen05 && c->D == 128 && n0_text + n0_vis == 0;
+  const bool tc5 = c->prefill_tcgen05 && c->D == 128 && (c->pool_map_ok || n0_text + n0_vis == 0);
   if (tc5) {
     if (make_prompt_tensor_map(&maps.q, q_dev, c->cfg.n_layers, n_tokens, c->hq) != QC_OK ||
         make_prompt_tensor_map(&maps.k, k_dev, c->cfg.n_layers, n_tokens, c->hkv) != QC_OK ||

@@ -108,6 +108,46 @@ def test_prefill_attend_full_size_sampled(name, mode):
     s.close()
 
 
+@pytest.mark.parametrize("name,mode,cut", [("llava15_7b", qc.QC_MODE_VLA_QC, 300), ("llava15_7b", qc.QC_MODE_GLA, 64),
+                                           ("qwen2vl_gqa", qc.QC_MODE_VLA_QC, 777)],
+                         ids=["llava15_7b-vla-300", "llava15_7b-gla-64", "qwen2vl_gqa-vla-777"])
+def test_prefill_attend_in_two_chunks_full_size(name, mode, cut):
+    """A full-size prompt given as two calls (the cut falls inside the image): the second call's
+    key tiles start with the cached text and visual tokens, read from the paged pool by the
+    tcgen05 kernel.  Both chunks' rows must equal the oracle's rows of ONE prefill over the whole
+    prompt, for sampled (layer, head) pairs, lazy layers and their leaders included."""
+    w = W.get_workload(name)
+    s = Session.for_workload(w, lazy_mode=mode)
+    seq = 2
+    kind, k, v = W.prefill_kv_torch(w, seq, s.device)
+    q = W.prefill_q_torch(w, seq, s.device)
+    T = len(kind)
+    out = torch.empty_like(q)
+    for a, b in ((0, cut), (cut, T)):
+        s.prefill_attend(0, kind[a:b], q[:, a:b].contiguous(), k[:, a:b].contiguous(), v[:, a:b].contiguous(),
+                         out_chunk := torch.empty_like(q[:, a:b].contiguous()))
+        out[:, a:b] = out_chunk
+    torch.cuda.synchronize()
+    assert torch.isfinite(out.float()).all()
+    kinds = w.layer_kind().tolist()
+    leaders = OP.leaders_of(kinds)
+    lz = list(w.lazy_layers)
+    samples = [(0, 0), (lz[0], 1), (lz[-1], w.n_q_heads - 1), (w.n_layers - 1, w.n_q_heads // 2)]
+    for layer, head in samples:
+        c = leaders[layer]
+        layers = [layer] if c == layer else [c, layer]
+        kv = head // w.group
+        qn = W.prefill_q_np(w, seq, layers=layers, heads=[head])
+        _, kn, vn = W.prefill_kv_np(w, seq, layers=layers, heads=[kv])
+        sub_kind = [0] if c == layer else [0, 1]
+        ref = OP.prefill_lazy_attention(f64(qn), f64(kn), f64(vn), kind, sub_kind, mode)[-1, :, 0]
+        got = bits_of(out[layer, :, head])
+        for t0 in range(0, T, 128):
+            assert_close(got[t0:t0 + 128], ref[t0:t0 + 128], f"{name} cut {cut} layer {layer} head {head} tokens {t0}..")
+    assert s.stats().device_error == 0
+    s.close()
+
+
 @pytest.mark.parametrize("name", ["llava_next_anyres", "qwen2vl_gqa"])
 def test_prefill_attend_repeats_bit_identically(name):
     """The kernel has no atomics and a fixed reduction order, so the same prompt gives the same
