@@ -476,6 +476,10 @@ constexpr int kTc5Threads = kTM + 64;   // 128 softmax threads (one per query ro
 // into the same buffer, so the issue warp waits for PV(kt) to complete before it issues S(kt+2)
 // (an earlier version relied on issue order alone and produced a corrupted tile now and then).
 // With two score buffers the softmax of tile kt+1 overlaps PV(kt) and S(kt+2).
+// When the sequence already holds tokens, the CTA's key tiles start with those (cached text, then
+// cached visual tokens, four pool pages per tile, all visible) before the prompt's own tiles.
+// CACHED = false is the instantiation for a prompt that starts a sequence: no code for cached tiles.
+template <bool CACHED>
 __global__ void __launch_bounds__(kTc5Threads, 2)
     prefill_attend_tcgen05_kernel(const __grid_constant__ PrefillArgs A, int32_t* err) {
   // No static shared memory: the dynamic window then starts on the 1024-byte boundary that the
@@ -513,7 +517,7 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
   // Key tiles, in order: the cached text tokens, the cached visual tokens (all visible, read from
   // the pool: a lazy layer's visual K -- and in GLA its text K -- are its leader's pages, which is
   // Eq. 5 / Eq. 7's selection for tokens already cached), then the new tokens (causal).
-  const int ct_text = (A.n0_text + kTN - 1) / kTN, ct_vis = (A.n0_vis + kTN - 1) / kTN;
+  const int ct_text = CACHED ? (A.n0_text + kTN - 1) / kTN : 0, ct_vis = CACHED ? (A.n0_vis + kTN - 1) / kTN : 0;
   const int n_cached = ct_text + ct_vis;
   const int n_ktiles = n_cached + min((A.T + kTN - 1) / kTN, (m0 + kTM + kTN - 1) / kTN);
 
@@ -563,7 +567,7 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
       const uint32_t c = kt < 32 ? codes[0] : (kt < 64 ? codes[1] : codes[2]);
       return static_cast<int>(__shfl_sync(0xffffffffu, c, kt & 31));
     };
-    const int k_text_layer = (A.n0_text && !(A.layer_flags[layer] & kLayerOwnsTextK)) ? lead : layer;
+    const int k_text_layer = (CACHED && A.n0_text && !(A.layer_flags[layer] & kLayerOwnsTextK)) ? lead : layer;
     // Where cached tile kt of the key (which = 1) or value (which = 2) sequence lives: source layer,
     // stream, first token and the stream's length.
     auto cached_tile = [&](int which, int kt, int& src, int& stream, int& ord0, int& n_valid) {
@@ -647,7 +651,7 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
     // tile kt of the CTA's tile sequence (cached tiles first).
     auto fetch_tile = [&](int which, int kt, uint32_t dst, uint32_t half, uint64_t* bar) {
       if (which != 0) {
-        if (kt < n_cached) {
+        if (CACHED && kt < n_cached) {
           fetch_cached(which, kt, dst, half, bar);
           return;
         }
@@ -808,7 +812,7 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
 #pragma unroll
         for (int j = 0; j < 32; ++j) p[j] = __uint_as_float(r0[j]), p[32 + j] = __uint_as_float(r1[j]);
       }
-      if (kt < n_cached) {   // cached tokens: all visible; only a stream's last tile is short
+      if (CACHED && kt < n_cached) {   // cached tokens: all visible; only a stream's last tile is short
         const int n_show = kt < ct_text ? A.n0_text - kt * kTN : A.n0_vis - (kt - ct_text) * kTN;
         if (n_show < kTN) {
 #pragma unroll
@@ -930,10 +934,16 @@ cudaError_t configure_prefill_kernels() {
   e = cudaFuncSetAttribute(prefill_attend_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            prefill_smem_bytes<64>());
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(prefill_attend_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  e = cudaFuncSetAttribute(prefill_attend_tcgen05_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            prefill_tcgen05_smem_bytes());
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(prefill_attend_tcgen05_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+  e = cudaFuncSetAttribute(prefill_attend_tcgen05_kernel<false>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                           cudaSharedmemCarveoutMaxShared);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(prefill_attend_tcgen05_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           prefill_tcgen05_smem_bytes());
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(prefill_attend_tcgen05_kernel<true>, cudaFuncAttributePreferredSharedMemoryCarveout,
                               cudaSharedmemCarveoutMaxShared);
 }
 
@@ -975,7 +985,10 @@ cudaError_t launch_prefill_attend(const Params& p, const uint8_t* kind_dev, cons
     a.tmap_o = maps->out;
     a.tile_code = tile_code_dev;
     const dim3 grid5((T + kTM - 1) / kTM, p.hq, p.n_layers);
-    prefill_attend_tcgen05_kernel<<<grid5, kTc5Threads, prefill_tcgen05_smem_bytes(), stream>>>(a, p.err);
+    if (n0_text + n0_vis > 0)
+      prefill_attend_tcgen05_kernel<true><<<grid5, kTc5Threads, prefill_tcgen05_smem_bytes(), stream>>>(a, p.err);
+    else
+      prefill_attend_tcgen05_kernel<false><<<grid5, kTc5Threads, prefill_tcgen05_smem_bytes(), stream>>>(a, p.err);
     return cudaGetLastError();
   }
   const dim3 grid((T + kBM - 1) / kBM, p.hq, p.n_layers);
