@@ -961,25 +961,42 @@ int decode_step_core(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, const 
   if (c->auto_split) {
     // Larger chunks mean fewer partial results to write and merge; smaller chunks mean more
     // work items to balance over the workers.  Take the largest chunk that still leaves
-    // every worker several items per launch.
-    // (one launch per layer: a launch is short, so its partial rows and their merge weigh more than
-    // the balance of its tail -- one and a half items per worker measured best, against five)
+    // every worker several items per launch: five when the step is one launch, one and a half
+    // when it is one launch per layer (a short launch's partial rows and their merge weigh more
+    // than the balance of its tail; 1, 2 and 3 were measured too).  With several launches per
+    // step, a long stream cut small also means many partial rows per output row for every one of
+    // those launches' merges: beyond 24 rows the chunk is doubled as long as one and a half items
+    // per worker remain.
+    const int64_t workers = static_cast<int64_t>(c->ctx->n_sms) * kAttendWarps * static_cast<int64_t>(c->groups.size());
+    auto items_at = [&](int cp, int* max_slots) {
+      int64_t cv = 0, ct = 0;
+      int slots = 0;
+      for (int i = 0; i < n_seqs; ++i) {
+        const SeqState& st = c->seqs[seq_ids[i]];
+        const int v = (pages_for(st.len_vis) + cp - 1) / cp, t = (pages_for(st.len_text) + cp - 1) / cp;
+        cv += v;
+        ct += t;
+        slots = std::max(slots, v + t);
+      }
+      if (max_slots) *max_slots = slots;
+      return (cv * c->n_visual_jobs + ct * c->n_text_jobs) * c->items_per_chunk;
+    };
     const int64_t twice_per_worker = c->plan_per < 0 ? 3 : 10;
-    const int64_t want =
-        twice_per_worker * c->ctx->n_sms * kAttendWarps * static_cast<int64_t>(c->groups.size()) / 2;
     // (a query group writes one partial row per head and chunk: its chunks stay at 128 keys or more)
     const int floor_pages = c->group > 1 ? std::max(c->min_chunk_pages, 8) : c->min_chunk_pages;
     int pick = floor_pages;
     for (int cp = kMaxChunkPages; cp > floor_pages; cp /= 2) {
-      int64_t cv = 0, ct = 0;
-      for (int i = 0; i < n_seqs; ++i) {
-        const SeqState& st = c->seqs[seq_ids[i]];
-        cv += (pages_for(st.len_vis) + cp - 1) / cp;
-        ct += (pages_for(st.len_text) + cp - 1) / cp;
-      }
-      if ((cv * c->n_visual_jobs + ct * c->n_text_jobs) * c->items_per_chunk >= want) {
+      if (2 * items_at(cp, nullptr) >= twice_per_worker * workers) {
         pick = cp;
         break;
+      }
+    }
+    if (c->groups.size() > 1) {
+      int slots = 0;
+      items_at(pick, &slots);
+      while (slots > 24 && pick * 2 <= kMaxChunkPages && 2 * items_at(pick * 2, nullptr) >= 3 * workers) {
+        pick *= 2;
+        items_at(pick, &slots);
       }
     }
     c->chunk_pages = pick;
