@@ -369,6 +369,7 @@ def run_prefill(args, w, mode, local_rank):
     dev = torch.device("cuda", local_rank)
     s = Session.for_workload(w, lazy_mode=mode, device=local_rank)
     s.set_option("prefill_tcgen05", 1 if args.prefill_kernel == "tcgen05" else 0)
+    s.set_option("prefill_shared_scores", 0 if args.no_prefill_sharing else 1)
     n_seqs = min(w.batch, max(4, args.warmup + 1))
     prompts = []
     for b in range(n_seqs):
@@ -417,6 +418,7 @@ def run_prefill(args, w, mode, local_rank):
         "metric": "prefill_attention_tokens_per_s", "value": n_seqs * T / (ms / 1e3), "unit": UNIT, "n_gpus": 1,
         "steps": n_seqs, "warmup": 1, "ms_per_step": ms / n_seqs, "higher_is_better": True, "dtype": "bf16",
         "data": "synthetic", "config": {"workload": w.name, "mode": args.mode, "prompt_tokens": T, "prompt_chunks": n_chunks,
+                                        "shared_score_passes": (args.mode == "gla" and not args.no_prefill_sharing),
                                         "n_layers": w.n_layers, "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads},
         "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                      "frac": achieved / peak, "traffic": None,
@@ -448,6 +450,9 @@ def main():
                     help="use this CUDA device on every rank (to exercise the multi-rank plumbing on one GPU)")
     ap.add_argument("--phase", default="decode", choices=["decode", "prefill"],
                     help="decode (the benchmark) or prefill (secondary: qc_prefill_attend over the prompts)")
+    ap.add_argument("--no-prefill-sharing", action="store_true",
+                    help="prefill phase, mode gla: one score pass per layer instead of one per run of up to three "
+                         "layers of a lazy block")
     ap.add_argument("--prefill-chunks", type=int, default=1,
                     help="prefill phase: give each prompt as this many consecutive calls (chunked prefill)")
     ap.add_argument("--prefill-kernel", default="tcgen05", choices=["tcgen05", "mma"],

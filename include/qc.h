@@ -245,8 +245,12 @@ int32_t qc_debug_read_row(qc_cache* cache, int32_t layer, int32_t stream, int32_
  * again; by Eq. 6 / the Q Cache rule the follower's scores are the leader's, so the result is the
  * one of the fused schedule.  VLA_EQ8 followers score with their own query and re-read the
  * leader's visual K.  0 = back to one launch per step.  qc_decode_step only),
- * "prefill_tcgen05" (0 = use the mma.sync prefill kernel), "profile" (1 = record CUDA events per
- * step). */
+ * "prefill_tcgen05" (0 = use the mma.sync prefill kernel), "prefill_shared_scores" (GLA only: by
+ * Eq. 5 the layers of a lazy block attend with the same Q and K, so qc_prefill_attend computes and
+ * normalises their scores once per run of up to three layers and applies them to each layer's V,
+ * bit-identically to one pass per layer; 0 = never, 1 = for prompts of 1536 tokens or more (the
+ * default: below that the pass's lower occupancy costs more than it saves), 2 = always),
+ * "profile" (1 = record CUDA events per step). */
 int32_t qc_set_option(qc_cache* cache, const char* key, int64_t value);
 
 /* Sum the recorded kernel times since the last call (synchronises), then reset them. */

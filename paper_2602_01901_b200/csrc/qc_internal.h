@@ -125,6 +125,15 @@ cudaError_t launch_prefill_scatter(const Params& p, const int32_t* tok_seq, cons
 // {128, heads, n_layers * T} read in boxes of 64 tokens x one head x 64 elements, and the output
 // as a 4-D tensor {128, hq, T, n_layers} written in boxes of 128 tokens x one head x 64 elements
 // (the token dimension of its own so that a store is clipped at the end of the prompt).
+// One launch unit of the tcgen05 kernel along blockIdx.z: n layers of one lazy block whose scores
+// are identical (GLA, Eq. 5: Q and K are the block's first layer's), so that they are computed and
+// normalised once and applied to each layer's own V; n = 1 is an ordinary single layer.
+struct PrefillPass {
+  int32_t n, v[3];
+};
+
+constexpr int kPrefillSharedLayers = 3;   // layers one shared-score pass feeds
+
 struct PrefillMaps {
   CUtensorMap q, k, v, out;
 };
@@ -132,6 +141,7 @@ cudaError_t launch_prefill_attend(const Params& p, const uint8_t* kind_dev, cons
                                   const uint8_t* leader_dev, const void* q, const void* k, const void* v, void* out,
                                   int32_t n_tokens, int32_t gla, const PrefillMaps* maps,
                                   const uint8_t* tile_code_dev, int32_t seq_id, int32_t n0_text, int32_t n0_vis,
+                                  const PrefillPass* passes_dev, int32_t n_single, int32_t n_shared,
                                   cudaStream_t stream);   // qc_prefill.cu; maps null or head_dim 64 = mma.sync kernel
 cudaError_t configure_prefill_kernels();
 cudaError_t launch_calibration(const Params& p, const int32_t* seq_ids_dev, const int32_t* len_text_dev,

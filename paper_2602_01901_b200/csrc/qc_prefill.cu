@@ -39,6 +39,7 @@ struct PrefillArgs {
   // tcgen05 kernel: q / k / v as 3-D tensors {D, heads, n_layers * T}, box {64, 1, 64}; the output as a
   // 4-D tensor {D, hq, T, n_layers}, box {64, 1, 128, 1}; 128-byte swizzle
   CUtensorMap tmap_q, tmap_k, tmap_v, tmap_o;
+  const PrefillPass* passes;   // device; tcgen05 kernel: what blockIdx.z stands for (null: layer blockIdx.z alone)
   CUtensorMap tmap_pool;   // the paged pool as a 2-D tensor [pages * hkv * 16 rows][D], box 16 rows x 64 elements
   int64_t n_pool_pages;    // bound for page ids read from the table
   const uint8_t* tile_code;    // [ceil(T / 64)] device: 0 = the 64-token tile is all text, 1 = all visual, 2 = mixed
@@ -479,18 +480,22 @@ constexpr int kTc5Threads = kTM + 64;   // 128 softmax threads (one per query ro
 // When the sequence already holds tokens, the CTA's key tiles start with those (cached text, then
 // cached visual tokens, four pool pages per tile, all visible) before the prompt's own tiles.
 // CACHED = false is the instantiation for a prompt that starts a sequence: no code for cached tiles.
-template <bool CACHED>
-__global__ void __launch_bounds__(kTc5Threads, 2)
+// NV > 1 is the instantiation for shared-score passes: up to NV layers' accumulators in tensor
+// memory (all 512 columns, so one CTA per SM), NV value tiles per key tile.
+template <bool CACHED, int NV>
+__global__ void __launch_bounds__(kTc5Threads, NV > 1 ? 1 : 2)
     prefill_attend_tcgen05_kernel(const __grid_constant__ PrefillArgs A, int32_t* err) {
+  static_assert(NV == 1 || !CACHED, "shared-score passes are for prompts that start a sequence");
+  constexpr uint32_t kCols = NV > 1 ? 512 : kTmemCols;
   // No static shared memory: the dynamic window then starts on the 1024-byte boundary that the
   // swizzled tiles need, and two CTAs fit an SM (2 x 112 KiB of tiles).  Checked below.
   extern __shared__ __align__(1024) uint8_t smem_dyn[];
   const uint32_t base = smem_u32(smem_dyn);
   const uint32_t sQ = base;                         // [2][128][128 B]  32 KiB
   const uint32_t sK = sQ + 2 * kTM * 128;           // two buffers of [2][64][128 B] 16 KiB
-  const uint32_t sV = sK + 2 * (2 * kTN * 128);     // two buffers
+  const uint32_t sV = sK + 2 * (2 * kTN * 128);     // two buffers per consumer: consumer x, buffer b at (2 x + b)
   constexpr uint32_t kKV = 2 * kTN * 128;
-  constexpr uint32_t kTiles = 2 * kTM * 128 + 4 * kKV;
+  constexpr uint32_t kTiles = 2 * kTM * 128 + 2 * kKV + NV * 2 * kKV;
   uint64_t* bar_s = reinterpret_cast<uint64_t*>(smem_dyn + kTiles);          // two: one per score buffer
   uint64_t* bar_p = reinterpret_cast<uint64_t*>(smem_dyn + kTiles + 16);          // two
   uint64_t* bar_k = reinterpret_cast<uint64_t*>(smem_dyn + kTiles + 32);          // two
@@ -499,6 +504,8 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
   uint32_t& tmem_base_slot = *reinterpret_cast<uint32_t*>(smem_dyn + kTiles + 80);
   volatile int32_t& failed = *reinterpret_cast<volatile int32_t*>(smem_dyn + kTiles + 84);
   uint64_t& bar_q = *reinterpret_cast<uint64_t*>(smem_dyn + kTiles + 88);   // the two 64-row halves of the Q tile
+  uint64_t& bar_e = *reinterpret_cast<uint64_t*>(smem_dyn + kTiles + 96);   // NV > 1: an output tile is staged
+  uint64_t& bar_r = *reinterpret_cast<uint64_t*>(smem_dyn + kTiles + 104);  // NV > 1: its store has read it
   if (base & 1023u) {   // cannot happen with the layout above; never run the tensor core on a misplaced tile
     if (threadIdx.x == 0) atomicMax(err, kErrBadPage);
     return;
@@ -507,7 +514,17 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_qtiles = (A.T + kTM - 1) / kTM;
   const int qt = n_qtiles - 1 - blockIdx.x;         // long rows first
-  const int head = blockIdx.y, layer = blockIdx.z;
+  const int head = blockIdx.y;
+  int n_cons = 1, v_layer[NV];
+  if (A.passes) {
+    const PrefillPass ps = A.passes[blockIdx.z];
+    n_cons = NV > 1 ? min(ps.n, NV) : 1;
+#pragma unroll
+    for (int x = 0; x < NV; ++x) v_layer[x] = ps.v[x < n_cons ? x : 0];
+  } else {
+    v_layer[0] = blockIdx.z;
+  }
+  const int layer = v_layer[0];   // decides where Q and K come from; with NV > 1 all consumers share that
   const int kvh = head / A.group;
   const bool lazy = A.layer_kind[layer] != 0;
   const int lead = A.leader[layer];
@@ -525,9 +542,11 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
     mbar_init(&bar_s[0], 1);
     mbar_init(&bar_s[1], 1);
     mbar_init(&bar_q, 2);
+    mbar_init(&bar_e, kTM);
+    mbar_init(&bar_r, 1);
     for (int b = 0; b < 2; ++b) {
       mbar_init(&bar_k[b], 1);
-      mbar_init(&bar_v[b], 1);
+      mbar_init(&bar_v[b], n_cons);
       mbar_init(&bar_o[b], 1);
       mbar_init(&bar_p[b], kTM);
     }
@@ -536,7 +555,7 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
   }
   if (warp == 4) {   // the score warp owns the TMEM allocation
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
-                 "r"(kTmemCols)
+                 "r"(kCols)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -649,7 +668,7 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
     };
     // `which`: 0 = 64 query rows (kt counts 64-row tiles of the prompt), 1 = key tile kt, 2 = value
     // tile kt of the CTA's tile sequence (cached tiles first).
-    auto fetch_tile = [&](int which, int kt, uint32_t dst, uint32_t half, uint64_t* bar) {
+    auto fetch_tile = [&](int which, int kt, uint32_t dst, uint32_t half, uint64_t* bar, int v_src = -1) {
       if (which != 0) {
         if (CACHED && kt < n_cached) {
           fetch_cached(which, kt, dst, half, bar);
@@ -657,7 +676,7 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
         }
         kt -= n_cached;   // a tile of new tokens
       }
-      int src = layer;
+      int src = (which == 2 && v_src >= 0) ? v_src : layer;
       bool mixed = false;
       if (which != 2 && lazy && kt * kTN < A.T) {   // queries and keys of a lazy layer: the leader's for visual rows
         if (gla) {
@@ -707,7 +726,12 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
       // ---------------- issue warp: S(kt) = Q K(kt)^T into score buffer kt & 1, O += P(kt) V(kt)
       const uint64_t qd = umma_desc(sQ, 16, 1024);
       const uint64_t kd0 = umma_desc(sK, 16, 1024), kd1 = umma_desc(sK + kKV, 16, 1024);
-      const uint64_t vd0 = umma_desc(sV, kTN * 128, 1024), vd1 = umma_desc(sV + kKV, kTN * 128, 1024);
+      uint64_t vd[NV][2];   // consumer x, buffer b
+#pragma unroll
+      for (int x = 0; x < NV; ++x) {
+        vd[x][0] = umma_desc(sV + (2 * x) * kKV, kTN * 128, 1024);
+        vd[x][1] = umma_desc(sV + (2 * x + 1) * kKV, kTN * 128, 1024);
+      }
       uint32_t ph_k[2] = {0, 0}, ph_v[2] = {0, 0}, ph_o[2] = {0, 0}, ph_p[2] = {0, 0};
       auto issue_scores = [&](int buf) {   // whole warp; one elected lane issues
         umma_scores<kTM * 128, kTN * 128>(tmem + kColS + buf * kTN, qd, buf ? kd1 : kd0, kIdescS);
@@ -731,7 +755,11 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
         if (!ok) break;
         {
           tc5_fence_after();
-          umma_values(tmem + kColO, tmem + kColS + buf * kTN, buf ? vd1 : vd0, kIdescO, kt > 0 ? 1u : 0u);
+#pragma unroll
+          for (int x = 0; x < NV; ++x)
+            if (x < n_cons)
+              umma_values(tmem + kColO + kTD * x, tmem + kColS + buf * kTN, buf ? vd[x][1] : vd[x][0], kIdescO,
+                          kt > 0 ? 1u : 0u);
           umma_commit(&bar_o[buf]);
         }
         if (kt + 2 < n_ktiles) {
@@ -752,10 +780,16 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
       fetch_tile(0, 2 * qt, sQ, kTM * 128, &bar_q);
       fetch_tile(1, 0, sK, kTN * 128, &bar_k[0]);
       fetch_tile(0, 2 * qt + 1, sQ + kTN * 128, kTM * 128, &bar_q);
-      fetch_tile(2, 0, sV, kTN * 128, &bar_v[0]);
+      auto fetch_values = [&](int kt) {   // one tile per consumer; bar_v[kt & 1] counts them all
+        const int b = kt & 1;
+#pragma unroll
+        for (int x = 0; x < NV; ++x)
+          if (x < n_cons) fetch_tile(2, kt, sV + (2 * x + b) * kKV, kTN * 128, &bar_v[b], v_layer[x]);
+      };
+      fetch_values(0);
       if (n_ktiles > 1) {
         fetch_tile(1, 1, sK + kKV, kTN * 128, &bar_k[1]);
-        fetch_tile(2, 1, sV + kKV, kTN * 128, &bar_v[1]);
+        fetch_values(1);
       }
       int k_next = 2, v_next = 2;
       uint32_t idle = 0;
@@ -774,7 +808,7 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
           const int b = v_next & 1;
           if (__all_sync(0xffffffffu, mbar_test_wait(&bar_o[b], ph_o[b]))) {
             ph_o[b] ^= 1u;
-            fetch_tile(2, v_next, sV + b * kKV, kTN * 128, &bar_v[b]);
+            fetch_values(v_next);
             ++v_next;
             progress = true;
           }
@@ -853,12 +887,17 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
         if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
         tc5_fence_after();
 #pragma unroll
-        for (int c = 0; c < kTD / 32; ++c) {
-          uint32_t r[32];
-          tmem_ld32(t_row + kColO + 32 * c, r);
+        for (int x = 0; x < NV; ++x) {
+          if (x < n_cons) {
 #pragma unroll
-          for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * corr);
-          tmem_st32(t_row + kColO + 32 * c, r);
+            for (int c = 0; c < kTD / 32; ++c) {
+              uint32_t r[32];
+              tmem_ld32(t_row + kColO + kTD * x + 32 * c, r);
+#pragma unroll
+              for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * corr);
+              tmem_st32(t_row + kColO + kTD * x + 32 * c, r);
+            }
+          }
         }
         asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
       }
@@ -875,17 +914,15 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
     }
     if (ok) ok = bounded_wait(&bar_o[(n_ktiles - 1) & 1], ((n_ktiles - 1) >> 1) & 1) && !failed;   // the last value product
     ok = __all_sync(0xffffffffu, ok);
-    if (ok) {
-      // every product has completed: the Q tile's shared memory is free and takes the output tile in
-      // the same swizzled layout, from where two tensor-map stores write it (clipped at token T)
-      tc5_fence_after();
-      const float inv = 1.f / l_sum;
+    // Scale the accumulator of consumer x and put the tile into the Q tile's shared memory (free: every
+    // product has completed) in the swizzled layout of a 128-row box.
+    auto stage_output = [&](int x, float inv) {
       const uint32_t orow = sQ + threadIdx.x * 128;
       const uint32_t sw = threadIdx.x & 7;
 #pragma unroll
       for (int c = 0; c < kTD / 32; ++c) {
         uint32_t r[32];
-        tmem_ld32(t_row + kColO + 32 * c, r);
+        tmem_ld32(t_row + kColO + kTD * x + 32 * c, r);
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           const int chunk = 4 * c + j;   // 16-byte chunk of the 256-byte row
@@ -898,6 +935,44 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
         }
       }
       fence_proxy_async();
+    };
+    if constexpr (NV > 1) {
+      // One output tile per consumer, one after the other through the same staging area: the 128
+      // threads arrive on bar_e when a tile is staged, thread 0 stores it and arrives on bar_r when
+      // the stores have read it (bounded waits throughout, as everywhere in this kernel).
+      if (ok) {
+        tc5_fence_after();
+        const float inv = 1.f / l_sum;
+        for (int x = 0; x < n_cons; ++x) {
+          if (x > 0) {
+            ok = bounded_wait(&bar_r, static_cast<uint32_t>(x - 1) & 1u) && !failed;
+            ok = __all_sync(0xffffffffu, ok);
+          }
+          if (!ok) break;
+          stage_output(x, inv);
+          mbar_arrive(&bar_e);
+          if (threadIdx.x == 0) {
+            if (bounded_wait(&bar_e, static_cast<uint32_t>(x) & 1u)) {
+              tensor_s2g_4d(&A.tmap_o, sQ, 0, head, m0, v_layer[x]);
+              tensor_s2g_4d(&A.tmap_o, sQ + kTM * 128, 64, head, m0, v_layer[x]);
+              asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+              asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // (also: shared memory is released at exit)
+              mbar_arrive(&bar_r);
+            } else {
+              failed = 1;
+            }
+          }
+          __syncwarp();
+        }
+      }
+      if (!ok) {
+        failed = 1;
+        if (lane == 0) atomicMax(err, kErrTimeout);
+      }
+    } else if (ok) {
+      // two tensor-map stores write the staged tile (clipped at token T)
+      tc5_fence_after();
+      stage_output(0, 1.f / l_sum);
       asm volatile("bar.sync 1, %0;" ::"n"(kTM) : "memory");   // the 128 softmax threads
       if (threadIdx.x == 0) {
         tensor_s2g_4d(&A.tmap_o, sQ, 0, head, m0, layer);
@@ -914,11 +989,12 @@ __global__ void __launch_bounds__(kTc5Threads, 2)
   tc5_fence_before();
   __syncthreads();
   if (warp == 4) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kCols) : "memory");
   }
 }
 
-constexpr int prefill_tcgen05_smem_bytes() { return 2 * kTM * 128 + 4 * (2 * kTN * 128) + 128; }
+constexpr int kSharedPassLayers = kPrefillSharedLayers;   // 3 x 128 + 2 x 64 columns = all of tensor memory
+constexpr int prefill_tcgen05_smem_bytes(int nv = 1) { return 2 * kTM * 128 + (2 + 2 * nv) * (2 * kTN * 128) + 128; }
 
 template <int D>
 constexpr int prefill_smem_bytes() {
@@ -934,23 +1010,30 @@ cudaError_t configure_prefill_kernels() {
   e = cudaFuncSetAttribute(prefill_attend_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            prefill_smem_bytes<64>());
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(prefill_attend_tcgen05_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  e = cudaFuncSetAttribute(prefill_attend_tcgen05_kernel<false, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            prefill_tcgen05_smem_bytes());
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(prefill_attend_tcgen05_kernel<false>, cudaFuncAttributePreferredSharedMemoryCarveout,
+  e = cudaFuncSetAttribute(prefill_attend_tcgen05_kernel<false, 1>, cudaFuncAttributePreferredSharedMemoryCarveout,
                            cudaSharedmemCarveoutMaxShared);
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(prefill_attend_tcgen05_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  e = cudaFuncSetAttribute(prefill_attend_tcgen05_kernel<true, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            prefill_tcgen05_smem_bytes());
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(prefill_attend_tcgen05_kernel<true>, cudaFuncAttributePreferredSharedMemoryCarveout,
-                              cudaSharedmemCarveoutMaxShared);
+  e = cudaFuncSetAttribute(prefill_attend_tcgen05_kernel<true, 1>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                           cudaSharedmemCarveoutMaxShared);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(prefill_attend_tcgen05_kernel<false, kSharedPassLayers>,
+                           cudaFuncAttributeMaxDynamicSharedMemorySize, prefill_tcgen05_smem_bytes(kSharedPassLayers));
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(prefill_attend_tcgen05_kernel<false, kSharedPassLayers>,
+                              cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
 }
 
 cudaError_t launch_prefill_attend(const Params& p, const uint8_t* kind_dev, const uint8_t* layer_kind_dev,
                                   const uint8_t* leader_dev, const void* q, const void* k, const void* v, void* out,
                                   int32_t T, int32_t gla, const PrefillMaps* maps,
                                   const uint8_t* tile_code_dev, int32_t seq_id, int32_t n0_text, int32_t n0_vis,
+                                  const PrefillPass* passes_dev, int32_t n_single, int32_t n_shared,
                                   cudaStream_t stream) {
   if (T <= 0) return cudaSuccess;
   PrefillArgs a{};
@@ -985,10 +1068,22 @@ cudaError_t launch_prefill_attend(const Params& p, const uint8_t* kind_dev, cons
     a.tmap_o = maps->out;
     a.tile_code = tile_code_dev;
     const dim3 grid5((T + kTM - 1) / kTM, p.hq, p.n_layers);
-    if (n0_text + n0_vis > 0)
-      prefill_attend_tcgen05_kernel<true><<<grid5, kTc5Threads, prefill_tcgen05_smem_bytes(), stream>>>(a, p.err);
-    else
-      prefill_attend_tcgen05_kernel<false><<<grid5, kTc5Threads, prefill_tcgen05_smem_bytes(), stream>>>(a, p.err);
+    if (n0_text + n0_vis > 0) {
+      prefill_attend_tcgen05_kernel<true, 1><<<grid5, kTc5Threads, prefill_tcgen05_smem_bytes(), stream>>>(a, p.err);
+    } else if (passes_dev && n_shared > 0) {
+      // the layers that share nothing, then the shared-score passes (passes_dev lists them in that order)
+      a.passes = passes_dev;
+      if (n_single > 0) {
+        const dim3 g1(grid5.x, grid5.y, n_single);
+        prefill_attend_tcgen05_kernel<false, 1><<<g1, kTc5Threads, prefill_tcgen05_smem_bytes(), stream>>>(a, p.err);
+      }
+      a.passes = passes_dev + n_single;
+      const dim3 g3(grid5.x, grid5.y, n_shared);
+      prefill_attend_tcgen05_kernel<false, kSharedPassLayers>
+          <<<g3, kTc5Threads, prefill_tcgen05_smem_bytes(kSharedPassLayers), stream>>>(a, p.err);
+    } else {
+      prefill_attend_tcgen05_kernel<false, 1><<<grid5, kTc5Threads, prefill_tcgen05_smem_bytes(), stream>>>(a, p.err);
+    }
     return cudaGetLastError();
   }
   const dim3 grid((T + kBM - 1) / kBM, p.hq, p.n_layers);

@@ -19,6 +19,10 @@ namespace {
 constexpr int kStageSlots = 8;       // pinned step-descriptor ring
 constexpr int kMaxProfileSteps = 16384;
 constexpr int kPrefillBatchTokens = 1 << 16;
+// Shared-score passes run one CTA per SM (three accumulators fill tensor memory); that pays once
+// a CTA has enough key tiles: measured -16 % / -10 % call time at 2048 / 3008 tokens, +4 % / +9 %
+// at 1120 / 675.
+constexpr int kPrefillShareMinTokens = 1536;
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -75,6 +79,10 @@ struct qc_cache {
   std::vector<cudaEvent_t> ev_in, ev_done;
   bool prefill_tcgen05 = true;    // head_dim 128: tcgen05 kernel; otherwise (or when switched off) mma.sync kernel
   bool pool_map_ok = false;       // c->tmap was encoded
+  int prefill_shared = 1;         // GLA prefill: layers of a block whose scores coincide share one score pass
+                                  // (0 never, 1 for prompts of kPrefillShareMinTokens or more, 2 always)
+  std::vector<PrefillPass> prefill_passes;   // singles first, then shared passes (GLA only; else empty)
+  int prefill_n_single = 0, prefill_n_shared = 0;
   int64_t n_pool_pages = 0;
   int layers_per_launch = 0;
   float scale = 0.f;
@@ -615,6 +623,22 @@ int32_t qc_alloc_cache(qc_ctx* ctx, const qc_config* cfg, void* pool_dev, size_t
   }
   build_jobs(&c->cfg, c->jobs, c->block_jobs, c->block_layers);
   build_layer_jobs(&c->cfg, c->layer_jobs, c->layer_job_range);
+  if (c->cfg.lazy_mode == QC_MODE_GLA) {
+    // Eq. 5: every layer of a lazy block attends with the block's first layer's Q and K, so runs
+    // of up to three of its layers share one score pass of the prefill kernel
+    std::vector<PrefillPass> shared;
+    for (const auto& bl : c->block_layers) {
+      for (int first = bl.first; first < bl.second; first += kPrefillSharedLayers) {
+        PrefillPass ps{};
+        ps.n = std::min(kPrefillSharedLayers, bl.second - first);
+        for (int x = 0; x < ps.n; ++x) ps.v[x] = first + x;
+        (ps.n > 1 ? shared : c->prefill_passes).push_back(ps);
+      }
+    }
+    c->prefill_n_single = static_cast<int>(c->prefill_passes.size());
+    c->prefill_n_shared = static_cast<int>(shared.size());
+    c->prefill_passes.insert(c->prefill_passes.end(), shared.begin(), shared.end());
+  }
   c->seqs.resize(cfg->max_seqs);
   c->table.assign(static_cast<size_t>(cfg->n_layers) * 4 * cfg->max_seqs * c->max_pages, -1);
   if (c->paged) {
@@ -785,7 +809,9 @@ int32_t qc_prefill_attend(qc_cache* c, int32_t seq_id, int32_t n_tokens, const u
   // tokens the sequence holds already (an earlier prompt chunk, generated tokens) precede the new ones
   const int n0_text = c->seqs[seq_id].active ? c->seqs[seq_id].len_text : 0;
   const int n0_vis = c->seqs[seq_id].active ? c->seqs[seq_id].len_vis : 0;
-  if (static_cast<size_t>(n_tokens) > static_cast<size_t>(kPrefillBatchTokens) * 3 * sizeof(int32_t))
+  const size_t tok_bytes = static_cast<size_t>(kPrefillBatchTokens) * 3 * sizeof(int32_t);   // kinds, tile codes, passes
+  if (align_up(n_tokens, 256) + align_up((n_tokens + 63) / 64, 256) + c->prefill_passes.size() * sizeof(PrefillPass) >
+      tok_bytes)
     return QC_ERR_INVALID_ARG;
   // store K/V first: this validates everything and leaves the cache unchanged on an error
   int st = qc_prefill_append(c, 1, &seq_id, &n_tokens, kind, k_dev, v_dev);
@@ -803,6 +829,12 @@ int32_t qc_prefill_attend(qc_cache* c, int32_t seq_id, int32_t n_tokens, const u
   uint8_t* codes_dev = kind_dev + align_up(n_tokens, 256);
   QC_CUDA(cudaMemcpyAsync(kind_dev, kind, n_tokens, cudaMemcpyHostToDevice, stream));
   QC_CUDA(cudaMemcpyAsync(codes_dev, codes.data(), n_tiles, cudaMemcpyHostToDevice, stream));
+  PrefillPass* passes_dev = reinterpret_cast<PrefillPass*>(codes_dev + align_up(n_tiles, 256));
+  const bool share = c->prefill_n_shared > 0 && n0_text + n0_vis == 0 &&
+                     (c->prefill_shared == 2 || (c->prefill_shared == 1 && n_tokens >= kPrefillShareMinTokens));
+  if (share)
+    QC_CUDA(cudaMemcpyAsync(passes_dev, c->prefill_passes.data(), c->prefill_passes.size() * sizeof(PrefillPass),
+                            cudaMemcpyHostToDevice, stream));
   QC_CUDA(cudaStreamSynchronize(stream));   // `kind` is the caller's host memory
   PrefillMaps maps;
   const bool tc5 = c->prefill_tcgen05 && c->D == 128 && (c->pool_map_ok || n0_text + n0_vis == 0);
@@ -828,14 +860,19 @@ int32_t qc_prefill_attend(qc_cache* c, int32_t seq_id, int32_t n_tokens, const u
   }
   QC_CUDA(launch_prefill_attend(p, kind_dev, c->ws + c->lay.layer_kind, c->ws + c->lay.leader, q_dev, k_dev, v_dev,
                                 out_dev, n_tokens, c->cfg.lazy_mode == QC_MODE_GLA ? 1 : 0, tc5 ? &maps : nullptr,
-                                codes_dev, seq_id, n0_text, n0_vis, stream));
+                                codes_dev, seq_id, n0_text, n0_vis, (tc5 && share) ? passes_dev : nullptr,
+                                c->prefill_n_single, c->prefill_n_shared, stream));
+  const bool shared_run = tc5 && share;
   if (ev) {
     QC_CUDA(cudaEventRecord(ev[1], stream));
     c->ev_prefill_calls++;
+    // executed arithmetic: 2 D flops per pair for the scores of every score pass, 2 D per pair for
+    // the value product of every layer
     const double pairs = 0.5 * n_tokens * (n_tokens + 1.0) + static_cast<double>(n_tokens) * (n0_text + n0_vis);
-    c->prof_prefill_flops += 4.0 * c->D * pairs * c->hq * c->cfg.n_layers;
+    const int score_passes = shared_run ? c->prefill_n_single + c->prefill_n_shared : c->cfg.n_layers;
+    c->prof_prefill_flops += 2.0 * c->D * pairs * c->hq * (score_passes + c->cfg.n_layers);
   }
-  c->kernel_launches++;
+  c->kernel_launches += (shared_run && c->prefill_n_single > 0) ? 2 : 1;
   return QC_OK;
 }
 
@@ -1314,6 +1351,11 @@ int32_t qc_set_option(qc_cache* c, const char* key, int64_t value) {
   if (k == "per_layer_logit_cache") {   // one launch per layer; followers take shared scores from the logit cache
     c->layers_per_launch = value ? -1 : 0;
     c->plan_dirty = true;
+    return QC_OK;
+  }
+  if (k == "prefill_shared_scores") {
+    if (value < 0 || value > 2) return QC_ERR_INVALID_ARG;
+    c->prefill_shared = static_cast<int>(value);
     return QC_OK;
   }
   if (k == "prefill_tcgen05") {

@@ -70,8 +70,10 @@ def test_prefill_attend_small(mode, case):
 
 
 @pytest.mark.parametrize("name,mode", [("llava15_7b", qc.QC_MODE_VLA_QC), ("llava15_7b", qc.QC_MODE_GLA),
-                                       ("qwen2vl_gqa", qc.QC_MODE_VLA_QC)],
-                         ids=["llava15_7b-vla", "llava15_7b-gla", "qwen2vl_gqa-vla"])
+                                       ("qwen2vl_gqa", qc.QC_MODE_VLA_QC), ("qwen2vl_gqa", qc.QC_MODE_GLA),
+                                       ("llava_next_2048_lazy22", qc.QC_MODE_GLA)],
+                         ids=["llava15_7b-vla", "llava15_7b-gla", "qwen2vl_gqa-vla", "qwen2vl_gqa-gla",
+                              "lazy22-gla"])
 def test_prefill_attend_full_size_sampled(name, mode):
     """One full-size prompt (all layers, all heads on the GPU); the oracle checks every row of
     sampled (layer, head) pairs, lazy layers and their leaders included."""
@@ -146,6 +148,31 @@ def test_prefill_attend_in_two_chunks_full_size(name, mode, cut):
             assert_close(got[t0:t0 + 128], ref[t0:t0 + 128], f"{name} cut {cut} layer {layer} head {head} tokens {t0}..")
     assert s.stats().device_error == 0
     s.close()
+
+
+@pytest.mark.parametrize("name", ["llava15_7b", "llava_next_2048_lazy22", "qwen2vl_gqa"])
+def test_prefill_gla_shared_score_passes_change_no_bit(name):
+    """GLA, Eq. 5: the layers of a lazy block attend with the same Q and K, so the kernel computes and
+    normalises their scores once per run of up to three layers and applies them to each layer's V.
+    That is the same arithmetic in the same order as one pass per layer: identical bits.
+    (blocks of two layers in the first workload, of four -- a pass of three and a single -- in the
+    second, query groups of seven in the third)"""
+    w = W.get_workload(name)
+    kind, q = None, None
+    outs = []
+    for shared in (2, 0):    # 2 = always (the default shares only from 1536 prompt tokens on)
+        s = Session.for_workload(w, lazy_mode=qc.QC_MODE_GLA)
+        s.set_option("prefill_shared_scores", shared)
+        kind, k, v = W.prefill_kv_torch(w, 1, s.device)
+        q = W.prefill_q_torch(w, 1, s.device)
+        out = torch.full_like(q, float("nan"))
+        s.prefill_attend(0, kind, q, k, v, out)
+        torch.cuda.synchronize()
+        assert s.stats().device_error == 0
+        outs.append(out)
+        s.close()
+    assert torch.isfinite(outs[0].float()).all()
+    assert torch.equal(outs[0].view(torch.int16), outs[1].view(torch.int16))
 
 
 @pytest.mark.parametrize("name", ["llava_next_anyres", "qwen2vl_gqa"])
