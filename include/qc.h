@@ -115,8 +115,10 @@ typedef struct qc_profile {
   int64_t items;              /* split-KV work items executed */
   int64_t prefill_calls;      /* qc_prefill_attend calls covered */
   double prefill_attend_ms;   /* summed duration of the prefill attention kernel */
-  double prefill_flops;       /* its arithmetic: 4 * head_dim flops per (query, visible key) pair,
-                                 every layer and query head */
+  double prefill_flops;       /* its executed arithmetic: per (query, visible key) pair and query head,
+                                 2 * head_dim flops for every score pass (one per layer, or one per
+                                 run of layers that share their scores) and 2 * head_dim for every
+                                 layer's value product */
 } qc_profile;
 
 /* Create a context on `device` that launches on `cuda_stream` (a cudaStream_t; NULL is the
