@@ -483,7 +483,7 @@ constexpr int kTc5Threads = kTM + 64;   // 128 softmax threads (one per query ro
 // NV > 1 is the instantiation for shared-score passes: up to NV layers' accumulators in tensor
 // memory (all 512 columns, so one CTA per SM), NV value tiles per key tile.
 template <bool CACHED, int NV>
-__global__ void __launch_bounds__(kTc5Threads, NV > 1 ? 1 : 2)
+__global__ void __launch_bounds__(NV > 1 ? kTc5Threads + 32 : kTc5Threads, NV > 1 ? 1 : 2)
     prefill_attend_tcgen05_kernel(const __grid_constant__ PrefillArgs A, int32_t* err) {
   static_assert(NV == 1 || !CACHED, "shared-score passes are for prompts that start a sequence");
   constexpr uint32_t kCols = NV > 1 ? 512 : kTmemCols;
@@ -722,7 +722,59 @@ __global__ void __launch_bounds__(kTc5Threads, NV > 1 ? 1 : 2)
         ok = __all_sync(0xffffffffu, bounded_wait(bar, phase) && !failed);
       phase ^= 1u;
     };
-    if (warp == 4) {
+    if (NV > 1 && warp != 5) {
+      // ---------------- shared-score passes: two issue warps.  Alone on its SM, the CTA has nothing
+      // else to hide one lane's issue time behind, so the score products (warp 4) and the value
+      // products of the NV consumers (warp 6) are issued in parallel; same hand-offs as below.
+      uint32_t ph_k[2] = {0, 0}, ph_v[2] = {0, 0}, ph_o[2] = {0, 0}, ph_p[2] = {0, 0};
+      if (warp == 4) {
+        const uint64_t qd = umma_desc(sQ, 16, 1024);
+        const uint64_t kd0 = umma_desc(sK, 16, 1024), kd1 = umma_desc(sK + kKV, 16, 1024);
+        auto issue_scores = [&](int buf) {
+          umma_scores<kTM * 128, kTN * 128>(tmem + kColS + buf * kTN, qd, buf ? kd1 : kd0, kIdescS);
+          umma_commit(&bar_s[buf]);
+        };
+        {
+          uint32_t ph_q = 0;
+          wait_on(&bar_q, ph_q);
+        }
+        for (int kt = 0; kt < 2 && kt < n_ktiles && ok; ++kt) {
+          wait_on(&bar_k[kt], ph_k[kt]);
+          if (ok) {
+            tc5_fence_after();
+            issue_scores(kt);
+          }
+        }
+        for (int kt = 0; kt + 2 < n_ktiles && ok; ++kt) {
+          const int buf = kt & 1;
+          wait_on(&bar_o[buf], ph_o[buf]);   // PV(kt) complete: the buffer's weights have been read
+          wait_on(&bar_k[buf], ph_k[buf]);   // K(kt+2) landed
+          if (!ok) break;
+          tc5_fence_after();
+          issue_scores(buf);
+        }
+      } else {
+        uint64_t vd[NV][2];   // consumer x, buffer b
+#pragma unroll
+        for (int x = 0; x < NV; ++x) {
+          vd[x][0] = umma_desc(sV + (2 * x) * kKV, kTN * 128, 1024);
+          vd[x][1] = umma_desc(sV + (2 * x + 1) * kKV, kTN * 128, 1024);
+        }
+        for (int kt = 0; kt < n_ktiles && ok; ++kt) {
+          const int buf = kt & 1;
+          wait_on(&bar_p[buf], ph_p[buf]);   // P(kt) is in tensor memory
+          wait_on(&bar_v[buf], ph_v[buf]);   // the consumers' V(kt) landed
+          if (!ok) break;
+          tc5_fence_after();
+#pragma unroll
+          for (int x = 0; x < NV; ++x)
+            if (x < n_cons)
+              umma_values(tmem + kColO + kTD * x, tmem + kColS + buf * kTN, buf ? vd[x][1] : vd[x][0], kIdescO,
+                          kt > 0 ? 1u : 0u);
+          umma_commit(&bar_o[buf]);
+        }
+      }
+    } else if (warp == 4) {
       // ---------------- issue warp: S(kt) = Q K(kt)^T into score buffer kt & 1, O += P(kt) V(kt)
       const uint64_t qd = umma_desc(sQ, 16, 1024);
       const uint64_t kd0 = umma_desc(sK, 16, 1024), kd1 = umma_desc(sK + kKV, 16, 1024);
@@ -1080,7 +1132,7 @@ cudaError_t launch_prefill_attend(const Params& p, const uint8_t* kind_dev, cons
       a.passes = passes_dev + n_single;
       const dim3 g3(grid5.x, grid5.y, n_shared);
       prefill_attend_tcgen05_kernel<false, kSharedPassLayers>
-          <<<g3, kTc5Threads, prefill_tcgen05_smem_bytes(kSharedPassLayers), stream>>>(a, p.err);
+          <<<g3, kTc5Threads + 32, prefill_tcgen05_smem_bytes(kSharedPassLayers), stream>>>(a, p.err);
     } else {
       prefill_attend_tcgen05_kernel<false, 1><<<grid5, kTc5Threads, prefill_tcgen05_smem_bytes(), stream>>>(a, p.err);
     }
