@@ -320,6 +320,20 @@ def _samples(w, n, rng):
     return out
 
 
+def test_options_reject_what_they_cannot_take():
+    w = _small_workload(128, 1, [0, 1], 24)
+    s = Session.for_workload(w, split_tokens=64)
+    for key, value in (("no_such_option", 1), ("layers_per_launch", -1), ("layers_per_launch", 3),
+                       ("prefill_shared_scores", 3), ("split_tokens", 24), ("split_tokens", 32), ("split_tokens", 1024)):
+        with pytest.raises(qc.QcError) as e:
+            s.set_option(key, value)
+        assert e.value.status == qc.QC_ERR_INVALID_ARG, (key, value)
+    for key, value in (("layers_per_launch", 1), ("per_layer_logit_cache", 1), ("per_layer_logit_cache", 0),
+                       ("prefill_shared_scores", 2), ("prefill_tcgen05", 0), ("split_tokens", 128), ("split_tokens", 0)):
+        s.set_option(key, value)
+    s.close()
+
+
 @pytest.mark.parametrize("mode", MODES, ids=MODE_IDS)
 def test_multi_turn_prefill_after_decode(mode):
     """A conversation with a second image: prompt, a few generated tokens, more prompt tokens
