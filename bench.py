@@ -204,6 +204,11 @@ def run_gpu(args, w, mode, rank, world, local_rank):
         s.set_option("layers_per_launch", args.blocks_per_launch)
     if args.per_layer:
         s.set_option("per_layer_logit_cache", 1)
+    if args.in_order:
+        s.set_option("in_order_launches", 1)
+    for kv in args.option:
+        key, value = kv.split("=")
+        s.set_option(key, int(value))
     inputs = _gen_inputs(w, 0, total_steps, dev, seq_offset)
     out = torch.empty(shape_o, dtype=torch.bfloat16, device=dev)
     for i in range(W_):
@@ -279,8 +284,11 @@ def run_gpu(args, w, mode, rank, world, local_rank):
         s2.close()
         return res
 
-    per_block = per_layer = None
-    if world == 1 and not args.no_per_block and not args.blocks_per_launch and not args.per_layer:
+    per_block = per_layer = in_order = None
+    if world == 1 and not args.no_per_block and not args.blocks_per_launch and not args.per_layer and not args.in_order:
+        in_order = ordered_arm("in_order_launches", 1,
+                               "one attention + merge launch per layer, layers in order; a leader's launch also "
+                               "sweeps its followers' cached V rows")
         per_block = ordered_arm("layers_per_launch", 1,
                                 "one attention + merge launch per lazy block, blocks in layer order")
         per_layer = ordered_arm("per_layer_logit_cache", 1,
@@ -352,6 +360,7 @@ def run_gpu(args, w, mode, rank, world, local_rank):
         "vs_all_full": all_full,
         "per_block_launches": per_block,
         "per_layer_launches": per_layer,
+        "in_order_launches": in_order,
         "step_ms_by_events": prof.step_ms / max(1, prof.steps),
         "paper_context": "paper reports ~35% KV saved and 1.5x-1.6x decode throughput for LLaVA-NeXT-7B on one 80GB A100 (whole model)",
     }
@@ -445,6 +454,9 @@ def main():
                     help="skip the comparison runs with one launch per lazy block / per layer")
     ap.add_argument("--per-layer", action="store_true",
                     help="run the main arm under the per-layer schedule with the logit cache (for profiling it)")
+    ap.add_argument("--in-order", action="store_true",
+                    help="run the main arm under the in-order schedule (for profiling it)")
+    ap.add_argument("--option", action="append", default=[], help="key=value passed to qc_set_option (main arm)")
     ap.add_argument("--dist-backend", default=None, help="torch.distributed backend (default: nccl on GPUs)")
     ap.add_argument("--force-device", type=int, default=-1,
                     help="use this CUDA device on every rank (to exercise the multi-rank plumbing on one GPU)")

@@ -47,7 +47,9 @@ enum {
   QC_ERR_OOM_PAGES = 3,   /* the pool has too few free pages for this call */
   QC_ERR_STATE = 4,       /* lazy layer 0, decode on an unknown sequence, duplicate id, ... */
   QC_ERR_CUDA = 5,        /* a CUDA runtime call failed */
-  QC_ERR_TIMEOUT = 6      /* a bounded wait inside a kernel ran out (device error word) */
+  QC_ERR_TIMEOUT = 6,     /* a bounded wait inside a kernel ran out (device error word) */
+  QC_ERR_BAD_PAGE = 7,    /* a kernel met a page id outside the pool and did not follow it (device error word) */
+  QC_ERR_PLAN = 8         /* a kernel met a work range outside the limits it was planned for (device error word) */
 };
 
 enum { QC_LAYER_FULL = 0, QC_LAYER_LAZY = 1 };

@@ -21,6 +21,8 @@ QC_ERR_OOM_PAGES = 3
 QC_ERR_STATE = 4
 QC_ERR_CUDA = 5
 QC_ERR_TIMEOUT = 6
+QC_ERR_BAD_PAGE = 7
+QC_ERR_PLAN = 8
 
 QC_LAYER_FULL, QC_LAYER_LAZY = 0, 1
 QC_MODE_VLA_QC, QC_MODE_VLA_EQ8, QC_MODE_GLA = 0, 1, 2

@@ -31,10 +31,6 @@ struct TcCtx {
   ItemPages ip;
 };
 
-__device__ __forceinline__ void load_tc_ctx(TcCtx& c, const Params& P, int item_idx, int lane) {
-  load_item_pages(c.ip, P, item_idx, lane);
-}
-
 // Byte offset of 16-byte chunk `chunk` (0 .. D/8-1) of row `row` inside a swizzled tile:
 // the tile is stored as column halves of 64 elements, each [16 rows][128 bytes], with the
 // chunk index inside a 128-byte row XORed with (row & 7).
@@ -48,12 +44,15 @@ __device__ __forceinline__ uint32_t swz(int row, int chunk) {
 // NQ == 1: every consumer shares the weights; NQ == NV: consumer x has its own queries.
 // MODE 1 (one query group, one consumer) also stores the scaled scores in the logit cache; MODE 2
 // takes them from there instead of reading K tiles (the ring then carries V tiles only).
-template <int D, int NQ, int NV, int MODE = 0>
+// SKIP (shared weights only): the consumers named in the item's skip_new mask leave out the
+// stream's last key (the step's new token): they get a copy of the weights with that key's set
+// to zero and their own sums.
+template <int D, int NQ, int NV, int MODE = 0, bool SKIP = false>
 __device__ __forceinline__ void process_item_tc(WorkerState& st, const TcCtx* ctx, uint32_t ring, uint64_t* full,
                                                 const Params& P, int lane) {
   constexpr int KS = D / 16;    // k-steps of the score product = m-tiles of the value product
-  auto ctx_of = [ctx](int k) -> const ItemPages& { return ctx[k & 1].ip; };
-  const Item& it = ctx[st.cons_k & 1].ip.item;
+  auto ctx_of = [ctx](int k) -> const ItemPages& { return ctx[k % kCtxSlots].ip; };
+  const Item& it = ctx[st.cons_k % kCtxSlots].ip.item;
   const int g = lane >> 2, t = lane & 3;
   const int n_heads = it.n_heads;
 
@@ -85,6 +84,9 @@ __device__ __forceinline__ void process_item_tc(WorkerState& st, const TcCtx* ct
 
   const int n_pages = it.n_pages;
   const int n_valid_last = it.n_valid_last;
+  const bool skip_here = SKIP && (it.flags & kFlagStreamEnd);
+  const uint32_t skip_mask = SKIP ? it.skip_new : 0u;
+  float l_skip[2] = {0.f, 0.f};
   // ldmatrix lane roles
   const int lrow = lane & 7, lmat = lane >> 3;
   const int k_row = lrow + ((lmat & 1) << 3), k_chunk = lmat >> 1;    // K: matrices (keys lo/hi) x (chunk +0/+1)
@@ -107,6 +109,8 @@ __device__ __forceinline__ void process_item_tc(WorkerState& st, const TcCtx* ct
   for (int pg = 0; pg < n_pages && !st.dead; ++pg) {
     const int nvalid = (pg == n_pages - 1) ? n_valid_last : kPage;
     uint32_t pb[NQ][2];
+    uint32_t pb_skip[2] = {0u, 0u};   // the weights without the new token (SKIP, last page only)
+    const bool skip_page = SKIP && skip_here && pg == n_pages - 1;
     // ---- K tile: scores of 16 keys for 8 heads
     {
       float s[NQ][4];
@@ -168,6 +172,18 @@ __device__ __forceinline__ void process_item_tc(WorkerState& st, const TcCtx* ct
         // weights as the B operand of the value product: keys 2t, 2t+1 (+8), head g
         pb[x][0] = movmatrix_trans(pack_bf16x2(p0, p1));
         pb[x][1] = movmatrix_trans(pack_bf16x2(p2, p3));
+        if (SKIP) {
+          float q0 = p0, q1 = p1, q2 = p2, q3 = p3;
+          if (skip_page) {
+            const int r_new = nvalid - 1;
+            if (g == r_new) q0 = q1 = 0.f;
+            if (g + 8 == r_new) q2 = q3 = 0.f;
+            pb_skip[0] = movmatrix_trans(pack_bf16x2(q0, q1));
+            pb_skip[1] = movmatrix_trans(pack_bf16x2(q2, q3));
+          }
+          l_skip[0] = fmaf(l_skip[0], c0, q0 + q2);
+          l_skip[1] = fmaf(l_skip[1], c1, q1 + q3);
+        }
         if (__any_sync(0xffffffffu, c0 != 1.f || c1 != 1.f)) {
 #pragma unroll
           for (int v = 0; v < NV; ++v) {
@@ -189,12 +205,14 @@ __device__ __forceinline__ void process_item_tc(WorkerState& st, const TcCtx* ct
     for (int v = 0; v < NV; ++v) {
       const uint32_t tile = wait_tile<D>(st, ring, full, P, lane);
       if (st.dead) break;
-      if (nvalid < kPage) {
+      const bool skipping = SKIP && skip_page && ((skip_mask >> v) & 1u);
+      const int nvalid_v = skipping ? nvalid - 1 : nvalid;
+      if (nvalid_v < kPage) {
         // rows past the end of the stream hold whatever the pool held: clear them, since a
         // zero weight does not cancel a NaN or an infinity
-        const int n_seg = (kPage - nvalid) * (D / 64);
+        const int n_seg = (kPage - nvalid_v) * (D / 64);
         for (int e = lane; e < n_seg * 8; e += 32) {
-          const int seg = e >> 3, half = seg / (kPage - nvalid), row = nvalid + seg % (kPage - nvalid);
+          const int seg = e >> 3, half = seg / (kPage - nvalid_v), row = nvalid_v + seg % (kPage - nvalid_v);
           asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(tile + (half << 11) + (row << 7) + ((e & 7) << 4)),
                        "r"(0u)
                        : "memory");
@@ -206,7 +224,8 @@ __device__ __forceinline__ void process_item_tc(WorkerState& st, const TcCtx* ct
       for (int i = 0; i < KS; ++i) {
         uint32_t a[4];
         ldmatrix_x4_trans(a, tile + swz<D>(v_row, 2 * i + v_chunk));
-        mma_bf16_16816(o[v][i], a, pb[NQ == 1 ? 0 : v]);
+        if (skipping) mma_bf16_16816(o[v][i], a, pb_skip);
+        else mma_bf16_16816(o[v][i], a, pb[NQ == 1 ? 0 : v]);
       }
       release_tile<kRingTc>(st);
       fill_ring<D, kRingTc, true>(st, ctx_of, ring, full, P, lane);
@@ -221,6 +240,13 @@ __device__ __forceinline__ void process_item_tc(WorkerState& st, const TcCtx* ct
     for (int off = 4; off < 32; off <<= 1) {
       l[x][0] += __shfl_xor_sync(0xffffffffu, l[x][0], off);
       l[x][1] += __shfl_xor_sync(0xffffffffu, l[x][1], off);
+    }
+  }
+  if (SKIP) {
+#pragma unroll
+    for (int off = 4; off < 32; off <<= 1) {
+      l_skip[0] += __shfl_xor_sync(0xffffffffu, l_skip[0], off);
+      l_skip[1] += __shfl_xor_sync(0xffffffffu, l_skip[1], off);
     }
   }
 #pragma unroll
@@ -239,9 +265,111 @@ __device__ __forceinline__ void process_item_tc(WorkerState& st, const TcCtx* ct
           dst[16 * i] = o[v][i][hh];
           dst[16 * i + 8] = o[v][i][2 + hh];
         }
-        if (g == 0) P.part_ml[row0 + hh] = make_float2(m[xq][hh], l[xq][hh]);
+        const bool skipped = SKIP && ((skip_mask >> v) & 1u);
+        if (g == 0) P.part_ml[row0 + hh] = make_float2(m[xq][hh], skipped ? l_skip[hh] : l[xq][hh]);
       }
     }
+  }
+  finish_rows<D>(P, ctx[st.cons_k % kCtxSlots].ip, lane);
+}
+
+// A worker's life: take items (claimed from the list, or the pieces of its static ranges), keep
+// the tile ring full across item boundaries, process each item.  While item k is processed the
+// ring already fetches tiles of item k + 1 and the context of item k + 2 (descriptor, page ids)
+// arrives by asynchronous copies.
+template <int D, bool STATIC>
+__device__ __forceinline__ void attend_tc_worker(const Params& P, TcCtx* ctx, uint32_t ring, uint64_t* full,
+                                                 RangeCursor* cursor, int wid, int lane) {
+  auto ctx_of = [ctx](int k) -> const ItemPages& { return ctx[k % kCtxSlots].ip; };
+  WorkerState st;
+  worker_init(st, 0);
+  Item it;
+  int issued = 0;
+  auto take = [&]() -> bool {   // the next item into `it`
+    if (STATIC) return cursor_step(cursor, P, it, lane);
+    const int idx = claim_take(P, issued);
+    if (idx < 0) return false;
+    it = load_item(P, idx);
+    return true;
+  };
+  // ---- ahead of the wait for the previous kernel: the first items and their page ids (from the
+  // launch plan, the step descriptors and the page tables, all written before that kernel
+  // started), and the first tiles unless they could hold the step's new token
+  if (STATIC) {
+    if (wid >= P.part_workers) return;
+    RangeCursor c;
+    const bool any = cursor_init(c, P, wid, lane);
+    if (lane == 0) *cursor = c;
+    __syncwarp();
+    if (!any) return;
+  } else {
+    issued = claim_issue(P, lane);
+  }
+  if (!take()) return;
+  begin_item_pages(ctx[0].ip, P, it, lane);
+  const Item first = it;
+  cp_async_wait_all();
+  __syncwarp();
+  st.n_my = 1;
+  const bool early_tiles = !(first.stream == 0 && (first.flags & kFlagStreamEnd) && first.n_pages <= kRingTc);
+  if (early_tiles) fill_ring<D, kRingTc, true>(st, ctx_of, ring, full, P, lane);
+  pdl_wait();
+  pdl_launch_dependents();
+  // ---- this layer's inputs; the rest of the first tiles; the second item's context while they fly
+  fill_ring<D, kRingTc, true>(st, ctx_of, ring, full, P, lane);
+  if (STATIC) record_row_slots(P, first, lane);
+  if (!STATIC) issued = claim_issue(P, lane);
+  bool more = take();
+  if (more) {
+    begin_item_pages(ctx[1].ip, P, it, lane);
+    if (STATIC) record_row_slots(P, it, lane);
+  }
+  cp_async_wait_all();
+  __syncwarp();
+  if (more) st.n_my = 2;
+  bool pending = false;   // a context is being filled for item st.n_my
+  if (!STATIC && more) issued = claim_issue(P, lane);
+
+  for (int k = 0; k < st.n_my && !st.dead; ++k) {
+    const Item& cur = ctx[k % kCtxSlots].ip.item;
+    const int nc = cur.n_cons;
+    const bool shared = cur.flags & kFlagShared;
+    if (more) {
+      // the third slot is free (it held the item before this one): start filling it with the item after next
+      more = take();
+      if (more) {
+        begin_item_pages(ctx[(k + 2) % kCtxSlots].ip, P, it, lane);
+        if (STATIC) record_row_slots(P, it, lane);
+        pending = true;
+      }
+    }
+    if (!STATIC && more) issued = claim_issue(P, lane);   // answered by the time the next item starts
+    if (nc == 1 && (cur.flags & kFlagReadLogits)) process_item_tc<D, 1, 1, 2>(st, ctx, ring, full, P, lane);
+    else if (nc == 1 && (cur.flags & kFlagWriteLogits)) process_item_tc<D, 1, 1, 1>(st, ctx, ring, full, P, lane);
+    else if (shared && cur.skip_new) {
+      if (nc == 1) process_item_tc<D, 1, 1, 0, true>(st, ctx, ring, full, P, lane);
+      else if (nc == 2) process_item_tc<D, 1, 2, 0, true>(st, ctx, ring, full, P, lane);
+      else if (nc == 3) process_item_tc<D, 1, 3, 0, true>(st, ctx, ring, full, P, lane);
+      else process_item_tc<D, 1, 4, 0, true>(st, ctx, ring, full, P, lane);
+    }
+    else if (nc == 1) process_item_tc<D, 1, 1>(st, ctx, ring, full, P, lane);
+    else if (shared && nc == 2) process_item_tc<D, 1, 2>(st, ctx, ring, full, P, lane);
+    else if (shared && nc == 3) process_item_tc<D, 1, 3>(st, ctx, ring, full, P, lane);
+    else if (shared) process_item_tc<D, 1, 4>(st, ctx, ring, full, P, lane);
+    else process_item_tc<D, 2, 2>(st, ctx, ring, full, P, lane);   // own-query sweeps feed at most two layers here
+    if (st.dead) break;
+    if (pending) {   // the context of item k + 2 has had this item's time to arrive
+      cp_async_wait_all();
+      __syncwarp();
+      st.n_my = k + 3;
+      pending = false;
+    }
+    st.cons_k = k + 1;
+    fill_ring<D, kRingTc, true>(st, ctx_of, ring, full, P, lane);
+  }
+  if (st.dead) {
+    cp_async_wait_all();
+    drain_ring<kRingTc>(st, full);
   }
 }
 
@@ -250,70 +378,31 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
   constexpr uint32_t kTile = kPage * D * 2;
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t full_all[kWarps][kRingTc];
+  __shared__ __align__(16) RangeCursor cursors[kWarps];
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // swizzled tiles must sit on 1024-byte boundaries
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
   const uint32_t ring = base + static_cast<uint32_t>(warp) * kRingTc * kTile;
-  TcCtx* ctx = reinterpret_cast<TcCtx*>(base_ptr + static_cast<size_t>(kWarps) * kRingTc * kTile) + warp * 2;
+  TcCtx* ctx = reinterpret_cast<TcCtx*>(base_ptr + static_cast<size_t>(kWarps) * kRingTc * kTile) + warp * kCtxSlots;
   uint64_t* full = full_all[warp];
-  auto ctx_of = [ctx](int k) -> const ItemPages& { return ctx[k & 1].ip; };
 
   if (lane == 0) {
     for (int s = 0; s < kRingTc; ++s) mbar_init(&full[s], 1);
     fence_mbar_init();
   }
   __syncthreads();
-  pdl_launch_dependents();
-  pdl_wait();
 
-  WorkerState st;
-  worker_init(st, 0);
-  int next = claim_take(P, claim_issue(P, lane));
-  if (next < 0) return;
-  load_tc_ctx(ctx[0], P, next, lane);
-  st.n_my = 1;
-  next = claim_take(P, claim_issue(P, lane));
-  if (next >= 0) {
-    load_tc_ctx(ctx[1], P, next, lane);
-    st.n_my = 2;
-  }
-  __syncwarp();
-  fill_ring<D, kRingTc, true>(st, ctx_of, ring, full, P, lane);
-
-  for (int k = 0; k < st.n_my && !st.dead; ++k) {
-    const Item& it = ctx[k & 1].ip.item;
-    const int nc = it.n_cons;
-    const bool shared = it.flags & kFlagShared;
-    // claim the item after next now; the answer is needed only when this item is done
-    const int issued = (next >= 0) ? claim_issue(P, lane) : 0;
-    if (nc == 1 && (it.flags & kFlagReadLogits)) process_item_tc<D, 1, 1, 2>(st, ctx, ring, full, P, lane);
-    else if (nc == 1 && (it.flags & kFlagWriteLogits)) process_item_tc<D, 1, 1, 1>(st, ctx, ring, full, P, lane);
-    else if (nc == 1) process_item_tc<D, 1, 1>(st, ctx, ring, full, P, lane);
-    else if (shared && nc == 2) process_item_tc<D, 1, 2>(st, ctx, ring, full, P, lane);
-    else if (shared && nc == 3) process_item_tc<D, 1, 3>(st, ctx, ring, full, P, lane);
-    else if (shared) process_item_tc<D, 1, 4>(st, ctx, ring, full, P, lane);
-    else process_item_tc<D, 2, 2>(st, ctx, ring, full, P, lane);   // own-query sweeps feed at most two layers here
-    if (st.dead) break;
-    __syncwarp();
-    if (next >= 0) {
-      next = claim_take(P, issued);
-      if (next >= 0) {   // the context slot of the item just finished receives the item after next
-        load_tc_ctx(ctx[k & 1], P, next, lane);
-        __syncwarp();
-        st.n_my = k + 3;
-      }
-    }
-    st.cons_k = k + 1;
-    fill_ring<D, kRingTc, true>(st, ctx_of, ring, full, P, lane);
-  }
-  if (st.dead) drain_ring<kRingTc>(st, full);
+  if (P.part_static)
+    attend_tc_worker<D, true>(P, ctx, ring, full, &cursors[warp], warp * gridDim.x + blockIdx.x, lane);
+  else
+    attend_tc_worker<D, false>(P, ctx, ring, full, &cursors[warp], 0, lane);
 }
 
 template <int D>
 constexpr int attend_tc_smem_bytes() {
-  return 1024 + kWarps * kRingTc * kPage * D * 2 + kWarps * 2 * static_cast<int>(sizeof(TcCtx));
+  return 1024 + kWarps * kRingTc * kPage * D * 2 + kWarps * kCtxSlots * static_cast<int>(sizeof(TcCtx));
 }
 
 }  // namespace
@@ -330,8 +419,8 @@ cudaError_t configure_kernels_tc(int* attend_smem) {
 
 cudaError_t launch_attend_tc(const Params& p, int n_sms, cudaStream_t stream) {
   const int n_items = p.item_end - p.item_begin;
-  if (n_items <= 0) return cudaSuccess;
-  const int grid = min(n_sms, (n_items + kWarps - 1) / kWarps);
+  if (!p.part_static && n_items <= 0) return cudaSuccess;
+  const int grid = p.part_static ? min(n_sms, p.part_workers) : min(n_sms, (n_items + kWarps - 1) / kWarps);
   if (p.d == 128)
     return launch_pdl(attend_tc_kernel<128>, dim3(grid), dim3(kThreads), attend_tc_smem_bytes<128>(), stream, p);
   return launch_pdl(attend_tc_kernel<64>, dim3(grid), dim3(kThreads), attend_tc_smem_bytes<64>(), stream, p);

@@ -16,8 +16,10 @@ constexpr int kWarps = kAttendWarps;
 constexpr int kThreads = kWarps * 32;
 constexpr uint32_t kSpinLimit = 1u << 22; // bounded mbarrier wait
 
+// values of the device error word (QC_ERR_* of the public header)
 constexpr int kErrTimeout = 6;
-constexpr int kErrBadPage = 5;
+constexpr int kErrBadPage = 7;
+constexpr int kErrPlan = 8;   // a work range did not fit the limits the host planned it for
 
 // ------------------------------------------------------------------------------------------
 // PTX helpers
@@ -52,11 +54,20 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint64_t* bar, uint32_t parity
 }
 // 1-D bulk copy global -> this CTA's shared memory, completion counted on an mbarrier.
 // Source, destination and size are multiples of 16 bytes by construction (whole page tiles).
-__device__ __forceinline__ void bulk_g2s(uint32_t dst_smem, const void* src, uint32_t bytes, uint64_t* bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                   dst_smem),
-               "l"(src), "r"(bytes), "r"(smem_u32(bar))
-               : "memory");
+// K/V tiles are read once per step: they are fetched with the evict-first L2 policy, so that the
+// stream of tiles does not push the page tables, the queries and the partial rows out of the L2.
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+  uint64_t policy;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+  return policy;
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst_smem, const void* src, uint32_t bytes, uint64_t* bar,
+                                         uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(
+          dst_smem),
+      "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(policy)
+      : "memory");
 }
 // 2-D tensor-map copy global -> this CTA's shared memory (the map applies the 128-byte
 // swizzle).  x is a multiple of 8 elements (16 bytes) by construction: 0 or 64.
@@ -68,11 +79,35 @@ __device__ __forceinline__ void tensor_g2s_2d(uint32_t dst_smem, const void* tma
       "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(smem_u32(bar))
       : "memory");
 }
+// the same with an L2 cache policy
+__device__ __forceinline__ void tensor_g2s_2d(uint32_t dst_smem, const void* tmap, int32_t x, int32_t y,
+                                              uint64_t* bar, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, "
+      "%3}], [%4], %5;" ::"r"(dst_smem),
+      "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(smem_u32(bar)), "l"(policy)
+      : "memory");
+}
+
+// Asynchronous global -> shared copies of 4 or 16 bytes (no registers held while in flight);
+// cp_async_wait_all() waits for the calling thread's own copies.
+__device__ __forceinline__ void cp_async_4(void* dst_smem, const void* src) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(dst_smem)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_16(void* dst_smem, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst_smem)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 
 // Programmatic dependent launch: the kernels of a decode step are launched back to back with
-// the programmatic-serialization attribute.  Each one first lets its successor start getting
-// scheduled, does its set-up that touches no global data, and then waits for its predecessor
-// to have completed (and its writes to be visible) before it reads or writes global memory.
+// the programmatic-serialization attribute.  Each one does the set-up that may run early, waits
+// for its predecessor to have completed (and its writes to be visible), and only then lets its
+// successor start getting scheduled.
+// Every kernel of the chain executes its wait BEFORE it lets its successor start, so when a kernel
+// starts running, the kernel before its predecessor -- and by induction everything earlier in
+// the stream -- has completed: what a kernel does ahead of its own wait may read anything that
+// was written two or more launches back (the attention kernels plan their first work items there,
+// from the launch plan, the step descriptors and the page tables).
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
@@ -161,6 +196,9 @@ __device__ __forceinline__ size_t table_row(const Params& P, int layer, int stre
 // Item descriptor and page ids of one item, as the ring needs them.
 struct ItemPages {
   Item item;
+  StepSeq sq;          // the item's sequence
+  int32_t kv_head;     // item.head / group
+  int32_t pad[3];
   int32_t pages[1 + kMaxCons][kMaxChunkPages];   // [0]: K pages, [1 + x]: V pages of consumer x
 };
 
@@ -173,6 +211,7 @@ struct WorkerState {
   uint32_t cons_phase;
   int in_flight;
   bool dead;           // a bounded wait ran out: stop fetching, drain, leave
+  uint64_t policy;     // L2 policy of the tile copies
 };
 
 __device__ __forceinline__ void worker_init(WorkerState& st, int n_my) {
@@ -183,6 +222,7 @@ __device__ __forceinline__ void worker_init(WorkerState& st, int n_my) {
   st.cons_phase = 0;
   st.in_flight = 0;
   st.dead = false;
+  st.policy = l2_evict_first_policy();
 }
 
 // Issue the copy of the next tile.  D: head dim; RING: slots; TMAP: copy through the tensor
@@ -207,12 +247,12 @@ __device__ __forceinline__ bool issue_one(WorkerState& st, CtxFn ctx, uint32_t r
     fence_proxy_async();   // the slot's earlier generic-proxy accesses precede this async write
     mbar_expect_tx(bar, kTile);
     if (TMAP) {
-      const int32_t row = (pid * P.hkv + c.item.kv_head) * kPage;
-      tensor_g2s_2d(dst, &P.tmap, 0, row, bar);
-      if (D == 128) tensor_g2s_2d(dst + kTile / 2, &P.tmap, 64, row, bar);
+      const int32_t row = (pid * P.hkv + c.kv_head) * kPage;
+      tensor_g2s_2d(dst, &P.tmap, 0, row, bar, st.policy);
+      if (D == 128) tensor_g2s_2d(dst + kTile / 2, &P.tmap, 64, row, bar, st.policy);
     } else {
-      const uint16_t* src = P.pool + (static_cast<size_t>(pid) * P.hkv + c.item.kv_head) * (kPage * D);
-      bulk_g2s(dst, src, kTile, bar);
+      const uint16_t* src = P.pool + (static_cast<size_t>(pid) * P.hkv + c.kv_head) * (kPage * D);
+      bulk_g2s(dst, src, kTile, bar, st.policy);
     }
   }
   st.iss_slot = (st.iss_slot + 1 == RING) ? 0 : st.iss_slot + 1;
@@ -276,23 +316,34 @@ __device__ __forceinline__ void drain_ring(WorkerState& st, uint64_t* full) {
   }
 }
 
-// Fetch an item's descriptor and page ids into the warp's context slot.  Returns the item.
-__device__ __forceinline__ Item load_item_pages(ItemPages& c, const Params& P, int item_idx, int lane) {
+// A warp keeps the contexts of three items: the one it consumes, the next one (whose tiles the ring
+// already fetches) and the one after, which is being filled by asynchronous copies meanwhile.
+constexpr int kCtxSlots = 3;
+
+// Start filling a context slot with an item and the page ids of its K stream and V streams
+// (asynchronous copies; cp_async_wait_all() + __syncwarp() completes them).
+__device__ __forceinline__ void begin_item_pages(ItemPages& c, const Params& P, const Item& it, int lane) {
+  __syncwarp();   // the slot's previous item is no longer read
+  if (lane == 0) {
+    c.item = it;
+    c.kv_head = it.head / P.group;
+  }
+  if (lane >= 30) cp_async_16(reinterpret_cast<uint4*>(&c.sq) + (lane - 30), reinterpret_cast<const uint4*>(P.seqs + it.seq_idx) + (lane - 30));
+  if (lane < it.n_pages) {
+    cp_async_4(&c.pages[0][lane], P.table + table_row(P, it.k_layer, it.stream, it.seq_id) + it.first_page + lane);
+    for (int x = 0; x < it.n_cons; ++x)
+      cp_async_4(&c.pages[1 + x][lane],
+                 P.table + table_row(P, it.v_layer[x], 2 + it.stream, it.seq_id) + it.first_page + lane);
+  }
+}
+
+// Fetch an item's descriptor from the item list.
+__device__ __forceinline__ Item load_item(const Params& P, int item_idx) {
   const uint4* ip = reinterpret_cast<const uint4*>(P.items + item_idx);
   uint4 a = __ldg(ip), b = __ldg(ip + 1);
-  __syncwarp();
-  if (lane == 0) {
-    reinterpret_cast<uint4*>(&c.item)[0] = a;
-    reinterpret_cast<uint4*>(&c.item)[1] = b;
-  }
   Item it;
   reinterpret_cast<uint4*>(&it)[0] = a;
   reinterpret_cast<uint4*>(&it)[1] = b;
-  if (lane < it.n_pages) {
-    c.pages[0][lane] = P.table[table_row(P, it.k_layer, it.stream, it.seq_id) + it.first_page + lane];
-    for (int x = 0; x < it.n_cons; ++x)
-      c.pages[1 + x][lane] = P.table[table_row(P, it.v_layer[x], 2 + it.stream, it.seq_id) + it.first_page + lane];
-  }
   return it;
 }
 
@@ -315,6 +366,379 @@ __device__ __forceinline__ float* logit_row(const Params& P, int stream, int seq
 __device__ __forceinline__ int claim_take(const Params& P, int issued) {
   const int idx = __shfl_sync(0xffffffffu, issued, 0);
   return idx < P.item_end - P.item_begin ? P.item_begin + idx : -1;
+}
+
+// ------------------------------------------------------------------------------------------
+// static partition of a launch
+// ------------------------------------------------------------------------------------------
+//
+// The work of a launch is laid out in tiles: plan positions of the launch in order, inside a
+// position the listed sequences, inside a sequence the rows (one per query head, or per query
+// group with GQA), inside a row its pages, each page worth w tiles (one K tile unless the scores
+// come from the logit cache, one V tile per consumer).  The space of T tiles is cut into ranges of
+// part_q tiles; a page belongs to the range its first tile falls into.  Physical worker i takes
+// ranges i*part_k .. i*part_k + part_k - 1, which are adjacent, so it walks rows forward from one
+// starting point.  The pages of a row that one range owns are one piece: an Item whose partial
+// result goes to slot (range - range owning the row's first page) of the row's stream.  The host
+// plans part_q so that a range is at least as long as any page (every range between a row's
+// first and last owns a page of it: no slot is left unwritten), a piece has at most
+// kMaxChunkPages pages and a row at most slots_per_stream pieces; T < 2^31.
+
+struct RangeCursor {
+  int32_t r0;        // tile offset of the current row
+  int32_t vw_end;    // first tile beyond the current range
+  int32_t vw, vw_stop;
+  int32_t pos, si, u;
+  int32_t row_pages, w;     // pages of the current row; tiles per page of its job
+  int32_t page;             // next page of the current row to hand out
+  int32_t owner0;           // range that owns the row's first page
+  int32_t len, seq_id;      // tokens of the row's stream; its sequence
+  int32_t pad;
+  Job job;
+};
+static_assert(sizeof(RangeCursor) == 72, "RangeCursor layout");
+
+__device__ __forceinline__ int job_tiles_per_page(const Job& j) {
+  return ((j.flags & kFlagReadLogits) ? 0 : 1) + j.n_cons;
+}
+
+// Load the job of plan position c.pos (if it changed) and the sequence c.si into the cursor.
+__device__ __forceinline__ void cursor_load_segment(RangeCursor& c, const Params& P, bool new_pos) {
+  if (new_pos) {
+    const uint4 raw = __ldg(reinterpret_cast<const uint4*>(P.plan + c.pos));
+    *reinterpret_cast<uint4*>(&c.job) = raw;
+    c.w = job_tiles_per_page(c.job);
+  }
+  const StepSeq sq = P.seqs[c.si];
+  c.len = c.job.stream ? sq.len_vis : sq.len_text;
+  c.seq_id = sq.seq_id;
+  c.row_pages = (c.len + kPage - 1) / kPage;
+}
+
+// Place the cursor of worker `wid` at its first range; false if the worker has no work.  All
+// lanes compute the same values.  Reads the launch plan and the step's sequence descriptors only,
+// the first 32 of each in one round of loads.
+__device__ __forceinline__ bool cursor_init(RangeCursor& c, const Params& P, int wid, int lane) {
+  const int32_t R = P.heads_per_item_dim;
+  c.vw = wid * P.part_k;
+  c.vw_stop = min(c.vw + P.part_k, P.part_vw);
+  if (c.vw >= c.vw_stop) return false;
+  const int32_t t0 = c.vw * P.part_q;
+  c.vw_end = t0 + P.part_q;
+  const int n_pos = P.pos_end - P.pos_begin;
+  uint4 pj_lo = make_uint4(0, 0, 0, 0);
+  int4 pj_hi = make_int4(0, 0, 0, 0);
+  int4 sq_lo = make_int4(0, 0, 0, 0), sq_hi = make_int4(0, 0, 0, 0);
+  if (lane < n_pos) {
+    pj_lo = __ldg(reinterpret_cast<const uint4*>(P.plan + P.pos_begin + lane));
+    pj_hi = __ldg(reinterpret_cast<const int4*>(P.plan + P.pos_begin + lane) + 1);
+  }
+  if (lane < P.n_seqs) {
+    sq_lo = reinterpret_cast<const int4*>(P.seqs + lane)[0];   // seq_id, len_text, len_vis, n_slots
+    sq_hi = reinterpret_cast<const int4*>(P.seqs + lane)[1];   // pre_v, pre_t, ncv, pad
+  }
+  // plan position: the last one of the launch that starts at or before t0
+  auto pos_base_of = [&](int wv_before, int wt_before) { return R * (wv_before * P.tp_v + wt_before * P.tp_t); };
+  int n_le = __popc(__ballot_sync(0xffffffffu, lane < n_pos && pos_base_of(pj_hi.z, pj_hi.w) <= t0));
+  int32_t pos_base;
+  if (n_le == 32 && n_pos > 32) {   // beyond the first round
+    for (int base = P.pos_begin + 32; base < P.pos_end; base += 32) {
+      const int idx = base + lane;
+      bool le = false;
+      if (idx < P.pos_end) {
+        const int4 hi = __ldg(reinterpret_cast<const int4*>(P.plan + idx) + 1);
+        le = pos_base_of(hi.z, hi.w) <= t0;
+      }
+      n_le += __popc(__ballot_sync(0xffffffffu, le));
+    }
+    c.pos = P.pos_begin + n_le - 1;
+    const PlanJob pj = P.plan[c.pos];
+    c.job = pj.job;
+    pos_base = pos_base_of(pj.wv_before, pj.wt_before);
+  } else {
+    const int src = max(n_le, 1) - 1;
+    c.pos = P.pos_begin + src;
+    uint4 j;
+    j.x = __shfl_sync(0xffffffffu, pj_lo.x, src);
+    j.y = __shfl_sync(0xffffffffu, pj_lo.y, src);
+    j.z = __shfl_sync(0xffffffffu, pj_lo.z, src);
+    j.w = __shfl_sync(0xffffffffu, pj_lo.w, src);
+    *reinterpret_cast<uint4*>(&c.job) = j;
+    pos_base = pos_base_of(__shfl_sync(0xffffffffu, pj_hi.z, src), __shfl_sync(0xffffffffu, pj_hi.w, src));
+  }
+  c.w = job_tiles_per_page(c.job);
+  // listed sequence: the last one whose rows start at or before t0
+  n_le = __popc(__ballot_sync(0xffffffffu, lane < P.n_seqs && pos_base + R * c.w * (c.job.stream ? sq_hi.x : sq_hi.y) <= t0));
+  int32_t my_pre;
+  if (n_le == 32 && P.n_seqs > 32) {
+    for (int base = 32; base < P.n_seqs; base += 32) {
+      const int idx = base + lane;
+      bool le = false;
+      if (idx < P.n_seqs) le = pos_base + R * c.w * (c.job.stream ? P.seqs[idx].pre_v : P.seqs[idx].pre_t) <= t0;
+      n_le += __popc(__ballot_sync(0xffffffffu, le));
+    }
+    c.si = n_le - 1;
+    const StepSeq sq = P.seqs[c.si];
+    c.len = c.job.stream ? sq.len_vis : sq.len_text;
+    c.seq_id = sq.seq_id;
+    my_pre = c.job.stream ? sq.pre_v : sq.pre_t;
+  } else {
+    const int src = max(n_le, 1) - 1;
+    c.si = src;
+    c.len = __shfl_sync(0xffffffffu, c.job.stream ? sq_lo.z : sq_lo.y, src);
+    c.seq_id = __shfl_sync(0xffffffffu, sq_lo.x, src);
+    my_pre = __shfl_sync(0xffffffffu, c.job.stream ? sq_hi.x : sq_hi.y, src);
+  }
+  c.row_pages = (c.len + kPage - 1) / kPage;
+  const int32_t seg_base = pos_base + R * c.w * my_pre;
+  c.u = 0;
+  c.r0 = seg_base;
+  c.page = 0;
+  if (c.row_pages > 0) {
+    const int32_t row_tiles = c.w * c.row_pages;
+    c.u = min(R - 1, (t0 - seg_base) / row_tiles);
+    c.r0 = seg_base + c.u * row_tiles;
+    c.page = (t0 - c.r0 + c.w - 1) / c.w;   // first page that starts at or after t0
+  }
+  c.owner0 = c.r0 / P.part_q;
+  c.pad = 0;
+  return true;
+}
+
+// Next piece of the worker's ranges, or false when they are used up.  Warp-uniform.
+__device__ __forceinline__ bool cursor_next(RangeCursor& c, const Params& P, Item& it) {
+  const int R = P.heads_per_item_dim;
+  for (;;) {
+    if (c.vw >= c.vw_stop) return false;
+    if (c.page >= c.row_pages) {   // next row
+      c.r0 += c.w * c.row_pages;
+      c.page = 0;
+      if (++c.u == R) {
+        c.u = 0;
+        bool new_pos = false;
+        if (++c.si == P.n_seqs) {
+          c.si = 0;
+          new_pos = true;
+          if (++c.pos >= P.pos_end) {
+            c.vw = c.vw_stop;
+            return false;
+          }
+        }
+        cursor_load_segment(c, P, new_pos);
+      }
+      c.owner0 = c.r0 / P.part_q;
+      continue;
+    }
+    const int32_t d = c.vw_end - c.r0;
+    const int lim = d <= 0 ? 0 : min(c.row_pages, (d + c.w - 1) / c.w);
+    if (c.page < lim) {
+      const int hpi = P.heads_per_item;
+      const int n_sub = (P.group + hpi - 1) / hpi;
+      const int kv_head = c.u / n_sub, sub = c.u - kv_head * n_sub;
+      const int slot = c.vw - c.owner0;
+      it.k_layer = c.job.k_layer;
+      it.stream = c.job.stream;
+      it.n_cons = c.job.n_cons;
+      it.flags = c.job.flags;
+#pragma unroll
+      for (int x = 0; x < kMaxCons; ++x) {
+        it.v_layer[x] = c.job.v_layer[x];
+        it.q_layer[x] = c.job.q_layer[x];
+      }
+      it.seq_id = static_cast<uint16_t>(c.seq_id);
+      it.seq_idx = static_cast<uint16_t>(c.si);
+      it.head = static_cast<uint16_t>(kv_head * P.group + sub * hpi);
+      it.slot = static_cast<uint16_t>((c.job.stream ? 0 : P.slots_per_stream) + slot);
+      it.first_page = static_cast<uint16_t>(c.page);
+      it.n_pages = static_cast<uint16_t>(lim - c.page);
+      const bool last = lim == c.row_pages;
+      if (last) it.flags |= kFlagStreamEnd;
+      it.n_valid_last = static_cast<uint16_t>(last ? c.len - (c.row_pages - 1) * kPage : kPage);
+      it.n_heads = static_cast<uint8_t>(min(hpi, P.group - sub * hpi));
+      it.skip_new = c.job.skip_new;
+      it.finish = c.job.finish;
+      it.pad1 = 0;
+      // the piece that holds a row's first page tells the merge how many pieces the row has
+      it.n_pieces = c.page == 0 ? static_cast<uint16_t>((c.r0 + c.w * (c.row_pages - 1)) / P.part_q - c.owner0 + 1) : 0;
+      if (lim - c.page > kMaxChunkPages || slot < 0 || slot >= P.slots_per_stream) {   // outside the plan's limits
+        atomicMax(P.err, kErrPlan);
+        c.vw = c.vw_stop;
+        return false;
+      }
+      c.page = lim;
+      return true;
+    }
+    // the current range owns nothing (more) of this row
+    ++c.vw;
+    c.vw_end += P.part_q;
+  }
+}
+
+// One step of a worker's cursor, kept in shared memory between items.  Warp-uniform.
+__device__ __forceinline__ bool cursor_step(RangeCursor* slot, const Params& P, Item& it, int lane) {
+  __syncwarp();
+  RangeCursor c = *slot;
+  const bool ok = cursor_next(c, P, it);
+  __syncwarp();
+  if (lane == 0) *slot = c;
+  __syncwarp();
+  return ok;
+}
+
+// Under the static partition, the piece that holds a row's first page records how many pieces
+// the row has: one entry per consumer layer and query head, visual and text streams side by side.
+__device__ __forceinline__ void record_row_slots(const Params& P, const Item& it, int lane) {
+  if (it.n_pieces == 0) return;
+  const int x = lane >> 3, h = lane & 7;
+  if (x < it.n_cons && h < it.n_heads) {
+    const size_t row = (static_cast<size_t>(it.v_layer[x]) * P.max_seqs + it.seq_idx) * P.hq + it.head + h;
+    P.row_slots[2 * row + (it.stream ? 0 : 1)] = it.n_pieces;
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// log-sum-exp merge of one output row's partials (one warp)
+// ------------------------------------------------------------------------------------------
+//
+// Used by the merge kernel and by the attention workers (the worker that delivers a row's last
+// partial merges it).  Partials may have been written by other SMs moments ago: they are read
+// past the L1 cache.  extra_leader >= 0 adds the step's new token as one more key (merge kernel,
+// rows of a GLA follower under the in-order schedule; Eq. 6).
+template <int D>
+__device__ __forceinline__ void merge_row(const Params& P, int layer, int si, int head, const StepSeq& sq, int lane,
+                                          int extra_leader) {
+  constexpr int VPL = D / 32;
+  const size_t base = (static_cast<size_t>(layer) * P.max_seqs + si) * P.max_slots;
+  // Partial rows of this output row: nv from the visual sweep in slots 0.., nt from the text
+  // sweep in slots text0...  With claimed items both counts follow from the stream lengths; under
+  // the static partition the sweeps recorded them.
+  int nv = sq.ncv, nt = sq.n_slots - sq.ncv, text0 = sq.ncv;
+  if (P.part_static) {
+    const size_t row = (static_cast<size_t>(layer) * P.max_seqs + si) * P.hq + head;
+    const uint32_t both = __ldcg(reinterpret_cast<const uint32_t*>(P.row_slots + 2 * row));
+    nv = sq.len_vis > 0 ? static_cast<int>(both & 0xffffu) : 0;
+    nt = static_cast<int>(both >> 16);
+    text0 = P.slots_per_stream;
+  }
+  const int n_slots = nv + nt;
+  auto phys = [&](int s) { return s < nv ? s : text0 + (s - nv); };
+
+  // Lane s holds the (max, sum) pair of slot s; the accumulator rows do not depend on them, so
+  // their loads are issued four at a time without waiting for the pairs.
+  float mmax = -INFINITY;
+  float2 my_ml = make_float2(-INFINITY, 0.f);
+  if (lane < n_slots) my_ml = __ldcg(P.part_ml + (base + phys(lane)) * P.hq + head);
+  mmax = my_ml.x;
+  for (int s = lane + 32; s < n_slots; s += 32) mmax = fmaxf(mmax, __ldcg(P.part_ml + (base + phys(s)) * P.hq + head).x);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xffffffffu, mmax, o));
+
+  float s_new = -INFINITY;
+  const uint16_t* v_new = nullptr;
+  if (extra_leader >= 0) {
+    const int kvh = head / P.group;
+    const uint16_t* qrow = P.qcache + ((static_cast<size_t>(extra_leader) * P.max_seqs + sq.seq_id) * P.hq + head) * D;
+    const uint16_t* krow = P.k + ((static_cast<size_t>(extra_leader) * P.n_seqs + si) * P.hkv + kvh) * D;
+    v_new = P.v + ((static_cast<size_t>(layer) * P.n_seqs + si) * P.hkv + kvh) * D + lane * VPL;
+    float dot = 0.f;
+#pragma unroll
+    for (int e = 0; e < VPL; ++e)
+      dot = fmaf(__uint_as_float(static_cast<uint32_t>(qrow[lane * VPL + e]) << 16),
+                 __uint_as_float(static_cast<uint32_t>(krow[lane * VPL + e]) << 16), dot);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+    s_new = dot * P.scale_log2;
+    mmax = fmaxf(mmax, s_new);
+  }
+
+  float lsum = 0.f;
+  float acc[VPL];
+#pragma unroll
+  for (int e = 0; e < VPL; ++e) acc[e] = 0.f;
+  if (v_new != nullptr) {
+    const float w = exp2f(s_new - mmax);
+    lsum = w;
+#pragma unroll
+    for (int e = 0; e < VPL; ++e) acc[e] = w * __uint_as_float(static_cast<uint32_t>(v_new[e]) << 16);
+  }
+  for (int s0 = 0; s0 < n_slots; s0 += 4) {
+    float v[4][VPL];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int s = phys(min(s0 + u, n_slots - 1));
+      const float* src = P.part_acc + ((base + s) * P.hq + head) * D + lane * VPL;
+      if (VPL == 4) {
+        const float4 a = __ldcg(reinterpret_cast<const float4*>(src));
+        v[u][0] = a.x, v[u][1] = a.y, v[u][2 % VPL] = a.z, v[u][3 % VPL] = a.w;
+      } else {
+        const float2 a = __ldcg(reinterpret_cast<const float2*>(src));
+        v[u][0] = a.x, v[u][1] = a.y;
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int s = s0 + u;
+      float2 ml;
+      if (s < 32) {
+        ml.x = __shfl_sync(0xffffffffu, my_ml.x, s & 31);
+        ml.y = __shfl_sync(0xffffffffu, my_ml.y, s & 31);
+      } else {
+        ml = __ldcg(P.part_ml + (base + phys(min(s, n_slots - 1))) * P.hq + head);
+      }
+      if (s < n_slots && ml.y > 0.f) {   // (a sweep that left out its only key has an empty partial)
+        const float w = exp2f(ml.x - mmax);
+        lsum = fmaf(ml.y, w, lsum);
+#pragma unroll
+        for (int e = 0; e < VPL; ++e) acc[e] = fmaf(v[u][e], w, acc[e]);
+      }
+    }
+  }
+  const float inv = 1.f / lsum;
+  const size_t orow = ((static_cast<size_t>(layer) * P.n_seqs + si) * P.hq + head);
+  uint16_t* dst = P.out + orow * D + lane * VPL;
+  if (VPL == 4) {
+    uint2 o;
+    o.x = f32_to_bf16_rne(acc[0] * inv) | (static_cast<uint32_t>(f32_to_bf16_rne(acc[1] * inv)) << 16);
+    o.y = f32_to_bf16_rne(acc[2 % VPL] * inv) | (static_cast<uint32_t>(f32_to_bf16_rne(acc[3 % VPL] * inv)) << 16);
+    *reinterpret_cast<uint2*>(dst) = o;
+  } else {
+    const uint32_t o = f32_to_bf16_rne(acc[0] * inv) | (static_cast<uint32_t>(f32_to_bf16_rne(acc[1] * inv)) << 16);
+    *reinterpret_cast<uint32_t*>(dst) = o;
+  }
+  if (P.lse != nullptr && lane == 0) P.lse[orow] = (mmax + log2f(lsum)) * 0.6931471805599453f;
+}
+
+// After an item's partial rows have been stored: count the item's pages towards the output rows
+// that this launch completes (the job's finish bits), and merge a row whose count is full.  The
+// count of a row is the pages of its visual and text streams, or of the item's stream alone when
+// only that stream is swept for the row in this launch.  Release / acquire: every lane fences its
+// stores before lane 0's atomic, and the merging warp fences again before it reads.
+template <int D>
+__device__ __forceinline__ void finish_rows(const Params& P, const ItemPages& c, int lane) {
+  const Item& it = c.item;
+  if ((it.finish & 0xf) == 0) return;
+  __threadfence();
+  __syncwarp();
+  const StepSeq sq = c.sq;
+  const int own_pages = ((it.stream ? sq.len_vis : sq.len_text) + kPage - 1) / kPage;
+  const int total = (it.finish & kFinishOwnStream)
+                        ? own_pages
+                        : (sq.len_vis + kPage - 1) / kPage + (sq.len_text + kPage - 1) / kPage;
+  // one counter per (consumer layer, sequence, first head of the item)
+  int old = 0;
+  if (lane < it.n_cons && ((it.finish >> lane) & 1)) {
+    const size_t row = (static_cast<size_t>(it.v_layer[lane]) * P.max_seqs + it.seq_idx) * P.hq + it.head;
+    old = atomicAdd(P.row_done + row, static_cast<int>(it.n_pages));
+  }
+  for (int x = 0; x < it.n_cons; ++x) {
+    if (!((it.finish >> x) & 1)) continue;
+    const int before = __shfl_sync(0xffffffffu, old, x);
+    if (before + it.n_pages != total) continue;
+    __threadfence();
+    const size_t row = (static_cast<size_t>(it.v_layer[x]) * P.max_seqs + it.seq_idx) * P.hq + it.head;
+    if (lane == 0) P.row_done[row] = 0;   // ready for the next step
+    for (int h = 0; h < it.n_heads; ++h) merge_row<D>(P, it.v_layer[x], it.seq_idx, it.head + h, sq, lane, -1);
+  }
 }
 
 }  // namespace

@@ -17,6 +17,7 @@ constexpr int kAttendWarps = 12;   // independent workers (warps) per attention 
 constexpr uint8_t kFlagShared = 1;      // one query scores for every consumer (same weights)
 constexpr uint8_t kFlagWriteLogits = 2; // the sweep also stores its scaled scores in the logit cache
 constexpr uint8_t kFlagReadLogits = 4;  // the sweep takes its scores from the logit cache: no K tile is read
+constexpr uint8_t kFlagStreamEnd = 8;   // (items only) the item's last page is the last page of its stream
 constexpr int kFlagCachedShift = 4;     // bit (4 + x): consumer x's query is read from the Q Cache
 
 // layer flags
@@ -29,15 +30,23 @@ struct Job {
   uint8_t k_layer, stream, n_cons, flags;
   uint8_t v_layer[kMaxCons];
   uint8_t q_layer[kMaxCons];
-  uint32_t pad;
+  uint8_t skip_new;   // bit x: consumer x leaves out the stream's last key (the step's new token, whose
+                      // value row of that layer does not exist yet when the sweep runs)
+  uint8_t finish;     // bit x: consumer x's output rows are complete once this launch's sweeps of them are
+                      // done, so the worker that delivers a row's last partial merges it (no merge launch);
+                      // kFinishOwnStream: only this job's stream contributes to those rows in this launch
+  uint8_t pad[2];
 };
+constexpr uint8_t kFinishOwnStream = 0x10;
 static_assert(sizeof(Job) == 16, "Job layout");
 
 // One position of the launch plan: a job plus how many visual-stream and text-stream jobs
-// precede it in the item list (all launches of a step share one list).  Static per cache.
+// precede it in the item list (all launches of a step share one list), and the tiles per page
+// (one K tile unless the scores come from the logit cache, one V tile per consumer) of the
+// visual-stream and text-stream jobs that precede it in its own launch.  Static per cache.
 struct __align__(16) PlanJob {
   Job job;
-  int32_t vis_before, text_before, pad0, pad1;
+  int32_t vis_before, text_before, wv_before, wt_before;
 };
 static_assert(sizeof(PlanJob) == 32, "PlanJob layout");
 
@@ -49,14 +58,17 @@ struct __align__(16) Item {
   uint16_t seq_id, seq_idx;
   uint16_t head, slot;
   uint16_t first_page, n_pages;
-  uint16_t n_valid_last, kv_head;
-  uint16_t n_heads, pad1;       // query heads head .. head + n_heads - 1 share the KV head (1 without GQA)
+  uint16_t n_valid_last;
+  uint8_t skip_new, finish;     // as in Job
+  uint8_t n_heads, pad1;        // query heads head .. head + n_heads - 1 share a KV head (head / group); 1 without GQA
+  uint16_t n_pieces;            // static partition, the piece with a row's first page: pieces of the row; else 0
 };
 static_assert(sizeof(Item) == 32, "Item layout");
 
 // One listed sequence of a step.  Lengths count the new token; ncv chunks of the visual stream
 // come first among the n_slots partial slots of an output row; pre_v / pre_t are the numbers
-// of items that the sequences listed before this one contribute to one visual / text job.
+// of items that the sequences listed before this one contribute to one visual / text job
+// (under the static partition of a launch: the pages of their visual / text streams).
 struct __align__(16) StepSeq {
   int32_t seq_id, len_text, len_vis, n_slots;
   int32_t pre_v, pre_t, ncv, pad;
@@ -92,6 +104,10 @@ struct Params {
   const uint8_t* layer_flags;
   int32_t* err;
   int32_t* work_counter;   // [n_layers] next unclaimed item of each attention launch of a step
+  uint16_t* row_slots;     // [n_layers][max_seqs][hq][2]: partial rows the visual / the text sweep left for an
+                           // output row (static partition only)
+  int32_t* row_done;       // [n_layers][max_seqs][hq]: pages of an output row swept so far in the current launch
+                           // (the worker that completes the count merges the row and resets it)
   int64_t n_pool_pages;    // bound for page ids (reads never leave the pool)
   int32_t n_layers, hq, hkv, d, group, max_seqs, max_pages, max_slots, chunk_pages;
   int32_t heads_per_item_dim;   // work items per (chunk, sequence): hq, or with GQA hkv * ceil(group / 8)
@@ -110,6 +126,18 @@ struct Params {
   int32_t item_begin, item_end;      // range handled by one attention launch
   int32_t launch_index;              // which work counter that launch uses
   int32_t layer_begin, layer_end;    // range handled by one merge launch
+  // static partition of an attention launch: the launch's work, counted in tiles in the order
+  // plan position -> listed sequence -> row (head or query group) -> page, is cut into part_vw
+  // ranges of part_q tiles; worker w takes ranges w * part_k .. w * part_k + part_k - 1.  A page
+  // belongs to the range its first tile falls into.
+  int32_t part_static;               // 0: items are claimed from the list
+  int32_t part_vw, part_k, part_workers;
+  int32_t part_q, part_tiles;        // tiles per range; tiles of the launch
+  int32_t tp_v, tp_t;                // pages of the visual / text streams, summed over the listed sequences
+  int32_t pos_begin, pos_end;        // plan positions of the launch
+  int32_t slots_per_stream;          // partial-row slots of one stream of an output row (text slots start here)
+  int32_t extra_key_leader;          // merge only, >= 0: the rows also take the step's new token as one more key,
+                                     // scored by that layer's Q Cache entry and new k (Eq. 6), valued by the own new v
 };
 
 // launchers (qc_kernels.cu); all asynchronous on `stream`

@@ -64,8 +64,7 @@ __device__ __forceinline__ void append_rows(const Params& P, const StepSeq& sq, 
 // n_layers blocks do the append.  (The append reads page ids from the table, so it is only
 // fused on steps without patches.)
 __global__ void setup_kernel(const __grid_constant__ Params P, const __grid_constant__ StepInline inl) {
-  pdl_launch_dependents();
-  pdl_wait();
+  pdl_wait();   // (no early start of the successor: it plans its work from what this kernel writes)
   const StepSeq* seqs = P.inline_seqs ? inl.seqs : P.seqs;
   const int n_expand = P.n_pos * P.n_seqs;
   const int n_house = (max(max(P.n_patches, P.n_layers), P.n_seqs * 8) + blockDim.x - 1) / blockDim.x;
@@ -120,10 +119,13 @@ __global__ void setup_kernel(const __grid_constant__ Params P, const __grid_cons
     it.first_page = static_cast<uint16_t>(first);
     it.n_pages = static_cast<uint16_t>(np);
     const bool last = (first + np == total_pages);
+    if (last) it.flags |= kFlagStreamEnd;
     it.n_valid_last = static_cast<uint16_t>(last ? len - (total_pages - 1) * kPage : kPage);
-    it.kv_head = static_cast<uint16_t>(kv_head);
-    it.n_heads = static_cast<uint16_t>(min(hpi, P.group - sub * hpi));
+    it.n_heads = static_cast<uint8_t>(min(hpi, P.group - sub * hpi));
+    it.skip_new = jb.skip_new;
+    it.finish = jb.finish;
     it.pad1 = 0;
+    it.n_pieces = 0;
     P.items[item_base + t] = it;
   }
 }
@@ -133,7 +135,6 @@ __global__ void setup_kernel(const __grid_constant__ Params P, const __grid_cons
 // ------------------------------------------------------------------------------------------
 
 __global__ void append_kernel(const __grid_constant__ Params P) {
-  pdl_launch_dependents();
   pdl_wait();
   append_rows(P, P.seqs[blockIdx.x], blockIdx.x, P.layer_begin + blockIdx.y);   // layers of one launch group
 }
@@ -180,10 +181,9 @@ struct WarpCtx {
   uint4 qraw[kMaxCons][D / 8];
 };
 
-// Fetch an item's descriptor, page ids and raw queries into the warp's context slot.
+// Start fetching the raw queries of the item in a context slot (asynchronous copies).
 template <int D>
-__device__ __forceinline__ void load_ctx(WarpCtx<D>& c, const Params& P, int item_idx, int lane) {
-  const Item it = load_item_pages(c.ip, P, item_idx, lane);
+__device__ __forceinline__ void begin_queries(WarpCtx<D>& c, const Params& P, const Item& it, int lane) {
   const int nq = (it.flags & kFlagShared) ? 1 : it.n_cons;
   if (lane < D / 8) {
     for (int x = 0; x < nq; ++x) {
@@ -191,23 +191,25 @@ __device__ __forceinline__ void load_ctx(WarpCtx<D>& c, const Params& P, int ite
       const uint16_t* src =
           cached ? P.qcache + ((static_cast<size_t>(it.q_layer[x]) * P.max_seqs + it.seq_id) * P.hq + it.head) * D
                  : P.q + ((static_cast<size_t>(it.q_layer[x]) * P.n_seqs + it.seq_idx) * P.hq + it.head) * D;
-      c.qraw[x][lane] = reinterpret_cast<const uint4*>(src)[lane];
+      cp_async_16(&c.qraw[x][lane], reinterpret_cast<const uint4*>(src) + lane);
     }
   }
-  __syncwarp();
 }
 
 // One item: NQ queries score the K tiles, NV value streams are accumulated.
 // NQ == 1: every consumer shares the weights; NQ == NV: consumer x has its own query.
 // MODE 1 (one query, one consumer) also stores the scaled scores in the logit cache; MODE 2 takes
 // them from there instead of reading K tiles (the ring then carries V tiles only).
-template <int D, int NQ, int NV, int MODE = 0>
+// SKIP (shared weights only): the consumers named in the item's skip_new mask leave out the
+// stream's last key -- the step's new token, whose value row of a follower does not exist yet when
+// its leader's launch runs (Eq. 6: V = [cached V, new v]); they get their own sum of weights.
+template <int D, int NQ, int NV, int MODE = 0, bool SKIP = false>
 __device__ __forceinline__ void process_item(WorkerState& st, const WarpCtx<D>* ctx, uint32_t ring, uint64_t* full,
                                              const Params& P, int lane) {
-  auto ctx_of = [ctx](int k) -> const ItemPages& { return ctx[k & 1].ip; };
+  auto ctx_of = [ctx](int k) -> const ItemPages& { return ctx[k % kCtxSlots].ip; };
   constexpr int EPL = D / 8;    // elements of a row held by one lane
   constexpr int LPR = D / 64;   // 16-byte loads per lane per row
-  const WarpCtx<D>& c = ctx[st.cons_k & 1];
+  const WarpCtx<D>& c = ctx[st.cons_k % kCtxSlots];
   const int kg = lane >> 3;     // which of 4 keys of a pass
   const int c8 = lane & 7;      // which 16-byte chunk of the row (and of its second half)
 
@@ -236,6 +238,10 @@ __device__ __forceinline__ void process_item(WorkerState& st, const WarpCtx<D>* 
 
   const int n_pages = c.ip.item.n_pages;
   const int n_valid_last = c.ip.item.n_valid_last;
+  // SKIP: the new token is key n_valid_last - 1 of the item's last page when that page ends the stream
+  const bool skip_here = SKIP && (c.ip.item.flags & kFlagStreamEnd);
+  const uint32_t skip_mask = SKIP ? c.ip.item.skip_new : 0u;
+  float l_skip = 0.f;       // sum of weights without the new token
   float* lg = nullptr;      // this item's first key in the logit cache
   float lg_next[4] = {0.f, 0.f, 0.f, 0.f};
   if (MODE != 0) {
@@ -307,6 +313,16 @@ __device__ __forceinline__ void process_item(WorkerState& st, const WarpCtx<D>* 
         psum += p[x][i];
       }
       l[x] = l[x] * corr + psum;
+      if (SKIP) {
+        float psum_skip = psum;
+        if (skip_here && pg == n_pages - 1) {
+          const int r_new = nvalid - 1;
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+            if (4 * i + kg == r_new) psum_skip -= p[x][i];
+        }
+        l_skip = l_skip * corr + psum_skip;
+      }
       m[x] = m_new;
       if (corr != 1.f) {
 #pragma unroll
@@ -323,10 +339,11 @@ __device__ __forceinline__ void process_item(WorkerState& st, const WarpCtx<D>* 
     for (int v = 0; v < NV; ++v) {
       const uint8_t* tile = static_cast<const uint8_t*>(__cvta_shared_to_generic(wait_tile<D>(st, ring, full, P, lane)));
       if (st.dead) break;
+      const int nvalid_v = (SKIP && skip_here && pg == n_pages - 1) ? nvalid - static_cast<int>((skip_mask >> v) & 1u) : nvalid;
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         const int r = 4 * i + kg;
-        if (r < nvalid) {
+        if (r < nvalid_v) {
           const uint4* row = reinterpret_cast<const uint4*>(tile + r * (D * 2));
           float vf[EPL];
 #pragma unroll
@@ -347,6 +364,10 @@ __device__ __forceinline__ void process_item(WorkerState& st, const WarpCtx<D>* 
   for (int x = 0; x < NQ; ++x) {
     l[x] += __shfl_xor_sync(0xffffffffu, l[x], 8);
     l[x] += __shfl_xor_sync(0xffffffffu, l[x], 16);
+  }
+  if (SKIP) {
+    l_skip += __shfl_xor_sync(0xffffffffu, l_skip, 8);
+    l_skip += __shfl_xor_sync(0xffffffffu, l_skip, 16);
   }
 #pragma unroll
   for (int v = 0; v < NV; ++v) {
@@ -369,53 +390,95 @@ __device__ __forceinline__ void process_item(WorkerState& st, const WarpCtx<D>* 
         d4[0] = make_float4(acc[v][8 * j + 0], acc[v][8 * j + 1], acc[v][8 * j + 2], acc[v][8 * j + 3]);
         d4[1] = make_float4(acc[v][8 * j + 4], acc[v][8 * j + 5], acc[v][8 * j + 6], acc[v][8 * j + 7]);
       }
-      if (c8 == 0) P.part_ml[row] = make_float2(m[NQ == 1 ? 0 : v], l[NQ == 1 ? 0 : v]);
+      const bool skipping = SKIP && ((skip_mask >> v) & 1u);
+      if (c8 == 0) P.part_ml[row] = make_float2(m[NQ == 1 ? 0 : v], skipping ? l_skip : l[NQ == 1 ? 0 : v]);
     }
   }
+  finish_rows<D>(P, c.ip, lane);
 }
 
-template <int D>
-__global__ void __launch_bounds__(kThreads, 1) attend_kernel(const __grid_constant__ Params P) {
-  constexpr uint32_t kTile = kPage * D * 2;
-  extern __shared__ __align__(128) uint8_t smem[];
-  __shared__ __align__(8) uint64_t full_all[kWarps][kRing];
-
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const uint32_t ring = smem_u32(smem) + static_cast<uint32_t>(warp) * kRing * kTile;
-  WarpCtx<D>* ctx = reinterpret_cast<WarpCtx<D>*>(smem + static_cast<size_t>(kWarps) * kRing * kTile) + warp * 2;
-  uint64_t* full = full_all[warp];
-  auto ctx_of = [ctx](int k) -> const ItemPages& { return ctx[k & 1].ip; };
-
-  if (lane == 0) {
-    for (int s = 0; s < kRing; ++s) mbar_init(&full[s], 1);
-    fence_mbar_init();
-  }
-  __syncthreads();
-  pdl_launch_dependents();
-  pdl_wait();
-
+// A worker's life: take items (claimed from the list, or the pieces of its static ranges), keep
+// the tile ring full across item boundaries, process each item.  While item k is processed the
+// ring already fetches tiles of item k + 1 and the context of item k + 2 (descriptor, page ids,
+// queries) arrives by asynchronous copies.
+template <int D, bool STATIC>
+__device__ __forceinline__ void attend_worker(const Params& P, WarpCtx<D>* ctx, uint32_t ring, uint64_t* full,
+                                              RangeCursor* cursor, int wid, int lane) {
+  auto ctx_of = [ctx](int k) -> const ItemPages& { return ctx[k % kCtxSlots].ip; };
   WorkerState st;
   worker_init(st, 0);
-  int next = claim_take(P, claim_issue(P, lane));
-  if (next < 0) return;
-  load_ctx<D>(ctx[0], P, next, lane);
-  st.n_my = 1;
-  next = claim_take(P, claim_issue(P, lane));
-  if (next >= 0) {
-    load_ctx<D>(ctx[1], P, next, lane);
-    st.n_my = 2;
+  Item it;
+  int issued = 0;
+  auto take = [&]() -> bool {   // the next item into `it`
+    if (STATIC) return cursor_step(cursor, P, it, lane);
+    const int idx = claim_take(P, issued);
+    if (idx < 0) return false;
+    it = load_item(P, idx);
+    return true;
+  };
+  // ---- ahead of the wait for the previous kernel: the first items and their page ids (from the
+  // launch plan, the step descriptors and the page tables, all written before that kernel
+  // started), and the first tiles unless they could hold the step's new token
+  if (STATIC) {
+    if (wid >= P.part_workers) return;
+    RangeCursor c;
+    const bool any = cursor_init(c, P, wid, lane);
+    if (lane == 0) *cursor = c;
+    __syncwarp();
+    if (!any) return;
+  } else {
+    issued = claim_issue(P, lane);
   }
+  if (!take()) return;
+  begin_item_pages(ctx[0].ip, P, it, lane);
+  const Item first = it;
+  cp_async_wait_all();
   __syncwarp();
+  st.n_my = 1;
+  const bool early_tiles = !(first.stream == 0 && (first.flags & kFlagStreamEnd) && first.n_pages <= kRing);
+  if (early_tiles) fill_ring<D, kRing, false>(st, ctx_of, ring, full, P, lane);
+  pdl_wait();
+  pdl_launch_dependents();
+  // ---- this layer's inputs; the rest of the first tiles; the second item's context while they fly
+  begin_queries<D>(ctx[0], P, first, lane);
   fill_ring<D, kRing, false>(st, ctx_of, ring, full, P, lane);
+  if (STATIC) record_row_slots(P, first, lane);
+  if (!STATIC) issued = claim_issue(P, lane);
+  bool more = take();
+  if (more) {
+    begin_item_pages(ctx[1].ip, P, it, lane);
+    begin_queries<D>(ctx[1], P, it, lane);
+    if (STATIC) record_row_slots(P, it, lane);
+  }
+  cp_async_wait_all();
+  __syncwarp();
+  if (more) st.n_my = 2;
+  bool pending = false;   // a context is being filled for item st.n_my
+  if (!STATIC && more) issued = claim_issue(P, lane);
 
   for (int k = 0; k < st.n_my && !st.dead; ++k) {
-    const Item& it = ctx[k & 1].ip.item;
-    const int nc = it.n_cons;
-    const bool shared = it.flags & kFlagShared;
-    // claim the item after next now; the answer is needed only when this item is done
-    const int issued = (next >= 0) ? claim_issue(P, lane) : 0;
-    if (nc == 1 && (it.flags & kFlagReadLogits)) process_item<D, 1, 1, 2>(st, ctx, ring, full, P, lane);
-    else if (nc == 1 && (it.flags & kFlagWriteLogits)) process_item<D, 1, 1, 1>(st, ctx, ring, full, P, lane);
+    const Item& cur = ctx[k % kCtxSlots].ip.item;
+    const int nc = cur.n_cons;
+    const bool shared = cur.flags & kFlagShared;
+    if (more) {
+      // the third slot is free (it held the item before this one): start filling it with the item after next
+      more = take();
+      if (more) {
+        begin_item_pages(ctx[(k + 2) % kCtxSlots].ip, P, it, lane);
+        begin_queries<D>(ctx[(k + 2) % kCtxSlots], P, it, lane);
+        if (STATIC) record_row_slots(P, it, lane);
+        pending = true;
+      }
+    }
+    if (!STATIC && more) issued = claim_issue(P, lane);   // answered by the time the next item starts
+    if (nc == 1 && (cur.flags & kFlagReadLogits)) process_item<D, 1, 1, 2>(st, ctx, ring, full, P, lane);
+    else if (nc == 1 && (cur.flags & kFlagWriteLogits)) process_item<D, 1, 1, 1>(st, ctx, ring, full, P, lane);
+    else if (shared && cur.skip_new) {
+      if (nc == 1) process_item<D, 1, 1, 0, true>(st, ctx, ring, full, P, lane);
+      else if (nc == 2) process_item<D, 1, 2, 0, true>(st, ctx, ring, full, P, lane);
+      else if (nc == 3) process_item<D, 1, 3, 0, true>(st, ctx, ring, full, P, lane);
+      else process_item<D, 1, 4, 0, true>(st, ctx, ring, full, P, lane);
+    }
     else if (nc == 1) process_item<D, 1, 1>(st, ctx, ring, full, P, lane);
     else if (shared && nc == 2) process_item<D, 1, 2>(st, ctx, ring, full, P, lane);
     else if (shared && nc == 3) process_item<D, 1, 3>(st, ctx, ring, full, P, lane);
@@ -424,83 +487,130 @@ __global__ void __launch_bounds__(kThreads, 1) attend_kernel(const __grid_consta
     else if (nc == 3) process_item<D, 3, 3>(st, ctx, ring, full, P, lane);
     else process_item<D, 4, 4>(st, ctx, ring, full, P, lane);
     if (st.dead) break;
-    __syncwarp();
-    if (next >= 0) {
-      next = claim_take(P, issued);
-      if (next >= 0) {   // the context slot of the item just finished receives the item after next
-        load_ctx<D>(ctx[k & 1], P, next, lane);
-        __syncwarp();
-        st.n_my = k + 3;
-      }
+    if (pending) {   // the context of item k + 2 has had this item's time to arrive
+      cp_async_wait_all();
+      __syncwarp();
+      st.n_my = k + 3;
+      pending = false;
     }
     st.cons_k = k + 1;
     fill_ring<D, kRing, false>(st, ctx_of, ring, full, P, lane);
   }
-  if (st.dead) drain_ring<kRing>(st, full);
+  if (st.dead) {
+    cp_async_wait_all();
+    drain_ring<kRing>(st, full);
+  }
+}
+
+template <int D>
+__global__ void __launch_bounds__(kThreads, 1) attend_kernel(const __grid_constant__ Params P) {
+  constexpr uint32_t kTile = kPage * D * 2;
+  extern __shared__ __align__(128) uint8_t smem[];
+  __shared__ __align__(8) uint64_t full_all[kWarps][kRing];
+  __shared__ __align__(16) RangeCursor cursors[kWarps];
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t ring = smem_u32(smem) + static_cast<uint32_t>(warp) * kRing * kTile;
+  WarpCtx<D>* ctx = reinterpret_cast<WarpCtx<D>*>(smem + static_cast<size_t>(kWarps) * kRing * kTile) + warp * kCtxSlots;
+  uint64_t* full = full_all[warp];
+
+  if (lane == 0) {
+    for (int s = 0; s < kRing; ++s) mbar_init(&full[s], 1);
+    fence_mbar_init();
+  }
+  __syncthreads();
+
+  if (P.part_static)
+    attend_worker<D, true>(P, ctx, ring, full, &cursors[warp], warp * gridDim.x + blockIdx.x, lane);
+  else
+    attend_worker<D, false>(P, ctx, ring, full, &cursors[warp], 0, lane);
 }
 
 // ------------------------------------------------------------------------------------------
 // merge: log-sum-exp combination of the partials of one (layer, sequence, head) per warp
 // ------------------------------------------------------------------------------------------
 
+// One warp per (layer, sequence, head).  Under the static partition the numbers of partial rows
+// are themselves data the attention kernel wrote, so the generic merge needs three dependent
+// rounds of loads (counts, then (max, sum) pairs, then rows).  When a row has at most 16 partials
+// per stream (the common case: a launch per layer leaves a handful) everything is requested in
+// one round instead: the counts, the pairs of the first 16 slots of either stream (lanes 0..15 /
+// 16..31) and the first four rows of either stream, whether written or not; what the counts then
+// rule out is ignored.  The step's sequence descriptor is read ahead of the wait for the
+// attention kernel (it was written when the step began).
 template <int D>
 __global__ void merge_kernel(const __grid_constant__ Params P) {
   constexpr int VPL = D / 32;
-  pdl_launch_dependents();
-  pdl_wait();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_layers = P.layer_end - P.layer_begin;
   const int idx = blockIdx.x * (blockDim.x >> 5) + warp;
-  if (idx >= n_layers * P.n_seqs * P.hq) return;
+  const bool live = idx < n_layers * P.n_seqs * P.hq;
   const int head = idx % P.hq;
   const int si = (idx / P.hq) % P.n_seqs;
   const int layer = P.layer_begin + idx / (P.hq * P.n_seqs);
-  const int n_slots = P.seqs[si].n_slots;
+  StepSeq sq{};
+  if (live) sq = P.seqs[si];
+  pdl_wait();
+  pdl_launch_dependents();
+  if (!live) return;
+  if (!P.part_static || P.extra_key_leader >= 0 || P.slots_per_stream < 4) {
+    merge_row<D>(P, layer, si, head, sq, lane, P.extra_key_leader);
+    return;
+  }
+  const int S = P.slots_per_stream;
+  const size_t row = (static_cast<size_t>(layer) * P.max_seqs + si) * P.hq + head;
   const size_t base = (static_cast<size_t>(layer) * P.max_seqs + si) * P.max_slots;
-
-  // Lane s holds the (max, sum) pair of slot s; the accumulator rows do not depend on them, so
-  // their loads are issued four at a time without waiting for the pairs.
-  float mmax = -INFINITY;
+  const uint32_t both = __ldcg(reinterpret_cast<const uint32_t*>(P.row_slots + 2 * row));
+  const int my_slot = lane < 16 ? lane : S + lane - 16;
   float2 my_ml = make_float2(-INFINITY, 0.f);
-  if (lane < n_slots) my_ml = P.part_ml[(base + lane) * P.hq + head];
-  mmax = my_ml.x;
-  for (int s = lane + 32; s < n_slots; s += 32) mmax = fmaxf(mmax, P.part_ml[(base + s) * P.hq + head].x);
+  if ((lane & 15) < S) my_ml = __ldcg(P.part_ml + (base + my_slot) * P.hq + head);
+  float v[8][VPL];   // rows of visual slots 0..3 and text slots 0..3
+#pragma unroll
+  for (int u = 0; u < 8; ++u) {
+    const int s = u < 4 ? u : S + u - 4;
+    const float* src = P.part_acc + ((base + s) * P.hq + head) * D + lane * VPL;
+    if (VPL == 4) {
+      const float4 a = __ldcg(reinterpret_cast<const float4*>(src));
+      v[u][0] = a.x, v[u][1] = a.y, v[u][2 % VPL] = a.z, v[u][3 % VPL] = a.w;
+    } else {
+      const float2 a = __ldcg(reinterpret_cast<const float2*>(src));
+      v[u][0] = a.x, v[u][1] = a.y;
+    }
+  }
+  const int nv = sq.len_vis > 0 ? static_cast<int>(both & 0xffffu) : 0;
+  const int nt = static_cast<int>(both >> 16);
+  if (nv > 16 || nt > 16) {
+    merge_row<D>(P, layer, si, head, sq, lane, -1);
+    return;
+  }
+  const bool mine = lane < 16 ? lane < nv : lane - 16 < nt;
+  if (!mine) my_ml = make_float2(-INFINITY, 0.f);
+  float mmax = my_ml.x;
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xffffffffu, mmax, o));
-
-  float lsum = 0.f;
+  const float my_w = my_ml.y > 0.f ? exp2f(my_ml.x - mmax) : 0.f;   // (an empty partial counts for nothing)
+  float lsum = my_ml.y * my_w;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) lsum += __shfl_xor_sync(0xffffffffu, lsum, o);
   float acc[VPL];
 #pragma unroll
   for (int e = 0; e < VPL; ++e) acc[e] = 0.f;
-  for (int s0 = 0; s0 < n_slots; s0 += 4) {
-    float v[4][VPL];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int s = min(s0 + u, n_slots - 1);
-      const float* src = P.part_acc + ((base + s) * P.hq + head) * D + lane * VPL;
-      if (VPL == 4) {
-        const float4 a = *reinterpret_cast<const float4*>(src);
-        v[u][0] = a.x, v[u][1] = a.y, v[u][2 % VPL] = a.z, v[u][3 % VPL] = a.w;
-      } else {
-        const float2 a = *reinterpret_cast<const float2*>(src);
-        v[u][0] = a.x, v[u][1] = a.y;
-      }
+  for (int u = 0; u < 8; ++u) {
+    const float w = __shfl_sync(0xffffffffu, my_w, u < 4 ? u : 12 + u);   // lanes 0..3 and 16..19
+    if (w > 0.f) {
+#pragma unroll
+      for (int e = 0; e < VPL; ++e) acc[e] = fmaf(v[u][e], w, acc[e]);
     }
+  }
+  for (int s = 4; s < max(nv, nt); ++s) {   // rows beyond the first four of a stream
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int s = s0 + u;
-      float2 ml;
-      if (s < 32) {
-        ml.x = __shfl_sync(0xffffffffu, my_ml.x, s & 31);
-        ml.y = __shfl_sync(0xffffffffu, my_ml.y, s & 31);
-      } else {
-        ml = P.part_ml[(base + min(s, n_slots - 1)) * P.hq + head];
-      }
-      if (s < n_slots) {
-        const float w = exp2f(ml.x - mmax);
-        lsum = fmaf(ml.y, w, lsum);
+    for (int t = 0; t < 2; ++t) {
+      const float w = __shfl_sync(0xffffffffu, my_w, (t ? 16 : 0) + s);
+      if (s < (t ? nt : nv) && w > 0.f) {
+        const float* src = P.part_acc + ((base + (t ? S : 0) + s) * P.hq + head) * D + lane * VPL;
 #pragma unroll
-        for (int e = 0; e < VPL; ++e) acc[e] = fmaf(v[u][e], w, acc[e]);
+        for (int e = 0; e < VPL; ++e) acc[e] = fmaf(__ldcg(src + e), w, acc[e]);
       }
     }
   }
@@ -521,7 +631,7 @@ __global__ void merge_kernel(const __grid_constant__ Params P) {
 
 template <int D>
 constexpr int attend_smem_bytes() {
-  return kWarps * kRing * kPage * D * 2 + kWarps * 2 * static_cast<int>(sizeof(WarpCtx<D>));
+  return kWarps * kRing * kPage * D * 2 + kWarps * kCtxSlots * static_cast<int>(sizeof(WarpCtx<D>));
 }
 
 }  // namespace
@@ -554,8 +664,9 @@ cudaError_t launch_append(const Params& p, cudaStream_t stream) {
 
 cudaError_t launch_attend(const Params& p, int n_sms, cudaStream_t stream) {
   const int n_items = p.item_end - p.item_begin;
-  if (n_items <= 0) return cudaSuccess;
-  const int grid = min(n_sms, (n_items + kWarps - 1) / kWarps);
+  if (!p.part_static && n_items <= 0) return cudaSuccess;
+  // static ranges: worker w is warp w / grid of CTA w % grid, so a launch with few workers still uses every SM
+  const int grid = p.part_static ? min(n_sms, p.part_workers) : min(n_sms, (n_items + kWarps - 1) / kWarps);
   if (p.d == 128)
     return launch_pdl(attend_kernel<128>, dim3(grid), dim3(kThreads), attend_smem_bytes<128>(), stream, p);
   return launch_pdl(attend_kernel<64>, dim3(grid), dim3(kThreads), attend_smem_bytes<64>(), stream, p);

@@ -35,11 +35,16 @@ struct SeqState {
 // One attention launch: a run of consecutive lazy blocks.
 struct LaunchGroup {
   int job_begin, job_end, layer_begin, layer_end;
+  int extra_key_leader;   // >= 0: the merge of these layers adds the step's new token (in-order schedule, GLA followers)
+  bool needs_merge;       // some output row of these layers is not merged by the attention kernel itself
+  int wv, wt;             // tiles per page summed over the launch's visual / text jobs
+  int w_min, w_max;       // smallest / largest tiles per page of a job of the launch
+  int w_max_v, w_max_t;   // largest tiles per page among its visual / text jobs
 };
 
 struct Layout {   // byte offsets into the workspace
-  size_t table, layer_flags, layer_kind, leader, jobs, plan, qcache, part_acc, part_ml, logits, items, step, err, counters, stage_q, stage_k, stage_v,
-      stage_out, stage_lse, tok, total;
+  size_t table, layer_flags, layer_kind, leader, jobs, plan, qcache, part_acc, part_ml, logits, items, step, err, counters, row_slots, row_done, stage_q,
+      stage_k, stage_v, stage_out, stage_lse, tok, total;
   size_t step_seqs, step_patches, step_bytes;   // offsets inside the step block
 };
 
@@ -100,6 +105,14 @@ struct qc_cache {
   std::vector<std::pair<int, int>> block_layers; // per lazy block: [layer_begin, layer_end)
   std::vector<Job> layer_jobs;                    // per-layer schedule (logit cache)
   std::vector<std::pair<int, int>> layer_job_range;   // per layer: [job_begin, job_end) in layer_jobs
+  std::vector<Job> inorder_jobs;                  // in-order schedule (a leader's launch also sweeps its followers' cached V)
+  std::vector<std::pair<int, int>> inorder_job_range;
+  std::vector<int> inorder_extra_key;             // per layer: the leader whose new token the merge adds, or -1
+  int slots_per_stream = 0;
+  int static_partition = -1;      // -1: static ranges when a step is several launches; 0 never; 1 always
+  bool fused_merge = false;       // the worker that delivers an output row's last partial merges it (no merge launch)
+  int static_min_tiles = 6;       // a static range is at least this long when the launch has the work for it
+                                  // (measured on launches of one layer: 3..8 equal, 12 and 16 slower)
   int text_streams_per_seq = 0;        // pages a sequence needs when its text crosses a page
 
   // pinned staging ring for step descriptors
@@ -174,6 +187,7 @@ void build_jobs(const qc_config* cfg, std::vector<Job>& jobs, std::vector<std::p
         j.stream = static_cast<uint8_t>(stream);
         j.n_cons = static_cast<uint8_t>(std::min(kMaxCons, e - first));
         j.flags = kFlagShared;
+        j.finish = static_cast<uint8_t>((1u << j.n_cons) - 1);   // a block's launch sweeps both streams of all its layers
         for (int x = 0; x < j.n_cons; ++x) {
           j.v_layer[x] = static_cast<uint8_t>(first + x);
           j.q_layer[x] = static_cast<uint8_t>(c);
@@ -189,6 +203,7 @@ void build_jobs(const qc_config* cfg, std::vector<Job>& jobs, std::vector<std::p
         j.stream = static_cast<uint8_t>(stream);
         j.n_cons = static_cast<uint8_t>(std::min(max_own, e - first));
         j.flags = (j.n_cons == 1) ? kFlagShared : 0;
+        j.finish = static_cast<uint8_t>((1u << j.n_cons) - 1);
         for (int x = 0; x < j.n_cons; ++x) {
           j.v_layer[x] = static_cast<uint8_t>(first + x);
           j.q_layer[x] = static_cast<uint8_t>(first + x);
@@ -203,6 +218,7 @@ void build_jobs(const qc_config* cfg, std::vector<Job>& jobs, std::vector<std::p
         j.stream = static_cast<uint8_t>(stream);
         j.n_cons = 1;
         j.flags = kFlagShared;
+        j.finish = 1;
         j.v_layer[0] = static_cast<uint8_t>(x);
         j.q_layer[0] = static_cast<uint8_t>(x);
         jobs.push_back(j);
@@ -247,6 +263,7 @@ void build_layer_jobs(const qc_config* cfg, std::vector<Job>& jobs, std::vector<
       j.stream = static_cast<uint8_t>(stream);
       j.n_cons = 1;
       j.flags = kFlagShared;
+      j.finish = 1;   // the layer's launch sweeps both of its streams
       j.v_layer[0] = static_cast<uint8_t>(l);
       j.q_layer[0] = static_cast<uint8_t>(l);
       j.k_layer = static_cast<uint8_t>(l);
@@ -267,8 +284,84 @@ void build_layer_jobs(const qc_config* cfg, std::vector<Job>& jobs, std::vector<
   }
 }
 
+// Jobs of the in-order schedule, layer by layer: the launch of layer l uses nothing of the layers
+// after l, as in a model where a layer's q/k/v only exist once the previous layer has run.  What a
+// follower shares with its leader are the scores (GLA: Q and K are the leader's, Eq. 6; VLA_QC: the
+// cached query on the leader's visual K), and the V rows they weight were cached before the step:
+// the visual stream never holds the new token, the text stream holds it last.  So the leader's
+// sweep also weights its followers' cached V rows, one K read and one set of weights for up to
+// kMaxCons layers, and leaves their partial rows behind.  A VLA_QC follower's own launch is its
+// text sweep (own q, own text K); a GLA follower has no sweep at all: its merge adds the new token
+// as one more key.  VLA_EQ8 followers score the leader's visual keys with their own query (Eq. 8
+// shares K only), in their own launch.
+void build_inorder_jobs(const qc_config* cfg, std::vector<Job>& jobs, std::vector<std::pair<int, int>>& layer_jobs,
+                        std::vector<int>& extra_key) {
+  const int N = cfg->n_layers;
+  extra_key.assign(N, -1);
+  int l = 0;
+  while (l < N) {
+    const int c = l;
+    int e = l + 1;
+    while (e < N && cfg->layer_kind[e] == QC_LAYER_LAZY) ++e;
+    auto own = [&](int layer, int k_layer, int stream, bool only_stream) {
+      Job j{};
+      j.k_layer = static_cast<uint8_t>(k_layer);
+      j.stream = static_cast<uint8_t>(stream);
+      j.n_cons = 1;
+      j.flags = kFlagShared;
+      j.finish = static_cast<uint8_t>(1 | (only_stream ? kFinishOwnStream : 0));
+      j.v_layer[0] = static_cast<uint8_t>(layer);
+      j.q_layer[0] = static_cast<uint8_t>(layer);
+      jobs.push_back(j);
+    };
+    auto shared = [&](int stream, bool skip_new) {   // the leader's query; consumers c .. e-1, kMaxCons per sweep
+      for (int first = c; first < e; first += kMaxCons) {
+        Job j{};
+        j.k_layer = static_cast<uint8_t>(c);
+        j.stream = static_cast<uint8_t>(stream);
+        j.n_cons = static_cast<uint8_t>(std::min(kMaxCons, e - first));
+        j.flags = kFlagShared;
+        for (int x = 0; x < j.n_cons; ++x) {
+          j.v_layer[x] = static_cast<uint8_t>(first + x);
+          j.q_layer[x] = static_cast<uint8_t>(c);
+          if (skip_new && first + x != c) j.skip_new |= static_cast<uint8_t>(1u << x);
+          if (first + x == c) j.finish |= static_cast<uint8_t>(1u << x);   // the followers' rows are completed later
+        }
+        jobs.push_back(j);
+      }
+    };
+    // the leader's launch
+    int job0 = static_cast<int>(jobs.size());
+    if (cfg->lazy_mode == QC_MODE_VLA_EQ8 || e - c == 1) {
+      own(c, c, 1, false);
+      own(c, c, 0, false);
+    } else if (cfg->lazy_mode == QC_MODE_VLA_QC) {
+      shared(1, false);
+      own(c, c, 0, false);
+    } else {
+      shared(1, false);
+      shared(0, true);
+    }
+    layer_jobs.emplace_back(job0, static_cast<int>(jobs.size()));
+    // the followers' launches
+    for (int f = c + 1; f < e; ++f) {
+      job0 = static_cast<int>(jobs.size());
+      if (cfg->lazy_mode == QC_MODE_VLA_EQ8) {
+        own(f, c, 1, false);
+        own(f, f, 0, false);
+      } else if (cfg->lazy_mode == QC_MODE_VLA_QC) {
+        own(f, f, 0, true);   // the visual partials are there already
+      } else {
+        extra_key[f] = c;
+      }
+      layer_jobs.emplace_back(job0, static_cast<int>(jobs.size()));
+    }
+    l = e;
+  }
+}
+
 struct Sizes {
-  int D, hq, hkv, max_pages, chunk_pages, max_slots;
+  int D, hq, hkv, max_pages, chunk_pages, max_slots, slots_per_stream;
   int64_t n_pool_pages;
   size_t page_bytes, pool_bytes, max_items, max_segs, max_patches;
   Layout lay;
@@ -283,7 +376,13 @@ int compute_sizes(const qc_config* cfg, Sizes* s) {
   s->max_pages = (cfg->max_tokens_per_seq + kPage - 1) / kPage;
   const int split = cfg->split_tokens ? cfg->split_tokens : 64;   // auto: the smallest chunk the per-step choice may take
   s->chunk_pages = split / kPage;
-  s->max_slots = 2 * ((s->max_pages + s->chunk_pages - 1) / s->chunk_pages);
+  // partial-row slots per stream of an output row: one per chunk when items are claimed.  Under the
+  // static partition a row of P pages at w tiles per page is cut into at most P w / q + 2 pieces by
+  // ranges of q tiles, and q may not exceed 30 pages of the launch's lightest job (a piece holds at
+  // most kMaxChunkPages page ids); tiles per page differ by at most 5x between the jobs of a launch
+  // (1 .. 1 + kMaxCons), so max_pages / 3 + 2 slots always leave room for a q within both bounds
+  s->slots_per_stream = std::max((s->max_pages + s->chunk_pages - 1) / s->chunk_pages, (s->max_pages + 2) / 3 + 2);
+  s->max_slots = 2 * s->slots_per_stream;
   s->page_bytes = static_cast<size_t>(s->hkv) * kPage * s->D * 2;
   if (cfg->page_size == 0)
     s->n_pool_pages = static_cast<int64_t>(cfg->n_layers) * 4 * cfg->max_seqs * s->max_pages;
@@ -298,7 +397,11 @@ int compute_sizes(const qc_config* cfg, Sizes* s) {
   std::vector<Job> layer_jobs;
   std::vector<std::pair<int, int>> lj;
   build_layer_jobs(cfg, layer_jobs, lj);
-  const size_t n_jobs = std::max(jobs.size(), layer_jobs.size());   // either schedule fits
+  std::vector<Job> inorder_jobs;
+  std::vector<int> extra;
+  lj.clear();
+  build_inorder_jobs(cfg, inorder_jobs, lj, extra);
+  const size_t n_jobs = std::max(std::max(jobs.size(), layer_jobs.size()), inorder_jobs.size());   // any schedule fits
   const size_t chunks_per_stream = (s->max_pages + s->chunk_pages - 1) / s->chunk_pages;
   s->max_segs = n_jobs * cfg->max_seqs;
   s->max_items = s->max_segs * chunks_per_stream * s->hq;
@@ -330,6 +433,8 @@ int compute_sizes(const qc_config* cfg, Sizes* s) {
   L.step = take(L.step_bytes);
   L.err = take(256);
   L.counters = take(N * sizeof(int32_t));
+  L.row_slots = take(N * S * s->hq * 2 * sizeof(uint16_t));
+  L.row_done = take(N * S * s->hq * sizeof(int32_t));
   L.stage_q = take(N * S * s->hq * s->D * 2);
   L.stage_k = take(N * S * s->hkv * s->D * 2);
   L.stage_v = take(N * S * s->hkv * s->D * 2);
@@ -362,6 +467,10 @@ Params base_params(const qc_cache* c) {
   p.layer_flags = c->ws + c->lay.layer_flags;
   p.err = reinterpret_cast<int32_t*>(c->ws + c->lay.err);
   p.work_counter = reinterpret_cast<int32_t*>(c->ws + c->lay.counters);
+  p.row_slots = reinterpret_cast<uint16_t*>(c->ws + c->lay.row_slots);
+  p.row_done = reinterpret_cast<int32_t*>(c->ws + c->lay.row_done);
+  p.slots_per_stream = c->slots_per_stream;
+  p.extra_key_leader = -1;
   p.n_pool_pages = c->n_pool_pages;
   p.n_layers = c->cfg.n_layers;
   p.hq = c->hq;
@@ -468,26 +577,28 @@ int rebuild_plan(qc_cache* c, int per_launch) {
   c->plan.clear();
   c->plan_vis_before.assign(1, 0);
   c->plan_text_before.assign(1, 0);
-  // per_launch < 0: the per-layer schedule (one launch per layer, logit cache); otherwise launches
-  // of `per_launch` lazy blocks (0 = all blocks in one launch)
+  // per_launch -1: the per-layer schedule with the logit cache; -2: the in-order schedule (one
+  // launch per layer, a leader's launch also sweeps its followers' cached V); otherwise launches of
+  // `per_launch` lazy blocks (0 = all blocks in one launch)
   const bool per_layer = per_launch < 0;
-  const std::vector<Job>& jobs = per_layer ? c->layer_jobs : c->jobs;
-  const int nb = static_cast<int>(per_layer ? c->layer_job_range.size() : c->block_jobs.size());
+  const std::vector<Job>& jobs = per_launch == -2 ? c->inorder_jobs : (per_launch == -1 ? c->layer_jobs : c->jobs);
+  const std::vector<std::pair<int, int>>& layer_range = per_launch == -2 ? c->inorder_job_range : c->layer_job_range;
+  const int nb = static_cast<int>(per_layer ? layer_range.size() : c->block_jobs.size());
   const int per = per_layer ? 1 : (per_launch == 0 ? nb : per_launch);
   c->n_visual_jobs = c->n_text_jobs = 0;
   c->visual_row_reads = c->text_row_reads = 0;
+  auto tiles_per_page = [](const Job& j) { return ((j.flags & kFlagReadLogits) ? 0 : 1) + j.n_cons; };
   for (const Job& j : jobs) {
     (j.stream ? c->n_visual_jobs : c->n_text_jobs)++;
-    (j.stream ? c->visual_row_reads : c->text_row_reads) += ((j.flags & kFlagReadLogits) ? 0 : 1) + j.n_cons;
+    (j.stream ? c->visual_row_reads : c->text_row_reads) += tiles_per_page(j);
   }
   std::vector<int> order;
   for (int b = 0; b < nb; b += per) {
     const int e = std::min(nb, b + per);
-    const LaunchGroup g = per_layer
-                              ? LaunchGroup{c->layer_job_range[b].first, c->layer_job_range[b].second, b, b + 1}
+    LaunchGroup g = per_layer ? LaunchGroup{layer_range[b].first, layer_range[b].second, b, b + 1}
                               : LaunchGroup{c->block_jobs[b].first, c->block_jobs[e - 1].second,
                                             c->block_layers[b].first, c->block_layers[e - 1].second};
-    c->groups.push_back(g);
+    g.extra_key_leader = per_launch == -2 ? c->inorder_extra_key[b] : -1;
     order.resize(g.job_end - g.job_begin);
     for (int j = g.job_begin; j < g.job_end; ++j) order[j - g.job_begin] = j;
     std::stable_sort(order.begin(), order.end(), [&](int x, int y) {
@@ -496,12 +607,28 @@ int rebuild_plan(qc_cache* c, int per_launch) {
       return jx.stream > jy.stream;
     });
     const int begin = static_cast<int>(c->plan.size());
+    g.wv = g.wt = g.w_max = g.w_max_v = g.w_max_t = 0;
+    g.w_min = 1 << 20;
+    std::vector<bool> finished(c->cfg.n_layers, false);
     for (int j : order) {
       const int vb = c->plan_vis_before.back(), tb = c->plan_text_before.back();
-      c->plan.push_back(PlanJob{jobs[j], vb, tb, 0, 0});
+      Job job = jobs[j];
+      if (!c->fused_merge) job.finish = 0;
+      for (int x = 0; x < job.n_cons; ++x)
+        if ((job.finish >> x) & 1) finished[job.v_layer[x]] = true;
+      c->plan.push_back(PlanJob{job, vb, tb, g.wv, g.wt});
       c->plan_vis_before.push_back(vb + (jobs[j].stream ? 1 : 0));
       c->plan_text_before.push_back(tb + (jobs[j].stream ? 0 : 1));
+      const int w = tiles_per_page(jobs[j]);
+      (jobs[j].stream ? g.wv : g.wt) += w;
+      int& w_max_s = jobs[j].stream ? g.w_max_v : g.w_max_t;
+      w_max_s = std::max(w_max_s, w);
+      g.w_min = std::min(g.w_min, w);
+      g.w_max = std::max(g.w_max, w);
     }
+    g.needs_merge = false;
+    for (int l = g.layer_begin; l < g.layer_end; ++l) g.needs_merge = g.needs_merge || !finished[l];
+    c->groups.push_back(g);
     c->group_pos.emplace_back(begin, static_cast<int>(c->plan.size()));
   }
   QC_CUDA(cudaMemcpyAsync(c->ws + c->lay.plan, c->plan.data(), c->plan.size() * sizeof(PlanJob),
@@ -534,6 +661,8 @@ const char* qc_status_string(int32_t s) {
     case QC_ERR_STATE: return "invalid state";
     case QC_ERR_CUDA: return "CUDA error";
     case QC_ERR_TIMEOUT: return "device wait timed out";
+    case QC_ERR_BAD_PAGE: return "page id outside the pool";
+    case QC_ERR_PLAN: return "work range outside its planned limits";
     default: return "unknown status";
   }
 }
@@ -600,6 +729,7 @@ int32_t qc_alloc_cache(qc_ctx* ctx, const qc_config* cfg, void* pool_dev, size_t
   c->chunk_pages = c->min_chunk_pages = s.chunk_pages;
   c->auto_split = cfg->split_tokens == 0;
   c->max_slots = s.max_slots;
+  c->slots_per_stream = s.slots_per_stream;
   c->n_pool_pages = s.n_pool_pages;
   c->scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / std::sqrt(static_cast<float>(s.D));
   c->ws = static_cast<uint8_t*>(workspace_dev);
@@ -623,6 +753,7 @@ int32_t qc_alloc_cache(qc_ctx* ctx, const qc_config* cfg, void* pool_dev, size_t
   }
   build_jobs(&c->cfg, c->jobs, c->block_jobs, c->block_layers);
   build_layer_jobs(&c->cfg, c->layer_jobs, c->layer_job_range);
+  build_inorder_jobs(&c->cfg, c->inorder_jobs, c->inorder_job_range, c->inorder_extra_key);
   if (c->cfg.lazy_mode == QC_MODE_GLA) {
     // Eq. 5: every layer of a lazy block attends with the block's first layer's Q and K, so runs
     // of up to three of its layers share one score pass of the prefill kernel
@@ -674,6 +805,7 @@ int32_t qc_alloc_cache(qc_ctx* ctx, const qc_config* cfg, void* pool_dev, size_t
   ok = ok && cudaMemcpyAsync(c->ws + c->lay.jobs, c->jobs.data(), c->jobs.size() * sizeof(Job),
                              cudaMemcpyHostToDevice, stream) == cudaSuccess;
   ok = ok && cudaMemsetAsync(c->ws + c->lay.err, 0, 256, stream) == cudaSuccess;
+  ok = ok && cudaMemsetAsync(c->ws + c->lay.row_done, 0, c->lay.stage_q - c->lay.row_done, stream) == cudaSuccess;
   ok = ok && cudaMemsetAsync(c->ws + c->lay.qcache, 0, c->lay.part_acc - c->lay.qcache, stream) == cudaSuccess;
   ok = ok && cudaStreamSynchronize(stream) == cudaSuccess;
   if (!ok) {
@@ -1054,21 +1186,41 @@ int decode_step_core(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, const 
     h_seqs = reinterpret_cast<StepSeq*>(hb + c->lay.step_seqs);
     if (n_patches) std::memcpy(hb + c->lay.step_patches, patches.data(), n_patches * sizeof(Patch));
   }
+  // Static partition: the step's launches cut their work into equal ranges instead of claiming
+  // items (by default whenever a step is several launches, whose short tails a few large items
+  // per worker would dominate).
+  bool use_static = c->static_partition == 1 || (c->static_partition < 0 && c->groups.size() > 1);
+  int64_t tp_v = 0, tp_t = 0;                     // pages of the visual / text streams over the listed sequences
+  int pmax_v = 0, pmax_t = 0;
+  for (int i = 0; i < n_seqs; ++i) {
+    const SeqState& st = c->seqs[seq_ids[i]];
+    const int pv = pages_for(st.len_vis), pt = pages_for(st.len_text);
+    tp_v += pv;
+    tp_t += pt;
+    pmax_v = std::max(pmax_v, pv);
+    pmax_t = std::max(pmax_t, pt);
+  }
+  for (const LaunchGroup& g : c->groups)   // tile offsets are 32-bit
+    if (static_cast<int64_t>(c->items_per_chunk) * (g.wv * tp_v + g.wt * tp_t) >= (1LL << 31)) use_static = false;
   int64_t tot_v = 0, tot_t = 0, step_rows = 0;   // step_rows: K/V rows the step has to read (for the profile)
+  int64_t pre_pv = 0, pre_pt = 0;
   for (int i = 0; i < n_seqs; ++i) {
     const int s = seq_ids[i];
     const SeqState& st = c->seqs[s];
-    const int ncv = (pages_for(st.len_vis) + c->chunk_pages - 1) / c->chunk_pages;
-    const int nct = (pages_for(st.len_text) + c->chunk_pages - 1) / c->chunk_pages;
-    h_seqs[i] = StepSeq{s, st.len_text, st.len_vis, ncv + nct, static_cast<int32_t>(tot_v),
-                        static_cast<int32_t>(tot_t), ncv, 0};
+    const int pv = pages_for(st.len_vis), pt = pages_for(st.len_text);
+    const int ncv = (pv + c->chunk_pages - 1) / c->chunk_pages;
+    const int nct = (pt + c->chunk_pages - 1) / c->chunk_pages;
+    h_seqs[i] = StepSeq{s, st.len_text, st.len_vis, ncv + nct, static_cast<int32_t>(use_static ? pre_pv : tot_v),
+                        static_cast<int32_t>(use_static ? pre_pt : tot_t), ncv, 0};
     tot_v += static_cast<int64_t>(ncv) * c->items_per_chunk;
     tot_t += static_cast<int64_t>(nct) * c->items_per_chunk;
+    pre_pv += pv;
+    pre_pt += pt;
     step_rows += st.len_vis * c->visual_row_reads + st.len_text * c->text_row_reads;
   }
   const int n_pos = static_cast<int>(c->plan.size());
   const int64_t n_items64 = c->plan_vis_before[n_pos] * tot_v + c->plan_text_before[n_pos] * tot_t;
-  const int n_items = static_cast<int>(n_items64);   // <= max_items: the item list was sized at allocation
+  const int n_items = use_static ? 0 : static_cast<int>(n_items64);   // <= max_items: the item list was sized at allocation
 
   // ---- enqueue
   if (!inline_step) {
@@ -1084,8 +1236,11 @@ int decode_step_core(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, const 
   p.out = static_cast<uint16_t*>(out_dev);
   p.lse = lse_out_dev;
   p.n_seqs = n_seqs;
-  p.n_pos = n_pos;
+  p.n_pos = use_static ? 0 : n_pos;   // static ranges need no item list
   p.n_items = n_items;
+  p.part_static = use_static ? 1 : 0;
+  p.tp_v = static_cast<int32_t>(tp_v);
+  p.tp_t = static_cast<int32_t>(tp_t);
   p.n_patches = n_patches;
   p.tot_v = static_cast<int32_t>(tot_v);
   p.tot_t = static_cast<int32_t>(tot_t);
@@ -1121,21 +1276,57 @@ int decode_step_core(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, const 
     p.layer_begin = c->groups[gi].layer_begin;
     p.layer_end = c->groups[gi].layer_end;
     p.launch_index = static_cast<int32_t>(gi);
+    p.pos_begin = pb;
+    p.pos_end = pe;
+    p.extra_key_leader = c->groups[gi].extra_key_leader;
+    bool has_work = p.item_end > p.item_begin;
+    if (use_static) {
+      const LaunchGroup& g = c->groups[gi];
+      const int64_t T = static_cast<int64_t>(c->items_per_chunk) * (g.wv * tp_v + g.wt * tp_t);
+      has_work = T > 0;
+      if (has_work) {
+        // tiles per page of the lightest / heaviest job that has any page, longest row in tiles
+        const int w_min = (tp_v > 0 && tp_t > 0) ? g.w_min : g.w_max_v * (tp_v > 0) + g.w_max_t * (tp_t > 0);
+        const int w_lo = std::max(1, std::min(w_min, g.w_min));
+        const int64_t row_max = std::max<int64_t>(static_cast<int64_t>(pmax_v) * g.w_max_v,
+                                                  static_cast<int64_t>(pmax_t) * g.w_max_t);
+        const int64_t q_max = 30LL * w_lo;
+        int64_t q_min = std::max<int64_t>(2LL * g.w_max, (row_max + c->slots_per_stream - 3) / (c->slots_per_stream - 2));
+        q_min = std::max<int64_t>(q_min, std::min<int64_t>(c->static_min_tiles, q_max / 2));
+        const int64_t W = static_cast<int64_t>(c->ctx->n_sms) * kAttendWarps;
+        int64_t k = 1, q;
+        if (T > W * q_max) {   // several ranges per worker, each as long as a piece may be
+          k = (T + W * q_max - 1) / (W * q_max);
+          q = (T + W * k - 1) / (W * k);
+        } else {
+          q = std::max<int64_t>(q_min, (T + W - 1) / W);
+        }
+        const int64_t vw = (T + q - 1) / q;
+        p.part_vw = static_cast<int32_t>(vw);
+        p.part_k = static_cast<int32_t>(k);
+        p.part_workers = static_cast<int32_t>((vw + k - 1) / k);
+        p.part_q = static_cast<int32_t>(q);
+        p.part_tiles = static_cast<int32_t>(T);
+      }
+    }
     if (pipe) {
       QC_CUDA(cudaStreamWaitEvent(stream, pipe->in[gi], 0));
       QC_CUDA(launch_append(p, stream));   // this group's layers only
       c->kernel_launches++;
     }
     if (ev && gi == 0) QC_CUDA(cudaEventRecord(ev[1], stream));
-    if (c->group > 1)
+    if (!has_work) {
+      // (a GLA follower of the in-order schedule: its merge does everything)
+    } else if (c->group > 1) {
       QC_CUDA(launch_attend_tc(p, c->ctx->n_sms, stream));
-    else
+    } else {
       QC_CUDA(launch_attend(p, c->ctx->n_sms, stream));
+    }
     if (ev && gi + 1 == c->groups.size()) QC_CUDA(cudaEventRecord(ev[2], stream));
-    QC_CUDA(launch_merge(p, stream));
+    if (c->groups[gi].needs_merge) QC_CUDA(launch_merge(p, stream));
     if (pipe) QC_CUDA(cudaEventRecord(pipe->done[gi], stream));
-    c->attend_launches++;
-    c->kernel_launches += 2;
+    c->attend_launches += has_work ? 1 : 0;
+    c->kernel_launches += (has_work ? 1 : 0) + (c->groups[gi].needs_merge ? 1 : 0);
   }
   if (ev) {
     QC_CUDA(cudaEventRecord(ev[3], stream));
@@ -1351,6 +1542,26 @@ int32_t qc_set_option(qc_cache* c, const char* key, int64_t value) {
   if (k == "per_layer_logit_cache") {   // one launch per layer; followers take shared scores from the logit cache
     c->layers_per_launch = value ? -1 : 0;
     c->plan_dirty = true;
+    return QC_OK;
+  }
+  if (k == "in_order_launches") {   // one launch per layer; a leader's launch also sweeps its followers' cached V
+    c->layers_per_launch = value ? -2 : 0;
+    c->plan_dirty = true;
+    return QC_OK;
+  }
+  if (k == "fused_merge") {   // 0: partial rows are merged by a launch of their own
+    c->fused_merge = value != 0;
+    c->plan_dirty = true;
+    return QC_OK;
+  }
+  if (k == "static_partition") {
+    if (value < -1 || value > 1) return QC_ERR_INVALID_ARG;
+    c->static_partition = static_cast<int>(value);
+    return QC_OK;
+  }
+  if (k == "static_min_tiles") {
+    if (value < 1 || value > 4096) return QC_ERR_INVALID_ARG;
+    c->static_min_tiles = static_cast<int>(value);
     return QC_OK;
   }
   if (k == "prefill_shared_scores") {

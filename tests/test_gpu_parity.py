@@ -174,6 +174,7 @@ def test_launch_grouping_and_host_entry_give_identical_bits():
     for variant in ("one_launch", "per_block", "host_buffers", "per_layer", "per_layer_set_then_host_buffers"):
         s = Session.for_workload(w, lazy_mode=qc.QC_MODE_VLA_QC, split_tokens=64)
         s.prefill_workload(w)
+        s.set_option("static_partition", 0)   # same chunks in every variant: the bits can then be compared
         if variant == "per_block":
             s.set_option("layers_per_launch", 1)
         if variant.startswith("per_layer"):
@@ -214,6 +215,7 @@ def test_per_layer_schedule_with_logit_cache(mode, case):
     for per_layer in (False, True):
         s = Session(w.n_layers, w.n_q_heads, w.n_kv_heads, head_dim, layer_kind, max_seqs=4, max_tokens_per_seq=256,
                     n_pages=w.n_layers * 4 * 3 * 17, lazy_mode=mode, split_tokens=split, poison_pool=True)
+        s.set_option("static_partition", 0)   # same chunks in both schedules
         if per_layer:
             s.set_option("per_layer_logit_cache", 1)
         sessions.append(s)
@@ -242,6 +244,61 @@ def test_per_layer_schedule_with_logit_cache(mode, case):
     for s in sessions:
         assert s.stats().device_error == 0
         s.close()
+
+
+SCHEDULES = {
+    # option settings that change how a step is cut into launches and work ranges, never its result
+    "one_launch_static_ranges": [("static_partition", 1)],
+    "per_block_static_ranges": [("layers_per_launch", 1)],
+    "per_layer_logit_cache_static_ranges": [("per_layer_logit_cache", 1)],
+    "in_order": [("in_order_launches", 1)],
+    "in_order_claimed_items": [("in_order_launches", 1), ("static_partition", 0)],
+    "in_order_short_ranges": [("in_order_launches", 1), ("static_min_tiles", 1)],
+    "in_order_merge_in_kernel": [("in_order_launches", 1), ("fused_merge", 1)],
+    "one_launch_merge_in_kernel": [("fused_merge", 1)],
+}
+
+
+@pytest.mark.parametrize("schedule", sorted(SCHEDULES))
+@pytest.mark.parametrize("mode", MODES, ids=MODE_IDS)
+@pytest.mark.parametrize("case", range(len(SMALL)))
+def test_schedules_against_the_oracle(mode, case, schedule):
+    """Every way of cutting a step into launches and work ranges gives the oracle's result: static
+    ranges instead of claimed items, one launch per lazy block, one launch per layer with the logit
+    cache, and the in-order schedule in which a leader's launch also sweeps its followers' cached V
+    rows (a VLA_QC follower's own launch is its text sweep; a GLA follower's is the merge, which
+    adds the new token as one more key, Eq. 6).  Ragged batch: a sequence without visual tokens,
+    different lengths, pages that fill up during the steps."""
+    head_dim, group, layer_kind, split = SMALL[case]
+    w = _small_workload(head_dim, group, layer_kind, 60 + case)
+    trunc = [w.n_prompt, 9, 70]
+    seq_ids = [2, 0, 3]
+    o = LazyAttentionOracle(w.n_layers, w.n_q_heads, w.n_kv_heads, head_dim, layer_kind, mode, n_seqs=3)
+    s = Session(w.n_layers, w.n_q_heads, w.n_kv_heads, head_dim, layer_kind, max_seqs=4, max_tokens_per_seq=256,
+                n_pages=w.n_layers * 4 * 3 * 17, lazy_mode=mode, split_tokens=split, poison_pool=True)
+    for key, value in SCHEDULES[schedule]:
+        s.set_option(key, value)
+    for b, sid in enumerate(seq_ids):
+        kind, k, v = W.prefill_kv_np(w, b)
+        T = trunc[b]
+        kind, k, v = kind[:T].copy(), k[:, :T], v[:, :T]
+        if b == 1:
+            kind[:] = 0
+        s.prefill_append([sid], [T], kind, _dev(k, s.device), _dev(v, s.device))
+        o.prefill_append(b, kind.tolist(), f64(k), f64(v))
+    out = torch.empty((w.n_layers, 3, w.n_q_heads, head_dim), dtype=torch.bfloat16, device=s.device)
+    lse = torch.empty((w.n_layers, 3, w.n_q_heads), dtype=torch.float32, device=s.device)
+    for step in range(w.decode_steps):
+        qn, kn, vn = W.decode_qkv_np(w, step)
+        s.decode_step(seq_ids, _dev(qn, s.device), _dev(kn, s.device), _dev(vn, s.device), out, lse)
+        got, got_lse = bits_of(out), lse.cpu().numpy()
+        for b in range(3):
+            ref, ref_lse = o.decode_step(b, f64(qn[:, b]), f64(kn[:, b]), f64(vn[:, b]))
+            for l in range(w.n_layers):
+                assert_close(got[l, b], ref[l], f"{schedule}: case {case} step {step} seq {b} layer {l}")
+            np.testing.assert_allclose(got_lse[:, b], ref_lse, atol=2e-3, rtol=0)
+    assert s.stats().device_error == 0
+    s.close()
 
 
 def test_split_size_changes_only_rounding():
@@ -451,21 +508,31 @@ FULL_CASES = [
     ("llava15_7b", qc.QC_MODE_VLA_QC, 16, "per_layer"),
     ("qwen2vl_gqa", qc.QC_MODE_VLA_QC, 16, "per_layer"),
     ("llava_next_2048_lazy22", qc.QC_MODE_GLA, 16, "per_layer"),
+    # the in-order schedule (the configuration bench.py's headline is timed on)
+    ("llava15_7b", qc.QC_MODE_VLA_QC, 24, "in_order"),
+    ("llava_next_anyres", qc.QC_MODE_VLA_QC, 16, "in_order"),
+    ("qwen2vl_gqa", qc.QC_MODE_VLA_QC, 24, "in_order"),
+    ("long_video_pruned", qc.QC_MODE_VLA_QC, 16, "in_order"),
+    ("llava15_7b", qc.QC_MODE_GLA, 16, "in_order"),
+    ("llava_next_2048_lazy22", qc.QC_MODE_GLA, 16, "in_order"),
+    ("llava_next_2048_lazy22", qc.QC_MODE_VLA_QC, 16, "in_order"),
 ]
 
 
 @pytest.mark.parametrize("case", FULL_CASES, ids=["-".join([c[0], MODE_IDS[c[1]]] + list(c[3:])) for c in FULL_CASES])
 def test_full_size_sampled(case):
     name, mode, n_samples = case[:3]
-    per_layer = len(case) > 3
+    launches = case[3] if len(case) > 3 else "one_launch"
     w = W.get_workload(name)
     rng = np.random.default_rng(w.seed)
     samples = _samples(w, n_samples, rng)
     oracles = [SampledOracle(w, mode, *t) for t in samples]
     schedule = set(step_schedule(w.decode_steps))
     s = Session.for_workload(w, lazy_mode=mode)
-    if per_layer:
+    if launches == "per_layer":
         s.set_option("per_layer_logit_cache", 1)
+    elif launches == "in_order":
+        s.set_option("in_order_launches", 1)
     s.prefill_workload(w)
     model = pg.PagedCacheModel(w.layer_kind().tolist(), mode, 16, s.cfg.n_pages, w.batch)
     for b in range(w.batch):

@@ -44,7 +44,7 @@ def test_random_call_sequences(trial):
     layer_kind = PATTERNS[trial % len(PATTERNS)]
     head_dim, group, hkv = SHAPES[(trial // 2) % len(SHAPES)]
     mode = int(rng.integers(3))
-    schedule = ["fused", "per_block", "per_layer"][trial % 3]
+    schedule = ["fused", "per_block", "per_layer", "in_order"][trial % 4]
     split = int(rng.choice([16, 32, 64, 128]))
     n_layers, hq = len(layer_kind), hkv * group
     n_pages = n_layers * 4 * MAX_SEQS * (MAX_TOKENS // 16 + 1)
@@ -54,6 +54,8 @@ def test_random_call_sequences(trial):
         s.set_option("layers_per_launch", 1)
     elif schedule == "per_layer":
         s.set_option("per_layer_logit_cache", 1)
+    elif schedule == "in_order":
+        s.set_option("in_order_launches", 1)
     model = pg.PagedCacheModel(layer_kind, mode, 16, n_pages, MAX_SEQS)
     oracles = {}      # live sequence id -> oracle of that lifetime
     lengths = {}      # live sequence id -> tokens held
