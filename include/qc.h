@@ -102,6 +102,8 @@ typedef struct qc_stats {
   int32_t device_error;           /* 0, or the QC_ERR_* code the device error word holds */
   int32_t n_active_seqs;
   int64_t kernel_launches;        /* kernels of this library launched for the cache so far */
+  int64_t kv_bytes_swept;         /* algorithmic K/V bytes of the decode steps so far: every stored row of the
+                                     listed sequences once per step */
 } qc_stats;
 
 /* Per-step kernel timing (CUDA events on the library's stream), for roofline accounting. */
@@ -121,6 +123,11 @@ typedef struct qc_profile {
                                  2 * head_dim flops for every score pass (one per layer, or one per
                                  run of layers that share their scores) and 2 * head_dim for every
                                  layer's value product */
+  double attend_kernel_ms;    /* option "profile" = 2: summed durations of the attention launches alone,
+                                 each between events of its own (events between launches end the
+                                 overlap of a launch's start with its predecessor's end: this mode is
+                                 for the kernel's time, not for the step's) */
+  int64_t attend_kernel_launches;
 } qc_profile;
 
 /* Create a context on `device` that launches on `cuda_stream` (a cudaStream_t; NULL is the
@@ -254,7 +261,18 @@ int32_t qc_debug_read_row(qc_cache* cache, int32_t layer, int32_t stream, int32_
  * normalises their scores once per run of up to three layers and applies them to each layer's V,
  * bit-identically to one pass per layer; 0 = never, 1 = for prompts of 1536 tokens or more (the
  * default: below that the pass's lower occupancy costs more than it saves), 2 = always),
- * "profile" (1 = record CUDA events per step). */
+ * "profile" (1 = record CUDA events per step; 2 = also around every attention launch), "in_order_launches"
+ * (1 = one launch per layer in layer order, each using nothing of later layers; what a follower
+ * shares with its leader are scores over rows cached before the step, so a leader's launch also
+ * weights its followers' cached V rows and leaves their partial rows behind; a VLA_QC follower's
+ * launch is its text sweep, a GLA follower's is the merge with the step's new token as one more
+ * key, Eq. 6; VLA_EQ8 followers sweep the leader's visual K with their own query), "static_partition"
+ * (-1 = a step of several launches cuts each launch's work into equal ranges of K/V tiles, one or a
+ * few per worker, instead of handing out chunk items; 0 = never; 1 = always), "static_min_tiles",
+ * "static_row_cost" (tuning of those ranges: shortest range, and what one more output row counts
+ * for, in 4 KiB tiles), "plan_ahead" (0 = workers locate their ranges themselves instead of reading
+ * starting points that one kernel per step works out for every launch), "fused_merge" (1 = the
+ * worker that delivers an output row's last partial merges it, instead of a merge launch). */
 int32_t qc_set_option(qc_cache* cache, const char* key, int64_t value);
 
 /* Sum the recorded kernel times since the last call (synchronises), then reset them. */

@@ -53,7 +53,7 @@ class qc_stats(C.Structure):
         ("kv_bytes_stored_paged", C.c_int64), ("kv_bytes_all_full_paged", C.c_int64),
         ("qcache_bytes", C.c_int64), ("decode_steps", C.c_int64), ("attend_launches", C.c_int64),
         ("device_error", C.c_int32), ("n_active_seqs", C.c_int32),
-        ("kernel_launches", C.c_int64),
+        ("kernel_launches", C.c_int64), ("kv_bytes_swept", C.c_int64),
     ]
 
 
@@ -62,6 +62,7 @@ class qc_profile(C.Structure):
         ("steps", C.c_int64), ("attend_ms", C.c_double), ("step_ms", C.c_double),
         ("kv_bytes_read", C.c_int64), ("items", C.c_int64),
         ("prefill_calls", C.c_int64), ("prefill_attend_ms", C.c_double), ("prefill_flops", C.c_double),
+        ("attend_kernel_ms", C.c_double), ("attend_kernel_launches", C.c_int64),
     ]
 
 

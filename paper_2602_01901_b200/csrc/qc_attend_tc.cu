@@ -279,7 +279,7 @@ __device__ __forceinline__ void process_item_tc(WorkerState& st, const TcCtx* ct
 // arrives by asynchronous copies.
 template <int D, bool STATIC>
 __device__ __forceinline__ void attend_tc_worker(const Params& P, TcCtx* ctx, uint32_t ring, uint64_t* full,
-                                                 RangeCursor* cursor, int wid, int lane) {
+                                                 RangeCursor* cursor, int32_t* stage, int wid, int lane) {
   auto ctx_of = [ctx](int k) -> const ItemPages& { return ctx[k % kCtxSlots].ip; };
   WorkerState st;
   worker_init(st, 0);
@@ -295,26 +295,42 @@ __device__ __forceinline__ void attend_tc_worker(const Params& P, TcCtx* ctx, ui
   // ---- ahead of the wait for the previous kernel: the first items and their page ids (from the
   // launch plan, the step descriptors and the page tables, all written before that kernel
   // started), and the first tiles unless they could hold the step's new token
-  if (STATIC) {
+  Item first;
+  if (STATIC && P.wdesc != nullptr) {
+    // planned ahead: one read gives the first item, its first page ids and the cursor
     if (wid >= P.part_workers) return;
-    RangeCursor c;
-    const bool any = cursor_init(c, P, wid, lane);
-    if (lane == 0) *cursor = c;
-    __syncwarp();
-    if (!any) return;
+    if (!load_worker_desc(P, wid, ctx[0].ip, cursor, stage, lane)) return;
+    first = ctx[0].ip.item;
+    st.n_my = 1;
+    const bool early_tiles = !(first.stream == 0 && (first.flags & kFlagStreamEnd) && first.n_pages <= kRingTc);
+    if (early_tiles) fill_ring<D, kRingTc, true>(st, ctx_of, ring, full, P, lane);
+    begin_item_pages(ctx[0].ip, P, first, lane);   // the whole page list, while the tiles fly
   } else {
-    issued = claim_issue(P, lane);
+    if (STATIC) {
+      if (wid >= P.part_workers) return;
+      RangeCursor c;
+      const bool any = cursor_init(c, part_view(P), wid, lane);
+      if (lane == 0) *cursor = c;
+      __syncwarp();
+      if (!any) return;
+    } else {
+      pdl_wait();   // the item list and the work counter are the previous kernel's
+      pdl_launch_dependents();
+      issued = claim_issue(P, lane);
+    }
+    if (!take()) return;
+    begin_item_pages(ctx[0].ip, P, it, lane);
+    first = it;
+    cp_async_wait_all();
+    __syncwarp();
+    st.n_my = 1;
+    const bool early_tiles = !(first.stream == 0 && (first.flags & kFlagStreamEnd) && first.n_pages <= kRingTc);
+    if (early_tiles) fill_ring<D, kRingTc, true>(st, ctx_of, ring, full, P, lane);
   }
-  if (!take()) return;
-  begin_item_pages(ctx[0].ip, P, it, lane);
-  const Item first = it;
-  cp_async_wait_all();
-  __syncwarp();
-  st.n_my = 1;
-  const bool early_tiles = !(first.stream == 0 && (first.flags & kFlagStreamEnd) && first.n_pages <= kRingTc);
-  if (early_tiles) fill_ring<D, kRingTc, true>(st, ctx_of, ring, full, P, lane);
-  pdl_wait();
-  pdl_launch_dependents();
+  if (STATIC) {
+    pdl_wait();
+    pdl_launch_dependents();
+  }
   // ---- this layer's inputs; the rest of the first tiles; the second item's context while they fly
   fill_ring<D, kRingTc, true>(st, ctx_of, ring, full, P, lane);
   if (STATIC) record_row_slots(P, first, lane);
@@ -373,12 +389,13 @@ __device__ __forceinline__ void attend_tc_worker(const Params& P, TcCtx* ctx, ui
   }
 }
 
-template <int D>
+template <int D, bool STATIC>
 __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_constant__ Params P) {
   constexpr uint32_t kTile = kPage * D * 2;
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t full_all[kWarps][kRingTc];
   __shared__ __align__(16) RangeCursor cursors[kWarps];
+  __shared__ __align__(16) int32_t stages[kWarps][12];
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // swizzled tiles must sit on 1024-byte boundaries
@@ -394,10 +411,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
   }
   __syncthreads();
 
-  if (P.part_static)
-    attend_tc_worker<D, true>(P, ctx, ring, full, &cursors[warp], warp * gridDim.x + blockIdx.x, lane);
-  else
-    attend_tc_worker<D, false>(P, ctx, ring, full, &cursors[warp], 0, lane);
+  attend_tc_worker<D, STATIC>(P, ctx, ring, full, &cursors[warp], stages[warp], warp * gridDim.x + blockIdx.x, lane);
 }
 
 template <int D>
@@ -408,10 +422,16 @@ constexpr int attend_tc_smem_bytes() {
 }  // namespace
 
 cudaError_t configure_kernels_tc(int* attend_smem) {
-  cudaError_t e = cudaFuncSetAttribute(attend_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaError_t e = cudaFuncSetAttribute(attend_tc_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        attend_tc_smem_bytes<128>());
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(attend_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  e = cudaFuncSetAttribute(attend_tc_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           attend_tc_smem_bytes<128>());
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(attend_tc_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           attend_tc_smem_bytes<64>());
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(attend_tc_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            attend_tc_smem_bytes<64>());
   if (attend_smem) *attend_smem = attend_tc_smem_bytes<128>();
   return e;
@@ -421,9 +441,14 @@ cudaError_t launch_attend_tc(const Params& p, int n_sms, cudaStream_t stream) {
   const int n_items = p.item_end - p.item_begin;
   if (!p.part_static && n_items <= 0) return cudaSuccess;
   const int grid = p.part_static ? min(n_sms, p.part_workers) : min(n_sms, (n_items + kWarps - 1) / kWarps);
-  if (p.d == 128)
-    return launch_pdl(attend_tc_kernel<128>, dim3(grid), dim3(kThreads), attend_tc_smem_bytes<128>(), stream, p);
-  return launch_pdl(attend_tc_kernel<64>, dim3(grid), dim3(kThreads), attend_tc_smem_bytes<64>(), stream, p);
+  if (p.d == 128) {
+    if (p.part_static)
+      return launch_pdl(attend_tc_kernel<128, true>, dim3(grid), dim3(kThreads), attend_tc_smem_bytes<128>(), stream, p);
+    return launch_pdl(attend_tc_kernel<128, false>, dim3(grid), dim3(kThreads), attend_tc_smem_bytes<128>(), stream, p);
+  }
+  if (p.part_static)
+    return launch_pdl(attend_tc_kernel<64, true>, dim3(grid), dim3(kThreads), attend_tc_smem_bytes<64>(), stream, p);
+  return launch_pdl(attend_tc_kernel<64, false>, dim3(grid), dim3(kThreads), attend_tc_smem_bytes<64>(), stream, p);
 }
 
 }  // namespace qc

@@ -211,7 +211,6 @@ struct WorkerState {
   uint32_t cons_phase;
   int in_flight;
   bool dead;           // a bounded wait ran out: stop fetching, drain, leave
-  uint64_t policy;     // L2 policy of the tile copies
 };
 
 __device__ __forceinline__ void worker_init(WorkerState& st, int n_my) {
@@ -222,7 +221,6 @@ __device__ __forceinline__ void worker_init(WorkerState& st, int n_my) {
   st.cons_phase = 0;
   st.in_flight = 0;
   st.dead = false;
-  st.policy = l2_evict_first_policy();
 }
 
 // Issue the copy of the next tile.  D: head dim; RING: slots; TMAP: copy through the tensor
@@ -246,13 +244,14 @@ __device__ __forceinline__ bool issue_one(WorkerState& st, CtxFn ctx, uint32_t r
     const uint32_t dst = ring + st.iss_slot * kTile;
     fence_proxy_async();   // the slot's earlier generic-proxy accesses precede this async write
     mbar_expect_tx(bar, kTile);
+    const uint64_t policy = l2_evict_first_policy();
     if (TMAP) {
       const int32_t row = (pid * P.hkv + c.kv_head) * kPage;
-      tensor_g2s_2d(dst, &P.tmap, 0, row, bar, st.policy);
-      if (D == 128) tensor_g2s_2d(dst + kTile / 2, &P.tmap, 64, row, bar, st.policy);
+      tensor_g2s_2d(dst, &P.tmap, 0, row, bar, policy);
+      if (D == 128) tensor_g2s_2d(dst + kTile / 2, &P.tmap, 64, row, bar, policy);
     } else {
       const uint16_t* src = P.pool + (static_cast<size_t>(pid) * P.hkv + c.kv_head) * (kPage * D);
-      bulk_g2s(dst, src, kTile, bar, st.policy);
+      bulk_g2s(dst, src, kTile, bar, policy);
     }
   }
   st.iss_slot = (st.iss_slot + 1 == RING) ? 0 : st.iss_slot + 1;
@@ -375,7 +374,8 @@ __device__ __forceinline__ int claim_take(const Params& P, int issued) {
 // The work of a launch is laid out in tiles: plan positions of the launch in order, inside a
 // position the listed sequences, inside a sequence the rows (one per query head, or per query
 // group with GQA), inside a row its pages, each page worth w tiles (one K tile unless the scores
-// come from the logit cache, one V tile per consumer).  The space of T tiles is cut into ranges of
+// come from the logit cache, one V tile per consumer) after a fixed part_row_cost per row (what
+// starting and finishing an item costs a worker).  The space of T tiles is cut into ranges of
 // part_q tiles; a page belongs to the range its first tile falls into.  Physical worker i takes
 // ranges i*part_k .. i*part_k + part_k - 1, which are adjacent, so it walks rows forward from one
 // starting point.  The pages of a row that one range owns are one piece: an Item whose partial
@@ -384,8 +384,8 @@ __device__ __forceinline__ int claim_take(const Params& P, int issued) {
 // first and last owns a page of it: no slot is left unwritten), a piece has at most
 // kMaxChunkPages pages and a row at most slots_per_stream pieces; T < 2^31.
 
-struct RangeCursor {
-  int32_t r0;        // tile offset of the current row
+struct __align__(16) RangeCursor {
+  int32_t r0;        // tile offset of the current row's first page
   int32_t vw_end;    // first tile beyond the current range
   int32_t vw, vw_stop;
   int32_t pos, si, u;
@@ -393,92 +393,134 @@ struct RangeCursor {
   int32_t page;             // next page of the current row to hand out
   int32_t owner0;           // range that owns the row's first page
   int32_t len, seq_id;      // tokens of the row's stream; its sequence
-  int32_t pad;
+  int32_t pad[3];
   Job job;
 };
-static_assert(sizeof(RangeCursor) == 72, "RangeCursor layout");
+static_assert(sizeof(RangeCursor) == 80, "RangeCursor layout");
+
+// What the partition of one launch is made of (the attention kernels take it from their
+// parameters, the kernel that plans every launch of a step ahead from its launch list).
+struct PartView {
+  const PlanJob* plan;
+  const StepSeq* seqs;
+  int32_t* err;
+  int32_t pos_begin, pos_end, n_seqs;
+  int32_t q, k, vw, row_cost;          // tiles per range, ranges per worker, ranges, fixed tiles per row
+  int32_t tp_v, tp_t;                  // pages of the visual / text streams over the listed sequences
+  int32_t rows, heads_per_item, group, slots_per_stream;   // rows per (position, sequence); query heads per row
+};
+
+__device__ __forceinline__ PartView part_view(const Params& P) {
+  PartView V;
+  V.plan = P.plan, V.seqs = P.seqs, V.err = P.err;
+  V.pos_begin = P.pos_begin, V.pos_end = P.pos_end, V.n_seqs = P.n_seqs;
+  V.q = P.part_q, V.k = P.part_k, V.vw = P.part_vw, V.row_cost = P.part_row_cost;
+  V.tp_v = P.tp_v, V.tp_t = P.tp_t;
+  V.rows = P.heads_per_item_dim, V.heads_per_item = P.heads_per_item, V.group = P.group;
+  V.slots_per_stream = P.slots_per_stream;
+  return V;
+}
 
 __device__ __forceinline__ int job_tiles_per_page(const Job& j) {
   return ((j.flags & kFlagReadLogits) ? 0 : 1) + j.n_cons;
 }
 
 // Load the job of plan position c.pos (if it changed) and the sequence c.si into the cursor.
-__device__ __forceinline__ void cursor_load_segment(RangeCursor& c, const Params& P, bool new_pos) {
+__device__ __forceinline__ void cursor_load_segment(RangeCursor& c, const PartView& V, bool new_pos) {
   if (new_pos) {
-    const uint4 raw = __ldg(reinterpret_cast<const uint4*>(P.plan + c.pos));
+    const uint4 raw = __ldg(reinterpret_cast<const uint4*>(V.plan + c.pos));
     *reinterpret_cast<uint4*>(&c.job) = raw;
     c.w = job_tiles_per_page(c.job);
   }
-  const StepSeq sq = P.seqs[c.si];
+  const StepSeq sq = V.seqs[c.si];
   c.len = c.job.stream ? sq.len_vis : sq.len_text;
   c.seq_id = sq.seq_id;
   c.row_pages = (c.len + kPage - 1) / kPage;
 }
 
+// Tile offset at which the rows of a plan position start (index: its place in the launch).
+__device__ __forceinline__ int32_t pos_base_of(const PartView& V, int wv_before, int wt_before, int index) {
+  return V.rows * (wv_before * V.tp_v + wt_before * V.tp_t + V.row_cost * V.n_seqs * index);
+}
+
+// With position, job, sequence and its length in place: the row and page at which tile t0 falls.
+__device__ __forceinline__ void cursor_place(RangeCursor& c, const PartView& V, int32_t t0, int32_t pos_base,
+                                             int32_t my_pre) {
+  c.w = job_tiles_per_page(c.job);
+  c.row_pages = (c.len + kPage - 1) / kPage;
+  const int32_t seg_base = pos_base + V.rows * (c.w * my_pre + V.row_cost * c.si);
+  // a row costs its fixed part and then its pages; r0 is where its first page starts
+  const int32_t row_cost = V.row_cost + c.w * c.row_pages;
+  c.u = row_cost > 0 ? min(V.rows - 1, (t0 - seg_base) / row_cost) : 0;
+  c.r0 = seg_base + c.u * row_cost + V.row_cost;
+  c.page = t0 > c.r0 ? (t0 - c.r0 + c.w - 1) / c.w : 0;   // first page that starts at or after t0
+  c.owner0 = c.r0 / V.q;
+  c.pad[0] = c.pad[1] = c.pad[2] = 0;
+}
+
 // Place the cursor of worker `wid` at its first range; false if the worker has no work.  All
-// lanes compute the same values.  Reads the launch plan and the step's sequence descriptors only,
-// the first 32 of each in one round of loads.
-__device__ __forceinline__ bool cursor_init(RangeCursor& c, const Params& P, int wid, int lane) {
-  const int32_t R = P.heads_per_item_dim;
-  c.vw = wid * P.part_k;
-  c.vw_stop = min(c.vw + P.part_k, P.part_vw);
+// lanes of a warp compute the same values.  Reads the launch plan and the step's sequence
+// descriptors only, the first 32 of each in one round of loads.
+__device__ __forceinline__ bool cursor_init(RangeCursor& c, const PartView& V, int wid, int lane) {
+  c.vw = wid * V.k;
+  c.vw_stop = min(c.vw + V.k, V.vw);
   if (c.vw >= c.vw_stop) return false;
-  const int32_t t0 = c.vw * P.part_q;
-  c.vw_end = t0 + P.part_q;
-  const int n_pos = P.pos_end - P.pos_begin;
+  const int32_t t0 = c.vw * V.q;
+  c.vw_end = t0 + V.q;
+  const int n_pos = V.pos_end - V.pos_begin;
   uint4 pj_lo = make_uint4(0, 0, 0, 0);
   int4 pj_hi = make_int4(0, 0, 0, 0);
   int4 sq_lo = make_int4(0, 0, 0, 0), sq_hi = make_int4(0, 0, 0, 0);
   if (lane < n_pos) {
-    pj_lo = __ldg(reinterpret_cast<const uint4*>(P.plan + P.pos_begin + lane));
-    pj_hi = __ldg(reinterpret_cast<const int4*>(P.plan + P.pos_begin + lane) + 1);
+    pj_lo = __ldg(reinterpret_cast<const uint4*>(V.plan + V.pos_begin + lane));
+    pj_hi = __ldg(reinterpret_cast<const int4*>(V.plan + V.pos_begin + lane) + 1);
   }
-  if (lane < P.n_seqs) {
-    sq_lo = reinterpret_cast<const int4*>(P.seqs + lane)[0];   // seq_id, len_text, len_vis, n_slots
-    sq_hi = reinterpret_cast<const int4*>(P.seqs + lane)[1];   // pre_v, pre_t, ncv, pad
+  if (lane < V.n_seqs) {
+    sq_lo = reinterpret_cast<const int4*>(V.seqs + lane)[0];   // seq_id, len_text, len_vis, n_slots
+    sq_hi = reinterpret_cast<const int4*>(V.seqs + lane)[1];   // pre_v, pre_t, ncv, pad
   }
   // plan position: the last one of the launch that starts at or before t0
-  auto pos_base_of = [&](int wv_before, int wt_before) { return R * (wv_before * P.tp_v + wt_before * P.tp_t); };
-  int n_le = __popc(__ballot_sync(0xffffffffu, lane < n_pos && pos_base_of(pj_hi.z, pj_hi.w) <= t0));
+  int n_le = __popc(__ballot_sync(0xffffffffu, lane < n_pos && pos_base_of(V, pj_hi.z, pj_hi.w, lane) <= t0));
   int32_t pos_base;
   if (n_le == 32 && n_pos > 32) {   // beyond the first round
-    for (int base = P.pos_begin + 32; base < P.pos_end; base += 32) {
+    for (int base = V.pos_begin + 32; base < V.pos_end; base += 32) {
       const int idx = base + lane;
       bool le = false;
-      if (idx < P.pos_end) {
-        const int4 hi = __ldg(reinterpret_cast<const int4*>(P.plan + idx) + 1);
-        le = pos_base_of(hi.z, hi.w) <= t0;
+      if (idx < V.pos_end) {
+        const int4 hi = __ldg(reinterpret_cast<const int4*>(V.plan + idx) + 1);
+        le = pos_base_of(V, hi.z, hi.w, idx - V.pos_begin) <= t0;
       }
       n_le += __popc(__ballot_sync(0xffffffffu, le));
     }
-    c.pos = P.pos_begin + n_le - 1;
-    const PlanJob pj = P.plan[c.pos];
+    c.pos = V.pos_begin + n_le - 1;
+    const PlanJob pj = V.plan[c.pos];
     c.job = pj.job;
-    pos_base = pos_base_of(pj.wv_before, pj.wt_before);
+    pos_base = pos_base_of(V, pj.wv_before, pj.wt_before, c.pos - V.pos_begin);
   } else {
     const int src = max(n_le, 1) - 1;
-    c.pos = P.pos_begin + src;
+    c.pos = V.pos_begin + src;
     uint4 j;
     j.x = __shfl_sync(0xffffffffu, pj_lo.x, src);
     j.y = __shfl_sync(0xffffffffu, pj_lo.y, src);
     j.z = __shfl_sync(0xffffffffu, pj_lo.z, src);
     j.w = __shfl_sync(0xffffffffu, pj_lo.w, src);
     *reinterpret_cast<uint4*>(&c.job) = j;
-    pos_base = pos_base_of(__shfl_sync(0xffffffffu, pj_hi.z, src), __shfl_sync(0xffffffffu, pj_hi.w, src));
+    pos_base = pos_base_of(V, __shfl_sync(0xffffffffu, pj_hi.z, src), __shfl_sync(0xffffffffu, pj_hi.w, src), src);
   }
-  c.w = job_tiles_per_page(c.job);
+  const int w = job_tiles_per_page(c.job);
   // listed sequence: the last one whose rows start at or before t0
-  n_le = __popc(__ballot_sync(0xffffffffu, lane < P.n_seqs && pos_base + R * c.w * (c.job.stream ? sq_hi.x : sq_hi.y) <= t0));
+  const int32_t rc = V.row_cost;
+  n_le = __popc(__ballot_sync(0xffffffffu, lane < V.n_seqs && pos_base + V.rows * (w * (c.job.stream ? sq_hi.x : sq_hi.y) + rc * lane) <= t0));
   int32_t my_pre;
-  if (n_le == 32 && P.n_seqs > 32) {
-    for (int base = 32; base < P.n_seqs; base += 32) {
+  if (n_le == 32 && V.n_seqs > 32) {
+    for (int base = 32; base < V.n_seqs; base += 32) {
       const int idx = base + lane;
       bool le = false;
-      if (idx < P.n_seqs) le = pos_base + R * c.w * (c.job.stream ? P.seqs[idx].pre_v : P.seqs[idx].pre_t) <= t0;
+      if (idx < V.n_seqs) le = pos_base + V.rows * (w * (c.job.stream ? V.seqs[idx].pre_v : V.seqs[idx].pre_t) + rc * idx) <= t0;
       n_le += __popc(__ballot_sync(0xffffffffu, le));
     }
     c.si = n_le - 1;
-    const StepSeq sq = P.seqs[c.si];
+    const StepSeq sq = V.seqs[c.si];
     c.len = c.job.stream ? sq.len_vis : sq.len_text;
     c.seq_id = sq.seq_id;
     my_pre = c.job.stream ? sq.pre_v : sq.pre_t;
@@ -489,51 +531,71 @@ __device__ __forceinline__ bool cursor_init(RangeCursor& c, const Params& P, int
     c.seq_id = __shfl_sync(0xffffffffu, sq_lo.x, src);
     my_pre = __shfl_sync(0xffffffffu, c.job.stream ? sq_hi.x : sq_hi.y, src);
   }
-  c.row_pages = (c.len + kPage - 1) / kPage;
-  const int32_t seg_base = pos_base + R * c.w * my_pre;
-  c.u = 0;
-  c.r0 = seg_base;
-  c.page = 0;
-  if (c.row_pages > 0) {
-    const int32_t row_tiles = c.w * c.row_pages;
-    c.u = min(R - 1, (t0 - seg_base) / row_tiles);
-    c.r0 = seg_base + c.u * row_tiles;
-    c.page = (t0 - c.r0 + c.w - 1) / c.w;   // first page that starts at or after t0
+  cursor_place(c, V, t0, pos_base, my_pre);
+  return true;
+}
+
+// The same by one thread alone (the kernel that plans a step's launches ahead).
+__device__ __forceinline__ bool cursor_init_scalar(RangeCursor& c, const PartView& V, int wid) {
+  c.vw = wid * V.k;
+  c.vw_stop = min(c.vw + V.k, V.vw);
+  if (c.vw >= c.vw_stop) return false;
+  const int32_t t0 = c.vw * V.q;
+  c.vw_end = t0 + V.q;
+  c.pos = V.pos_begin;
+  int32_t pos_base = 0;
+  for (int p = V.pos_begin + 1; p < V.pos_end; ++p) {
+    const int4 hi = __ldg(reinterpret_cast<const int4*>(V.plan + p) + 1);
+    const int32_t b = pos_base_of(V, hi.z, hi.w, p - V.pos_begin);
+    if (b > t0) break;
+    c.pos = p;
+    pos_base = b;
   }
-  c.owner0 = c.r0 / P.part_q;
-  c.pad = 0;
+  c.job = V.plan[c.pos].job;
+  const int w = job_tiles_per_page(c.job);
+  int lo = 0, hi = V.n_seqs - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    const int32_t pre = c.job.stream ? V.seqs[mid].pre_v : V.seqs[mid].pre_t;
+    if (pos_base + V.rows * (w * pre + V.row_cost * mid) <= t0) lo = mid;
+    else hi = mid - 1;
+  }
+  c.si = lo;
+  const StepSeq sq = V.seqs[c.si];
+  c.len = c.job.stream ? sq.len_vis : sq.len_text;
+  c.seq_id = sq.seq_id;
+  cursor_place(c, V, t0, pos_base, c.job.stream ? sq.pre_v : sq.pre_t);
   return true;
 }
 
 // Next piece of the worker's ranges, or false when they are used up.  Warp-uniform.
-__device__ __forceinline__ bool cursor_next(RangeCursor& c, const Params& P, Item& it) {
-  const int R = P.heads_per_item_dim;
+__device__ __forceinline__ bool cursor_next(RangeCursor& c, const PartView& V, Item& it) {
   for (;;) {
     if (c.vw >= c.vw_stop) return false;
     if (c.page >= c.row_pages) {   // next row
-      c.r0 += c.w * c.row_pages;
+      c.r0 += c.w * c.row_pages + V.row_cost;
       c.page = 0;
-      if (++c.u == R) {
+      if (++c.u == V.rows) {
         c.u = 0;
         bool new_pos = false;
-        if (++c.si == P.n_seqs) {
+        if (++c.si == V.n_seqs) {
           c.si = 0;
           new_pos = true;
-          if (++c.pos >= P.pos_end) {
+          if (++c.pos >= V.pos_end) {
             c.vw = c.vw_stop;
             return false;
           }
         }
-        cursor_load_segment(c, P, new_pos);
+        cursor_load_segment(c, V, new_pos);
       }
-      c.owner0 = c.r0 / P.part_q;
+      c.owner0 = c.r0 / V.q;
       continue;
     }
     const int32_t d = c.vw_end - c.r0;
     const int lim = d <= 0 ? 0 : min(c.row_pages, (d + c.w - 1) / c.w);
     if (c.page < lim) {
-      const int hpi = P.heads_per_item;
-      const int n_sub = (P.group + hpi - 1) / hpi;
+      const int hpi = V.heads_per_item;
+      const int n_sub = (V.group + hpi - 1) / hpi;
       const int kv_head = c.u / n_sub, sub = c.u - kv_head * n_sub;
       const int slot = c.vw - c.owner0;
       it.k_layer = c.job.k_layer;
@@ -547,21 +609,21 @@ __device__ __forceinline__ bool cursor_next(RangeCursor& c, const Params& P, Ite
       }
       it.seq_id = static_cast<uint16_t>(c.seq_id);
       it.seq_idx = static_cast<uint16_t>(c.si);
-      it.head = static_cast<uint16_t>(kv_head * P.group + sub * hpi);
-      it.slot = static_cast<uint16_t>((c.job.stream ? 0 : P.slots_per_stream) + slot);
+      it.head = static_cast<uint16_t>(kv_head * V.group + sub * hpi);
+      it.slot = static_cast<uint16_t>((c.job.stream ? 0 : V.slots_per_stream) + slot);
       it.first_page = static_cast<uint16_t>(c.page);
       it.n_pages = static_cast<uint16_t>(lim - c.page);
       const bool last = lim == c.row_pages;
       if (last) it.flags |= kFlagStreamEnd;
       it.n_valid_last = static_cast<uint16_t>(last ? c.len - (c.row_pages - 1) * kPage : kPage);
-      it.n_heads = static_cast<uint8_t>(min(hpi, P.group - sub * hpi));
+      it.n_heads = static_cast<uint8_t>(min(hpi, V.group - sub * hpi));
       it.skip_new = c.job.skip_new;
       it.finish = c.job.finish;
       it.pad1 = 0;
       // the piece that holds a row's first page tells the merge how many pieces the row has
-      it.n_pieces = c.page == 0 ? static_cast<uint16_t>((c.r0 + c.w * (c.row_pages - 1)) / P.part_q - c.owner0 + 1) : 0;
-      if (lim - c.page > kMaxChunkPages || slot < 0 || slot >= P.slots_per_stream) {   // outside the plan's limits
-        atomicMax(P.err, kErrPlan);
+      it.n_pieces = c.page == 0 ? static_cast<uint16_t>((c.r0 + c.w * (c.row_pages - 1)) / V.q - c.owner0 + 1) : 0;
+      if (lim - c.page > kMaxChunkPages || slot < 0 || slot >= V.slots_per_stream) {   // outside the plan's limits
+        atomicMax(V.err, kErrPlan);
         c.vw = c.vw_stop;
         return false;
       }
@@ -570,7 +632,7 @@ __device__ __forceinline__ bool cursor_next(RangeCursor& c, const Params& P, Ite
     }
     // the current range owns nothing (more) of this row
     ++c.vw;
-    c.vw_end += P.part_q;
+    c.vw_end += V.q;
   }
 }
 
@@ -578,11 +640,29 @@ __device__ __forceinline__ bool cursor_next(RangeCursor& c, const Params& P, Ite
 __device__ __forceinline__ bool cursor_step(RangeCursor* slot, const Params& P, Item& it, int lane) {
   __syncwarp();
   RangeCursor c = *slot;
-  const bool ok = cursor_next(c, P, it);
+  const bool ok = cursor_next(c, part_view(P), it);
   __syncwarp();
   if (lane == 0) *slot = c;
   __syncwarp();
   return ok;
+}
+
+// Start of a worker from the descriptor planned for it when the step began: the first item goes
+// into the context slot together with the page ids of its first two pages, the cursor into the
+// worker's cursor slot.  False if the worker has no work.  `stage`: 48 bytes of shared memory.
+__device__ __forceinline__ bool load_worker_desc(const Params& P, int wid, ItemPages& c0, RangeCursor* cursor,
+                                                 int32_t* stage, int lane) {
+  const uint4* d = reinterpret_cast<const uint4*>(P.wdesc + static_cast<size_t>(P.launch_index) * kPlanWorkers + wid);
+  if (lane < 2) cp_async_16(reinterpret_cast<uint4*>(&c0.item) + lane, d + lane);
+  else if (lane < 5) cp_async_16(reinterpret_cast<uint4*>(stage) + (lane - 2), d + lane);
+  else if (lane < 10) cp_async_16(reinterpret_cast<uint4*>(cursor) + (lane - 5), d + lane);
+  cp_async_wait_all();
+  __syncwarp();
+  if (c0.item.n_pages == 0) return false;
+  if (lane < 2 * (1 + kMaxCons)) c0.pages[lane >> 1][lane & 1] = stage[lane];
+  if (lane == 0) c0.kv_head = c0.item.head / P.group;
+  __syncwarp();
+  return true;
 }
 
 // Under the static partition, the piece that holds a row's first page records how many pieces

@@ -85,6 +85,30 @@ struct Patch {
   int32_t index, page;
 };
 
+// Static partition of one attention launch, as the kernel that plans a step ahead needs it.
+struct LaunchDesc {
+  int32_t pos_begin, pos_end;
+  int32_t part_q, part_k, part_vw, part_workers, part_row_cost, pad;
+};
+static_assert(sizeof(LaunchDesc) == 32, "LaunchDesc layout");
+constexpr int kMaxPlanLaunches = 128;   // launches of a step that can be planned ahead (a launch per layer fits)
+constexpr int kPlanWorkers = 2048;      // worker descriptors kept per launch
+struct LaunchList {
+  LaunchDesc launch[kMaxPlanLaunches];
+};
+
+// Where a worker of a statically partitioned launch starts: its first item, the page ids of that
+// item's first two pages (K stream, then the V stream of each consumer) so that the first tiles
+// can be requested at once, and the cursor from which its later items follow.  Written for every
+// launch of a step by one kernel when the step begins; a worker then starts from one 160-byte read.
+struct __align__(16) WorkerDesc {
+  Item item;                        // n_pages == 0: the worker has no work
+  int32_t pids[1 + kMaxCons][2];
+  int32_t pad[2];
+  int32_t cursor[20];               // a RangeCursor
+};
+static_assert(sizeof(WorkerDesc) == 160, "WorkerDesc layout");
+
 // Kernel parameter block.
 struct Params {
   // cache-lifetime
@@ -106,6 +130,7 @@ struct Params {
   int32_t* work_counter;   // [n_layers] next unclaimed item of each attention launch of a step
   uint16_t* row_slots;     // [n_layers][max_seqs][hq][2]: partial rows the visual / the text sweep left for an
                            // output row (static partition only)
+  const WorkerDesc* wdesc; // [launches of the step][kPlanWorkers] planned ahead, or null: workers find their own start
   int32_t* row_done;       // [n_layers][max_seqs][hq]: pages of an output row swept so far in the current launch
                            // (the worker that completes the count merges the row and resets it)
   int64_t n_pool_pages;    // bound for page ids (reads never leave the pool)
@@ -133,6 +158,7 @@ struct Params {
   int32_t part_static;               // 0: items are claimed from the list
   int32_t part_vw, part_k, part_workers;
   int32_t part_q, part_tiles;        // tiles per range; tiles of the launch
+  int32_t part_row_cost;             // what a row counts for besides its pages, in tiles
   int32_t tp_v, tp_t;                // pages of the visual / text streams, summed over the listed sequences
   int32_t pos_begin, pos_end;        // plan positions of the launch
   int32_t slots_per_stream;          // partial-row slots of one stream of an output row (text slots start here)
@@ -143,6 +169,7 @@ struct Params {
 // launchers (qc_kernels.cu); all asynchronous on `stream`
 cudaError_t launch_setup(const Params& p, const StepInline* inl, cudaStream_t stream);
 cudaError_t launch_append(const Params& p, cudaStream_t stream);
+cudaError_t launch_plan(const Params& p, const LaunchList& list, int n_launches, cudaStream_t stream);   // writes p.wdesc
 cudaError_t launch_attend(const Params& p, int n_sms, cudaStream_t stream);      // one query head per item
 cudaError_t launch_attend_tc(const Params& p, int n_sms, cudaStream_t stream);   // query-group items (GQA)
 cudaError_t launch_merge(const Params& p, cudaStream_t stream);

@@ -64,7 +64,11 @@ __device__ __forceinline__ void append_rows(const Params& P, const StepSeq& sq, 
 // n_layers blocks do the append.  (The append reads page ids from the table, so it is only
 // fused on steps without patches.)
 __global__ void setup_kernel(const __grid_constant__ Params P, const __grid_constant__ StepInline inl) {
-  pdl_wait();   // (no early start of the successor: it plans its work from what this kernel writes)
+  // With claimed items the attention kernel touches nothing before its own wait, so it may be
+  // scheduled while this kernel runs; under the static partition it plans its first work ahead of
+  // its wait from what this kernel writes, and must not start early.
+  if (!P.part_static) pdl_launch_dependents();
+  pdl_wait();
   const StepSeq* seqs = P.inline_seqs ? inl.seqs : P.seqs;
   const int n_expand = P.n_pos * P.n_seqs;
   const int n_house = (max(max(P.n_patches, P.n_layers), P.n_seqs * 8) + blockDim.x - 1) / blockDim.x;
@@ -137,6 +141,46 @@ __global__ void setup_kernel(const __grid_constant__ Params P, const __grid_cons
 __global__ void append_kernel(const __grid_constant__ Params P) {
   pdl_wait();
   append_rows(P, P.seqs[blockIdx.x], blockIdx.x, P.layer_begin + blockIdx.y);   // layers of one launch group
+}
+
+// ------------------------------------------------------------------------------------------
+// plan: where every worker of every statically partitioned launch of the step starts
+// ------------------------------------------------------------------------------------------
+
+__global__ void plan_kernel(const __grid_constant__ Params P, const __grid_constant__ LaunchList list) {
+  pdl_wait();   // the page tables and the sequence descriptors are final
+  const int g = blockIdx.y, wid = blockIdx.x * blockDim.x + threadIdx.x;
+  const LaunchDesc L = list.launch[g];
+  if (wid >= kPlanWorkers) return;
+  WorkerDesc* out = const_cast<WorkerDesc*>(P.wdesc) + static_cast<size_t>(g) * kPlanWorkers + wid;
+  PartView V = part_view(P);
+  V.pos_begin = L.pos_begin, V.pos_end = L.pos_end;
+  V.q = L.part_q, V.k = L.part_k, V.vw = L.part_vw, V.row_cost = L.part_row_cost;
+  WorkerDesc d;
+  d.item.n_pages = 0;
+  RangeCursor c;
+  if (wid < L.part_workers && cursor_init_scalar(c, V, wid) && cursor_next(c, V, d.item)) {
+    const Item& it = d.item;
+    for (int j = 0; j < 2; ++j) {
+      const int pg = it.first_page + min(j, it.n_pages - 1);
+      d.pids[0][j] = P.table[table_row(P, it.k_layer, it.stream, it.seq_id) + pg];
+      for (int x = 0; x < kMaxCons; ++x)
+        d.pids[1 + x][j] = x < it.n_cons ? P.table[table_row(P, it.v_layer[x], 2 + it.stream, it.seq_id) + pg] : 0;
+    }
+    d.pad[0] = d.pad[1] = 0;
+    *reinterpret_cast<RangeCursor*>(d.cursor) = c;
+  } else {
+    d.item.n_pages = 0;
+  }
+  const uint4* src = reinterpret_cast<const uint4*>(&d);
+  uint4* dst = reinterpret_cast<uint4*>(out);
+  if (d.item.n_pages == 0) {   // no work: an all-zero item says so
+    dst[0] = make_uint4(0, 0, 0, 0);
+    dst[1] = make_uint4(0, 0, 0, 0);
+    return;
+  }
+#pragma unroll
+  for (int i = 0; i < 10; ++i) dst[i] = src[i];
 }
 
 // ------------------------------------------------------------------------------------------
@@ -403,7 +447,7 @@ __device__ __forceinline__ void process_item(WorkerState& st, const WarpCtx<D>* 
 // queries) arrives by asynchronous copies.
 template <int D, bool STATIC>
 __device__ __forceinline__ void attend_worker(const Params& P, WarpCtx<D>* ctx, uint32_t ring, uint64_t* full,
-                                              RangeCursor* cursor, int wid, int lane) {
+                                              RangeCursor* cursor, int32_t* stage, int wid, int lane) {
   auto ctx_of = [ctx](int k) -> const ItemPages& { return ctx[k % kCtxSlots].ip; };
   WorkerState st;
   worker_init(st, 0);
@@ -419,26 +463,42 @@ __device__ __forceinline__ void attend_worker(const Params& P, WarpCtx<D>* ctx, 
   // ---- ahead of the wait for the previous kernel: the first items and their page ids (from the
   // launch plan, the step descriptors and the page tables, all written before that kernel
   // started), and the first tiles unless they could hold the step's new token
-  if (STATIC) {
+  Item first;
+  if (STATIC && P.wdesc != nullptr) {
+    // planned ahead: one read gives the first item, its first page ids and the cursor
     if (wid >= P.part_workers) return;
-    RangeCursor c;
-    const bool any = cursor_init(c, P, wid, lane);
-    if (lane == 0) *cursor = c;
-    __syncwarp();
-    if (!any) return;
+    if (!load_worker_desc(P, wid, ctx[0].ip, cursor, stage, lane)) return;
+    first = ctx[0].ip.item;
+    st.n_my = 1;
+    const bool early_tiles = !(first.stream == 0 && (first.flags & kFlagStreamEnd) && first.n_pages <= kRing);
+    if (early_tiles) fill_ring<D, kRing, false>(st, ctx_of, ring, full, P, lane);
+    begin_item_pages(ctx[0].ip, P, first, lane);   // the whole page list, while the tiles fly
   } else {
-    issued = claim_issue(P, lane);
+    if (STATIC) {
+      if (wid >= P.part_workers) return;
+      RangeCursor c;
+      const bool any = cursor_init(c, part_view(P), wid, lane);
+      if (lane == 0) *cursor = c;
+      __syncwarp();
+      if (!any) return;
+    } else {
+      pdl_wait();   // the item list and the work counter are the previous kernel's
+      pdl_launch_dependents();
+      issued = claim_issue(P, lane);
+    }
+    if (!take()) return;
+    begin_item_pages(ctx[0].ip, P, it, lane);
+    first = it;
+    cp_async_wait_all();
+    __syncwarp();
+    st.n_my = 1;
+    const bool early_tiles = !(first.stream == 0 && (first.flags & kFlagStreamEnd) && first.n_pages <= kRing);
+    if (early_tiles) fill_ring<D, kRing, false>(st, ctx_of, ring, full, P, lane);
   }
-  if (!take()) return;
-  begin_item_pages(ctx[0].ip, P, it, lane);
-  const Item first = it;
-  cp_async_wait_all();
-  __syncwarp();
-  st.n_my = 1;
-  const bool early_tiles = !(first.stream == 0 && (first.flags & kFlagStreamEnd) && first.n_pages <= kRing);
-  if (early_tiles) fill_ring<D, kRing, false>(st, ctx_of, ring, full, P, lane);
-  pdl_wait();
-  pdl_launch_dependents();
+  if (STATIC) {
+    pdl_wait();
+    pdl_launch_dependents();
+  }
   // ---- this layer's inputs; the rest of the first tiles; the second item's context while they fly
   begin_queries<D>(ctx[0], P, first, lane);
   fill_ring<D, kRing, false>(st, ctx_of, ring, full, P, lane);
@@ -502,12 +562,13 @@ __device__ __forceinline__ void attend_worker(const Params& P, WarpCtx<D>* ctx, 
   }
 }
 
-template <int D>
+template <int D, bool STATIC>
 __global__ void __launch_bounds__(kThreads, 1) attend_kernel(const __grid_constant__ Params P) {
   constexpr uint32_t kTile = kPage * D * 2;
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ __align__(8) uint64_t full_all[kWarps][kRing];
   __shared__ __align__(16) RangeCursor cursors[kWarps];
+  __shared__ __align__(16) int32_t stages[kWarps][12];
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t ring = smem_u32(smem) + static_cast<uint32_t>(warp) * kRing * kTile;
@@ -520,10 +581,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_kernel(const __grid_consta
   }
   __syncthreads();
 
-  if (P.part_static)
-    attend_worker<D, true>(P, ctx, ring, full, &cursors[warp], warp * gridDim.x + blockIdx.x, lane);
-  else
-    attend_worker<D, false>(P, ctx, ring, full, &cursors[warp], 0, lane);
+  attend_worker<D, STATIC>(P, ctx, ring, full, &cursors[warp], stages[warp], warp * gridDim.x + blockIdx.x, lane);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -641,10 +699,14 @@ constexpr int attend_smem_bytes() {
 // ------------------------------------------------------------------------------------------
 
 cudaError_t configure_kernels(int* attend_smem) {
-  cudaError_t e = cudaFuncSetAttribute(attend_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaError_t e = cudaFuncSetAttribute(attend_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        attend_smem_bytes<128>());
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(attend_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, attend_smem_bytes<64>());
+  e = cudaFuncSetAttribute(attend_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, attend_smem_bytes<128>());
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(attend_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, attend_smem_bytes<64>());
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(attend_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, attend_smem_bytes<64>());
   if (attend_smem) *attend_smem = attend_smem_bytes<128>();
   return e;
 }
@@ -657,6 +719,11 @@ cudaError_t launch_setup(const Params& p, const StepInline* inl, cudaStream_t st
   return launch_pdl(setup_kernel, dim3(blocks), dim3(kBlock), 0, stream, p, inl ? *inl : kNone);
 }
 
+cudaError_t launch_plan(const Params& p, const LaunchList& list, int n_launches, cudaStream_t stream) {
+  if (n_launches <= 0) return cudaSuccess;
+  return launch_pdl(plan_kernel, dim3(kPlanWorkers / 128, n_launches), dim3(128), 0, stream, p, list);
+}
+
 cudaError_t launch_append(const Params& p, cudaStream_t stream) {
   dim3 grid(p.n_seqs, p.layer_end - p.layer_begin);
   return launch_pdl(append_kernel, grid, dim3(128), 0, stream, p);
@@ -667,9 +734,14 @@ cudaError_t launch_attend(const Params& p, int n_sms, cudaStream_t stream) {
   if (!p.part_static && n_items <= 0) return cudaSuccess;
   // static ranges: worker w is warp w / grid of CTA w % grid, so a launch with few workers still uses every SM
   const int grid = p.part_static ? min(n_sms, p.part_workers) : min(n_sms, (n_items + kWarps - 1) / kWarps);
-  if (p.d == 128)
-    return launch_pdl(attend_kernel<128>, dim3(grid), dim3(kThreads), attend_smem_bytes<128>(), stream, p);
-  return launch_pdl(attend_kernel<64>, dim3(grid), dim3(kThreads), attend_smem_bytes<64>(), stream, p);
+  if (p.d == 128) {
+    if (p.part_static)
+      return launch_pdl(attend_kernel<128, true>, dim3(grid), dim3(kThreads), attend_smem_bytes<128>(), stream, p);
+    return launch_pdl(attend_kernel<128, false>, dim3(grid), dim3(kThreads), attend_smem_bytes<128>(), stream, p);
+  }
+  if (p.part_static)
+    return launch_pdl(attend_kernel<64, true>, dim3(grid), dim3(kThreads), attend_smem_bytes<64>(), stream, p);
+  return launch_pdl(attend_kernel<64, false>, dim3(grid), dim3(kThreads), attend_smem_bytes<64>(), stream, p);
 }
 
 cudaError_t launch_merge(const Params& p, cudaStream_t stream) {

@@ -43,7 +43,7 @@ struct LaunchGroup {
 };
 
 struct Layout {   // byte offsets into the workspace
-  size_t table, layer_flags, layer_kind, leader, jobs, plan, qcache, part_acc, part_ml, logits, items, step, err, counters, row_slots, row_done, stage_q,
+  size_t table, layer_flags, layer_kind, leader, jobs, plan, qcache, part_acc, part_ml, logits, items, step, err, counters, row_slots, row_done, wdesc, stage_q,
       stage_k, stage_v, stage_out, stage_lse, tok, total;
   size_t step_seqs, step_patches, step_bytes;   // offsets inside the step block
 };
@@ -111,6 +111,8 @@ struct qc_cache {
   int slots_per_stream = 0;
   int static_partition = -1;      // -1: static ranges when a step is several launches; 0 never; 1 always
   bool fused_merge = false;       // the worker that delivers an output row's last partial merges it (no merge launch)
+  bool plan_ahead = true;         // one kernel per step works out where every worker of every launch starts
+  int static_row_cost = 4;        // tiles a row counts for besides its pages (a worker's cost of one more item)
   int static_min_tiles = 6;       // a static range is at least this long when the launch has the work for it
                                   // (measured on launches of one layer: 3..8 equal, 12 and 16 slower)
   int text_streams_per_seq = 0;        // pages a sequence needs when its text crosses a page
@@ -122,7 +124,9 @@ struct qc_cache {
   int stage_next = 0;
 
   // profiling
-  bool profile = false;
+  int profile = 0;                     // 1: events per step; 2: also around every attention launch
+  std::vector<cudaEvent_t> ev_launch;  // profile 2: begin / end of every attention launch
+  int ev_launches = 0;
   std::vector<cudaEvent_t> ev;         // 4 per step: step begin, attend begin, attend end, step end
   int ev_steps = 0;
   int64_t prof_bytes = 0, prof_items = 0;
@@ -130,7 +134,7 @@ struct qc_cache {
   int ev_prefill_calls = 0;
   double prof_prefill_flops = 0.0;
 
-  int64_t decode_steps = 0, attend_launches = 0, kernel_launches = 0;
+  int64_t decode_steps = 0, attend_launches = 0, kernel_launches = 0, kv_bytes_swept = 0;
 };
 
 namespace {
@@ -435,6 +439,7 @@ int compute_sizes(const qc_config* cfg, Sizes* s) {
   L.counters = take(N * sizeof(int32_t));
   L.row_slots = take(N * S * s->hq * 2 * sizeof(uint16_t));
   L.row_done = take(N * S * s->hq * sizeof(int32_t));
+  L.wdesc = take(std::min<size_t>(N, kMaxPlanLaunches) * kPlanWorkers * sizeof(WorkerDesc));
   L.stage_q = take(N * S * s->hq * s->D * 2);
   L.stage_k = take(N * S * s->hkv * s->D * 2);
   L.stage_v = take(N * S * s->hkv * s->D * 2);
@@ -723,6 +728,9 @@ int32_t qc_alloc_cache(qc_ctx* ctx, const qc_config* cfg, void* pool_dev, size_t
   c->hkv = s.hkv;
   c->group = s.hq / s.hkv;
   c->heads_per_item = c->group > 1 ? 8 : 1;
+  // what one more item costs a worker, in tiles: a query-group item fetches its query fragments when it
+  // starts and leaves up to eight partial rows (measured on launches of one layer: 4 resp. 8 best)
+  c->static_row_cost = c->group > 1 ? 8 : 4;
   c->items_per_chunk = c->group > 1 ? s.hkv * ((c->group + 7) / 8) : s.hq;
   c->paged = cfg->page_size == 16;
   c->max_pages = s.max_pages;
@@ -805,7 +813,7 @@ int32_t qc_alloc_cache(qc_ctx* ctx, const qc_config* cfg, void* pool_dev, size_t
   ok = ok && cudaMemcpyAsync(c->ws + c->lay.jobs, c->jobs.data(), c->jobs.size() * sizeof(Job),
                              cudaMemcpyHostToDevice, stream) == cudaSuccess;
   ok = ok && cudaMemsetAsync(c->ws + c->lay.err, 0, 256, stream) == cudaSuccess;
-  ok = ok && cudaMemsetAsync(c->ws + c->lay.row_done, 0, c->lay.stage_q - c->lay.row_done, stream) == cudaSuccess;
+  ok = ok && cudaMemsetAsync(c->ws + c->lay.row_done, 0, c->lay.wdesc - c->lay.row_done, stream) == cudaSuccess;
   ok = ok && cudaMemsetAsync(c->ws + c->lay.qcache, 0, c->lay.part_acc - c->lay.qcache, stream) == cudaSuccess;
   ok = ok && cudaStreamSynchronize(stream) == cudaSuccess;
   if (!ok) {
@@ -825,6 +833,7 @@ int32_t qc_free(qc_ctx* ctx, qc_cache* cache) {
     for (int i = 0; i < kStageSlots; ++i)
       if (cache->stage_done[i]) cudaEventDestroy(cache->stage_done[i]);
     for (cudaEvent_t e : cache->ev) cudaEventDestroy(e);
+    for (cudaEvent_t e : cache->ev_launch) cudaEventDestroy(e);
     for (cudaEvent_t e : cache->ev_in) cudaEventDestroy(e);
     for (cudaEvent_t e : cache->ev_done) cudaEventDestroy(e);
     if (cache->copy_in) cudaStreamDestroy(cache->copy_in);
@@ -1201,7 +1210,8 @@ int decode_step_core(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, const 
     pmax_t = std::max(pmax_t, pt);
   }
   for (const LaunchGroup& g : c->groups)   // tile offsets are 32-bit
-    if (static_cast<int64_t>(c->items_per_chunk) * (g.wv * tp_v + g.wt * tp_t) >= (1LL << 31)) use_static = false;
+    if (static_cast<int64_t>(c->items_per_chunk) * (g.wv * tp_v + g.wt * tp_t + 64LL * n_seqs * (g.job_end - g.job_begin)) >= (1LL << 31))
+      use_static = false;
   int64_t tot_v = 0, tot_t = 0, step_rows = 0;   // step_rows: K/V rows the step has to read (for the profile)
   int64_t pre_pv = 0, pre_pt = 0;
   for (int i = 0; i < n_seqs; ++i) {
@@ -1249,6 +1259,49 @@ int decode_step_core(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, const 
   // the host pipe has copied them)
   p.fused_append = (n_patches == 0 && !pipe) ? 1 : 0;
 
+  // static partition of every launch of the step (part_workers == 0: the launch has nothing to sweep)
+  auto partition_of = [&](size_t gi) {
+    const LaunchGroup& g = c->groups[gi];
+    const int pb = c->group_pos[gi].first, pe = c->group_pos[gi].second;
+    LaunchDesc L{};
+    L.pos_begin = pb;
+    L.pos_end = pe;
+    L.part_row_cost = c->static_row_cost;
+    const int64_t kv_tiles = static_cast<int64_t>(c->items_per_chunk) * (g.wv * tp_v + g.wt * tp_t);
+    if (kv_tiles <= 0) return L;
+    const int64_t T = kv_tiles + static_cast<int64_t>(c->items_per_chunk) * c->static_row_cost * n_seqs * (pe - pb);
+    // tiles per page of the lightest / heaviest job that has any page, longest row in tiles
+    const int w_min = (tp_v > 0 && tp_t > 0) ? g.w_min : g.w_max_v * (tp_v > 0) + g.w_max_t * (tp_t > 0);
+    const int w_lo = std::max(1, std::min(w_min, g.w_min));
+    const int64_t row_max = std::max<int64_t>(static_cast<int64_t>(pmax_v) * g.w_max_v,
+                                              static_cast<int64_t>(pmax_t) * g.w_max_t);
+    const int64_t q_max = 30LL * w_lo;
+    int64_t q_min = std::max<int64_t>(2LL * g.w_max, (row_max + c->slots_per_stream - 3) / (c->slots_per_stream - 2));
+    q_min = std::max<int64_t>(q_min, std::min<int64_t>(c->static_min_tiles, q_max / 2));
+    const int64_t W = static_cast<int64_t>(c->ctx->n_sms) * kAttendWarps;
+    int64_t k = 1, q;
+    if (T > W * q_max) {   // several ranges per worker, each as long as a piece may be
+      k = (T + W * q_max - 1) / (W * q_max);
+      q = (T + W * k - 1) / (W * k);
+    } else {
+      q = std::max<int64_t>(q_min, (T + W - 1) / W);
+    }
+    const int64_t vw = (T + q - 1) / q;
+    L.part_vw = static_cast<int32_t>(vw);
+    L.part_k = static_cast<int32_t>(k);
+    L.part_workers = static_cast<int32_t>((vw + k - 1) / k);
+    L.part_q = static_cast<int32_t>(q);
+    return L;
+  };
+  LaunchList launches;
+  const bool planned = use_static && c->plan_ahead && c->groups.size() <= static_cast<size_t>(kMaxPlanLaunches) &&
+                       c->groups.size() <= static_cast<size_t>(std::min(c->cfg.n_layers, kMaxPlanLaunches)) &&
+                       c->ctx->n_sms * kAttendWarps <= kPlanWorkers;
+  if (use_static)
+    for (size_t gi = 0; gi < c->groups.size() && gi < static_cast<size_t>(kMaxPlanLaunches); ++gi)
+      launches.launch[gi] = partition_of(gi);
+  p.wdesc = planned ? reinterpret_cast<const WorkerDesc*>(c->ws + c->lay.wdesc) : nullptr;
+
   cudaEvent_t* ev = nullptr;
   if (c->profile && c->ev_steps < kMaxProfileSteps) {
     if (static_cast<int>(c->ev.size()) < 4 * (c->ev_steps + 1)) {
@@ -1269,6 +1322,10 @@ int decode_step_core(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, const 
     QC_CUDA(launch_append(p, stream));
     c->kernel_launches++;
   }
+  if (planned) {
+    QC_CUDA(launch_plan(p, launches, static_cast<int>(c->groups.size()), stream));
+    c->kernel_launches++;
+  }
   for (size_t gi = 0; gi < c->groups.size(); ++gi) {
     const int pb = c->group_pos[gi].first, pe = c->group_pos[gi].second;
     p.item_begin = static_cast<int32_t>(c->plan_vis_before[pb] * tot_v + c->plan_text_before[pb] * tot_t);
@@ -1281,33 +1338,15 @@ int decode_step_core(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, const 
     p.extra_key_leader = c->groups[gi].extra_key_leader;
     bool has_work = p.item_end > p.item_begin;
     if (use_static) {
-      const LaunchGroup& g = c->groups[gi];
-      const int64_t T = static_cast<int64_t>(c->items_per_chunk) * (g.wv * tp_v + g.wt * tp_t);
-      has_work = T > 0;
-      if (has_work) {
-        // tiles per page of the lightest / heaviest job that has any page, longest row in tiles
-        const int w_min = (tp_v > 0 && tp_t > 0) ? g.w_min : g.w_max_v * (tp_v > 0) + g.w_max_t * (tp_t > 0);
-        const int w_lo = std::max(1, std::min(w_min, g.w_min));
-        const int64_t row_max = std::max<int64_t>(static_cast<int64_t>(pmax_v) * g.w_max_v,
-                                                  static_cast<int64_t>(pmax_t) * g.w_max_t);
-        const int64_t q_max = 30LL * w_lo;
-        int64_t q_min = std::max<int64_t>(2LL * g.w_max, (row_max + c->slots_per_stream - 3) / (c->slots_per_stream - 2));
-        q_min = std::max<int64_t>(q_min, std::min<int64_t>(c->static_min_tiles, q_max / 2));
-        const int64_t W = static_cast<int64_t>(c->ctx->n_sms) * kAttendWarps;
-        int64_t k = 1, q;
-        if (T > W * q_max) {   // several ranges per worker, each as long as a piece may be
-          k = (T + W * q_max - 1) / (W * q_max);
-          q = (T + W * k - 1) / (W * k);
-        } else {
-          q = std::max<int64_t>(q_min, (T + W - 1) / W);
-        }
-        const int64_t vw = (T + q - 1) / q;
-        p.part_vw = static_cast<int32_t>(vw);
-        p.part_k = static_cast<int32_t>(k);
-        p.part_workers = static_cast<int32_t>((vw + k - 1) / k);
-        p.part_q = static_cast<int32_t>(q);
-        p.part_tiles = static_cast<int32_t>(T);
-      }
+      const LaunchDesc& L = launches.launch[gi < kMaxPlanLaunches ? gi : 0];
+      const LaunchDesc one = gi < kMaxPlanLaunches ? L : partition_of(gi);
+      has_work = one.part_workers > 0;
+      p.part_q = one.part_q;
+      p.part_k = one.part_k;
+      p.part_vw = one.part_vw;
+      p.part_workers = one.part_workers;
+      p.part_row_cost = one.part_row_cost;
+      p.part_tiles = 0;
     }
     if (pipe) {
       QC_CUDA(cudaStreamWaitEvent(stream, pipe->in[gi], 0));
@@ -1315,6 +1354,18 @@ int decode_step_core(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, const 
       c->kernel_launches++;
     }
     if (ev && gi == 0) QC_CUDA(cudaEventRecord(ev[1], stream));
+    cudaEvent_t* evl = nullptr;
+    if (ev && c->profile == 2 && has_work && c->ev_launches < 64 * kMaxProfileSteps) {
+      if (static_cast<int>(c->ev_launch.size()) < 2 * (c->ev_launches + 1)) {
+        for (int i = 0; i < 2; ++i) {
+          cudaEvent_t e;
+          QC_CUDA(cudaEventCreate(&e));
+          c->ev_launch.push_back(e);
+        }
+      }
+      evl = &c->ev_launch[2 * c->ev_launches++];
+      QC_CUDA(cudaEventRecord(evl[0], stream));
+    }
     if (!has_work) {
       // (a GLA follower of the in-order schedule: its merge does everything)
     } else if (c->group > 1) {
@@ -1322,6 +1373,7 @@ int decode_step_core(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, const 
     } else {
       QC_CUDA(launch_attend(p, c->ctx->n_sms, stream));
     }
+    if (evl) QC_CUDA(cudaEventRecord(evl[1], stream));
     if (ev && gi + 1 == c->groups.size()) QC_CUDA(cudaEventRecord(ev[2], stream));
     if (c->groups[gi].needs_merge) QC_CUDA(launch_merge(p, stream));
     if (pipe) QC_CUDA(cudaEventRecord(pipe->done[gi], stream));
@@ -1335,6 +1387,7 @@ int decode_step_core(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, const 
     c->prof_items += n_items;
   }
   c->decode_steps++;
+  c->kv_bytes_swept += step_rows * c->hkv * c->D * 2;
   return QC_OK;
 }
 
@@ -1463,6 +1516,7 @@ int32_t qc_get_stats(qc_cache* c, qc_stats* out) {
   out->decode_steps = c->decode_steps;
   out->attend_launches = c->attend_launches;
   out->kernel_launches = c->kernel_launches;
+  out->kv_bytes_swept = c->kv_bytes_swept;
   QC_CUDA(cudaSetDevice(c->ctx->device));
   int32_t err = 0;
   QC_CUDA(cudaMemcpyAsync(&err, c->ws + c->lay.err, sizeof(err), cudaMemcpyDeviceToHost, c->ctx->stream));
@@ -1559,6 +1613,15 @@ int32_t qc_set_option(qc_cache* c, const char* key, int64_t value) {
     c->static_partition = static_cast<int>(value);
     return QC_OK;
   }
+  if (k == "plan_ahead") {
+    c->plan_ahead = value != 0;
+    return QC_OK;
+  }
+  if (k == "static_row_cost") {
+    if (value < 0 || value > 64) return QC_ERR_INVALID_ARG;
+    c->static_row_cost = static_cast<int>(value);
+    return QC_OK;
+  }
   if (k == "static_min_tiles") {
     if (value < 1 || value > 4096) return QC_ERR_INVALID_ARG;
     c->static_min_tiles = static_cast<int>(value);
@@ -1574,7 +1637,8 @@ int32_t qc_set_option(qc_cache* c, const char* key, int64_t value) {
     return QC_OK;
   }
   if (k == "profile") {
-    c->profile = value != 0;
+    if (value < 0 || value > 2) return QC_ERR_INVALID_ARG;
+    c->profile = static_cast<int>(value);
     return QC_OK;
   }
   return QC_ERR_INVALID_ARG;
@@ -1601,6 +1665,13 @@ int32_t qc_get_profile(qc_cache* c, qc_profile* out) {
   out->prefill_flops = c->prof_prefill_flops;
   c->ev_prefill_calls = 0;
   c->prof_prefill_flops = 0.0;
+  for (int i = 0; i < c->ev_launches; ++i) {
+    float a = 0.f;
+    QC_CUDA(cudaEventElapsedTime(&a, c->ev_launch[2 * i], c->ev_launch[2 * i + 1]));
+    out->attend_kernel_ms += a;
+  }
+  out->attend_kernel_launches = c->ev_launches;
+  c->ev_launches = 0;
   out->steps = c->ev_steps;
   out->kv_bytes_read = c->prof_bytes;
   out->items = c->prof_items;

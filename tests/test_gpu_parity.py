@@ -253,7 +253,8 @@ SCHEDULES = {
     "per_layer_logit_cache_static_ranges": [("per_layer_logit_cache", 1)],
     "in_order": [("in_order_launches", 1)],
     "in_order_claimed_items": [("in_order_launches", 1), ("static_partition", 0)],
-    "in_order_short_ranges": [("in_order_launches", 1), ("static_min_tiles", 1)],
+    "in_order_short_ranges": [("in_order_launches", 1), ("static_min_tiles", 1), ("static_row_cost", 0)],
+    "in_order_costly_rows": [("in_order_launches", 1), ("static_row_cost", 5)],
     "in_order_merge_in_kernel": [("in_order_launches", 1), ("fused_merge", 1)],
     "one_launch_merge_in_kernel": [("fused_merge", 1)],
 }
