@@ -5,10 +5,13 @@
 
 A step is one qc_decode_step over the whole batch (append + Q Cache write + split-KV partial
 attention + log-sum-exp merge, all layers).  `value` is decode tokens/s with inputs resident
-in HBM; `e2e` is the same through qc_decode_step_host with pinned HOST buffers (q, k, v copied
-in, out copied back, inside the timed region).  With N > 1 (torchrun) every rank runs its own
-batch of the same shape on its own GPU (independent sequences: no collective on the data
-path); the time is the maximum over ranks.
+in HBM under the in-order schedule (one launch per layer, each using nothing of later layers);
+`e2e` is the same through qc_decode_step_host with pinned HOST buffers (q, k, v copied in, out
+copied back, inside the timed region).  Without --workload the headline is the largest
+configuration and `per_config` holds a record for each of the other model-shaped ones.  With
+N > 1 every rank runs its own batch of the same shape on its own GPU (independent sequences: no
+collective on the data path); the time is the maximum over ranks.  `--gpus N` starts the N
+ranks itself unless a launcher already did.
 """
 
 from __future__ import annotations
@@ -31,8 +34,7 @@ UNIT = "tokens/s"
 MODES = {"vla_qc": 0, "vla_eq8": 1, "gla": 2}
 
 # (dram__bytes_read.sum + dram__bytes_write.sum) / algorithmic K/V bytes of one attention launch,
-# from the ncu captures of small cases summarised in profiles/attend_kernels_small_cases_ncu_full.md.
-# Traffic grows in proportion to the K/V bytes swept (every tile is fetched once; partial results are
+# from ncu captures of small cases.  Traffic grows in proportion to the K/V bytes swept (every tile is fetched once; partial results are
 # written once per chunk), so a full launch's traffic is this ratio times its algorithmic bytes.
 NCU_TRAFFIC_RATIO = {"attend_kernel": 1.069, "attend_tc_kernel": 1.070}
 
@@ -110,55 +112,81 @@ def _physical_gpu_index(local: int) -> int:
 
 
 # ------------------------------------------------------------------------------------------
-# CPU oracle leg (bounded sample)
+# CPU oracle leg (bounded, fixed sample)
 # ------------------------------------------------------------------------------------------
 
-def cpu_oracle_sample(w, mode: int, first_step: int, budget_s: float = 12.0):
-    """Time the fp64 oracle, as it stands, on a bounded sample of the workload.
+ORACLE_STEPS = 16         # decode steps each sampled sub-problem is advanced through
 
-    Sample: whole-stack sub-problems (all layers, one sequence, one KV head with its query
-    heads), each advanced through decode steps starting at `first_step` context length, until
-    the time budget is used.  One generated token of the full workload costs n_kv_heads such
-    sub-problem steps, so tokens/s = sub-problem steps per second / n_kv_heads.
-    """
+
+def _host_cores() -> int:
+    try:
+        return max(1, len(os.sched_getaffinity(0)))
+    except AttributeError:
+        return max(1, os.cpu_count() or 1)
+
+
+def _oracle_unit(job):
+    """One sampled sub-problem on one core: the whole layer stack of one (sequence, KV head) with its
+    query heads, advanced through ORACLE_STEPS decode steps.  Returns the seconds spent inside the
+    oracle's decode_step (input generation is not the oracle's work)."""
+    name, mode, first_step, unit = job
     from threadpoolctl import threadpool_limits
 
     from oracle.lazy_attention import LazyAttentionOracle
     from paper_2602_01901_b200 import workloads as W
 
+    w = W.get_workload(name)
     f64 = W.bf16_bits_to_f64
     g = w.group
-    done, spent, units = 0, 0.0, 0
+    seq, kvh = unit % w.batch, (unit // w.batch) % w.n_kv_heads
+    heads = list(range(kvh * g, (kvh + 1) * g))
+    spent = 0.0
     with threadpool_limits(limits=1):
-        unit = 0
-        while spent < budget_s and unit < w.batch * w.n_kv_heads:
-            seq, kvh = unit % w.batch, (unit // w.batch) % w.n_kv_heads
-            heads = list(range(kvh * g, (kvh + 1) * g))
-            o = LazyAttentionOracle(w.n_layers, g, 1, w.head_dim, w.layer_kind().tolist(), mode, n_seqs=1)
-            kind, k, v = W.prefill_kv_np(w, seq, heads=[kvh])
-            o.prefill_append(0, kind.tolist(), f64(k), f64(v))
-            # untimed catch-up to the benchmark's first timed step (appends only matter)
-            for step in range(first_step):
-                q, kk, vv = W.decode_qkv_np(w, step, seqs=[seq], q_heads=heads, kv_heads=[kvh])
-                for l in range(w.n_layers):
-                    o.V_T[l][0].append(f64(vv[l, 0]))
-                    if o.K_T[l][0] is not None:
-                        o.K_T[l][0].append(f64(kk[l, 0]))
-            for step in range(first_step, first_step + 16):
-                q, kk, vv = W.decode_qkv_np(w, step, seqs=[seq], q_heads=heads, kv_heads=[kvh])
-                qf, kf, vf = f64(q[:, 0]), f64(kk[:, 0]), f64(vv[:, 0])
-                t0 = time.perf_counter()
-                o.decode_step(0, qf, kf, vf)
-                spent += time.perf_counter() - t0
-                done += 1
-            unit += 1
-            units += 1
-    tokens_per_s = done / spent / w.n_kv_heads
+        o = LazyAttentionOracle(w.n_layers, g, 1, w.head_dim, w.layer_kind().tolist(), mode, n_seqs=1)
+        kind, k, v = W.prefill_kv_np(w, seq, heads=[kvh])
+        o.prefill_append(0, kind.tolist(), f64(k), f64(v))
+        for step in range(first_step):   # untimed catch-up to the first timed context (only the appends matter)
+            q, kk, vv = W.decode_qkv_np(w, step, seqs=[seq], q_heads=heads, kv_heads=[kvh])
+            for l in range(w.n_layers):
+                o.V_T[l][0].append(f64(vv[l, 0]))
+                if o.K_T[l][0] is not None:
+                    o.K_T[l][0].append(f64(kk[l, 0]))
+        for step in range(first_step, first_step + ORACLE_STEPS):
+            q, kk, vv = W.decode_qkv_np(w, step, seqs=[seq], q_heads=heads, kv_heads=[kvh])
+            qf, kf, vf = f64(q[:, 0]), f64(kk[:, 0]), f64(vv[:, 0])
+            t0 = time.perf_counter()
+            o.decode_step(0, qf, kf, vf)
+            spent += time.perf_counter() - t0
+    return spent
+
+
+def cpu_oracle_sample(w, mode: int, first_step: int):
+    """Time the fp64 oracle, as it stands, on a fixed sample of the workload, on all host cores.
+
+    Sample: four whole-stack sub-problems per core (all layers, one sequence, one KV head with its
+    query heads; sub-problem i is sequence i mod batch, KV head i div batch), each advanced through
+    ORACLE_STEPS decode steps from the context of the benchmark's first timed step, one process per
+    core.  One generated token of the workload costs n_kv_heads sub-problem steps, so tokens/s =
+    sub-problem steps / (the busiest core's seconds inside the oracle) / n_kv_heads.
+    """
+    import multiprocessing as mp
+
+    cores = _host_cores()
+    n_units = min(4 * cores, w.batch * w.n_kv_heads)
+    cores = min(cores, n_units)
+    jobs = [(w.name, mode, first_step, u) for u in range(n_units)]
+    ctx = mp.get_context("spawn")
+    with ctx.Pool(cores) as pool:
+        spent = pool.map(_oracle_unit, jobs, chunksize=1)
+    # with equal costs per sub-problem the busiest core did ceil(n / cores) of them
+    per_core = -(-n_units // cores)
+    busiest = per_core * max(spent)
+    tokens_per_s = n_units * ORACLE_STEPS / busiest / w.n_kv_heads
     return {
-        "value": tokens_per_s, "unit": UNIT, "cores": 1, "kind": "oracle",
-        "sample": f"{units} (sequence, KV head) sub-problems x all {w.n_layers} layers x 16 decode steps from "
-                  f"context {w.n_prompt + first_step}; {done} sub-problem steps in {spent:.1f} s, "
-                  f"scaled by 1/{w.n_kv_heads} KV heads per token",
+        "value": tokens_per_s, "unit": UNIT, "cores": cores, "kind": "oracle",
+        "sample": f"{n_units} (sequence, KV head) sub-problems x all {w.n_layers} layers x {ORACLE_STEPS} decode steps "
+                  f"from context {w.n_prompt + first_step} of {w.name}, one process per core; slowest sub-problem "
+                  f"{max(spent):.2f} s inside the oracle, {per_core} per core; scaled by 1/{w.n_kv_heads} KV heads per token",
     }
 
 
@@ -172,199 +200,276 @@ def _gen_inputs(w, first, count, device, seq_offset=0):
     return [W.decode_qkv_torch(w, s, device, seq_offset) for s in range(first, first + count)]
 
 
-def run_gpu(args, w, mode, rank, world, local_rank):
-    import torch
+class _Arms:
+    """The timed arms of one workload on one GPU, all on one cache: consecutive decode steps under
+    different schedules (a schedule changes how a step is cut into launches, never its result)."""
 
-    from paper_2602_01901_b200 import binding as qc
-    from paper_2602_01901_b200.session import Session
+    def __init__(self, args, w, mode, group, local_rank, seq_offset, all_full=False):
+        import torch
 
-    from paper_2602_01901_b200.ranks import RankGroup
+        from paper_2602_01901_b200 import binding as qc
+        from paper_2602_01901_b200.session import Session
 
-    group = RankGroup(backend=args.dist_backend)   # NCCL when launched by torchrun with WORLD_SIZE > 1
-    seq_offset = rank * w.batch  # every rank serves its own sequences of the global batch
+        self.torch, self.w, self.group, self.args = torch, w, group, args
+        self.dev = torch.device("cuda", local_rank)
+        self.s = Session.for_workload(w, lazy_mode=mode, device=local_rank, split_tokens=args.split_tokens,
+                                      all_full=all_full)
+        self.s.prefill_workload(w, seq_offset)
+        self.ids = qc._i32_array(list(range(w.batch)))
+        self.out = torch.empty((w.n_layers, w.batch, w.n_q_heads, w.head_dim), dtype=torch.bfloat16, device=self.dev)
+        self.step = 0
+        self.seq_offset = seq_offset
 
-    def barrier():
-        group.barrier()
-        torch.cuda.synchronize()
+    def barrier(self):
+        self.group.barrier()
+        self.torch.cuda.synchronize()
 
-    max_over_ranks = group.max_over_ranks
+    def set(self, options):
+        for key, value in options:
+            self.s.set_option(key, value)
 
-    W_, K = args.warmup, args.steps
-    total_steps = W_ + K
-    if total_steps > w.decode_steps:
-        raise SystemExit(f"warmup + steps = {total_steps} exceeds the workload's {w.decode_steps} decode steps")
-    ids = qc._i32_array(list(range(w.batch)))
-    dev = torch.device("cuda", local_rank)
-    shape_o = (w.n_layers, w.batch, w.n_q_heads, w.head_dim)
+    def run(self, n, timed=True, profile=0):
+        """n consecutive decode steps; returns ms per step (max over ranks), K/V bytes per step, the
+        library's profile of the region (if asked for) and its kernel launches."""
+        torch = self.torch
+        if self.step + n > self.w.decode_steps:
+            raise SystemExit(f"{self.w.name}: the arms need more than the workload's {self.w.decode_steps} decode steps")
+        inputs = _gen_inputs(self.w, self.step, n, self.dev, self.seq_offset)
+        self.s.set_option("profile", profile)
+        st0 = self.s.stats()
+        self.barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(n):
+            self.s.decode_step(self.ids, *inputs[i], self.out)
+        e1.record()
+        self.barrier()
+        ms = self.group.max_over_ranks(e0.elapsed_time(e1)) / n
+        prof = self.s.profile() if profile else None
+        self.s.set_option("profile", 0)
+        st1 = self.s.stats()
+        if st1.device_error:
+            raise SystemExit(f"device error word = {st1.device_error}")
+        self.step += n
+        return {"ms_per_step": ms, "kv_bytes_per_step": (st1.kv_bytes_swept - st0.kv_bytes_swept) / n,
+                "launches_per_step": (st1.kernel_launches - st0.kernel_launches) / n,
+                "context_first": self.w.n_prompt + self.step - n + 1, "context_last": self.w.n_prompt + self.step,
+                "prof": prof}
 
-    # ---- arm 1: inputs resident in HBM ---------------------------------------------------
-    s = Session.for_workload(w, lazy_mode=mode, device=local_rank, split_tokens=args.split_tokens)
-    s.prefill_workload(w, seq_offset)
-    if args.blocks_per_launch:
-        s.set_option("layers_per_launch", args.blocks_per_launch)
-    if args.per_layer:
-        s.set_option("per_layer_logit_cache", 1)
-    if args.in_order:
-        s.set_option("in_order_launches", 1)
+    def run_host(self, n):
+        """n steps through qc_decode_step_host with pinned host buffers; returns tokens/s inputs."""
+        torch = self.torch
+        dev_in = _gen_inputs(self.w, self.step, n, self.dev, self.seq_offset)
+        host_in = [tuple(t.cpu().pin_memory() for t in step) for step in dev_in]
+        host_out = torch.empty(self.out.shape, dtype=torch.bfloat16).pin_memory()
+        del dev_in
+        self.barrier()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        g0.record()
+        for i in range(n):
+            self.s.decode_step_host(self.ids, *host_in[i], host_out)   # returns after the copy back has finished
+        g1.record()
+        self.barrier()
+        ms = self.group.max_over_ranks(g0.elapsed_time(g1)) / n
+        self.step += n
+        return {"ms_per_step": ms, "h2d": sum(t.numel() * 2 for t in host_in[0]), "d2h": host_out.numel() * 2}
+
+    def check_output(self):
+        checksum = float(self.out.float().abs().sum().item())
+        if not np.isfinite(checksum) or checksum == 0.0:
+            raise SystemExit("output is not finite / all zero")
+
+    def close(self):
+        st = self.s.stats()
+        self.s.close()
+        del self.s, self.out
+        self.torch.cuda.empty_cache()
+        return st
+
+
+IN_ORDER = [("in_order_launches", 1)]
+ONE_LAUNCH = [("in_order_launches", 0), ("layers_per_launch", 0)]
+
+
+def measure_workload(args, w, mode, group, local_rank, world, rank, K, W_, Ke, extra_arms):
+    """All arms of one workload.  The headline arm is the in-order schedule (one launch per layer,
+    each using nothing of later layers: what a model that computes layer after layer can issue),
+    timed with the library's profiling off; the same schedule is then run with events around every
+    attention launch for the kernel's own time.  The one-launch schedule (every layer's q/k/v known
+    up front, which only a harness has) is reported beside it."""
+    peak, peak_kind = _peaks()
+    kernel = "attend_tc_kernel" if w.group > 1 else "attend_kernel"
+    a = _Arms(args, w, mode, group, local_rank, rank * w.batch)
+    a.set(IN_ORDER)
     for kv in args.option:
         key, value = kv.split("=")
-        s.set_option(key, int(value))
-    inputs = _gen_inputs(w, 0, total_steps, dev, seq_offset)
-    out = torch.empty(shape_o, dtype=torch.bfloat16, device=dev)
-    for i in range(W_):
-        s.decode_step(ids, *inputs[i], out)
-    s.set_option("profile", 1)
-    launches_before = s.stats().kernel_launches
-    barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.s.set_option(key, int(value))
+    a.run(W_, timed=False)
+    launches0 = a.s.stats().kernel_launches
     with ClockSampler(_physical_gpu_index(local_rank)) as clocks:
-        e0.record()
-        for i in range(W_, total_steps):
-            s.decode_step(ids, *inputs[i], out)
-        e1.record()
-        barrier()
-    ms = max_over_ranks(e0.elapsed_time(e1))
-    prof = s.profile()
-    s.set_option("profile", 0)
-    st = s.stats()
-    if st.device_error:
-        raise SystemExit(f"device error word = {st.device_error}")
-    checksum = float(out.float().abs().sum().item())
-    if not np.isfinite(checksum) or checksum == 0.0:
-        raise SystemExit("output is not finite / all zero")
-    s.close()
-    del s
+        main = a.run(K)
+    gpu_launches = int(a.s.stats().kernel_launches - launches0)
+    a.check_output()
+    kp = a.run(min(K, 16), profile=2)           # the kernel's own time, launch by launch
+    prof = kp["prof"]
+    n_launch = max(1, prof.attend_kernel_launches)
+    kernel_gbs = prof.kv_bytes_read / (prof.attend_kernel_ms / 1e3) / 1e9
+    a.set(ONE_LAUNCH)
+    a.run(3, timed=False)
+    one = a.run(K)
+    onep = a.run(min(K, 16), profile=1)["prof"]
+    one_attend_ms = onep.attend_ms / max(1, onep.steps)
+    one_gbs = onep.kv_bytes_read / (onep.attend_ms / 1e3) / 1e9
+    extra = {}
+    if extra_arms and world == 1:
+        a.set([("layers_per_launch", 1)])
+        a.run(3, timed=False)
+        pb = a.run(min(K, 32))
+        extra["per_block_launches"] = {
+            "ms_per_step": pb["ms_per_step"], "kv_gb_per_s_whole_step": pb["kv_bytes_per_step"] / pb["ms_per_step"] / 1e6,
+            "note": "one attention + merge launch per lazy block, blocks in layer order (needs a block's q/k/v at once)"}
+        a.set([("per_layer_logit_cache", 1)])
+        a.run(3, timed=False)
+        pl = a.run(min(K, 32))
+        extra["per_layer_logit_cache"] = {
+            "ms_per_step": pl["ms_per_step"], "kv_gb_per_s_whole_step": pl["kv_bytes_per_step"] / pl["ms_per_step"] / 1e6,
+            "note": "one launch per layer; followers sweep their V with the leader's scores from a logit cache"}
+        a.set(IN_ORDER)
+    a.set(IN_ORDER)
+    a.run(3, timed=False)
+    host = a.run_host(Ke)
+    st = a.close()
+    tokens = w.batch * world
+    res = {
+        "workload": w.name, "mode": args.mode, "schedule": "in_order (one launch per layer, layers in order)",
+        "tokens_per_s": tokens / (main["ms_per_step"] / 1e3), "ms_per_step": main["ms_per_step"],
+        "context": [main["context_first"], main["context_last"]],
+        "kv_bytes_per_step": main["kv_bytes_per_step"],
+        "whole_step_gb_per_s": main["kv_bytes_per_step"] / main["ms_per_step"] / 1e6,
+        "whole_step_frac": main["kv_bytes_per_step"] / main["ms_per_step"] / 1e6 / peak,
+        "attend_launches_per_step": n_launch / max(1, prof.steps),
+        "attend_ms_per_step": prof.attend_kernel_ms / max(1, prof.steps),
+        "algorithmic_bytes_per_launch": prof.kv_bytes_read / n_launch,
+        "avg_launch_ms": prof.attend_kernel_ms / n_launch,
+        "kernel_gb_per_s": kernel_gbs, "frac": kernel_gbs / peak, "frac_of_nominal_8TBs": kernel_gbs / 8000.0,
+        "kernel": kernel, "gpu_launches": gpu_launches, "launches_per_step": main["launches_per_step"],
+        "one_launch": {"harness_only": True, "ms_per_step": one["ms_per_step"],
+                       "tokens_per_s": tokens / (one["ms_per_step"] / 1e3), "attend_ms": one_attend_ms,
+                       "kernel_gb_per_s": one_gbs, "frac": one_gbs / peak, "context": [one["context_first"], one["context_last"]],
+                       "note": "all layers in one attention launch: needs every layer's q/k/v before the step starts"},
+        "e2e": {"value": tokens / (host["ms_per_step"] / 1e3), "unit": UNIT, "h2d_bytes_per_step": host["h2d"],
+                "d2h_bytes_per_step": host["d2h"], "steps": Ke, "ms_per_step": host["ms_per_step"]},
+        "kv_saved": {"token_exact": 1 - st.kv_bytes_stored / st.kv_bytes_all_full,
+                     "paged": 1 - st.kv_bytes_stored_paged / st.kv_bytes_all_full_paged,
+                     "bytes_stored": st.kv_bytes_stored, "bytes_all_full": st.kv_bytes_all_full,
+                     "qcache_bytes": st.qcache_bytes},
+        "clocks": clocks.summary(),
+    }
+    res["e2e"]["over_value"] = res["e2e"]["value"] / res["tokens_per_s"]
+    res.update(extra)
+    if extra_arms and world == 1 and not args.no_all_full:
+        # the same steps on a cache whose layers are all ordinary (Eq. 2 only), same schedule
+        f = _Arms(args, w, mode, group, local_rank, rank * w.batch, all_full=True)
+        f.set(IN_ORDER)
+        f.run(W_, timed=False)
+        full = f.run(K)
+        stf = f.close()
+        res["vs_all_full"] = {"ms_per_step": full["ms_per_step"], "tokens_per_s": tokens / (full["ms_per_step"] / 1e3),
+                              "kv_bytes_stored": stf.kv_bytes_stored, "speedup_of_lazy": full["ms_per_step"] / main["ms_per_step"],
+                              "context": [full["context_first"], full["context_last"]],
+                              "note": "same inputs, steps and schedule, every layer ordinary (Eq. 2 only)"}
+    return res
 
-    # ---- arm 1b (one GPU only): the same steps on a cache whose layers are all ordinary -------
-    all_full = None
-    if world == 1 and not args.no_all_full:
-        s = Session.for_workload(w, lazy_mode=mode, device=local_rank, split_tokens=args.split_tokens, all_full=True)
-        s.prefill_workload(w, seq_offset)
-        for i in range(W_):
-            s.decode_step(ids, *inputs[i], out)
-        torch.cuda.synchronize()
-        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        f0.record()
-        for i in range(W_, total_steps):
-            s.decode_step(ids, *inputs[i], out)
-        f1.record()
-        torch.cuda.synchronize()
-        ms_full = f0.elapsed_time(f1)
-        st_full = s.stats()
-        s.close()
-        del s
-        all_full = {"ms_per_step": ms_full / K, "tokens_per_s": w.batch * K / (ms_full / 1e3),
-                    "kv_bytes_stored": st_full.kv_bytes_stored, "speedup_of_lazy": ms_full / ms,
-                    "note": "same inputs and steps, every layer ordinary (Eq. 2 only)"}
-    # ---- arms 1c, 1d (one GPU only): the same steps under the two schedules that issue layers in order.
-    # per_block: one attention + merge launch per lazy block (needs a block's q/k/v at once).
-    # per_layer: one launch pair per layer, followers reading the leader's scores from the logit
-    # cache: the schedule of a model in which a layer's q/k/v only exist after the previous layer.
-    def ordered_arm(option, value, note):
-        s2 = Session.for_workload(w, lazy_mode=mode, device=local_rank, split_tokens=args.split_tokens)
-        s2.prefill_workload(w, seq_offset)
-        s2.set_option(option, value)
-        for i in range(W_):
-            s2.decode_step(ids, *inputs[i], out)
-        s2.set_option("profile", 1)
-        torch.cuda.synchronize()
-        launches0 = s2.stats().kernel_launches
-        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        f0.record()
-        for i in range(W_, total_steps):
-            s2.decode_step(ids, *inputs[i], out)
-        f1.record()
-        torch.cuda.synchronize()
-        ms2 = f0.elapsed_time(f1)
-        prof2 = s2.profile()
-        res = {"ms_per_step": ms2 / K, "tokens_per_s": w.batch * K / (ms2 / 1e3),
-               "gpu_launches": int(s2.stats().kernel_launches - launches0),
-               "kv_gb_per_s_whole_step": prof2.kv_bytes_read / (ms2 / 1e3) / 1e9,
-               "kv_bytes_read_per_step": prof2.kv_bytes_read / max(1, prof2.steps), "note": note}
-        s2.close()
-        return res
 
-    per_block = per_layer = in_order = None
-    if world == 1 and not args.no_per_block and not args.blocks_per_launch and not args.per_layer and not args.in_order:
-        in_order = ordered_arm("in_order_launches", 1,
-                               "one attention + merge launch per layer, layers in order; a leader's launch also "
-                               "sweeps its followers' cached V rows")
-        per_block = ordered_arm("layers_per_launch", 1,
-                                "one attention + merge launch per lazy block, blocks in layer order")
-        per_layer = ordered_arm("per_layer_logit_cache", 1,
-                                "one attention + merge launch per layer, layers in order; followers take the "
-                                "leader's scores from the logit cache instead of reading its K")
-    del inputs
-    torch.cuda.empty_cache()
+def measure_tiny(args, mode, group, local_rank):
+    """The small contiguous workload: launch-latency-bound (1.4 MB per layer), reported in us per step."""
+    from paper_2602_01901_b200 import workloads as W
 
-    # ---- arm 2: host buffers through qc_decode_step_host -----------------------------------
-    Ke = min(K, args.e2e_steps)
-    s = Session.for_workload(w, lazy_mode=mode, device=local_rank, split_tokens=args.split_tokens)
-    s.prefill_workload(w, seq_offset)
-    dev_in = _gen_inputs(w, 0, W_ + Ke, dev, seq_offset)
-    for i in range(W_):
-        s.decode_step(ids, *dev_in[i], out)
-    host_in = [tuple(t.cpu().pin_memory() for t in dev_in[i]) for i in range(W_, W_ + Ke)]
-    host_out = torch.empty(shape_o, dtype=torch.bfloat16).pin_memory()
-    del dev_in
-    barrier()
-    g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    g0.record()
-    for i in range(Ke):
-        s.decode_step_host(ids, *host_in[i], host_out)     # returns after the copy back has finished
-    g1.record()
-    barrier()
-    e2e_s = max_over_ranks(g0.elapsed_time(g1)) / 1e3
-    h2d = sum(t.numel() * 2 for t in host_in[0])
-    d2h = host_out.numel() * 2
-    s.close()
+    w = W.get_workload("tiny")
+    a = _Arms(args, w, mode, group, local_rank, 0)
+    a.set(IN_ORDER)
+    a.run(3, timed=False)
+    io = a.run(5)
+    a.set(ONE_LAUNCH)
+    a.run(3, timed=False)
+    one = a.run(5)
+    a.close()
+    return {"workload": "tiny", "us_per_step": io["ms_per_step"] * 1e3, "us_per_step_one_launch": one["ms_per_step"] * 1e3,
+            "note": "L2-resident, launch-latency-bound: no HBM fraction is meaningful"}
 
+
+HEADLINE = "llava_next_anyres"                       # the largest configuration by bytes per step
+OTHERS = ("llava15_7b", "qwen2vl_gqa", "long_video_pruned")
+
+
+def run_gpu(args, rank, world, local_rank):
+    from paper_2602_01901_b200 import workloads as W
+    from paper_2602_01901_b200.ranks import RankGroup
+
+    group = RankGroup(backend=args.dist_backend)   # NCCL when launched with WORLD_SIZE > 1
+    mode = MODES[args.mode]
+    W_, K, Ke = args.warmup, args.steps, min(args.steps, args.e2e_steps)
+    single = args.workload is not None
+    head_w = _shape(args, W.get_workload(args.workload or HEADLINE))
+    head = measure_workload(args, head_w, mode, group, local_rank, world, rank, K, W_, Ke,
+                            extra_arms=single and not args.no_per_block)
+    per_config, tiny = [], None
+    if not single and world == 1:
+        for name in OTHERS:
+            w = W.get_workload(name)
+            k = min(K, 48)
+            per_config.append(measure_workload(args, w, mode, group, local_rank, world, rank, k, W_, min(Ke, 16),
+                                               extra_arms=(name == "llava15_7b" and not args.no_per_block)))
+        tiny = measure_tiny(args, mode, group, local_rank)
     group.close()
     if rank != 0:
         return None
     peak, peak_kind = _peaks()
-    tokens = w.batch * K * world
-    attend_s = prof.attend_ms / 1e3
-    achieved = prof.kv_bytes_read / attend_s / 1e9
-    launches_attend = K
-    kernel = "attend_tc_kernel" if w.group > 1 else "attend_kernel"
-    traffic = NCU_TRAFFIC_RATIO[kernel] * prof.kv_bytes_read / launches_attend
+    traffic = NCU_TRAFFIC_RATIO[head["kernel"]] * head["algorithmic_bytes_per_launch"]
     line = {
-        "metric": METRIC, "value": tokens / (ms / 1e3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W_,
-        "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "metric": METRIC, "value": head["tokens_per_s"], "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W_,
+        "ms_per_step": head["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": {
-            "workload": w.name, "mode": args.mode, "batch_per_gpu": w.batch, "n_layers": w.n_layers,
-            "lazy_layers": len(w.lazy_layers), "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads,
-            "head_dim": w.head_dim, "context_first_timed_step": w.n_prompt + W_ + 1,
-            "context_last_timed_step": w.n_prompt + total_steps, "page_tokens": w.page_size,
-            "l2": "inputs larger than L2: every step streams the whole KV cache", "arithmetic": "bf16 storage, fp32 accumulate",
+            "workload": head_w.name, "mode": args.mode, "schedule": head["schedule"], "batch_per_gpu": head_w.batch,
+            "n_layers": head_w.n_layers, "lazy_layers": len(head_w.lazy_layers), "q_heads": head_w.n_q_heads,
+            "kv_heads": head_w.n_kv_heads, "head_dim": head_w.head_dim, "context_first_timed_step": head["context"][0],
+            "context_last_timed_step": head["context"][1], "page_tokens": head_w.page_size,
+            "l2": "inputs larger than L2: every step streams the whole KV cache",
+            "arithmetic": "bf16 storage, fp32 accumulate",
         },
         "roofline": {
-            "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-            "traffic": traffic, "traffic_source": "ncu dram bytes of a small case, scaled by K/V bytes per launch",
-            "peak_kind": f"of {peak_kind}", "kernel": kernel,
-            "algorithmic_bytes_per_launch": prof.kv_bytes_read / launches_attend,
-            "avg_launch_ms": prof.attend_ms / launches_attend, "frac_of_nominal_8TBs": achieved / 8000.0,
+            "bound": "hbm", "achieved": head["kernel_gb_per_s"], "peak": peak, "unit": "GB/s", "frac": head["frac"],
+            "traffic": traffic, "traffic_source": "ncu dram bytes of a small case scaled by the K/V bytes of a launch "
+                                                  "(an upper estimate: the small case writes more partial rows per byte)",
+            "peak_kind": f"of {peak_kind}", "kernel": head["kernel"],
+            "algorithmic_bytes_per_launch": head["algorithmic_bytes_per_launch"], "avg_launch_ms": head["avg_launch_ms"],
+            "launches_per_step": head["attend_launches_per_step"], "frac_of_nominal_8TBs": head["frac_of_nominal_8TBs"],
+            "whole_step_frac": head["whole_step_frac"],
+            "note": "achieved = K/V bytes of the attention launches / their summed durations (events around every "
+                    "launch, second pass); whole_step_frac = the same bytes / the profiling-off step time",
         },
-        "e2e": {"value": w.batch * Ke * world / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
-                "d2h_bytes_per_step": d2h, "steps": Ke},
-        "gpu_launches": int(st.kernel_launches - launches_before),
-        "clocks": clocks.summary(),
-        "kv_cache": {
-            "bytes_stored": st.kv_bytes_stored, "bytes_all_full": st.kv_bytes_all_full,
-            "saved_frac_token_exact": 1 - st.kv_bytes_stored / st.kv_bytes_all_full,
-            "saved_frac_paged": 1 - st.kv_bytes_stored_paged / st.kv_bytes_all_full_paged,
-            "qcache_bytes": st.qcache_bytes,
-        },
-        "vs_all_full": all_full,
-        "per_block_launches": per_block,
-        "per_layer_launches": per_layer,
-        "in_order_launches": in_order,
-        "step_ms_by_events": prof.step_ms / max(1, prof.steps),
+        "e2e": head["e2e"], "gpu_launches": head["gpu_launches"], "clocks": head["clocks"],
+        "kv_cache": head["kv_saved"], "one_launch": head["one_launch"],
+        "per_config": per_config, "tiny": tiny,
         "paper_context": "paper reports ~35% KV saved and 1.5x-1.6x decode throughput for LLaVA-NeXT-7B on one 80GB A100 (whole model)",
     }
+    for key in ("vs_all_full", "per_block_launches", "per_layer_logit_cache"):
+        if key in head:
+            line[key] = head[key]
     return line
+
+
+def _shape(args, w):
+    if not (args.layers or args.batch):
+        return w
+    # a smaller case of the same shape, e.g. for a profiler capture that must stay a few GB
+    import dataclasses
+
+    n_layers = args.layers or w.n_layers
+    batch = args.batch or w.batch
+    return dataclasses.replace(w, name=f"{w.name}[layers={n_layers},batch={batch}]", n_layers=n_layers, batch=batch,
+                               lazy_layers=tuple(l for l in w.lazy_layers if l < n_layers))
 
 
 def run_prefill(args, w, mode, local_rank):
@@ -439,24 +544,36 @@ def run_prefill(args, w, mode, local_rank):
     }
 
 
+def _self_launch(argv, n):
+    """`python bench.py --gpus N` without a launcher: start N ranks of this script on this node."""
+    import socket
+    import subprocess
+
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr",
+           "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + argv
+    return subprocess.call(cmd)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=240)
+    ap.add_argument("--steps", type=int, default=48)
     ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="llava15_7b")
+    ap.add_argument("--workload", default=None,
+                    help="one workload only (default: the headline on the largest configuration plus a record per "
+                         "other model-shaped configuration and the tiny one)")
     ap.add_argument("--mode", default="vla_qc", choices=sorted(MODES))
-    ap.add_argument("--e2e-steps", type=int, default=64)
+    ap.add_argument("--e2e-steps", type=int, default=32)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-all-full", action="store_true", help="skip the all-ordinary-layers comparison run")
     ap.add_argument("--no-per-block", action="store_true",
-                    help="skip the comparison runs with one launch per lazy block / per layer")
-    ap.add_argument("--per-layer", action="store_true",
-                    help="run the main arm under the per-layer schedule with the logit cache (for profiling it)")
-    ap.add_argument("--in-order", action="store_true",
-                    help="run the main arm under the in-order schedule (for profiling it)")
-    ap.add_argument("--option", action="append", default=[], help="key=value passed to qc_set_option (main arm)")
+                    help="skip the comparison arms (one launch per lazy block, per layer with the logit cache, "
+                         "all layers ordinary)")
+    ap.add_argument("--option", action="append", default=[], help="key=value passed to qc_set_option (headline arm)")
     ap.add_argument("--dist-backend", default=None, help="torch.distributed backend (default: nccl on GPUs)")
     ap.add_argument("--force-device", type=int, default=-1,
                     help="use this CUDA device on every rank (to exercise the multi-rank plumbing on one GPU)")
@@ -470,25 +587,16 @@ def main():
     ap.add_argument("--prefill-kernel", default="tcgen05", choices=["tcgen05", "mma"],
                     help="prefill phase, head_dim 128: tcgen05 kernel (default) or the mma.sync kernel")
     ap.add_argument("--split-tokens", type=int, default=0, help="keys per split-KV work item (0 = library default)")
-    ap.add_argument("--blocks-per-launch", type=int, default=0,
-                    help="0 = one attention launch per step; k = one launch per k lazy blocks, in layer order")
     ap.add_argument("--layers", type=int, default=0, help="cut the stack to its first N layers (profiling-size case)")
     ap.add_argument("--batch", type=int, default=0, help="override the batch (profiling-size case)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(_self_launch(sys.argv[1:], args.gpus))
 
     from paper_2602_01901_b200 import workloads as W
 
-    w = W.get_workload(args.workload)
-    if args.layers or args.batch:
-        # a smaller case of the same shape, e.g. for a profiler capture that must stay a few GB
-        import dataclasses
-
-        n_layers = args.layers or w.n_layers
-        batch = args.batch or w.batch
-        w = dataclasses.replace(w, name=f"{w.name}[layers={n_layers},batch={batch}]", n_layers=n_layers, batch=batch,
-                                lazy_layers=tuple(l for l in w.lazy_layers if l < n_layers))
     mode = MODES[args.mode]
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -497,12 +605,20 @@ def main():
         local_rank = args.force_device
 
     if args.impl == "reference":
+        # the oracle on the host cores; under a multi-rank launch rank 0 alone works, the others only
+        # answer the roll call that fills n_gpus
+        from paper_2602_01901_b200.ranks import RankGroup
+
+        group = RankGroup(backend=args.dist_backend or "gloo")
+        ranks = int(group.sum_over_ranks(1.0))
+        group.close()
         if rank != 0:
             return
+        w = _shape(args, W.get_workload(args.workload or HEADLINE))
         t0 = time.perf_counter()
-        base = cpu_oracle_sample(w, mode, args.warmup, budget_s=20.0)
+        base = cpu_oracle_sample(w, mode, args.warmup)
         line = {
-            "impl": "reference", "metric": METRIC, "value": base["value"], "unit": UNIT, "n_gpus": args.gpus,
+            "impl": "reference", "metric": METRIC, "value": base["value"], "unit": UNIT, "n_gpus": ranks,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * w.batch / base["value"],
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": w.name, "mode": args.mode, "batch_per_gpu": w.batch},
@@ -515,11 +631,13 @@ def main():
 
     if args.phase == "prefill":
         if rank == 0:
+            w = _shape(args, W.get_workload(args.workload or "llava15_7b"))
             print(json.dumps(run_prefill(args, w, mode, local_rank)))
         return
-    line = run_gpu(args, w, mode, rank, world, local_rank)
+    line = run_gpu(args, rank, world, local_rank)
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:
+            w = _shape(args, W.get_workload(args.workload or HEADLINE))
             line["cpu_baseline"] = cpu_oracle_sample(w, mode, args.warmup)
         print(json.dumps(line))
 
