@@ -13,7 +13,12 @@
  *
  * Conventions common to every call
  *   - Every function returns an int32 status (QC_OK == 0).  Nothing throws, aborts or prints.
- *     On an error status the cache is unchanged and no output is written.
+ *     On an error status the cache is unchanged and no output is written, with two exceptions:
+ *     QC_ERR_CUDA (a CUDA call failed part-way: free the cache) and the device error word.  A
+ *     kernel that gives up (a bounded wait that ran out, a page id or work range outside its
+ *     limits) ends normally, leaves its part of the output unwritten and records a code in the
+ *     device error word, mirrored into mapped host memory: qc_get_stats reports it, and every later
+ *     qc_decode_step / qc_decode_step_host on that cache returns it instead of running.
  *   - "dev" pointers are CUDA device pointers on the context's device; "host" pointers are
  *     ordinary host memory.  All device memory is owned by the caller: the pool and the
  *     workspace are handed in at qc_alloc_cache and must outlive the cache.  The library
@@ -272,7 +277,11 @@ int32_t qc_debug_read_row(qc_cache* cache, int32_t layer, int32_t stream, int32_
  * "static_row_cost" (tuning of those ranges: shortest range, and what one more output row counts
  * for, in 4 KiB tiles), "plan_ahead" (0 = workers locate their ranges themselves instead of reading
  * starting points that one kernel per step works out for every launch), "fused_merge" (1 = the
- * worker that delivers an output row's last partial merges it, instead of a merge launch). */
+ * worker that delivers an output row's last partial merges it, instead of a merge launch),
+ * "debug_drop_tile" (test hook for the error path: 1 = every worker of an attention launch leaves
+ * out the copy of its first tile and waits for it with a short limit; nothing is in flight for that
+ * wait, so it runs out, the worker records QC_ERR_TIMEOUT and returns, and the kernel ends normally
+ * with its rows unwritten). */
 int32_t qc_set_option(qc_cache* cache, const char* key, int64_t value);
 
 /* Sum the recorded kernel times since the last call (synchronises), then reset them. */
@@ -302,8 +311,11 @@ int32_t qc_get_profile(qc_cache* cache, qc_profile* out);
  * launches nothing.
  *
  * The call performs no device or pinned-host allocation and frees nothing.  Its first call
- * on a device looks up the scratch array's device address (once per device); make that first
- * call outside any stream capture.  All calls share the one array, and it keeps whatever
+ * on a device looks up the scratch array's device address (once per device).  That look-up, or
+ * the first launch, may be the moment the CUDA runtime loads the library's device code onto the
+ * GPU, scratch array included -- the one thing here that does take device memory -- so make one
+ * call per device at start-up, while memory may still be taken, and outside any stream capture.
+ * The calling thread's current device is the same after the call as before.  All calls share the one array, and it keeps whatever
  * the previous call left there: each call overwrites every entry it later reads, so nothing
  * needs clearing, but two calls whose kernels overlap on the GPU (different streams, or
  * different host threads) race on it.  Serialise them on one stream.  Asynchronous on

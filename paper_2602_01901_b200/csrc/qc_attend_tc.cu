@@ -283,6 +283,7 @@ __device__ __forceinline__ void attend_tc_worker(const Params& P, TcCtx* ctx, ui
   auto ctx_of = [ctx](int k) -> const ItemPages& { return ctx[k % kCtxSlots].ip; };
   WorkerState st;
   worker_init(st, 0);
+  st.drop_next = P.debug_drop_tile != 0;   // (test hook)
   Item it;
   int issued = 0;
   auto take = [&]() -> bool {   // the next item into `it`
@@ -385,7 +386,7 @@ __device__ __forceinline__ void attend_tc_worker(const Params& P, TcCtx* ctx, ui
   }
   if (st.dead) {
     cp_async_wait_all();
-    drain_ring<kRingTc>(st, full);
+    drain_ring<kRingTc>(st, full, P.debug_drop_tile ? kDebugSpinLimit : kSpinLimit);
   }
 }
 

@@ -20,6 +20,7 @@ constexpr uint32_t kSpinLimit = 1u << 22; // bounded mbarrier wait
 constexpr int kErrTimeout = 6;
 constexpr int kErrBadPage = 7;
 constexpr int kErrPlan = 8;   // a work range did not fit the limits the host planned it for
+constexpr uint32_t kDebugSpinLimit = 1u << 12;   // wait limit under the test hook that drops a tile copy
 
 // ------------------------------------------------------------------------------------------
 // PTX helpers
@@ -178,6 +179,15 @@ __device__ __forceinline__ uint16_t f32_to_bf16_rne(float x) {
   return static_cast<uint16_t>(u >> 16);
 }
 
+// Record an error: the device word (largest code wins) and its mirror in mapped host memory.
+__device__ __forceinline__ void report_error(int32_t* err, int32_t* err_host, int code) {
+  atomicMax(err, code);
+  if (err_host != nullptr) {
+    *reinterpret_cast<volatile int32_t*>(err_host) = code;
+    __threadfence_system();
+  }
+}
+
 __device__ __forceinline__ size_t table_row(const Params& P, int layer, int stream, int seq_id) {
   return ((static_cast<size_t>(layer) * 4 + stream) * P.max_seqs + seq_id) * P.max_pages;
 }
@@ -211,6 +221,7 @@ struct WorkerState {
   uint32_t cons_phase;
   int in_flight;
   bool dead;           // a bounded wait ran out: stop fetching, drain, leave
+  bool drop_next;      // test hook: the next tile's copy is left out
 };
 
 __device__ __forceinline__ void worker_init(WorkerState& st, int n_my) {
@@ -221,6 +232,7 @@ __device__ __forceinline__ void worker_init(WorkerState& st, int n_my) {
   st.cons_phase = 0;
   st.in_flight = 0;
   st.dead = false;
+  st.drop_next = false;
 }
 
 // Issue the copy of the next tile.  D: head dim; RING: slots; TMAP: copy through the tensor
@@ -236,10 +248,13 @@ __device__ __forceinline__ bool issue_one(WorkerState& st, CtxFn ctx, uint32_t r
   if (st.iss_which == 0 && (c.item.flags & kFlagReadLogits)) st.iss_which = 1;   // scores come from the logit cache
   int pid = c.pages[st.iss_which][st.iss_page];
   if (static_cast<uint32_t>(pid) >= static_cast<uint64_t>(P.n_pool_pages)) {   // never read outside the pool
-    if (lane == 0) atomicMax(P.err, kErrBadPage);
+    if (lane == 0) report_error(P.err, P.err_host, kErrBadPage);
     pid = 0;
   }
-  if (lane == 0) {
+  if (P.debug_drop_tile && st.drop_next) {
+    // test hook: count the tile as in flight without requesting it; its wait will run out
+    st.drop_next = false;
+  } else if (lane == 0) {
     uint64_t* bar = &full[st.iss_slot];
     const uint32_t dst = ring + st.iss_slot * kTile;
     fence_proxy_async();   // the slot's earlier generic-proxy accesses precede this async write
@@ -281,9 +296,10 @@ __device__ __forceinline__ uint32_t wait_tile(WorkerState& st, uint32_t ring, ui
   constexpr uint32_t kTile = kPage * D * 2;
   uint64_t* bar = &full[st.cons_slot];
   uint32_t done = mbar_try_wait(bar, st.cons_phase);
-  for (uint32_t spin = 0; !done && spin < kSpinLimit; ++spin) done = mbar_try_wait(bar, st.cons_phase);
+  const uint32_t limit = P.debug_drop_tile ? kDebugSpinLimit : kSpinLimit;
+  for (uint32_t spin = 0; !done && spin < limit; ++spin) done = mbar_try_wait(bar, st.cons_phase);
   if (!done) {
-    if (lane == 0) atomicMax(P.err, kErrTimeout);
+    if (lane == 0) report_error(P.err, P.err_host, kErrTimeout);
     st.dead = true;
   }
   return ring + st.cons_slot * kTile;
@@ -302,11 +318,11 @@ __device__ __forceinline__ void release_tile(WorkerState& st) {
 // After a failed wait: copies still in flight write into this CTA's shared memory; give them
 // a bounded chance to land before the warp leaves.
 template <int RING>
-__device__ __forceinline__ void drain_ring(WorkerState& st, uint64_t* full) {
+__device__ __forceinline__ void drain_ring(WorkerState& st, uint64_t* full, uint32_t limit = kSpinLimit) {
   while (st.in_flight > 0) {
     uint64_t* bar = &full[st.cons_slot];
     uint32_t done = 0;
-    for (uint32_t spin = 0; !done && spin < kSpinLimit; ++spin) done = mbar_try_wait(bar, st.cons_phase);
+    for (uint32_t spin = 0; !done && spin < limit; ++spin) done = mbar_try_wait(bar, st.cons_phase);
     st.in_flight--;
     if (++st.cons_slot == RING) {
       st.cons_slot = 0;
@@ -404,6 +420,7 @@ struct PartView {
   const PlanJob* plan;
   const StepSeq* seqs;
   int32_t* err;
+  int32_t* err_host;
   int32_t pos_begin, pos_end, n_seqs;
   int32_t q, k, vw, row_cost;          // tiles per range, ranges per worker, ranges, fixed tiles per row
   int32_t tp_v, tp_t;                  // pages of the visual / text streams over the listed sequences
@@ -412,7 +429,7 @@ struct PartView {
 
 __device__ __forceinline__ PartView part_view(const Params& P) {
   PartView V;
-  V.plan = P.plan, V.seqs = P.seqs, V.err = P.err;
+  V.plan = P.plan, V.seqs = P.seqs, V.err = P.err, V.err_host = P.err_host;
   V.pos_begin = P.pos_begin, V.pos_end = P.pos_end, V.n_seqs = P.n_seqs;
   V.q = P.part_q, V.k = P.part_k, V.vw = P.part_vw, V.row_cost = P.part_row_cost;
   V.tp_v = P.tp_v, V.tp_t = P.tp_t;
@@ -623,7 +640,7 @@ __device__ __forceinline__ bool cursor_next(RangeCursor& c, const PartView& V, I
       // the piece that holds a row's first page tells the merge how many pieces the row has
       it.n_pieces = c.page == 0 ? static_cast<uint16_t>((c.r0 + c.w * (c.row_pages - 1)) / V.q - c.owner0 + 1) : 0;
       if (lim - c.page > kMaxChunkPages || slot < 0 || slot >= V.slots_per_stream) {   // outside the plan's limits
-        atomicMax(V.err, kErrPlan);
+        report_error(V.err, V.err_host, kErrPlan);
         c.vw = c.vw_stop;
         return false;
       }

@@ -127,6 +127,7 @@ struct Params {
   const Patch* patches;
   const uint8_t* layer_flags;
   int32_t* err;
+  int32_t* err_host;       // the same word in mapped host memory: the host sees an error without a copy
   int32_t* work_counter;   // [n_layers] next unclaimed item of each attention launch of a step
   uint16_t* row_slots;     // [n_layers][max_seqs][hq][2]: partial rows the visual / the text sweep left for an
                            // output row (static partition only)
@@ -162,6 +163,8 @@ struct Params {
   int32_t tp_v, tp_t;                // pages of the visual / text streams, summed over the listed sequences
   int32_t pos_begin, pos_end;        // plan positions of the launch
   int32_t slots_per_stream;          // partial-row slots of one stream of an output row (text slots start here)
+  int32_t debug_drop_tile;           // test hook: every worker of an attention launch leaves out the copy of its first
+                                     // tile and waits for it with a short limit (nothing in flight, nothing faults)
   int32_t extra_key_leader;          // merge only, >= 0: the rows also take the step's new token as one more key,
                                      // scored by that layer's Q Cache entry and new k (Eq. 6), valued by the own new v
 };

@@ -451,6 +451,7 @@ __device__ __forceinline__ void attend_worker(const Params& P, WarpCtx<D>* ctx, 
   auto ctx_of = [ctx](int k) -> const ItemPages& { return ctx[k % kCtxSlots].ip; };
   WorkerState st;
   worker_init(st, 0);
+  st.drop_next = P.debug_drop_tile != 0;   // (test hook)
   Item it;
   int issued = 0;
   auto take = [&]() -> bool {   // the next item into `it`
@@ -558,7 +559,7 @@ __device__ __forceinline__ void attend_worker(const Params& P, WarpCtx<D>* ctx, 
   }
   if (st.dead) {
     cp_async_wait_all();
-    drain_ring<kRing>(st, full);
+    drain_ring<kRing>(st, full, P.debug_drop_tile ? kDebugSpinLimit : kSpinLimit);
   }
 }
 

@@ -119,6 +119,9 @@ struct qc_cache {
 
   // pinned staging ring for step descriptors
   uint8_t* pinned = nullptr;
+  int32_t* err_host = nullptr;        // mapped host word the kernels mirror the device error word into
+  int32_t* err_host_dev = nullptr;    // its device address
+  int debug_drop_tile = 0;
   cudaEvent_t stage_done[kStageSlots]{};
   bool stage_used[kStageSlots]{};
   int stage_next = 0;
@@ -471,6 +474,8 @@ Params base_params(const qc_cache* c) {
   p.patches = reinterpret_cast<const Patch*>(c->ws + c->lay.step + c->lay.step_patches);
   p.layer_flags = c->ws + c->lay.layer_flags;
   p.err = reinterpret_cast<int32_t*>(c->ws + c->lay.err);
+  p.err_host = c->err_host_dev;
+  p.debug_drop_tile = c->debug_drop_tile;
   p.work_counter = reinterpret_cast<int32_t*>(c->ws + c->lay.counters);
   p.row_slots = reinterpret_cast<uint16_t*>(c->ws + c->lay.row_slots);
   p.row_done = reinterpret_cast<int32_t*>(c->ws + c->lay.row_done);
@@ -801,6 +806,11 @@ int32_t qc_alloc_cache(qc_ctx* ctx, const qc_config* cfg, void* pool_dev, size_t
                           cudaHostAllocDefault) == cudaSuccess;
   for (int i = 0; ok && i < kStageSlots; ++i)
     ok = cudaEventCreateWithFlags(&c->stage_done[i], cudaEventDisableTiming) == cudaSuccess;
+  ok = ok && cudaHostAlloc(reinterpret_cast<void**>(&c->err_host), 64, cudaHostAllocMapped) == cudaSuccess;
+  if (ok) {
+    *c->err_host = 0;
+    ok = cudaHostGetDevicePointer(reinterpret_cast<void**>(&c->err_host_dev), c->err_host, 0) == cudaSuccess;
+  }
   ok = ok && cudaMemcpyAsync(c->ws + c->lay.table, c->table.data(), c->table.size() * sizeof(int32_t),
                              cudaMemcpyHostToDevice, stream) == cudaSuccess;
   ok = ok && cudaMemcpyAsync(c->ws + c->lay.layer_flags, c->layer_flags.data(), c->layer_flags.size(),
@@ -840,6 +850,7 @@ int32_t qc_free(qc_ctx* ctx, qc_cache* cache) {
     if (cache->copy_out) cudaStreamDestroy(cache->copy_out);
     for (cudaEvent_t e : cache->ev_prefill) cudaEventDestroy(e);
     if (cache->pinned) cudaFreeHost(cache->pinned);
+    if (cache->err_host) cudaFreeHost(cache->err_host);
     delete cache;
   }
   if (ctx) delete ctx;
@@ -954,7 +965,17 @@ int32_t qc_prefill_attend(qc_cache* c, int32_t seq_id, int32_t n_tokens, const u
   if (align_up(n_tokens, 256) + align_up((n_tokens + 63) / 64, 256) + c->prefill_passes.size() * sizeof(PrefillPass) >
       tok_bytes)
     return QC_ERR_INVALID_ARG;
-  // store K/V first: this validates everything and leaves the cache unchanged on an error
+  // what can fail without touching the cache comes first: the tensor maps over the caller's tensors
+  PrefillMaps maps;
+  const bool tc5 = c->prefill_tcgen05 && c->D == 128 && (c->pool_map_ok || n0_text + n0_vis == 0);
+  if (tc5) {
+    if (make_prompt_tensor_map(&maps.q, q_dev, c->cfg.n_layers, n_tokens, c->hq) != QC_OK ||
+        make_prompt_tensor_map(&maps.k, k_dev, c->cfg.n_layers, n_tokens, c->hkv) != QC_OK ||
+        make_prompt_tensor_map(&maps.v, v_dev, c->cfg.n_layers, n_tokens, c->hkv) != QC_OK ||
+        make_output_tensor_map(&maps.out, out_dev, c->cfg.n_layers, n_tokens, c->hq) != QC_OK)
+      return QC_ERR_CUDA;
+  }
+  // store K/V: this validates the rest and leaves the cache unchanged on an error
   int st = qc_prefill_append(c, 1, &seq_id, &n_tokens, kind, k_dev, v_dev);
   if (st != QC_OK) return st;
   cudaStream_t stream = c->ctx->stream;
@@ -977,15 +998,6 @@ int32_t qc_prefill_attend(qc_cache* c, int32_t seq_id, int32_t n_tokens, const u
     QC_CUDA(cudaMemcpyAsync(passes_dev, c->prefill_passes.data(), c->prefill_passes.size() * sizeof(PrefillPass),
                             cudaMemcpyHostToDevice, stream));
   QC_CUDA(cudaStreamSynchronize(stream));   // `kind` is the caller's host memory
-  PrefillMaps maps;
-  const bool tc5 = c->prefill_tcgen05 && c->D == 128 && (c->pool_map_ok || n0_text + n0_vis == 0);
-  if (tc5) {
-    if (make_prompt_tensor_map(&maps.q, q_dev, c->cfg.n_layers, n_tokens, c->hq) != QC_OK ||
-        make_prompt_tensor_map(&maps.k, k_dev, c->cfg.n_layers, n_tokens, c->hkv) != QC_OK ||
-        make_prompt_tensor_map(&maps.v, v_dev, c->cfg.n_layers, n_tokens, c->hkv) != QC_OK ||
-        make_output_tensor_map(&maps.out, out_dev, c->cfg.n_layers, n_tokens, c->hq) != QC_OK)
-      return QC_ERR_CUDA;
-  }
   const Params p = base_params(c);
   cudaEvent_t* ev = nullptr;
   if (c->profile && c->ev_prefill_calls < kMaxProfileSteps) {
@@ -1097,6 +1109,7 @@ int decode_step_core(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, const 
   const void* ptrs[4] = {q_dev, k_dev, v_dev, out_dev};
   for (const void* ptr : ptrs)
     if (reinterpret_cast<uintptr_t>(ptr) & 15) return QC_ERR_INVALID_ARG;
+  if (const int32_t dev_err = *static_cast<volatile int32_t*>(c->err_host)) return dev_err;   // an earlier kernel gave up
   const int N = c->cfg.n_layers;
   // ---- validate, count pages
   int64_t need = 0;
@@ -1611,6 +1624,10 @@ int32_t qc_set_option(qc_cache* c, const char* key, int64_t value) {
   if (k == "static_partition") {
     if (value < -1 || value > 1) return QC_ERR_INVALID_ARG;
     c->static_partition = static_cast<int>(value);
+    return QC_OK;
+  }
+  if (k == "debug_drop_tile") {   // test hook, see qc.h
+    c->debug_drop_tile = value != 0;
     return QC_OK;
   }
   if (k == "plan_ahead") {

@@ -200,6 +200,13 @@ extern "C" int32_t qc_attend_static(int32_t device, void* cuda_stream, const voi
   const void* ptrs[4] = {q_dev, k_dev, v_dev, out_dev};
   for (const void* p : ptrs)
     if (reinterpret_cast<uintptr_t>(p) & 15) return QC_ERR_INVALID_ARG;
+  // launch on `device`, then give the calling thread its own current device back
+  int caller_device = -1;
+  if (cudaGetDevice(&caller_device) != cudaSuccess) return QC_ERR_CUDA;
+  struct Restore {
+    int device;
+    ~Restore() { cudaSetDevice(device); }
+  } restore{caller_device};
   if (cudaSetDevice(device) != cudaSuccess) return QC_ERR_CUDA;
 
   float* scratch = nullptr;

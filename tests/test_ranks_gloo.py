@@ -70,3 +70,21 @@ def test_single_process_is_identity():
     assert sum(parts, []) == list(range(10)) and max(map(len, parts)) - min(map(len, parts)) <= 1
     with pytest.raises(ValueError):
         owned_sequences(4, 2, 2)
+
+
+def test_bench_starts_its_own_ranks_when_no_launcher_did():
+    """`python bench.py --gpus 2` without torchrun re-launches itself as two ranks; the reference arm
+    (the CPU oracle; needs no GPU) answers with the number of ranks that took part."""
+    import json
+    import subprocess
+
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_PORT")}
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2",
+                          "--dist-backend", "gloo", "--workload", "tiny"], capture_output=True, text=True, timeout=600,
+                         env=env, cwd=ROOT)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [l for l in res.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1                       # rank 0 alone prints
+    line = json.loads(lines[0])
+    assert line["impl"] == "reference" and line["n_gpus"] == 2
+    assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] >= 1

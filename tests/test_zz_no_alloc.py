@@ -4,17 +4,21 @@ A serving loop with a frozen memory budget, or code running inside another frame
 callback, cannot create a workspace for the library.  qc_attend_static serves them from a
 scratch array built into the library.  This test drives it through the C ABI twice in a row
 (the second call sees the scratch contents the first one left behind) and checks each result
-against qc_decode_step on a one-layer cache fed with the same tensors, within the same
-tolerances as the other GPU tests.  It also checks that oversized requests are refused.
+against the fp64 oracle's softmax attention on the same bits (Eq. 2) and against qc_decode_step
+on a one-layer cache fed with the same tensors, within the same tolerances as the other GPU
+tests.  It also checks that oversized requests are refused.
 
 The file name sorts last so that a run which stops at the first failure has already run
 every other test.
 """
 
+import math
+
 import numpy as np
 import pytest
 import torch
 
+from oracle.lazy_attention import softmax_attention
 from paper_2602_01901_b200 import binding as qc
 from paper_2602_01901_b200 import workloads as W
 from paper_2602_01901_b200.session import Session, bits_of
@@ -57,6 +61,16 @@ def test_static_scratch_entry_point_matches_decode_step(head_dim, n_q, n_kv, n_p
         assert np.all(np.isfinite(got))
         assert float(np.max(np.abs(got - ref))) <= MAX_ABS
         assert float(np.linalg.norm(got - ref) / np.linalg.norm(ref)) <= REL_L2
+        # and against the oracle: plain softmax attention of every head over its whole history
+        group = n_q // n_kv
+        want = np.empty_like(got)
+        for b in range(n_seqs):
+            kb, vb = f64(hist_k[b]), f64(hist_v[b])
+            for h in range(n_q):
+                want[b, h] = softmax_attention([(f64(qn[0, b, h]), kb[:, h // group])], vb[:, h // group],
+                                               1.0 / math.sqrt(head_dim))[0]
+        assert float(np.max(np.abs(got - want))) <= MAX_ABS
+        assert float(np.linalg.norm(got - want) / np.linalg.norm(want)) <= REL_L2
     assert s.stats().device_error == 0
     s.close()
 
