@@ -662,14 +662,29 @@ __global__ void merge_kernel(const __grid_constant__ Params P) {
       for (int e = 0; e < VPL; ++e) acc[e] = fmaf(v[u][e], w, acc[e]);
     }
   }
-  for (int s = 4; s < max(nv, nt); ++s) {   // rows beyond the first four of a stream
+  // rows beyond the first four of a stream: four of either stream per round of loads
+  for (int s0 = 4; s0 < max(nv, nt); s0 += 4) {
+    float r[8][VPL];
 #pragma unroll
-    for (int t = 0; t < 2; ++t) {
-      const float w = __shfl_sync(0xffffffffu, my_w, (t ? 16 : 0) + s);
+    for (int u = 0; u < 8; ++u) {
+      const int s = s0 + (u & 3), t = u >> 2;
+      const bool have = s < (t ? nt : nv);
+      const float* src = P.part_acc + ((base + (t ? S : 0) + (have ? s : 0)) * P.hq + head) * D + lane * VPL;
+      if (VPL == 4) {
+        const float4 a = __ldcg(reinterpret_cast<const float4*>(src));
+        r[u][0] = a.x, r[u][1] = a.y, r[u][2 % VPL] = a.z, r[u][3 % VPL] = a.w;
+      } else {
+        const float2 a = __ldcg(reinterpret_cast<const float2*>(src));
+        r[u][0] = a.x, r[u][1] = a.y;
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int s = s0 + (u & 3), t = u >> 2;
+      const float w = __shfl_sync(0xffffffffu, my_w, (t ? 16 : 0) + (s & 15));
       if (s < (t ? nt : nv) && w > 0.f) {
-        const float* src = P.part_acc + ((base + (t ? S : 0) + s) * P.hq + head) * D + lane * VPL;
 #pragma unroll
-        for (int e = 0; e < VPL; ++e) acc[e] = fmaf(__ldcg(src + e), w, acc[e]);
+        for (int e = 0; e < VPL; ++e) acc[e] = fmaf(r[u][e], w, acc[e]);
       }
     }
   }

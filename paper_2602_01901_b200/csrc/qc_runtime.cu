@@ -1222,7 +1222,18 @@ int decode_step_core(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, const 
     pmax_v = std::max(pmax_v, pv);
     pmax_t = std::max(pmax_t, pt);
   }
-  for (const LaunchGroup& g : c->groups)   // tile offsets are 32-bit
+  // Static ranges pay off for launches that leave a worker one or two ranges' worth of tiles (a
+  // launch per layer or per lazy block); on larger launches claimed 512-key items were measured
+  // faster (config 2, five blocks per launch: 0.89 against 1.05 ms per step; two blocks: 1.04
+  // against 1.12).  Tile offsets are 32-bit.
+  if (c->static_partition < 0) {
+    const int64_t workers = static_cast<int64_t>(c->ctx->n_sms) * kAttendWarps;
+    for (const LaunchGroup& g : c->groups) {
+      const int64_t tiles = static_cast<int64_t>(c->items_per_chunk) * (g.wv * tp_v + g.wt * tp_t);
+      if (tiles > workers * 60 * std::max(1, g.w_min)) use_static = false;
+    }
+  }
+  for (const LaunchGroup& g : c->groups)
     if (static_cast<int64_t>(c->items_per_chunk) * (g.wv * tp_v + g.wt * tp_t + 64LL * n_seqs * (g.job_end - g.job_begin)) >= (1LL << 31))
       use_static = false;
   int64_t tot_v = 0, tot_t = 0, step_rows = 0;   // step_rows: K/V rows the step has to read (for the profile)
