@@ -734,8 +734,10 @@ int32_t qc_alloc_cache(qc_ctx* ctx, const qc_config* cfg, void* pool_dev, size_t
   c->group = s.hq / s.hkv;
   c->heads_per_item = c->group > 1 ? 8 : 1;
   // what one more item costs a worker, in tiles: a query-group item fetches its query fragments when it
-  // starts and leaves up to eight partial rows (measured on launches of one layer: 4 resp. 8 best)
-  c->static_row_cost = c->group > 1 ? 8 : 4;
+  // starts and leaves up to eight partial rows (measured on launches of one layer: 4 resp. 12 best,
+  // with ranges of at least 6 resp. 4 tiles)
+  c->static_row_cost = c->group > 1 ? 12 : 4;
+  c->static_min_tiles = c->group > 1 ? 4 : 6;
   c->items_per_chunk = c->group > 1 ? s.hkv * ((c->group + 7) / 8) : s.hq;
   c->paged = cfg->page_size == 16;
   c->max_pages = s.max_pages;
