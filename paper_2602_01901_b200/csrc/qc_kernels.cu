@@ -6,12 +6,15 @@
 //   append_kernel   writes the new token's k / v rows into the text streams and every
 //                   ordinary layer's q into the Q Cache (a launch of its own on steps with patches
 //                   and per launch group of the host-buffer entry point)
+//   plan_kernel     for a step whose launches are cut into static tile ranges: where every worker of
+//                   every launch starts (first item, its first page ids, the cursor for the rest)
 //   attend_kernel   persistent split-KV partial attention, one query head per work item (MHA):
-//                   each warp is an independent worker that claims items from a counter, streams
-//                   K/V page tiles through its own shared-memory ring with bulk asynchronous
-//                   copies and keeps an online softmax in registers; under the per-layer
-//                   schedule a leader's sweep also stores its scaled scores in the logit cache
-//                   and a follower's sweep reads them there instead of any K tile
+//                   each warp is an independent worker that takes items -- claimed from a counter,
+//                   or the pieces of its static range of the launch's tiles -- streams K/V page
+//                   tiles through its own shared-memory ring with bulk asynchronous copies and
+//                   keeps an online softmax in registers; a leader's sweep can weight several
+//                   layers' V rows with one set of scores, store its scaled scores in the logit
+//                   cache, or leave out the step's new token for its followers
 //                   (the grouped-query variant on tensor cores is in qc_attend_tc.cu)
 //   merge_kernel    log-sum-exp merge of the partials, bf16 output
 //   prefill_scatter_kernel  stores prompt K/V rows into their pages
