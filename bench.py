@@ -169,7 +169,7 @@ def cpu_oracle_sample(w, mode: int, first_step: int):
     query heads; sub-problem i is sequence i mod batch, KV head i div batch), each advanced through
     ORACLE_STEPS decode steps from the context of the benchmark's first timed step, one process per
     core.  One generated token of the workload costs n_kv_heads sub-problem steps, so tokens/s =
-    sub-problem steps / (the busiest core's seconds inside the oracle) / n_kv_heads.
+    sub-problem steps / (core-seconds inside the oracle / cores) / n_kv_heads.
     """
     import multiprocessing as mp
 
@@ -180,15 +180,15 @@ def cpu_oracle_sample(w, mode: int, first_step: int):
     ctx = mp.get_context("spawn")
     with ctx.Pool(cores) as pool:
         spent = pool.map(_oracle_unit, jobs, chunksize=1)
-    # with equal costs per sub-problem the busiest core did ceil(n / cores) of them
-    per_core = -(-n_units // cores)
-    busiest = per_core * max(spent)
-    tokens_per_s = n_units * ORACLE_STEPS / busiest / w.n_kv_heads
+    # throughput of the cores together: sub-problem steps per core-second inside the oracle, times the cores
+    # (the mean over sub-problems, so that one straggler on a shared host does not decide the figure)
+    core_seconds = float(sum(spent))
+    tokens_per_s = n_units * ORACLE_STEPS / (core_seconds / cores) / w.n_kv_heads
     return {
         "value": tokens_per_s, "unit": UNIT, "cores": cores, "kind": "oracle",
         "sample": f"{n_units} (sequence, KV head) sub-problems x all {w.n_layers} layers x {ORACLE_STEPS} decode steps "
-                  f"from context {w.n_prompt + first_step} of {w.name}, one process per core; slowest sub-problem "
-                  f"{max(spent):.2f} s inside the oracle, {per_core} per core; scaled by 1/{w.n_kv_heads} KV heads per token",
+                  f"from context {w.n_prompt + first_step} of {w.name}, one process per core; {core_seconds:.1f} core-seconds "
+                  f"inside the oracle (slowest sub-problem {max(spent):.2f} s); scaled by 1/{w.n_kv_heads} KV heads per token",
     }
 
 
