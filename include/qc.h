@@ -214,6 +214,25 @@ int32_t qc_lazy_blocks(const float* similarity, int32_t n_layers, float eps, int
 int32_t qc_decode_step(qc_cache* cache, int32_t n_seqs, const int32_t* seq_ids, const void* q_dev,
                        const void* k_dev, const void* v_dev, void* out_dev, float* lse_out_dev);
 
+/* The same step issued layer by layer, for a caller whose layer l+1 inputs only exist after layer l's
+ * output (a model that computes layer after layer).  qc_decode_begin does the step's page planning
+ * for the listed sequences (distinct, active) and plans every layer's launch; then exactly n_layers
+ * calls of qc_decode_layer follow, for layer 0, 1, ... in order, each with that layer's slices
+ *   q_dev bf16 [n_seqs][n_q_heads][head_dim], k_dev / v_dev bf16 [n_seqs][n_kv_heads][head_dim],
+ *   out_dev bf16 [n_seqs][n_q_heads][head_dim], lse_out_dev optional fp32 [n_seqs][n_q_heads].
+ * A call appends the layer's k/v (and refreshes the Q Cache from an ordinary layer's q), runs the
+ * layer's attention launch and its merge, asynchronously; out_dev is complete when the stream
+ * has executed the call.  The launches are those of the in-order schedule ("in_order_launches"):
+ * a leader's call also weights its followers' cached V rows, so a follower's call is short (VLA_QC:
+ * its text sweep; GLA: the merge with the new token as one more key; k_dev of a GLA follower is
+ * ignored).  Results equal qc_decode_step's.  While a step is open (begun, layers left), every call
+ * that would change the cache returns QC_ERR_STATE; a step cannot be abandoned: the sequences'
+ * lengths and pages were committed by qc_decode_begin.  Errors: as qc_decode_step; a layer out of
+ * order or without an open step is QC_ERR_STATE. */
+int32_t qc_decode_begin(qc_cache* cache, int32_t n_seqs, const int32_t* seq_ids);
+int32_t qc_decode_layer(qc_cache* cache, int32_t layer, const void* q_dev, const void* k_dev, const void* v_dev,
+                        void* out_dev, float* lse_out_dev);
+
 /* Same step with HOST buffers of the same layouts.  The step runs as up to four launch groups of
  * consecutive lazy blocks; on two internal copy streams the inputs of a group are copied to
  * staging in the workspace while the previous group computes, and its outputs are copied back

@@ -33,7 +33,7 @@ EXPORTS = (
     "qc_init", "qc_cache_bytes_required", "qc_alloc_cache", "qc_prefill_append", "qc_prefill_attend", "qc_decode_step",
     "qc_decode_step_host", "qc_layer_similarity", "qc_lazy_blocks", "qc_free_seq", "qc_free", "qc_get_stats", "qc_debug_page_table",
     "qc_debug_read_qcache", "qc_debug_read_row", "qc_set_option", "qc_get_profile", "qc_status_string",
-    "qc_attend_static",
+    "qc_attend_static", "qc_decode_begin", "qc_decode_layer",
 )
 
 
@@ -98,6 +98,8 @@ def load() -> C.CDLL:
         "qc_layer_similarity": [vp, i32, pi32, vp, vp, i32, C.POINTER(C.c_float)],
         "qc_lazy_blocks": [C.POINTER(C.c_float), i32, C.c_float, i32, pu8],
         "qc_decode_step_host": [vp, i32, pi32, vp, vp, vp, vp, vp],
+        "qc_decode_begin": [vp, i32, pi32],
+        "qc_decode_layer": [vp, i32, vp, vp, vp, vp, vp],
         "qc_free_seq": [vp, i32],
         "qc_free": [vp, vp],
         "qc_get_stats": [vp, C.POINTER(qc_stats)],
@@ -196,6 +198,16 @@ def qc_decode_step(cache, seq_ids, q_ptr: int, k_ptr: int, v_ptr: int, out_ptr: 
     ids = seq_ids if isinstance(seq_ids, C.Array) else _i32_array(seq_ids)
     _check(load().qc_decode_step(cache, len(ids), ids, C.c_void_p(q_ptr), C.c_void_p(k_ptr), C.c_void_p(v_ptr),
                                  C.c_void_p(out_ptr), C.c_void_p(lse_ptr or None)), "qc_decode_step")
+
+
+def qc_decode_begin(cache, seq_ids) -> None:
+    ids = seq_ids if isinstance(seq_ids, C.Array) else _i32_array(seq_ids)
+    _check(load().qc_decode_begin(cache, len(ids), ids), "qc_decode_begin")
+
+
+def qc_decode_layer(cache, layer: int, q_ptr: int, k_ptr: int, v_ptr: int, out_ptr: int, lse_ptr: int = 0) -> None:
+    _check(load().qc_decode_layer(cache, layer, C.c_void_p(q_ptr), C.c_void_p(k_ptr), C.c_void_p(v_ptr),
+                                  C.c_void_p(out_ptr), C.c_void_p(lse_ptr or None)), "qc_decode_layer")
 
 
 def qc_decode_step_host(cache, seq_ids, q_ptr: int, k_ptr: int, v_ptr: int, out_ptr: int, lse_ptr: int = 0) -> None:

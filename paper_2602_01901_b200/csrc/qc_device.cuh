@@ -735,7 +735,14 @@ __device__ __forceinline__ void merge_row(const Params& P, int layer, int si, in
   if (extra_leader >= 0) {
     const int kvh = head / P.group;
     const uint16_t* qrow = P.qcache + ((static_cast<size_t>(extra_leader) * P.max_seqs + sq.seq_id) * P.hq + head) * D;
-    const uint16_t* krow = P.k + ((static_cast<size_t>(extra_leader) * P.n_seqs + si) * P.hkv + kvh) * D;
+    // the leader's new k: the last row of its text K stream (appended before this kernel ran)
+    const int pos = sq.len_text - 1;
+    int pid = P.table[table_row(P, extra_leader, 0, sq.seq_id) + pos / kPage];
+    if (static_cast<uint32_t>(pid) >= static_cast<uint64_t>(P.n_pool_pages)) {   // never read outside the pool
+      if (lane == 0) report_error(P.err, P.err_host, kErrBadPage);
+      pid = 0;
+    }
+    const uint16_t* krow = P.pool + ((static_cast<size_t>(pid) * P.hkv + kvh) * kPage + pos % kPage) * D;
     v_new = P.v + ((static_cast<size_t>(layer) * P.n_seqs + si) * P.hkv + kvh) * D + lane * VPL;
     float dot = 0.f;
 #pragma unroll

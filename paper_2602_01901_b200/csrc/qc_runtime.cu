@@ -42,6 +42,16 @@ struct LaunchGroup {
   int w_max_v, w_max_t;   // largest tiles per page among its visual / text jobs
 };
 
+// A step opened by qc_decode_begin: what its layer-by-layer launches need.
+struct OpenStep {
+  bool active = false;
+  Params p{};
+  LaunchList launches{};
+  bool use_static = false;
+  int64_t tot_v = 0, tot_t = 0, bytes = 0;
+  int next_layer = 0;
+};
+
 struct Layout {   // byte offsets into the workspace
   size_t table, layer_flags, layer_kind, leader, jobs, plan, qcache, part_acc, part_ml, logits, items, step, err, counters, row_slots, row_done, wdesc, stage_q,
       stage_k, stage_v, stage_out, stage_lse, tok, total;
@@ -138,6 +148,7 @@ struct qc_cache {
   double prof_prefill_flops = 0.0;
 
   int64_t decode_steps = 0, attend_launches = 0, kernel_launches = 0, kv_bytes_swept = 0;
+  OpenStep open;
 };
 
 namespace {
@@ -862,6 +873,7 @@ int32_t qc_free(qc_ctx* ctx, qc_cache* cache) {
 int32_t qc_prefill_append(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, const int32_t* n_tokens,
                           const uint8_t* kind, const void* k_dev, const void* v_dev) {
   if (!c || n_seqs < 0 || (n_seqs > 0 && (!seq_ids || !n_tokens))) return QC_ERR_INVALID_ARG;
+  if (c->open.active) return QC_ERR_STATE;   // a decode step is open
   if (n_seqs == 0) return QC_OK;
   if (!k_dev || !v_dev) return QC_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(k_dev) & 15) || (reinterpret_cast<uintptr_t>(v_dev) & 15)) return QC_ERR_INVALID_ARG;
@@ -1102,11 +1114,72 @@ struct HostPipe {
   cudaEvent_t* done;
 };
 
+// One attention launch of a step (group gi of the launch plan) with its merge; optionally the
+// append of the group's layers first (host-buffer entry point, per-layer entry point).
+int run_group(qc_cache* c, Params& p, size_t gi, const LaunchList& launches, bool use_static, int64_t tot_v,
+              int64_t tot_t, bool append_first, cudaEvent_t wait_in, cudaEvent_t record_done, cudaEvent_t* ev,
+              cudaStream_t stream) {
+  const int pb = c->group_pos[gi].first, pe = c->group_pos[gi].second;
+  p.item_begin = static_cast<int32_t>(c->plan_vis_before[pb] * tot_v + c->plan_text_before[pb] * tot_t);
+  p.item_end = static_cast<int32_t>(c->plan_vis_before[pe] * tot_v + c->plan_text_before[pe] * tot_t);
+  p.layer_begin = c->groups[gi].layer_begin;
+  p.layer_end = c->groups[gi].layer_end;
+  p.launch_index = static_cast<int32_t>(gi);
+  p.pos_begin = pb;
+  p.pos_end = pe;
+  p.extra_key_leader = c->groups[gi].extra_key_leader;
+  bool has_work = p.item_end > p.item_begin;
+  if (use_static) {   // (a step has at most n_layers <= 127 launches: every one has its entry)
+    const LaunchDesc& one = launches.launch[gi];
+    has_work = one.part_workers > 0;
+    p.part_q = one.part_q;
+    p.part_k = one.part_k;
+    p.part_vw = one.part_vw;
+    p.part_workers = one.part_workers;
+    p.part_row_cost = one.part_row_cost;
+    p.part_tiles = 0;
+  }
+  if (wait_in) QC_CUDA(cudaStreamWaitEvent(stream, wait_in, 0));
+  if (append_first) {
+    QC_CUDA(launch_append(p, stream));   // this group's layers only
+    c->kernel_launches++;
+  }
+  if (ev && gi == 0) QC_CUDA(cudaEventRecord(ev[1], stream));
+  cudaEvent_t* evl = nullptr;
+  if (ev && c->profile == 2 && has_work && c->ev_launches < 64 * kMaxProfileSteps) {
+    if (static_cast<int>(c->ev_launch.size()) < 2 * (c->ev_launches + 1)) {
+      for (int i = 0; i < 2; ++i) {
+        cudaEvent_t e;
+        QC_CUDA(cudaEventCreate(&e));
+        c->ev_launch.push_back(e);
+      }
+    }
+    evl = &c->ev_launch[2 * c->ev_launches++];
+    QC_CUDA(cudaEventRecord(evl[0], stream));
+  }
+  if (!has_work) {
+    // (a GLA follower of the in-order schedule: its merge does everything)
+  } else if (c->group > 1) {
+    QC_CUDA(launch_attend_tc(p, c->ctx->n_sms, stream));
+  } else {
+    QC_CUDA(launch_attend(p, c->ctx->n_sms, stream));
+  }
+  if (evl) QC_CUDA(cudaEventRecord(evl[1], stream));
+  if (ev && gi + 1 == c->groups.size()) QC_CUDA(cudaEventRecord(ev[2], stream));
+  if (c->groups[gi].needs_merge) QC_CUDA(launch_merge(p, stream));
+  if (record_done) QC_CUDA(cudaEventRecord(record_done, stream));
+  c->attend_launches += has_work ? 1 : 0;
+  c->kernel_launches += (has_work ? 1 : 0) + (c->groups[gi].needs_merge ? 1 : 0);
+  return QC_OK;
+}
+
 int decode_step_core(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, const void* q_dev, const void* k_dev,
-                     const void* v_dev, void* out_dev, float* lse_out_dev, const HostPipe* pipe) {
+                     const void* v_dev, void* out_dev, float* lse_out_dev, const HostPipe* pipe,
+                     bool open_only = false) {
   if (!c || n_seqs < 0 || (n_seqs > 0 && !seq_ids)) return QC_ERR_INVALID_ARG;
-  if (n_seqs == 0) return QC_OK;
-  if (!q_dev || !k_dev || !v_dev || !out_dev) return QC_ERR_INVALID_ARG;
+  if (c->open.active) return QC_ERR_STATE;   // a step opened by qc_decode_begin has layers left
+  if (n_seqs == 0) return open_only ? QC_ERR_INVALID_ARG : QC_OK;
+  if (!open_only && (!q_dev || !k_dev || !v_dev || !out_dev)) return QC_ERR_INVALID_ARG;
   if (n_seqs > c->cfg.max_seqs) return QC_ERR_INVALID_ARG;
   const void* ptrs[4] = {q_dev, k_dev, v_dev, out_dev};
   for (const void* ptr : ptrs)
@@ -1130,7 +1203,7 @@ int decode_step_core(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, const 
   QC_CUDA(cudaSetDevice(c->ctx->device));
   cudaStream_t stream = c->ctx->stream;
 
-  const int want_per = pipe ? pipe->per_launch : c->layers_per_launch;
+  const int want_per = open_only ? -2 : (pipe ? pipe->per_launch : c->layers_per_launch);
   if (c->plan_dirty || c->plan_per != want_per) {
     const int st = rebuild_plan(c, want_per);
     if (st != QC_OK) return st;
@@ -1283,7 +1356,7 @@ int decode_step_core(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, const 
   p.inline_seqs = inline_step ? 1 : 0;
   // the append reads the page table (not beside its patches) and every layer's k/v (not before
   // the host pipe has copied them)
-  p.fused_append = (n_patches == 0 && !pipe) ? 1 : 0;
+  p.fused_append = (n_patches == 0 && !pipe && !open_only) ? 1 : 0;
 
   // static partition of every launch of the step (part_workers == 0: the launch has nothing to sweep)
   auto partition_of = [&](size_t gi) {
@@ -1329,7 +1402,7 @@ int decode_step_core(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, const 
   p.wdesc = planned ? reinterpret_cast<const WorkerDesc*>(c->ws + c->lay.wdesc) : nullptr;
 
   cudaEvent_t* ev = nullptr;
-  if (c->profile && c->ev_steps < kMaxProfileSteps) {
+  if (c->profile && !open_only && c->ev_steps < kMaxProfileSteps) {
     if (static_cast<int>(c->ev.size()) < 4 * (c->ev_steps + 1)) {
       for (int i = 0; i < 4; ++i) {
         cudaEvent_t e;
@@ -1342,7 +1415,7 @@ int decode_step_core(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, const 
   }
   QC_CUDA(launch_setup(p, inline_step ? &inl : nullptr, stream));
   c->kernel_launches++;
-  if (!p.fused_append && !pipe) {
+  if (!p.fused_append && !pipe && !open_only) {
     p.layer_begin = 0;
     p.layer_end = N;
     QC_CUDA(launch_append(p, stream));
@@ -1352,59 +1425,22 @@ int decode_step_core(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, const 
     QC_CUDA(launch_plan(p, launches, static_cast<int>(c->groups.size()), stream));
     c->kernel_launches++;
   }
+  if (open_only) {   // qc_decode_begin: the launches follow layer by layer (qc_decode_layer)
+    OpenStep& o = c->open;
+    o.p = p;
+    o.launches = launches;
+    o.use_static = use_static;
+    o.tot_v = tot_v;
+    o.tot_t = tot_t;
+    o.next_layer = 0;
+    o.bytes = step_rows * c->hkv * c->D * 2;
+    o.active = true;
+    return QC_OK;
+  }
   for (size_t gi = 0; gi < c->groups.size(); ++gi) {
-    const int pb = c->group_pos[gi].first, pe = c->group_pos[gi].second;
-    p.item_begin = static_cast<int32_t>(c->plan_vis_before[pb] * tot_v + c->plan_text_before[pb] * tot_t);
-    p.item_end = static_cast<int32_t>(c->plan_vis_before[pe] * tot_v + c->plan_text_before[pe] * tot_t);
-    p.layer_begin = c->groups[gi].layer_begin;
-    p.layer_end = c->groups[gi].layer_end;
-    p.launch_index = static_cast<int32_t>(gi);
-    p.pos_begin = pb;
-    p.pos_end = pe;
-    p.extra_key_leader = c->groups[gi].extra_key_leader;
-    bool has_work = p.item_end > p.item_begin;
-    if (use_static) {
-      const LaunchDesc& L = launches.launch[gi < kMaxPlanLaunches ? gi : 0];
-      const LaunchDesc one = gi < kMaxPlanLaunches ? L : partition_of(gi);
-      has_work = one.part_workers > 0;
-      p.part_q = one.part_q;
-      p.part_k = one.part_k;
-      p.part_vw = one.part_vw;
-      p.part_workers = one.part_workers;
-      p.part_row_cost = one.part_row_cost;
-      p.part_tiles = 0;
-    }
-    if (pipe) {
-      QC_CUDA(cudaStreamWaitEvent(stream, pipe->in[gi], 0));
-      QC_CUDA(launch_append(p, stream));   // this group's layers only
-      c->kernel_launches++;
-    }
-    if (ev && gi == 0) QC_CUDA(cudaEventRecord(ev[1], stream));
-    cudaEvent_t* evl = nullptr;
-    if (ev && c->profile == 2 && has_work && c->ev_launches < 64 * kMaxProfileSteps) {
-      if (static_cast<int>(c->ev_launch.size()) < 2 * (c->ev_launches + 1)) {
-        for (int i = 0; i < 2; ++i) {
-          cudaEvent_t e;
-          QC_CUDA(cudaEventCreate(&e));
-          c->ev_launch.push_back(e);
-        }
-      }
-      evl = &c->ev_launch[2 * c->ev_launches++];
-      QC_CUDA(cudaEventRecord(evl[0], stream));
-    }
-    if (!has_work) {
-      // (a GLA follower of the in-order schedule: its merge does everything)
-    } else if (c->group > 1) {
-      QC_CUDA(launch_attend_tc(p, c->ctx->n_sms, stream));
-    } else {
-      QC_CUDA(launch_attend(p, c->ctx->n_sms, stream));
-    }
-    if (evl) QC_CUDA(cudaEventRecord(evl[1], stream));
-    if (ev && gi + 1 == c->groups.size()) QC_CUDA(cudaEventRecord(ev[2], stream));
-    if (c->groups[gi].needs_merge) QC_CUDA(launch_merge(p, stream));
-    if (pipe) QC_CUDA(cudaEventRecord(pipe->done[gi], stream));
-    c->attend_launches += has_work ? 1 : 0;
-    c->kernel_launches += (has_work ? 1 : 0) + (c->groups[gi].needs_merge ? 1 : 0);
+    const int st = run_group(c, p, gi, launches, use_static, tot_v, tot_t, pipe != nullptr,
+                             pipe ? pipe->in[gi] : nullptr, pipe ? pipe->done[gi] : nullptr, ev, stream);
+    if (st != QC_OK) return st;
   }
   if (ev) {
     QC_CUDA(cudaEventRecord(ev[3], stream));
@@ -1424,6 +1460,42 @@ extern "C" {
 int32_t qc_decode_step(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, const void* q_dev, const void* k_dev,
                        const void* v_dev, void* out_dev, float* lse_out_dev) {
   return decode_step_core(c, n_seqs, seq_ids, q_dev, k_dev, v_dev, out_dev, lse_out_dev, nullptr);
+}
+
+int32_t qc_decode_begin(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids) {
+  return decode_step_core(c, n_seqs, seq_ids, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, true);
+}
+
+int32_t qc_decode_layer(qc_cache* c, int32_t layer, const void* q_dev, const void* k_dev, const void* v_dev,
+                        void* out_dev, float* lse_out_dev) {
+  if (!c || !q_dev || !k_dev || !v_dev || !out_dev) return QC_ERR_INVALID_ARG;
+  const void* ptrs[4] = {q_dev, k_dev, v_dev, out_dev};
+  for (const void* ptr : ptrs)
+    if (reinterpret_cast<uintptr_t>(ptr) & 15) return QC_ERR_INVALID_ARG;
+  OpenStep& o = c->open;
+  if (!o.active || layer != o.next_layer) return QC_ERR_STATE;
+  if (const int32_t dev_err = *static_cast<volatile int32_t*>(c->err_host)) return dev_err;
+  QC_CUDA(cudaSetDevice(c->ctx->device));
+  // the kernels index a step's tensors as [layer][sequence]...: hand them this layer's slices at that place
+  Params p = o.p;
+  const uintptr_t q_off = static_cast<uintptr_t>(layer) * p.n_seqs * c->hq * c->D * 2;
+  const uintptr_t kv_off = static_cast<uintptr_t>(layer) * p.n_seqs * c->hkv * c->D * 2;
+  p.q = reinterpret_cast<const uint16_t*>(reinterpret_cast<uintptr_t>(q_dev) - q_off);
+  p.k = reinterpret_cast<const uint16_t*>(reinterpret_cast<uintptr_t>(k_dev) - kv_off);
+  p.v = reinterpret_cast<const uint16_t*>(reinterpret_cast<uintptr_t>(v_dev) - kv_off);
+  p.out = reinterpret_cast<uint16_t*>(reinterpret_cast<uintptr_t>(out_dev) - q_off);
+  p.lse = lse_out_dev ? reinterpret_cast<float*>(reinterpret_cast<uintptr_t>(lse_out_dev) -
+                                                  static_cast<uintptr_t>(layer) * p.n_seqs * c->hq * sizeof(float))
+                      : nullptr;
+  const int st = run_group(c, p, static_cast<size_t>(layer), o.launches, o.use_static, o.tot_v, o.tot_t, true, nullptr,
+                           nullptr, nullptr, c->ctx->stream);
+  if (st != QC_OK) return st;
+  if (++o.next_layer == c->cfg.n_layers) {
+    o.active = false;
+    c->decode_steps++;
+    c->kv_bytes_swept += o.bytes;
+  }
+  return QC_OK;
 }
 
 int32_t qc_decode_step_host(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, const void* q_host,
@@ -1498,7 +1570,7 @@ int32_t qc_decode_step_host(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids,
 int32_t qc_free_seq(qc_cache* c, int32_t seq_id) {
   if (!c || seq_id < 0 || seq_id >= c->cfg.max_seqs) return QC_ERR_INVALID_ARG;
   SeqState& st = c->seqs[seq_id];
-  if (!st.active) return QC_ERR_STATE;
+  if (!st.active || c->open.active) return QC_ERR_STATE;
   if (c->paged) {
     for (auto it = st.alloc_order.rbegin(); it != st.alloc_order.rend(); ++it) c->free_stack.push_back(*it);
     for (int l = 0; l < c->cfg.n_layers; ++l)

@@ -65,6 +65,14 @@ class Session:
         qc.qc_decode_step(self.cache, seq_ids, q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
                           lse.data_ptr() if lse is not None else 0)
 
+    def decode_begin(self, seq_ids):
+        qc.qc_decode_begin(self.cache, seq_ids)
+
+    def decode_layer(self, layer: int, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, out: torch.Tensor,
+                     lse: Optional[torch.Tensor] = None):
+        qc.qc_decode_layer(self.cache, layer, q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
+                           lse.data_ptr() if lse is not None else 0)
+
     def decode_step_host(self, seq_ids, q, k, v, out, lse=None):
         qc.qc_decode_step_host(self.cache, seq_ids, q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
                                lse.data_ptr() if lse is not None else 0)
