@@ -204,7 +204,9 @@ def _gen_inputs(w, first, count, device, seq_offset=0):
 
 class _Arms:
     """The timed arms of one workload on one GPU, all on one cache: consecutive decode steps under
-    different schedules (a schedule changes how a step is cut into launches, never its result)."""
+    different schedules (a schedule changes how a step is cut into launches, never its result).  The
+    context grows by one token per step, so a later arm sweeps more bytes per step than an earlier one:
+    every record carries its context range, and GB/s figures are the ones to compare across arms."""
 
     def __init__(self, args, w, mode, group, local_rank, seq_offset, all_full=False):
         import torch
@@ -257,6 +259,43 @@ class _Arms:
                 "launches_per_step": (st1.kernel_launches - st0.kernel_launches) / n,
                 "context_first": self.w.n_prompt + self.step - n + 1, "context_last": self.w.n_prompt + self.step,
                 "prof": prof}
+
+    def run_layer_calls(self, n):
+        """n steps through qc_decode_begin / qc_decode_layer, every layer's tensors passed on their own."""
+        torch = self.torch
+        inputs = _gen_inputs(self.w, self.step, n + 2, self.dev, self.seq_offset)
+        outs = [torch.empty(self.out.shape[1:], dtype=torch.bfloat16, device=self.dev) for _ in range(self.w.n_layers)]
+
+        from paper_2602_01901_b200 import binding as qc
+
+        # raw pointers of every (step, layer) slice, taken ahead of the timed loop: the loop itself is
+        # one C call per layer, as a model's runtime would make them
+        ptrs = [[(q[l].data_ptr(), k[l].data_ptr(), v[l].data_ptr(), outs[l].data_ptr()) for l in range(self.w.n_layers)]
+                for q, k, v in inputs]
+        cache, ids = self.s.cache, self.ids
+
+        def step(i):
+            qc.qc_decode_begin(cache, ids)
+            for l, (qp, kp, vp, op) in enumerate(ptrs[i]):
+                qc.qc_decode_layer(cache, l, qp, kp, vp, op)
+
+        for i in range(2):
+            step(i)
+        st0 = self.s.stats()
+        self.barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(2, n + 2):
+            step(i)
+        e1.record()
+        self.barrier()
+        ms = self.group.max_over_ranks(e0.elapsed_time(e1)) / n
+        st1 = self.s.stats()
+        if st1.device_error:
+            raise SystemExit(f"device error word = {st1.device_error}")
+        self.step += n + 2
+        return {"ms_per_step": ms, "kv_bytes_per_step": (st1.kv_bytes_swept - st0.kv_bytes_swept) / n,
+                "context_first": self.w.n_prompt + self.step - n + 1, "context_last": self.w.n_prompt + self.step}
 
     def run_host(self, n):
         """n steps through qc_decode_step_host with pinned host buffers; returns tokens/s inputs."""
@@ -326,17 +365,25 @@ def measure_workload(args, w, mode, group, local_rank, world, rank, K, W_, Ke, e
     if extra_arms and world == 1:
         a.set([("layers_per_launch", 1)])
         a.run(3, timed=False)
-        pb = a.run(min(K, 32))
+        pb = a.run(min(K, 24))
         extra["per_block_launches"] = {
             "ms_per_step": pb["ms_per_step"], "kv_gb_per_s_whole_step": pb["kv_bytes_per_step"] / pb["ms_per_step"] / 1e6,
+            "context": [pb["context_first"], pb["context_last"]],
             "note": "one attention + merge launch per lazy block, blocks in layer order (needs a block's q/k/v at once)"}
         a.set([("per_layer_logit_cache", 1)])
         a.run(3, timed=False)
-        pl = a.run(min(K, 32))
+        pl = a.run(min(K, 24))
         extra["per_layer_logit_cache"] = {
             "ms_per_step": pl["ms_per_step"], "kv_gb_per_s_whole_step": pl["kv_bytes_per_step"] / pl["ms_per_step"] / 1e6,
+            "context": [pl["context_first"], pl["context_last"]],
             "note": "one launch per layer; followers sweep their V with the leader's scores from a logit cache"}
         a.set(IN_ORDER)
+        lc = a.run_layer_calls(min(K, 24))
+        extra["layer_calls"] = {
+            "ms_per_step": lc["ms_per_step"], "kv_gb_per_s_whole_step": lc["kv_bytes_per_step"] / lc["ms_per_step"] / 1e6,
+            "context": [lc["context_first"], lc["context_last"]],
+            "note": "the in-order step through qc_decode_begin + one qc_decode_layer per layer (each call gets only "
+                    "that layer's q/k/v and also appends them: one more small launch per layer)"}
     a.set(IN_ORDER)
     a.run(3, timed=False)
     host = a.run_host(Ke)
@@ -456,7 +503,7 @@ def run_gpu(args, rank, world, local_rank):
         "per_config": per_config, "tiny": tiny,
         "paper_context": "paper reports ~35% KV saved and 1.5x-1.6x decode throughput for LLaVA-NeXT-7B on one 80GB A100 (whole model)",
     }
-    for key in ("vs_all_full", "per_block_launches", "per_layer_logit_cache"):
+    for key in ("vs_all_full", "per_block_launches", "per_layer_logit_cache", "layer_calls"):
         if key in head:
             line[key] = head[key]
     return line

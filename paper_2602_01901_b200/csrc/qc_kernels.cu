@@ -143,6 +143,9 @@ __global__ void setup_kernel(const __grid_constant__ Params P, const __grid_cons
 
 __global__ void append_kernel(const __grid_constant__ Params P) {
   pdl_wait();
+  // what the next kernel does ahead of its own wait reads nothing this kernel writes (an attention
+  // worker's early tiles leave out the page that can hold the new token)
+  pdl_launch_dependents();
   append_rows(P, P.seqs[blockIdx.x], blockIdx.x, P.layer_begin + blockIdx.y);   // layers of one launch group
 }
 
