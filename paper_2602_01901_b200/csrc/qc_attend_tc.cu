@@ -125,6 +125,28 @@ __device__ __forceinline__ void process_item_tc(WorkerState& st, const TcCtx* ct
       } else {
         const uint32_t tile = wait_tile<D>(st, ring, full, P, lane);
         if (st.dead) break;
+        if (holds_new_token(P, it, pg)) {
+          // the new token's k row comes from the step's input: into the (swizzled) tile, and into the pool
+          const ItemPages& ip = ctx[st.cons_k % kCtxSlots].ip;
+          if (lane < D / 8) {
+            const uint4 val = ip.new_k[lane];
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(tile + swz<D>(nvalid - 1, lane)), "r"(val.x),
+                         "r"(val.y), "r"(val.z), "r"(val.w)
+                         : "memory");
+            const int pid = ip.pages[0][pg];
+            if (static_cast<uint32_t>(pid) < static_cast<uint64_t>(P.n_pool_pages))
+              reinterpret_cast<uint4*>(P.pool + ((static_cast<size_t>(pid) * P.hkv + ip.kv_head) * kPage + (nvalid - 1)) * D)[lane] = val;
+          }
+          // an ordinary layer's queries go to the Q Cache
+          if (it.q_layer[0] == it.k_layer && !((it.flags >> kFlagCachedShift) & 1) && (P.layer_flags[it.k_layer] & kLayerWritesQCache)) {
+            const uint4* src = reinterpret_cast<const uint4*>(
+                P.q + ((static_cast<size_t>(it.k_layer) * P.n_seqs + it.seq_idx) * P.hq + it.head) * D);
+            uint4* dst = reinterpret_cast<uint4*>(
+                P.qcache + ((static_cast<size_t>(it.k_layer) * P.max_seqs + it.seq_id) * P.hq + it.head) * D);
+            for (int e = lane; e < n_heads * (D / 8); e += 32) dst[e] = src[e];
+          }
+          __syncwarp();
+        }
 #pragma unroll
         for (int x = 0; x < NQ; ++x) s[x][0] = s[x][1] = s[x][2] = s[x][3] = 0.f;
 #pragma unroll
@@ -207,6 +229,24 @@ __device__ __forceinline__ void process_item_tc(WorkerState& st, const TcCtx* ct
       if (st.dead) break;
       const bool skipping = SKIP && skip_page && ((skip_mask >> v) & 1u);
       const int nvalid_v = skipping ? nvalid - 1 : nvalid;
+      if (!skipping && holds_new_token(P, it, pg)) {
+        // this consumer's new v row, likewise
+        const ItemPages& ip = ctx[st.cons_k % kCtxSlots].ip;
+        if (lane < D / 8) {
+          const uint4 val = v == first_taker(it)
+                                ? ip.new_v[lane]
+                                : reinterpret_cast<const uint4*>(
+                                      P.v + ((static_cast<size_t>(it.v_layer[v]) * P.n_seqs + it.seq_idx) * P.hkv + ip.kv_head) * D)[lane];
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(tile + swz<D>(nvalid - 1, lane)), "r"(val.x),
+                       "r"(val.y), "r"(val.z), "r"(val.w)
+                       : "memory");
+          const int pid = ip.pages[1 + v][pg];
+          if (static_cast<uint32_t>(pid) < static_cast<uint64_t>(P.n_pool_pages))
+            reinterpret_cast<uint4*>(P.pool + ((static_cast<size_t>(pid) * P.hkv + ip.kv_head) * kPage + (nvalid - 1)) * D)[lane] = val;
+        }
+        fence_proxy_async();
+        __syncwarp();
+      }
       if (nvalid_v < kPage) {
         // rows past the end of the stream hold whatever the pool held: clear them, since a
         // zero weight does not cancel a NaN or an infinity
@@ -333,12 +373,14 @@ __device__ __forceinline__ void attend_tc_worker(const Params& P, TcCtx* ctx, ui
     pdl_launch_dependents();
   }
   // ---- this layer's inputs; the rest of the first tiles; the second item's context while they fly
+  begin_new_rows(ctx[0].ip, P, first, lane, D);
   fill_ring<D, kRingTc, true>(st, ctx_of, ring, full, P, lane);
   if (STATIC) record_row_slots(P, first, lane);
   if (!STATIC) issued = claim_issue(P, lane);
   bool more = take();
   if (more) {
     begin_item_pages(ctx[1].ip, P, it, lane);
+    begin_new_rows(ctx[1].ip, P, it, lane, D);
     if (STATIC) record_row_slots(P, it, lane);
   }
   cp_async_wait_all();
@@ -356,6 +398,7 @@ __device__ __forceinline__ void attend_tc_worker(const Params& P, TcCtx* ctx, ui
       more = take();
       if (more) {
         begin_item_pages(ctx[(k + 2) % kCtxSlots].ip, P, it, lane);
+        begin_new_rows(ctx[(k + 2) % kCtxSlots].ip, P, it, lane, D);
         if (STATIC) record_row_slots(P, it, lane);
         pending = true;
       }

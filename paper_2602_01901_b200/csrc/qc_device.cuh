@@ -209,6 +209,8 @@ struct ItemPages {
   StepSeq sq;          // the item's sequence
   int32_t kv_head;     // item.head / group
   int32_t pad[3];
+  uint4 new_k[16];     // folded append: the new token's k row of the item's K layer and the v row of its
+  uint4 new_v[16];     // first consumer that takes the new token (fetched with the queries)
   int32_t pages[1 + kMaxCons][kMaxChunkPages];   // [0]: K pages, [1 + x]: V pages of consumer x
 };
 
@@ -664,6 +666,31 @@ __device__ __forceinline__ bool cursor_step(RangeCursor* slot, const Params& P, 
   return ok;
 }
 
+// Folded append: is page `pg` of the item the page that receives the step's new token?
+__device__ __forceinline__ bool holds_new_token(const Params& P, const Item& it, int pg) {
+  return P.fold_append && it.stream == 0 && (it.flags & kFlagStreamEnd) && pg == it.n_pages - 1;
+}
+
+// Folded append: start fetching the new token's rows of an item that ends its layer's text stream
+// (this layer's inputs: after the wait for the previous kernel, with the queries).
+__device__ __forceinline__ int first_taker(const Item& it) {   // first consumer that does not leave out the new token
+  for (int x = 0; x < it.n_cons; ++x)
+    if (!((it.skip_new >> x) & 1)) return x;
+  return -1;
+}
+__device__ __forceinline__ void begin_new_rows(ItemPages& c, const Params& P, const Item& it, int lane, int d) {
+  if (!(P.fold_append && it.stream == 0 && (it.flags & kFlagStreamEnd))) return;
+  const int n_vec = d / 8, kv_head = it.head / P.group;
+  if (lane < n_vec)
+    cp_async_16(&c.new_k[lane], reinterpret_cast<const uint4*>(
+                                    P.k + ((static_cast<size_t>(it.k_layer) * P.n_seqs + it.seq_idx) * P.hkv + kv_head) * d) + lane);
+  const int x = first_taker(it);
+  if (x >= 0 && lane >= 16 && lane - 16 < n_vec)
+    cp_async_16(&c.new_v[lane - 16],
+                reinterpret_cast<const uint4*>(
+                    P.v + ((static_cast<size_t>(it.v_layer[x]) * P.n_seqs + it.seq_idx) * P.hkv + kv_head) * d) + (lane - 16));
+}
+
 // Start of a worker from the descriptor planned for it when the step began: the first item goes
 // into the context slot together with the page ids of its first two pages, the cursor into the
 // worker's cursor slot.  False if the worker has no work.  `stage`: 48 bytes of shared memory.
@@ -753,6 +780,17 @@ __device__ __forceinline__ void merge_row(const Params& P, int layer, int si, in
     for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
     s_new = dot * P.scale_log2;
     mmax = fmaxf(mmax, s_new);
+    if (P.fold_append && head % P.group == 0) {
+      // this layer's new v row has no sweep to store it: the merge warp of the KV head's first query head does
+      int pid_v = P.table[table_row(P, layer, 2, sq.seq_id) + pos / kPage];
+      if (static_cast<uint32_t>(pid_v) < static_cast<uint64_t>(P.n_pool_pages)) {
+        uint16_t* dst_v = P.pool + ((static_cast<size_t>(pid_v) * P.hkv + kvh) * kPage + pos % kPage) * D + lane * VPL;
+#pragma unroll
+        for (int e = 0; e < VPL; ++e) dst_v[e] = v_new[e];
+      } else if (lane == 0) {
+        report_error(P.err, P.err_host, kErrBadPage);
+      }
+    }
   }
 
   float lsum = 0.f;

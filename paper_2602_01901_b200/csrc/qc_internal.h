@@ -163,6 +163,10 @@ struct Params {
   int32_t tp_v, tp_t;                // pages of the visual / text streams, summed over the listed sequences
   int32_t pos_begin, pos_end;        // plan positions of the launch
   int32_t slots_per_stream;          // partial-row slots of one stream of an output row (text slots start here)
+  int32_t fold_append;               // in-order schedule: the new token's k/v rows (and an ordinary layer's q for the
+                                     // Q Cache) are taken from the step's inputs by the attention worker (or the
+                                     // merge warp) that meets the end of the layer's text stream, which also stores
+                                     // them: no append launch, nothing of a layer is touched before its own launch
   int32_t debug_drop_tile;           // test hook: every worker of an attention launch leaves out the copy of its first
                                      // tile and waits for it with a short limit (nothing in flight, nothing faults)
   int32_t extra_key_leader;          // merge only, >= 0: the rows also take the step's new token as one more key,

@@ -317,6 +317,22 @@ __device__ __forceinline__ void process_item(WorkerState& st, const WarpCtx<D>* 
       // ---- K tile: scores of 16 keys
       const uint8_t* tile = static_cast<const uint8_t*>(__cvta_shared_to_generic(wait_tile<D>(st, ring, full, P, lane)));
       if (st.dead) break;
+      if (holds_new_token(P, c.ip.item, pg)) {
+        // the new token's k row comes from the step's input: into the tile, and into the pool for later steps
+        const Item& it = c.ip.item;
+        if (lane < D / 8) {
+          const uint4 val = c.ip.new_k[lane];
+          reinterpret_cast<uint4*>(const_cast<uint8_t*>(tile) + (nvalid - 1) * (D * 2))[lane] = val;
+          const int pid = c.ip.pages[0][pg];
+          if (static_cast<uint32_t>(pid) < static_cast<uint64_t>(P.n_pool_pages))
+            reinterpret_cast<uint4*>(P.pool + ((static_cast<size_t>(pid) * P.hkv + c.ip.kv_head) * kPage + (nvalid - 1)) * D)[lane] = val;
+          // an ordinary layer's query goes to the Q Cache
+          if (it.q_layer[0] == it.k_layer && !((it.flags >> kFlagCachedShift) & 1) && (P.layer_flags[it.k_layer] & kLayerWritesQCache))
+            reinterpret_cast<uint4*>(P.qcache + ((static_cast<size_t>(it.k_layer) * P.max_seqs + it.seq_id) * P.hq + it.head) * D)[lane] =
+                c.qraw[0][lane];
+        }
+        __syncwarp();
+      }
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         const int r = 4 * i + kg;
@@ -390,6 +406,21 @@ __device__ __forceinline__ void process_item(WorkerState& st, const WarpCtx<D>* 
       const uint8_t* tile = static_cast<const uint8_t*>(__cvta_shared_to_generic(wait_tile<D>(st, ring, full, P, lane)));
       if (st.dead) break;
       const int nvalid_v = (SKIP && skip_here && pg == n_pages - 1) ? nvalid - static_cast<int>((skip_mask >> v) & 1u) : nvalid;
+      if (nvalid_v == nvalid && holds_new_token(P, c.ip.item, pg)) {
+        // this consumer's new v row, likewise
+        const Item& it = c.ip.item;
+        if (lane < D / 8) {
+          const uint4 val = v == first_taker(it)
+                                ? c.ip.new_v[lane]
+                                : reinterpret_cast<const uint4*>(
+                                      P.v + ((static_cast<size_t>(it.v_layer[v]) * P.n_seqs + it.seq_idx) * P.hkv + c.ip.kv_head) * D)[lane];
+          reinterpret_cast<uint4*>(const_cast<uint8_t*>(tile) + (nvalid - 1) * (D * 2))[lane] = val;
+          const int pid = c.ip.pages[1 + v][pg];
+          if (static_cast<uint32_t>(pid) < static_cast<uint64_t>(P.n_pool_pages))
+            reinterpret_cast<uint4*>(P.pool + ((static_cast<size_t>(pid) * P.hkv + c.ip.kv_head) * kPage + (nvalid - 1)) * D)[lane] = val;
+        }
+        __syncwarp();
+      }
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         const int r = 4 * i + kg;
@@ -508,6 +539,7 @@ __device__ __forceinline__ void attend_worker(const Params& P, WarpCtx<D>* ctx, 
   }
   // ---- this layer's inputs; the rest of the first tiles; the second item's context while they fly
   begin_queries<D>(ctx[0], P, first, lane);
+  begin_new_rows(ctx[0].ip, P, first, lane, D);
   fill_ring<D, kRing, false>(st, ctx_of, ring, full, P, lane);
   if (STATIC) record_row_slots(P, first, lane);
   if (!STATIC) issued = claim_issue(P, lane);
@@ -515,6 +547,7 @@ __device__ __forceinline__ void attend_worker(const Params& P, WarpCtx<D>* ctx, 
   if (more) {
     begin_item_pages(ctx[1].ip, P, it, lane);
     begin_queries<D>(ctx[1], P, it, lane);
+    begin_new_rows(ctx[1].ip, P, it, lane, D);
     if (STATIC) record_row_slots(P, it, lane);
   }
   cp_async_wait_all();
@@ -533,6 +566,7 @@ __device__ __forceinline__ void attend_worker(const Params& P, WarpCtx<D>* ctx, 
       if (more) {
         begin_item_pages(ctx[(k + 2) % kCtxSlots].ip, P, it, lane);
         begin_queries<D>(ctx[(k + 2) % kCtxSlots], P, it, lane);
+        begin_new_rows(ctx[(k + 2) % kCtxSlots].ip, P, it, lane, D);
         if (STATIC) record_row_slots(P, it, lane);
         pending = true;
       }

@@ -121,6 +121,7 @@ struct qc_cache {
   int slots_per_stream = 0;
   int static_partition = -1;      // -1: static ranges when a step is several launches; 0 never; 1 always
   bool fused_merge = false;       // the worker that delivers an output row's last partial merges it (no merge launch)
+  bool fold_append = true;        // in-order schedule: new rows are taken and stored by the layer's own launch
   bool plan_ahead = true;         // one kernel per step works out where every worker of every launch starts
   int static_row_cost = 4;        // tiles a row counts for besides its pages (a worker's cost of one more item)
   int static_min_tiles = 6;       // a static range is at least this long when the launch has the work for it
@@ -1356,7 +1357,11 @@ int decode_step_core(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, const 
   p.inline_seqs = inline_step ? 1 : 0;
   // the append reads the page table (not beside its patches) and every layer's k/v (not before
   // the host pipe has copied them)
-  p.fused_append = (n_patches == 0 && !pipe && !open_only) ? 1 : 0;
+  // in-order schedule: nothing of a layer is touched before its own launch (the worker that meets
+  // the end of the layer's text stream takes the new rows from the inputs and stores them)
+  const bool fold = want_per == -2 && c->fold_append;
+  p.fold_append = fold ? 1 : 0;
+  p.fused_append = (n_patches == 0 && !pipe && !open_only && !fold) ? 1 : 0;
 
   // static partition of every launch of the step (part_workers == 0: the launch has nothing to sweep)
   auto partition_of = [&](size_t gi) {
@@ -1415,7 +1420,7 @@ int decode_step_core(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, const 
   }
   QC_CUDA(launch_setup(p, inline_step ? &inl : nullptr, stream));
   c->kernel_launches++;
-  if (!p.fused_append && !pipe && !open_only) {
+  if (!p.fused_append && !pipe && !open_only && !fold) {
     p.layer_begin = 0;
     p.layer_end = N;
     QC_CUDA(launch_append(p, stream));
@@ -1487,8 +1492,8 @@ int32_t qc_decode_layer(qc_cache* c, int32_t layer, const void* q_dev, const voi
   p.lse = lse_out_dev ? reinterpret_cast<float*>(reinterpret_cast<uintptr_t>(lse_out_dev) -
                                                   static_cast<uintptr_t>(layer) * p.n_seqs * c->hq * sizeof(float))
                       : nullptr;
-  const int st = run_group(c, p, static_cast<size_t>(layer), o.launches, o.use_static, o.tot_v, o.tot_t, true, nullptr,
-                           nullptr, nullptr, c->ctx->stream);
+  const int st = run_group(c, p, static_cast<size_t>(layer), o.launches, o.use_static, o.tot_v, o.tot_t,
+                           !p.fold_append, nullptr, nullptr, nullptr, c->ctx->stream);
   if (st != QC_OK) return st;
   if (++o.next_layer == c->cfg.n_layers) {
     o.active = false;
@@ -1713,6 +1718,10 @@ int32_t qc_set_option(qc_cache* c, const char* key, int64_t value) {
   }
   if (k == "debug_drop_tile") {   // test hook, see qc.h
     c->debug_drop_tile = value != 0;
+    return QC_OK;
+  }
+  if (k == "fold_append") {
+    c->fold_append = value != 0;
     return QC_OK;
   }
   if (k == "plan_ahead") {

@@ -17,6 +17,7 @@ from paper_2602_01901_b200 import binding as qc
 from paper_2602_01901_b200 import workloads as W
 from paper_2602_01901_b200.session import Session, bits_of
 
+from oracle.lazy_attention import leaders_of as pg_leaders
 from parity_util import MAX_ABS, REL_L2, SampledOracle, assert_close, f64, full_oracle, step_schedule
 
 pytestmark = pytest.mark.gpu
@@ -255,6 +256,7 @@ SCHEDULES = {
     "in_order_claimed_items": [("in_order_launches", 1), ("static_partition", 0)],
     "in_order_short_ranges": [("in_order_launches", 1), ("static_min_tiles", 1), ("static_row_cost", 0)],
     "in_order_costly_rows": [("in_order_launches", 1), ("static_row_cost", 5)],
+    "in_order_append_at_step_start": [("in_order_launches", 1), ("fold_append", 0)],
     "in_order_merge_in_kernel": [("in_order_launches", 1), ("fused_merge", 1)],
     "one_launch_merge_in_kernel": [("fused_merge", 1)],
 }
@@ -298,6 +300,16 @@ def test_schedules_against_the_oracle(mode, case, schedule):
             for l in range(w.n_layers):
                 assert_close(got[l, b], ref[l], f"{schedule}: case {case} step {step} seq {b} layer {l}")
             np.testing.assert_allclose(got_lse[:, b], ref_lse, atol=2e-3, rtol=0)
+    # what the last step left in the cache, whichever launch stored it: the new rows and the Q Cache, bit for bit
+    leaders = pg_leaders(layer_kind)
+    for b, sid in enumerate(seq_ids):
+        _, n_text, _ = s.page_table(0, qc.QC_STREAM_V_TEXT, sid)
+        for l in range(w.n_layers):
+            assert np.array_equal(s.read_row(l, qc.QC_STREAM_V_TEXT, sid, n_text - 1, 1), vn[l, b, 1])
+            owner = l if (layer_kind[l] == 0 or mode != qc.QC_MODE_GLA) else leaders[l]
+            assert np.array_equal(s.read_row(l, qc.QC_STREAM_K_TEXT, sid, n_text - 1, 1), kn[owner, b, 1])
+            if layer_kind[l]:
+                assert np.array_equal(s.read_qcache(l)[sid], qn[leaders[l], b])
     assert s.stats().device_error == 0
     s.close()
 
