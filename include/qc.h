@@ -220,8 +220,9 @@ int32_t qc_decode_step(qc_cache* cache, int32_t n_seqs, const int32_t* seq_ids, 
  * calls of qc_decode_layer follow, for layer 0, 1, ... in order, each with that layer's slices
  *   q_dev bf16 [n_seqs][n_q_heads][head_dim], k_dev / v_dev bf16 [n_seqs][n_kv_heads][head_dim],
  *   out_dev bf16 [n_seqs][n_q_heads][head_dim], lse_out_dev optional fp32 [n_seqs][n_q_heads].
- * A call appends the layer's k/v (and refreshes the Q Cache from an ordinary layer's q), runs the
- * layer's attention launch and its merge, asynchronously; out_dev is complete when the stream
+ * A call appends the layer's k/v (and refreshes the Q Cache from an ordinary layer's q) and runs the
+ * layer's attention launch and its merge, asynchronously (the append is part of the attention
+ * launch: no launch of its own); out_dev is complete when the stream
  * has executed the call.  The launches are those of the in-order schedule ("in_order_launches"):
  * a leader's call also weights its followers' cached V rows, so a follower's call is short (VLA_QC:
  * its text sweep; GLA: the merge with the new token as one more key; k_dev of a GLA follower is
@@ -297,6 +298,9 @@ int32_t qc_debug_read_row(qc_cache* cache, int32_t layer, int32_t stream, int32_
  * for, in 4 KiB tiles), "plan_ahead" (0 = workers locate their ranges themselves instead of reading
  * starting points that one kernel per step works out for every launch), "fused_merge" (1 = the
  * worker that delivers an output row's last partial merges it, instead of a merge launch),
+ * "fold_append" (in-order schedule and qc_decode_layer; 1, the default = a layer's new k/v rows and an
+ * ordinary layer's q are taken from the inputs and stored by that layer's own launch; 0 = by an
+ * append when the step begins, resp. an append launch per layer call),
  * "debug_drop_tile" (test hook for the error path: 1 = every worker of an attention launch leaves
  * out the copy of its first tile and waits for it with a short limit; nothing is in flight for that
  * wait, so it runs out, the worker records QC_ERR_TIMEOUT and returns, and the kernel ends normally
