@@ -106,6 +106,7 @@ __device__ __forceinline__ void process_item_tc(WorkerState& st, const TcCtx* ct
     }
   }
 
+  const int new_pg = holds_new_token(P, it, n_pages - 1) ? n_pages - 1 : -1;   // folded append: page of the new token
   for (int pg = 0; pg < n_pages && !st.dead; ++pg) {
     const int nvalid = (pg == n_pages - 1) ? n_valid_last : kPage;
     uint32_t pb[NQ][2];
@@ -125,7 +126,7 @@ __device__ __forceinline__ void process_item_tc(WorkerState& st, const TcCtx* ct
       } else {
         const uint32_t tile = wait_tile<D>(st, ring, full, P, lane);
         if (st.dead) break;
-        if (holds_new_token(P, it, pg)) {
+        if (pg == new_pg) {
           // the new token's k row comes from the step's input: into the (swizzled) tile, and into the pool
           const ItemPages& ip = ctx[st.cons_k % kCtxSlots].ip;
           if (lane < D / 8) {
@@ -229,7 +230,7 @@ __device__ __forceinline__ void process_item_tc(WorkerState& st, const TcCtx* ct
       if (st.dead) break;
       const bool skipping = SKIP && skip_page && ((skip_mask >> v) & 1u);
       const int nvalid_v = skipping ? nvalid - 1 : nvalid;
-      if (!skipping && holds_new_token(P, it, pg)) {
+      if (pg == new_pg && !skipping) {
         // this consumer's new v row, likewise
         const ItemPages& ip = ctx[st.cons_k % kCtxSlots].ip;
         if (lane < D / 8) {
@@ -335,7 +336,8 @@ __device__ __forceinline__ void attend_tc_worker(const Params& P, TcCtx* ctx, ui
   };
   // ---- ahead of the wait for the previous kernel: the first items and their page ids (from the
   // launch plan, the step descriptors and the page tables, all written before that kernel
-  // started), and the first tiles unless they could hold the step's new token
+  // started), and the first tiles unless they could hold a new token that an earlier launch of the
+  // step stores (with the folded append the worker patches the new token's row itself)
   Item first;
   if (STATIC && P.wdesc != nullptr) {
     // planned ahead: one read gives the first item, its first page ids and the cursor
@@ -343,7 +345,7 @@ __device__ __forceinline__ void attend_tc_worker(const Params& P, TcCtx* ctx, ui
     if (!load_worker_desc(P, wid, ctx[0].ip, cursor, stage, lane)) return;
     first = ctx[0].ip.item;
     st.n_my = 1;
-    const bool early_tiles = !(first.stream == 0 && (first.flags & kFlagStreamEnd) && first.n_pages <= kRingTc);
+    const bool early_tiles = P.fold_append || !(first.stream == 0 && (first.flags & kFlagStreamEnd) && first.n_pages <= kRingTc);
     if (early_tiles) fill_ring<D, kRingTc, true>(st, ctx_of, ring, full, P, lane);
     begin_item_pages(ctx[0].ip, P, first, lane);   // the whole page list, while the tiles fly
   } else {
@@ -365,7 +367,7 @@ __device__ __forceinline__ void attend_tc_worker(const Params& P, TcCtx* ctx, ui
     cp_async_wait_all();
     __syncwarp();
     st.n_my = 1;
-    const bool early_tiles = !(first.stream == 0 && (first.flags & kFlagStreamEnd) && first.n_pages <= kRingTc);
+    const bool early_tiles = P.fold_append || !(first.stream == 0 && (first.flags & kFlagStreamEnd) && first.n_pages <= kRingTc);
     if (early_tiles) fill_ring<D, kRingTc, true>(st, ctx_of, ring, full, P, lane);
   }
   if (STATIC) {

@@ -302,6 +302,7 @@ __device__ __forceinline__ void process_item(WorkerState& st, const WarpCtx<D>* 
     }
   }
 
+  const int new_pg = holds_new_token(P, c.ip.item, n_pages - 1) ? n_pages - 1 : -1;   // folded append: page of the new token
   for (int pg = 0; pg < n_pages && !st.dead; ++pg) {
     const int nvalid = (pg == n_pages - 1) ? n_valid_last : kPage;
     float p[NQ][4];
@@ -317,7 +318,7 @@ __device__ __forceinline__ void process_item(WorkerState& st, const WarpCtx<D>* 
       // ---- K tile: scores of 16 keys
       const uint8_t* tile = static_cast<const uint8_t*>(__cvta_shared_to_generic(wait_tile<D>(st, ring, full, P, lane)));
       if (st.dead) break;
-      if (holds_new_token(P, c.ip.item, pg)) {
+      if (pg == new_pg) {
         // the new token's k row comes from the step's input: into the tile, and into the pool for later steps
         const Item& it = c.ip.item;
         if (lane < D / 8) {
@@ -406,7 +407,7 @@ __device__ __forceinline__ void process_item(WorkerState& st, const WarpCtx<D>* 
       const uint8_t* tile = static_cast<const uint8_t*>(__cvta_shared_to_generic(wait_tile<D>(st, ring, full, P, lane)));
       if (st.dead) break;
       const int nvalid_v = (SKIP && skip_here && pg == n_pages - 1) ? nvalid - static_cast<int>((skip_mask >> v) & 1u) : nvalid;
-      if (nvalid_v == nvalid && holds_new_token(P, c.ip.item, pg)) {
+      if (pg == new_pg && nvalid_v == nvalid) {
         // this consumer's new v row, likewise
         const Item& it = c.ip.item;
         if (lane < D / 8) {
@@ -500,7 +501,8 @@ __device__ __forceinline__ void attend_worker(const Params& P, WarpCtx<D>* ctx, 
   };
   // ---- ahead of the wait for the previous kernel: the first items and their page ids (from the
   // launch plan, the step descriptors and the page tables, all written before that kernel
-  // started), and the first tiles unless they could hold the step's new token
+  // started), and the first tiles unless they could hold a new token that an earlier launch of the
+  // step stores (with the folded append the worker patches the new token's row itself)
   Item first;
   if (STATIC && P.wdesc != nullptr) {
     // planned ahead: one read gives the first item, its first page ids and the cursor
@@ -508,7 +510,7 @@ __device__ __forceinline__ void attend_worker(const Params& P, WarpCtx<D>* ctx, 
     if (!load_worker_desc(P, wid, ctx[0].ip, cursor, stage, lane)) return;
     first = ctx[0].ip.item;
     st.n_my = 1;
-    const bool early_tiles = !(first.stream == 0 && (first.flags & kFlagStreamEnd) && first.n_pages <= kRing);
+    const bool early_tiles = P.fold_append || !(first.stream == 0 && (first.flags & kFlagStreamEnd) && first.n_pages <= kRing);
     if (early_tiles) fill_ring<D, kRing, false>(st, ctx_of, ring, full, P, lane);
     begin_item_pages(ctx[0].ip, P, first, lane);   // the whole page list, while the tiles fly
   } else {
@@ -530,7 +532,7 @@ __device__ __forceinline__ void attend_worker(const Params& P, WarpCtx<D>* ctx, 
     cp_async_wait_all();
     __syncwarp();
     st.n_my = 1;
-    const bool early_tiles = !(first.stream == 0 && (first.flags & kFlagStreamEnd) && first.n_pages <= kRing);
+    const bool early_tiles = P.fold_append || !(first.stream == 0 && (first.flags & kFlagStreamEnd) && first.n_pages <= kRing);
     if (early_tiles) fill_ring<D, kRing, false>(st, ctx_of, ring, full, P, lane);
   }
   if (STATIC) {
