@@ -47,7 +47,13 @@ __device__ __forceinline__ uint32_t swz(int row, int chunk) {
 // SKIP (shared weights only): the consumers named in the item's skip_new mask leave out the
 // stream's last key (the step's new token): they get a copy of the weights with that key's set
 // to zero and their own sums.
-template <int D, int NQ, int NV, int MODE = 0, bool SKIP = false>
+// FOLD: the item may end its layer's text stream under the folded append (the new token's rows come
+// from the step's inputs).  Launches without the folded append use the instantiation without it,
+// whose page loop then carries none of this (with it in every instantiation the one-launch step was
+// 3.5 % slower); under the folded append every single-consumer item of a launch takes this one
+// (sending only the items that end a stream here made the workers alternate between two copies of
+// the loop: 1.20 against 1.09 ms per step at config 2).
+template <int D, int NQ, int NV, int MODE = 0, bool SKIP = false, bool FOLD = false>
 __device__ __forceinline__ void process_item_tc(WorkerState& st, const TcCtx* ctx, uint32_t ring, uint64_t* full,
                                                 const Params& P, int lane) {
   constexpr int KS = D / 16;    // k-steps of the score product = m-tiles of the value product
@@ -106,7 +112,8 @@ __device__ __forceinline__ void process_item_tc(WorkerState& st, const TcCtx* ct
     }
   }
 
-  const int new_pg = holds_new_token(P, it, n_pages - 1) ? n_pages - 1 : -1;   // folded append: page of the new token
+  constexpr bool kMayFold = FOLD || SKIP;
+  const int new_pg = (kMayFold && holds_new_token(P, it, n_pages - 1)) ? n_pages - 1 : -1;   // folded append: page of the new token
   for (int pg = 0; pg < n_pages && !st.dead; ++pg) {
     const int nvalid = (pg == n_pages - 1) ? n_valid_last : kPage;
     uint32_t pb[NQ][2];
@@ -126,7 +133,7 @@ __device__ __forceinline__ void process_item_tc(WorkerState& st, const TcCtx* ct
       } else {
         const uint32_t tile = wait_tile<D>(st, ring, full, P, lane);
         if (st.dead) break;
-        if (pg == new_pg) {
+        if (kMayFold && pg == new_pg) {
           // the new token's k row comes from the step's input: into the (swizzled) tile, and into the pool
           const ItemPages& ip = ctx[st.cons_k % kCtxSlots].ip;
           if (lane < D / 8) {
@@ -230,7 +237,7 @@ __device__ __forceinline__ void process_item_tc(WorkerState& st, const TcCtx* ct
       if (st.dead) break;
       const bool skipping = SKIP && skip_page && ((skip_mask >> v) & 1u);
       const int nvalid_v = skipping ? nvalid - 1 : nvalid;
-      if (pg == new_pg && !skipping) {
+      if (kMayFold && pg == new_pg && !skipping) {
         // this consumer's new v row, likewise
         const ItemPages& ip = ctx[st.cons_k % kCtxSlots].ip;
         if (lane < D / 8) {
@@ -414,6 +421,7 @@ __device__ __forceinline__ void attend_tc_worker(const Params& P, TcCtx* ctx, ui
       else if (nc == 3) process_item_tc<D, 1, 3, 0, true>(st, ctx, ring, full, P, lane);
       else process_item_tc<D, 1, 4, 0, true>(st, ctx, ring, full, P, lane);
     }
+    else if (nc == 1 && P.fold_append) process_item_tc<D, 1, 1, 0, false, true>(st, ctx, ring, full, P, lane);   // (one code path per launch)
     else if (nc == 1) process_item_tc<D, 1, 1>(st, ctx, ring, full, P, lane);
     else if (shared && nc == 2) process_item_tc<D, 1, 2>(st, ctx, ring, full, P, lane);
     else if (shared && nc == 3) process_item_tc<D, 1, 3>(st, ctx, ring, full, P, lane);

@@ -253,7 +253,13 @@ __device__ __forceinline__ void begin_queries(WarpCtx<D>& c, const Params& P, co
 // SKIP (shared weights only): the consumers named in the item's skip_new mask leave out the
 // stream's last key -- the step's new token, whose value row of a follower does not exist yet when
 // its leader's launch runs (Eq. 6: V = [cached V, new v]); they get their own sum of weights.
-template <int D, int NQ, int NV, int MODE = 0, bool SKIP = false>
+// FOLD: the item may end its layer's text stream under the folded append (the new token's rows come
+// from the step's inputs).  Launches without the folded append use the instantiation without it,
+// whose page loop then carries none of this (with it in every instantiation the one-launch step was
+// 3.5 % slower); under the folded append every single-consumer item of a launch takes this one
+// (sending only the items that end a stream here made the workers alternate between two copies of
+// the loop: 1.20 against 1.09 ms per step at config 2).
+template <int D, int NQ, int NV, int MODE = 0, bool SKIP = false, bool FOLD = false>
 __device__ __forceinline__ void process_item(WorkerState& st, const WarpCtx<D>* ctx, uint32_t ring, uint64_t* full,
                                              const Params& P, int lane) {
   auto ctx_of = [ctx](int k) -> const ItemPages& { return ctx[k % kCtxSlots].ip; };
@@ -302,7 +308,8 @@ __device__ __forceinline__ void process_item(WorkerState& st, const WarpCtx<D>* 
     }
   }
 
-  const int new_pg = holds_new_token(P, c.ip.item, n_pages - 1) ? n_pages - 1 : -1;   // folded append: page of the new token
+  constexpr bool kMayFold = FOLD || SKIP;
+  const int new_pg = (kMayFold && holds_new_token(P, c.ip.item, n_pages - 1)) ? n_pages - 1 : -1;   // folded append: page of the new token
   for (int pg = 0; pg < n_pages && !st.dead; ++pg) {
     const int nvalid = (pg == n_pages - 1) ? n_valid_last : kPage;
     float p[NQ][4];
@@ -318,7 +325,7 @@ __device__ __forceinline__ void process_item(WorkerState& st, const WarpCtx<D>* 
       // ---- K tile: scores of 16 keys
       const uint8_t* tile = static_cast<const uint8_t*>(__cvta_shared_to_generic(wait_tile<D>(st, ring, full, P, lane)));
       if (st.dead) break;
-      if (pg == new_pg) {
+      if (kMayFold && pg == new_pg) {
         // the new token's k row comes from the step's input: into the tile, and into the pool for later steps
         const Item& it = c.ip.item;
         if (lane < D / 8) {
@@ -407,7 +414,7 @@ __device__ __forceinline__ void process_item(WorkerState& st, const WarpCtx<D>* 
       const uint8_t* tile = static_cast<const uint8_t*>(__cvta_shared_to_generic(wait_tile<D>(st, ring, full, P, lane)));
       if (st.dead) break;
       const int nvalid_v = (SKIP && skip_here && pg == n_pages - 1) ? nvalid - static_cast<int>((skip_mask >> v) & 1u) : nvalid;
-      if (pg == new_pg && nvalid_v == nvalid) {
+      if (kMayFold && pg == new_pg && nvalid_v == nvalid) {
         // this consumer's new v row, likewise
         const Item& it = c.ip.item;
         if (lane < D / 8) {
@@ -582,6 +589,7 @@ __device__ __forceinline__ void attend_worker(const Params& P, WarpCtx<D>* ctx, 
       else if (nc == 3) process_item<D, 1, 3, 0, true>(st, ctx, ring, full, P, lane);
       else process_item<D, 1, 4, 0, true>(st, ctx, ring, full, P, lane);
     }
+    else if (nc == 1 && P.fold_append) process_item<D, 1, 1, 0, false, true>(st, ctx, ring, full, P, lane);   // (one code path per launch)
     else if (nc == 1) process_item<D, 1, 1>(st, ctx, ring, full, P, lane);
     else if (shared && nc == 2) process_item<D, 1, 2>(st, ctx, ring, full, P, lane);
     else if (shared && nc == 3) process_item<D, 1, 3>(st, ctx, ring, full, P, lane);
