@@ -533,6 +533,9 @@ def run_prefill(args, w, mode, local_rank):
     s = Session.for_workload(w, lazy_mode=mode, device=local_rank)
     s.set_option("prefill_tcgen05", 1 if args.prefill_kernel == "tcgen05" else 0)
     s.set_option("prefill_shared_scores", 0 if args.no_prefill_sharing else 1)
+    for kv in args.option:
+        key, _, val = kv.partition("=")
+        s.set_option(key, int(val))
     n_seqs = min(w.batch, max(4, args.warmup + 1))
     prompts = []
     for b in range(n_seqs):

@@ -286,6 +286,8 @@ int32_t qc_debug_read_row(qc_cache* cache, int32_t layer, int32_t stream, int32_
  * normalises their scores once per run of up to three layers and applies them to each layer's V,
  * bit-identically to one pass per layer; 0 = never, 1 = for prompts of 1536 tokens or more (the
  * default: below that the pass's lower occupancy costs more than it saves), 2 = always),
+ * "prefill_pair_min_tokens" (n > 0: prompts of n tokens or more that start a sequence run on the
+ * prefill kernel with two query tiles per CTA and 128-key tiles; 0, the default: never),
  * "profile" (1 = record CUDA events per step; 2 = also around every attention launch), "in_order_launches"
  * (1 = one launch per layer in layer order, each using nothing of later layers; what a follower
  * shares with its leader are scores over rows cached before the step, so a leader's launch also

@@ -204,7 +204,7 @@ cudaError_t launch_prefill_attend(const Params& p, const uint8_t* kind_dev, cons
                                   int32_t n_tokens, int32_t gla, const PrefillMaps* maps,
                                   const uint8_t* tile_code_dev, int32_t seq_id, int32_t n0_text, int32_t n0_vis,
                                   const PrefillPass* passes_dev, int32_t n_single, int32_t n_shared,
-                                  cudaStream_t stream);   // qc_prefill.cu; maps null or head_dim 64 = mma.sync kernel
+                                  int32_t pair_min_tokens, cudaStream_t stream);   // qc_prefill.cu; maps null or head_dim 64 = mma.sync kernel
 cudaError_t configure_prefill_kernels();
 cudaError_t launch_calibration(const Params& p, const int32_t* seq_ids_dev, const int32_t* len_text_dev,
                                const int32_t* len_vis_dev, float* rows_dev, int32_t max_len, float* js_dev,

@@ -1045,6 +1045,421 @@ __global__ void __launch_bounds__(NV > 1 ? kTc5Threads + 32 : kTc5Threads, NV > 
   }
 }
 
+// ------------------------------------------------------------------------------------------
+// Two query tiles per CTA, key tiles of 128 tokens
+// ------------------------------------------------------------------------------------------
+//
+// For prompts that start a sequence.  One CTA = 256 query rows (two tiles of 128) of one (layer,
+// query head), alone on its SM with all 512 columns of tensor memory: per query tile t one score
+// buffer S_t[128 x 128] and one accumulator O_t[128 x 128].  Per 128-key tile and query tile:
+//     S_t = Q_t . K^T     8 x tcgen05.mma (M 128, N 128, K 16)
+//     O_t += P_t . V      2 x 4 tcgen05.mma (M 128, N 128, K 16), P_t (bf16) read from the first 64 columns of S_t
+// so a key costs half as many products, barrier round trips and tensor-memory transfers as with
+// 64-key tiles, and a score product reads 8 KiB of shared memory for 64 cycles of arithmetic
+// instead of 6 KiB for 32.  The two query tiles alternate on the tensor core: while the 128
+// softmax threads of one tile work, the products of the other tile run.
+// Warps 0-3 / 4-7: softmax of query tile 0 / 1, one thread per row.  Warp 8 issues the score
+// products, warp 9 the value products, warp 10 fetches (warps 8-11 give registers to the others).  Hand-offs (mbarriers, all waits bounded):
+//   bar_q[t]            copies -> warp 8          query tile t landed
+//   bar_k[b], bar_v[b]  copies -> warps 8 / 9     K / V tile landed in buffer b
+//   bar_s[t]            tensor core -> softmax t  S_t(kt) complete
+//   bar_p[t], bar_pb[t] softmax t -> warp 9       the weights P_t(kt) of keys 0..63 / 64..127 are written
+//   bar_o[t]            tensor core -> warp 8, softmax t    PV_t(kt) complete: S_t may be overwritten, O_t rescaled
+//   bar_kf[b], bar_vf[b]  tensor core -> warp 10  both tiles' products on buffer b are complete
+// No barrier can run two completions ahead of a waiter: each next completion needs something the
+// waiter produces after it has seen the previous one.
+constexpr int kPN = 128;                             // keys per tile
+constexpr int kPairThreads = 2 * kTM + 4 * 32;   // warp 11 only completes the warpgroup whose registers are handed over
+constexpr uint32_t kPairQT = 2 * kTM * 128;          // one query tile: two 64-column halves of 128 rows
+constexpr uint32_t kPairKT = 2 * kPN * 128;          // one key or value tile
+constexpr uint32_t kPairHalf = kPN * 128;            // distance between the two column halves of a tile (kTM == kPN)
+constexpr uint32_t kPairTiles = 2 * kPairQT + 4 * kPairKT;
+constexpr int prefill_pair_smem_bytes() { return kPairTiles + 176; }
+
+__global__ void __launch_bounds__(kPairThreads, 1)
+    prefill_attend_pair_kernel(const __grid_constant__ PrefillArgs A, int32_t* err) {
+  extern __shared__ __align__(1024) uint8_t smem_dyn[];
+  const uint32_t base = smem_u32(smem_dyn);
+  const uint32_t sQ = base, sK = sQ + 2 * kPairQT, sV = sK + 2 * kPairKT;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem_dyn + kPairTiles);
+  uint64_t *bar_q = bars, *bar_k = bars + 2, *bar_v = bars + 4, *bar_s = bars + 6, *bar_p = bars + 8, *bar_o = bars + 10,
+           *bar_kf = bars + 12, *bar_vf = bars + 14, *bar_pb = bars + 16;
+  uint32_t& tmem_base_slot = *reinterpret_cast<uint32_t*>(smem_dyn + kPairTiles + 144);
+  volatile int32_t& failed = *reinterpret_cast<volatile int32_t*>(smem_dyn + kPairTiles + 148);
+  if (base & 1023u) {   // cannot happen with the layout above; never run the tensor core on a misplaced tile
+    if (threadIdx.x == 0) atomicMax(err, kErrBadPage);
+    return;
+  }
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n_pairs = (A.T + 2 * kTM - 1) / (2 * kTM);
+  const int qp = n_pairs - 1 - blockIdx.x;          // long rows first
+  const int head = blockIdx.y;
+  const int layer = A.passes ? A.passes[blockIdx.z].v[0] : static_cast<int>(blockIdx.z);
+  const int kvh = head / A.group;
+  const bool lazy = A.layer_kind[layer] != 0;
+  const int lead = A.leader[layer];
+  const bool gla = A.gla != 0;
+  // query tile t covers rows (2 qp + t) * 128 .. + 127 and sees key tiles 0 .. n_kt<t> - 1
+  const int n_all = (A.T + kPN - 1) / kPN;
+  const int n_kt0 = min(n_all, 2 * qp + 1), n_kt1 = (2 * qp + 1) * kTM < A.T ? min(n_all, 2 * qp + 2) : 0;
+  const int n_ktiles = max(n_kt0, n_kt1);
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&bar_q[i], 2);
+      mbar_init(&bar_k[i], 2);
+      mbar_init(&bar_v[i], 2);
+      mbar_init(&bar_s[i], 1);
+      mbar_init(&bar_p[i], kTM);
+      mbar_init(&bar_pb[i], kTM);
+      mbar_init(&bar_o[i], 1);
+      mbar_init(&bar_kf[i], 1);
+      mbar_init(&bar_vf[i], 1);
+    }
+    fence_mbar_init();
+    failed = 0;
+  }
+  if (warp == 8) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
+                 "r"(512u)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc5_fence_before();
+  __syncthreads();
+  tc5_fence_after();
+  const uint32_t tmem = tmem_base_slot;
+  // tensor memory columns: S_0, S_1, O_0, O_1
+  constexpr uint32_t kIdescS = (1u << 4) | (1u << 7) | (1u << 10) | ((kPN >> 3) << 17) | ((kTM >> 4) << 24);
+  constexpr uint32_t kIdescO = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((kTD >> 3) << 17) | ((kTM >> 4) << 24);
+
+  if (warp >= 8) {
+    // the issuing and fetching warps need few registers; the softmax threads hold a row of 128 scores
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;" ::: "memory");
+    bool ok = true;
+    auto wait_on = [&](uint64_t* bar, uint32_t& phase) {   // warp-uniform bounded wait
+      if (ok && !__all_sync(0xffffffffu, mbar_try_wait(bar, phase)))
+        ok = __all_sync(0xffffffffu, bounded_wait(bar, phase) && !failed);
+      phase ^= 1u;
+    };
+    if (warp == 11) {
+      // nothing
+    } else if (warp == 8) {
+      // ---------------- score products: S_t(kt) once K(kt) has landed and PV_t(kt - 1) is complete
+      const uint64_t qd0 = umma_desc(sQ, 16, 1024), qd1 = umma_desc(sQ + kPairQT, 16, 1024);
+      const uint64_t kd0 = umma_desc(sK, 16, 1024), kd1 = umma_desc(sK + kPairKT, 16, 1024);
+      uint32_t ph_q = 0, ph_k = 0, ph_o = 0;   // bit b / bit t: the phase of barrier b / t
+      auto wait_bit = [&](uint64_t* bar, uint32_t& phases, int i) {
+        uint32_t ph = (phases >> i) & 1u;
+        wait_on(bar, ph);
+        phases ^= 1u << i;
+      };
+      for (int kt = 0; kt < n_ktiles && ok; ++kt) {
+        const int b = kt & 1;
+        wait_bit(&bar_k[b], ph_k, b);
+#pragma unroll
+        for (int t = 0; t < 2; ++t) {
+          if (kt >= (t ? n_kt1 : n_kt0)) continue;
+          if (kt == 0) wait_bit(&bar_q[t], ph_q, t);
+          else wait_bit(&bar_o[t], ph_o, t);
+          if (!ok) break;
+          tc5_fence_after();
+          umma_scores<kPairHalf, kPairHalf>(tmem + t * kPN, t ? qd1 : qd0, b ? kd1 : kd0, kIdescS);
+          umma_commit(&bar_s[t]);
+        }
+        if (ok) umma_commit(&bar_kf[b]);
+      }
+    } else if (warp == 9) {
+      // ---------------- value products: PV_t(kt) once P_t(kt) is written and V(kt) has landed
+      const uint64_t vd0 = umma_desc(sV, kPairHalf, 1024), vd1 = umma_desc(sV + kPairKT, kPairHalf, 1024);
+      uint32_t ph_p = 0, ph_pb = 0, ph_v = 0;
+      auto wait_bit = [&](uint64_t* bar, uint32_t& phases, int i) {
+        uint32_t ph = (phases >> i) & 1u;
+        wait_on(bar, ph);
+        phases ^= 1u << i;
+      };
+      for (int kt = 0; kt < n_ktiles && ok; ++kt) {
+        const int b = kt & 1;
+        bool first = true;
+#pragma unroll
+        for (int t = 0; t < 2; ++t) {
+          if (kt >= (t ? n_kt1 : n_kt0)) continue;
+          wait_bit(&bar_p[t], ph_p, t);
+          if (first) {
+            wait_bit(&bar_v[b], ph_v, b);
+            first = false;
+          }
+          if (!ok) break;
+          tc5_fence_after();
+          umma_values(tmem + 2 * kPN + t * kTD, tmem + t * kPN, b ? vd1 : vd0, kIdescO, kt > 0 ? 1u : 0u);
+          wait_bit(&bar_pb[t], ph_pb, t);   // the weights of keys 64..127
+          if (!ok) break;
+          tc5_fence_after();
+          umma_values(tmem + 2 * kPN + t * kTD, tmem + t * kPN + 32, (b ? vd1 : vd0) + 512, kIdescO, 1u);
+          umma_commit(&bar_o[t]);
+        }
+        if (ok) umma_commit(&bar_vf[b]);
+      }
+    } else {
+      // ---------------- load warp.  64 rows per request: rows of one layer by two tensor-map copies,
+      // a tile mixing text and visual rows of a VLA lazy layer row by row.
+      uint32_t codes[3] = {0u, 0u, 0u};
+      if (lazy && !gla) {
+        const int n_tiles = (A.T + kTN - 1) / kTN;
+#pragma unroll
+        for (int i = 0; i < 3; ++i)
+          if (lane + 32 * i < n_tiles) codes[i] = A.tile_code[lane + 32 * i];
+      }
+      auto code_of = [&](int kt) -> int {   // whole warp
+        if (kt >= 96) return A.tile_code[kt];
+        const uint32_t c = kt < 32 ? codes[0] : (kt < 64 ? codes[1] : codes[2]);
+        return static_cast<int>(__shfl_sync(0xffffffffu, c, kt & 31));
+      };
+      // which: 0 = query rows, 1 = key rows, 2 = value rows; kt64 counts 64-token tiles of the prompt
+      auto fetch64 = [&](int which, int kt64, uint32_t dst, uint64_t* bar) {
+        int src = layer;
+        bool mixed = false;
+        if (which != 2 && lazy && kt64 * kTN < A.T) {
+          if (gla) {
+            src = lead;
+          } else {
+            const int code = code_of(kt64);
+            mixed = code == 2;
+            src = code == 1 ? lead : layer;
+          }
+        }
+        if (!mixed) {
+          if (lane == 0) {
+            const void* tm = which == 0 ? static_cast<const void*>(&A.tmap_q)
+                                        : (which == 1 ? static_cast<const void*>(&A.tmap_k) : static_cast<const void*>(&A.tmap_v));
+            const int h = which == 0 ? head : kvh;
+            mbar_expect_tx(bar, 2 * kTN * 128);
+            tensor_g2s_3d(dst, tm, 0, h, src * A.T + kt64 * kTN, bar);
+            tensor_g2s_3d(dst + kPairHalf, tm, 64, h, src * A.T + kt64 * kTN, bar);
+          }
+        } else {
+          const uint16_t* from = which == 0 ? A.q : A.k;
+          const int heads = which == 0 ? A.hq : A.hkv, h = which == 0 ? head : kvh;
+          for (int e = lane; e < kTN * (kTD / 8); e += 32) {
+            const int r = e >> 4, c = e & 15, t = kt64 * kTN + r;
+            const uint32_t d = dst + (c >> 3) * kPairHalf + r * 128 + (((c & 7) ^ (r & 7)) << 4);
+            if (t < A.T) {
+              const int l = A.kind[t] ? lead : layer;
+              cp_async16(d, from + ((static_cast<size_t>(l) * A.T + t) * heads + h) * kTD + c * 8);
+            } else {
+              asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(d), "r"(0u) : "memory");
+            }
+          }
+          cp_async_commit();
+          cp_async_wait<0>();
+          fence_proxy_async();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar);
+        }
+      };
+      auto fetch128 = [&](int which, int tile, uint32_t dst, uint64_t* bar) {
+        fetch64(which, 2 * tile, dst, bar);
+        fetch64(which, 2 * tile + 1, dst + kTN * 128, bar);
+      };
+      fetch128(0, 2 * qp, sQ, &bar_q[0]);
+      fetch128(1, 0, sK, &bar_k[0]);
+      if (n_kt1 > 0) fetch128(0, 2 * qp + 1, sQ + kPairQT, &bar_q[1]);
+      fetch128(2, 0, sV, &bar_v[0]);
+      if (n_ktiles > 1) {
+        fetch128(1, 1, sK + kPairKT, &bar_k[1]);
+        fetch128(2, 1, sV + kPairKT, &bar_v[1]);
+      }
+      int k_next = 2, v_next = 2;
+      uint32_t ph_kf = 0, ph_vf = 0, idle = 0;   // bit b: the phase of barrier b
+      while ((k_next < n_ktiles || v_next < n_ktiles) && ok) {
+        bool progress = false;
+        if (k_next < n_ktiles) {
+          const int b = k_next & 1;
+          if (__all_sync(0xffffffffu, mbar_test_wait(&bar_kf[b], (ph_kf >> b) & 1u))) {
+            ph_kf ^= 1u << b;
+            fetch128(1, k_next, sK + b * kPairKT, &bar_k[b]);
+            ++k_next;
+            progress = true;
+          }
+        }
+        if (v_next < n_ktiles) {
+          const int b = v_next & 1;
+          if (__all_sync(0xffffffffu, mbar_test_wait(&bar_vf[b], (ph_vf >> b) & 1u))) {
+            ph_vf ^= 1u << b;
+            fetch128(2, v_next, sV + b * kPairKT, &bar_v[b]);
+            ++v_next;
+            progress = true;
+          }
+        }
+        if (progress) {
+          idle = 0;
+        } else if (++idle > (1u << 20) || ((idle & 1023u) == 0 && failed)) {
+          ok = false;
+        }
+      }
+    }
+    if (!ok) failed = 1;
+    __syncwarp();
+  } else {
+    // ------------------------------------------------------------------ softmax threads of query tile t
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 224;" ::: "memory");
+    const int t = warp >> 2, tid = threadIdx.x & (kTM - 1);
+    const int n_mine = t ? n_kt1 : n_kt0;
+    const int m0 = (2 * qp + t) * kTM;
+    const int row = m0 + tid;
+    const uint32_t t_row = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);   // this warp's 32 TMEM lanes
+    const uint32_t cS = t * kPN, cO = 2 * kPN + t * kTD;
+    float m_ref = -INFINITY, l_sum = 0.f;
+    uint32_t ph_s = 0;
+    bool ok = true;
+    // The two tiles take turns at the softmax arithmetic (named barriers 3 + t: tile t may start its
+    // iteration kt once the other tile has finished the iteration before it in the order (0, 0),
+    // (1, 0), (0, 1), (1, 1), ...), so that one tile's exponentials run while the other tile's
+    // products do; left to themselves both tiles' scores complete together and the tensor core idles
+    // while both compute.  A tile with no predecessor left does not wait.
+    const int n_other = t ? n_kt0 : n_kt1;
+    auto pass_turn = [&]() {
+      if (t == 0) asm volatile("bar.arrive 4, %0;" ::"n"(2 * kTM) : "memory");
+      else asm volatile("bar.arrive 3, %0;" ::"n"(2 * kTM) : "memory");
+    };
+    for (int kt = 0; kt < n_mine; ++kt) {
+      if (failed) { ok = false; break; }
+      if (!__all_sync(0xffffffffu, mbar_try_wait(&bar_s[t], ph_s))) {
+        ok = bounded_wait(&bar_s[t], ph_s) && !failed;
+        if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+      }
+      ph_s ^= 1u;
+      if (t == 0) {
+        if (kt > 0 && n_other > 0) asm volatile("bar.sync 3, %0;" ::"n"(2 * kTM) : "memory");
+      } else {
+        if (kt < n_other) asm volatile("bar.sync 4, %0;" ::"n"(2 * kTM) : "memory");
+      }
+      tc5_fence_after();
+      float p[kPN];
+      {
+        uint32_t r0[32], r1[32], r2[32], r3[32];
+        tmem_ld32_nowait(t_row + cS, r0);
+        tmem_ld32_nowait(t_row + cS + 32, r1);
+        tmem_ld32_nowait(t_row + cS + 64, r2);
+        tmem_ld32_nowait(t_row + cS + 96, r3);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          p[j] = __uint_as_float(r0[j]), p[32 + j] = __uint_as_float(r1[j]);
+          p[64 + j] = __uint_as_float(r2[j]), p[96 + j] = __uint_as_float(r3[j]);
+        }
+      }
+      const int n0 = kt * kPN;
+      if (n0 + kPN - 1 > m0 || n0 + kPN > A.T) {   // only tiles on the diagonal or at the end of the prompt need the mask
+#pragma unroll
+        for (int j = 0; j < kPN; ++j) {
+          const int key = n0 + j;
+          if (!(key <= row && key < A.T)) p[j] = -INFINITY;
+        }
+      }
+      float mx[4] = {p[0], p[1], p[2], p[3]};
+#pragma unroll
+      for (int j = 4; j < kPN; ++j) mx[j & 3] = fmaxf(mx[j & 3], p[j]);
+      const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * A.scale_log2;   // the scale is positive
+      float corr = 1.f;
+      if (m_tile > m_ref + kRescaleThreshold || m_ref == -INFINITY) {
+        if (m_tile != -INFINITY) {
+          corr = exp2f(m_ref - m_tile);     // 0 on the first tile
+          m_ref = m_tile;
+        }
+      }
+      const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
+      if (kt > 0 && __any_sync(0xffffffffu, corr != 1.f)) {   // rare: move the accumulator to the new reference
+        ok = bounded_wait(&bar_o[t], static_cast<uint32_t>(kt - 1) & 1u) && !failed;   // PV_t(kt - 1) complete
+        if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+        tc5_fence_after();
+#pragma unroll
+        for (int c = 0; c < kTD / 32; ++c) {
+          uint32_t r[32];
+          tmem_ld32(t_row + cO + 32 * c, r);
+#pragma unroll
+          for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * corr);
+          tmem_st32(t_row + cO + 32 * c, r);
+        }
+        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+      }
+      // ---- weights as the A operand, in place of the scores just read: 128 bf16 = 64 columns of this row's
+      // lane, handed over in two halves so that the value products of keys 0..63 run during the
+      // exponentials of keys 64..127
+      float ps[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+#pragma unroll
+        for (int j = 64 * h; j < 64 * h + 64; ++j) {
+          p[j] = ex2_approx(fmaf(p[j], A.scale_log2, neg_m));
+          ps[j & 3] += p[j];
+        }
+        if (h == 1 && (t == 0 ? n_other > 0 : kt + 1 < n_other)) pass_turn();   // the other tile's next iteration may start
+        uint32_t w[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) w[j] = pack_bf16x2(p[64 * h + 2 * j], p[64 * h + 2 * j + 1]);
+        tmem_st32(t_row + cS + 32 * h, w);
+        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+        tc5_fence_before();
+        mbar_arrive(h ? &bar_pb[t] : &bar_p[t]);
+      }
+      l_sum = l_sum * corr + ((ps[0] + ps[1]) + (ps[2] + ps[3]));
+    }
+    if (!ok) {   // leaving early: the other tile must not wait for this one's turn
+      failed = 1;
+      __threadfence_block();
+      pass_turn();
+    }
+    if (n_mine > 0) {
+      if (ok) ok = bounded_wait(&bar_o[t], static_cast<uint32_t>(n_mine - 1) & 1u) && !failed;   // the last value product
+      ok = __all_sync(0xffffffffu, ok);
+      if (ok) {
+        // scale the accumulator and put the tile into query tile t's shared memory (free: every product
+        // of the tile has completed) in the swizzled layout of a 128-row box; two tensor-map stores
+        tc5_fence_after();
+        const float inv = 1.f / l_sum;
+        const uint32_t sQt = sQ + t * kPairQT;
+        const uint32_t orow = sQt + tid * 128;
+        const uint32_t sw = tid & 7;
+#pragma unroll
+        for (int c = 0; c < kTD / 32; ++c) {
+          uint32_t r[32];
+          tmem_ld32(t_row + cO + 32 * c, r);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int chunk = 4 * c + j;   // 16-byte chunk of the 256-byte row
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(orow + (chunk >> 3) * kPairHalf + (((chunk & 7) ^ sw) << 4)),
+                         "r"(pack_bf16x2(__uint_as_float(r[8 * j + 0]) * inv, __uint_as_float(r[8 * j + 1]) * inv)),
+                         "r"(pack_bf16x2(__uint_as_float(r[8 * j + 2]) * inv, __uint_as_float(r[8 * j + 3]) * inv)),
+                         "r"(pack_bf16x2(__uint_as_float(r[8 * j + 4]) * inv, __uint_as_float(r[8 * j + 5]) * inv)),
+                         "r"(pack_bf16x2(__uint_as_float(r[8 * j + 6]) * inv, __uint_as_float(r[8 * j + 7]) * inv))
+                         : "memory");
+          }
+        }
+        fence_proxy_async();
+        if (t == 0) asm volatile("bar.sync 1, %0;" ::"n"(kTM) : "memory");   // the tile's 128 softmax threads
+        else asm volatile("bar.sync 2, %0;" ::"n"(kTM) : "memory");
+        if (tid == 0) {
+          tensor_s2g_4d(&A.tmap_o, sQt, 0, head, m0, layer);
+          tensor_s2g_4d(&A.tmap_o, sQt + kPairHalf, 64, head, m0, layer);
+          asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+          asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // shared memory is released at exit
+        }
+      } else {
+        failed = 1;
+        if (lane == 0) atomicMax(err, kErrTimeout);
+        if (t == 0) asm volatile("bar.arrive 1, %0;" ::"n"(kTM) : "memory");   // do not hold the tile's other softmax warps
+        else asm volatile("bar.arrive 2, %0;" ::"n"(kTM) : "memory");
+      }
+    }
+  }
+  tc5_fence_before();
+  __syncthreads();
+  if (warp == 8) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+  }
+}
+
 constexpr int kSharedPassLayers = kPrefillSharedLayers;   // 3 x 128 + 2 x 64 columns = all of tensor memory
 constexpr int prefill_tcgen05_smem_bytes(int nv = 1) { return 2 * kTM * 128 + (2 + 2 * nv) * (2 * kTN * 128) + 128; }
 
@@ -1074,6 +1489,9 @@ cudaError_t configure_prefill_kernels() {
   e = cudaFuncSetAttribute(prefill_attend_tcgen05_kernel<true, 1>, cudaFuncAttributePreferredSharedMemoryCarveout,
                            cudaSharedmemCarveoutMaxShared);
   if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(prefill_attend_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           prefill_pair_smem_bytes());
+  if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(prefill_attend_tcgen05_kernel<false, kSharedPassLayers>,
                            cudaFuncAttributeMaxDynamicSharedMemorySize, prefill_tcgen05_smem_bytes(kSharedPassLayers));
   if (e != cudaSuccess) return e;
@@ -1086,7 +1504,7 @@ cudaError_t launch_prefill_attend(const Params& p, const uint8_t* kind_dev, cons
                                   int32_t T, int32_t gla, const PrefillMaps* maps,
                                   const uint8_t* tile_code_dev, int32_t seq_id, int32_t n0_text, int32_t n0_vis,
                                   const PrefillPass* passes_dev, int32_t n_single, int32_t n_shared,
-                                  cudaStream_t stream) {
+                                  int32_t pair_min_tokens, cudaStream_t stream) {
   if (T <= 0) return cudaSuccess;
   PrefillArgs a{};
   a.q = static_cast<const uint16_t*>(q);
@@ -1120,12 +1538,18 @@ cudaError_t launch_prefill_attend(const Params& p, const uint8_t* kind_dev, cons
     a.tmap_o = maps->out;
     a.tile_code = tile_code_dev;
     const dim3 grid5((T + kTM - 1) / kTM, p.hq, p.n_layers);
+    // prompts that start a sequence, from pair_min_tokens on: two query tiles per CTA, 128-key tiles
+    const bool pair = pair_min_tokens > 0 && T >= pair_min_tokens;
+    const dim3 gridp((T + 2 * kTM - 1) / (2 * kTM), p.hq, p.n_layers);
     if (n0_text + n0_vis > 0) {
       prefill_attend_tcgen05_kernel<true, 1><<<grid5, kTc5Threads, prefill_tcgen05_smem_bytes(), stream>>>(a, p.err);
     } else if (passes_dev && n_shared > 0) {
       // the layers that share nothing, then the shared-score passes (passes_dev lists them in that order)
       a.passes = passes_dev;
-      if (n_single > 0) {
+      if (n_single > 0 && pair) {
+        const dim3 g1(gridp.x, gridp.y, n_single);
+        prefill_attend_pair_kernel<<<g1, kPairThreads, prefill_pair_smem_bytes(), stream>>>(a, p.err);
+      } else if (n_single > 0) {
         const dim3 g1(grid5.x, grid5.y, n_single);
         prefill_attend_tcgen05_kernel<false, 1><<<g1, kTc5Threads, prefill_tcgen05_smem_bytes(), stream>>>(a, p.err);
       }
@@ -1133,6 +1557,8 @@ cudaError_t launch_prefill_attend(const Params& p, const uint8_t* kind_dev, cons
       const dim3 g3(grid5.x, grid5.y, n_shared);
       prefill_attend_tcgen05_kernel<false, kSharedPassLayers>
           <<<g3, kTc5Threads + 32, prefill_tcgen05_smem_bytes(kSharedPassLayers), stream>>>(a, p.err);
+    } else if (pair) {
+      prefill_attend_pair_kernel<<<gridp, kPairThreads, prefill_pair_smem_bytes(), stream>>>(a, p.err);
     } else {
       prefill_attend_tcgen05_kernel<false, 1><<<grid5, kTc5Threads, prefill_tcgen05_smem_bytes(), stream>>>(a, p.err);
     }

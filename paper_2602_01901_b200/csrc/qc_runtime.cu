@@ -94,6 +94,7 @@ struct qc_cache {
   std::vector<cudaEvent_t> ev_in, ev_done;
   bool prefill_tcgen05 = true;    // head_dim 128: tcgen05 kernel; otherwise (or when switched off) mma.sync kernel
   bool pool_map_ok = false;       // c->tmap was encoded
+  int prefill_pair_min_tokens = 0;   // prompts this long that start a sequence run two query tiles per CTA (0: never)
   int prefill_shared = 1;         // GLA prefill: layers of a block whose scores coincide share one score pass
                                   // (0 never, 1 for prompts of kPrefillShareMinTokens or more, 2 always)
   std::vector<PrefillPass> prefill_passes;   // singles first, then shared passes (GLA only; else empty)
@@ -1029,7 +1030,7 @@ int32_t qc_prefill_attend(qc_cache* c, int32_t seq_id, int32_t n_tokens, const u
   QC_CUDA(launch_prefill_attend(p, kind_dev, c->ws + c->lay.layer_kind, c->ws + c->lay.leader, q_dev, k_dev, v_dev,
                                 out_dev, n_tokens, c->cfg.lazy_mode == QC_MODE_GLA ? 1 : 0, tc5 ? &maps : nullptr,
                                 codes_dev, seq_id, n0_text, n0_vis, (tc5 && share) ? passes_dev : nullptr,
-                                c->prefill_n_single, c->prefill_n_shared, stream));
+                                c->prefill_n_single, c->prefill_n_shared, c->prefill_pair_min_tokens, stream));
   const bool shared_run = tc5 && share;
   if (ev) {
     QC_CUDA(cudaEventRecord(ev[1], stream));
@@ -1741,6 +1742,11 @@ int32_t qc_set_option(qc_cache* c, const char* key, int64_t value) {
   if (k == "prefill_shared_scores") {
     if (value < 0 || value > 2) return QC_ERR_INVALID_ARG;
     c->prefill_shared = static_cast<int>(value);
+    return QC_OK;
+  }
+  if (k == "prefill_pair_min_tokens") {
+    if (value < 0) return QC_ERR_INVALID_ARG;
+    c->prefill_pair_min_tokens = static_cast<int>(std::min<int64_t>(value, 1 << 30));
     return QC_OK;
   }
   if (k == "prefill_tcgen05") {

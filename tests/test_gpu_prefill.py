@@ -69,6 +69,45 @@ def test_prefill_attend_small(mode, case):
     s.close()
 
 
+PAIR_CASES = [
+    # (group, layer_kind, n_text_before, n_visual, n_text_after): head_dim 128, two query tiles per CTA
+    (1, [0, 1, 0, 1, 1], 5, 150, 22),            # 177 tokens: one pair, second tile ragged
+    (7, [0, 1], 9, 40, 8),                       # 57 tokens: the second tile of the pair has no row
+    (2, [0, 1, 1, 0], 17, 290, 78),              # 385 tokens: two pairs, the last with one row in its first tile
+    (1, [0, 1], 3, 500, 9),                      # 512 tokens: two full pairs
+    (2, [0, 1, 1], 40, 0, 260),                  # text only, 300 tokens
+    (1, [0, 0, 1], 0, 700, 69),                  # 769 tokens: four pairs, starts with a visual token
+]
+
+
+@pytest.mark.parametrize("mode", MODES, ids=MODE_IDS)
+@pytest.mark.parametrize("case", range(len(PAIR_CASES)))
+def test_prefill_attend_two_query_tiles_per_cta_small(mode, case):
+    """The kernel for long prompts (two query tiles per CTA, 128-key tiles), forced onto short
+    prompts so that the oracle checks every row: ragged tails, a pair whose second tile is empty,
+    tiles that mix text and visual rows of a VLA lazy layer."""
+    group, layer_kind, nb, nv, na = PAIR_CASES[case]
+    D = 128
+    lazy = tuple(i for i, k in enumerate(layer_kind) if k)
+    w = W.Workload(70 + case, f"prefill_pair{case}", len(layer_kind), 2 * group, 2, D, 16, 2, nb, nv, nv, na, 4, lazy)
+    s = Session.for_workload(w, lazy_mode=mode, poison_pool=True)
+    s.set_option("prefill_pair_min_tokens", 1)
+    s.set_option("prefill_shared_scores", 0)
+    for b in range(w.batch):
+        kind, k, v = W.prefill_kv_np(w, b)
+        q = W.prefill_q_np(w, b)
+        out = torch.full((w.n_layers, len(kind), w.n_q_heads, D), float("nan"), dtype=torch.bfloat16, device=s.device)
+        s.prefill_attend(b, kind, _dev(q, s.device), _dev(k, s.device), _dev(v, s.device), out)
+        torch.cuda.synchronize()
+        assert s.stats().device_error == 0
+        ref = OP.prefill_lazy_attention(f64(q), f64(k), f64(v), kind, layer_kind, mode)
+        got = bits_of(out)
+        for l in range(w.n_layers):
+            for t0 in range(0, len(kind), 64):
+                assert_close(got[l, t0:t0 + 64], ref[l, t0:t0 + 64], f"pair case {case} seq {b} layer {l} tokens {t0}..")
+    s.close()
+
+
 @pytest.mark.parametrize("name,mode", [("llava15_7b", qc.QC_MODE_VLA_QC), ("llava15_7b", qc.QC_MODE_GLA),
                                        ("qwen2vl_gqa", qc.QC_MODE_VLA_QC), ("qwen2vl_gqa", qc.QC_MODE_GLA),
                                        ("llava_next_2048_lazy22", qc.QC_MODE_GLA)],
