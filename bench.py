@@ -677,7 +677,10 @@ def main():
             "impl": "reference", "metric": METRIC, "value": base["value"], "unit": UNIT, "n_gpus": ranks,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * w.batch / base["value"],
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": w.name, "mode": args.mode, "batch_per_gpu": w.batch},
+            "config": {"workload": w.name, "mode": args.mode, "schedule": "oracle (one layer, sequence and head at a time)",
+                       "batch_per_gpu": w.batch, "n_layers": w.n_layers, "lazy_layers": len(w.lazy_layers),
+                       "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads, "head_dim": w.head_dim,
+                       "page_tokens": w.page_size, "arithmetic": "fp64"},
             "cpu_baseline": base,
             "e2e": {"value": base["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "wall_s": time.perf_counter() - t0,
