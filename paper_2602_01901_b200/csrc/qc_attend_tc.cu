@@ -465,7 +465,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
   }
   __syncthreads();
 
-  attend_tc_worker<D, STATIC>(P, ctx, ring, full, &cursors[warp], stages[warp], warp * gridDim.x + blockIdx.x, lane);
+  attend_tc_worker<D, STATIC>(P, ctx, ring, full, &cursors[warp], stages[warp], worker_index(P, warp, kWarps), lane);
 }
 
 template <int D>
@@ -494,7 +494,7 @@ cudaError_t configure_kernels_tc(int* attend_smem) {
 cudaError_t launch_attend_tc(const Params& p, int n_sms, cudaStream_t stream) {
   const int n_items = p.item_end - p.item_begin;
   if (!p.part_static && n_items <= 0) return cudaSuccess;
-  const int grid = p.part_static ? min(n_sms, p.part_workers) : min(n_sms, (n_items + kWarps - 1) / kWarps);
+  const int grid = min(n_sms, ((p.part_static ? p.part_workers : n_items) + kWarps - 1) / kWarps);
   if (p.d == 128) {
     if (p.part_static)
       return launch_pdl(attend_tc_kernel<128, true>, dim3(grid), dim3(kThreads), attend_tc_smem_bytes<128>(), stream, p);

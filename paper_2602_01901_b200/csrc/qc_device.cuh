@@ -709,6 +709,16 @@ __device__ __forceinline__ bool load_worker_desc(const Params& P, int wid, ItemP
   return true;
 }
 
+// Which worker of a launch a warp is.  Under the static partition the warps of a CTA are adjacent
+// workers (adjacent ranges: the same rows, page-table lines and queries), and a launch with fewer
+// workers than warps fills the first CTAs and leaves the other SMs to the next launch's early
+// part.  Measured against one worker of every CTA first (same call, in-order step): config 2
+// 1.117 -> 1.078 ms, configs 3 / 4 / 5 within 0.6 %; runs of adjacent workers spread over all CTAs: 1.092.
+__device__ __forceinline__ int worker_index(const Params& P, int warp, int warps_per_cta) {
+  if (!P.part_static) return warp * gridDim.x + blockIdx.x;
+  return static_cast<int>(blockIdx.x) * warps_per_cta + warp;
+}
+
 // Under the static partition, the piece that holds a row's first page records how many pieces
 // the row has: one entry per consumer layer and query head, visual and text streams side by side.
 __device__ __forceinline__ void record_row_slots(const Params& P, const Item& it, int lane) {

@@ -632,7 +632,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_kernel(const __grid_consta
   }
   __syncthreads();
 
-  attend_worker<D, STATIC>(P, ctx, ring, full, &cursors[warp], stages[warp], warp * gridDim.x + blockIdx.x, lane);
+  attend_worker<D, STATIC>(P, ctx, ring, full, &cursors[warp], stages[warp], worker_index(P, warp, kWarps), lane);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -799,7 +799,7 @@ cudaError_t launch_attend(const Params& p, int n_sms, cudaStream_t stream) {
   const int n_items = p.item_end - p.item_begin;
   if (!p.part_static && n_items <= 0) return cudaSuccess;
   // static ranges: worker w is warp w / grid of CTA w % grid, so a launch with few workers still uses every SM
-  const int grid = p.part_static ? min(n_sms, p.part_workers) : min(n_sms, (n_items + kWarps - 1) / kWarps);
+  const int grid = min(n_sms, ((p.part_static ? p.part_workers : n_items) + kWarps - 1) / kWarps);
   if (p.d == 128) {
     if (p.part_static)
       return launch_pdl(attend_kernel<128, true>, dim3(grid), dim3(kThreads), attend_smem_bytes<128>(), stream, p);
