@@ -38,7 +38,7 @@ MODES = {"vla_qc": 0, "vla_eq8": 1, "gla": 2}
 # 181-257 MB for the MHA kernel, 74-107 MB for the GQA kernel).  Every tile is fetched once and the
 # partial rows are written once per piece, so traffic grows in proportion to the K/V bytes swept and a
 # full-size launch's traffic is this ratio times its algorithmic bytes.
-NCU_TRAFFIC_RATIO = {"attend_kernel": 1.031, "attend_tc_kernel": 1.059}
+NCU_TRAFFIC_RATIO = {"attend_kernel": 1.028, "attend_tc_kernel": 1.057}
 
 
 def _peaks():
