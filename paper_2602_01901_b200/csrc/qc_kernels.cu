@@ -644,8 +644,10 @@ __global__ void __launch_bounds__(kThreads, 1) attend_kernel(const __grid_consta
 // rounds of loads (counts, then (max, sum) pairs, then rows).  When a row has at most 16 partials
 // per stream (the common case: a launch per layer leaves a handful) everything is requested in
 // one round instead: the counts, the pairs of the first 16 slots of either stream (lanes 0..15 /
-// 16..31) and the first four rows of either stream, whether written or not; what the counts then
-// rule out is ignored.  The step's sequence descriptor is read ahead of the wait for the
+// 16..31) and the first rows (up to four) of either stream that a guess at the counts names; what
+// the counts then rule out is ignored, and what they add beyond four is one more round per stream
+// (eight visual rows in the first round were measured slower: rows never written are not in the
+// L2).  The step's sequence descriptor is read ahead of the wait for the
 // attention kernel (it was written when the step began).
 template <int D>
 __global__ void merge_kernel(const __grid_constant__ Params P) {
@@ -659,36 +661,49 @@ __global__ void merge_kernel(const __grid_constant__ Params P) {
   const int layer = P.layer_begin + idx / (P.hq * P.n_seqs);
   StepSeq sq{};
   if (live) sq = P.seqs[si];
+  const bool fast = P.part_static && P.extra_key_leader < 0 && P.slots_per_stream >= 4;
+  const size_t row = (static_cast<size_t>(layer) * P.max_seqs + si) * P.hq + head;
+  // A guess at the row's piece counts, read while the attention kernel may still run: its workers
+  // record the counts when they start a row, and the entry keeps the previous step's counts until
+  // then, which are nearly always the same.  The guess only decides which rows the first round of
+  // loads asks for (rows never written are not in the L2); the counts used are read after the wait.
+  uint32_t guess = 0;
+  if (live && fast) guess = __ldcg(reinterpret_cast<const uint32_t*>(P.row_slots + 2 * row));
   pdl_wait();
   pdl_launch_dependents();
   if (!live) return;
-  if (!P.part_static || P.extra_key_leader >= 0 || P.slots_per_stream < 4) {
+  if (!fast) {
     merge_row<D>(P, layer, si, head, sq, lane, P.extra_key_leader);
     return;
   }
   const int S = P.slots_per_stream;
-  const size_t row = (static_cast<size_t>(layer) * P.max_seqs + si) * P.hq + head;
   const size_t base = (static_cast<size_t>(layer) * P.max_seqs + si) * P.max_slots;
   const uint32_t both = __ldcg(reinterpret_cast<const uint32_t*>(P.row_slots + 2 * row));
   const int my_slot = lane < 16 ? lane : S + lane - 16;
   float2 my_ml = make_float2(-INFINITY, 0.f);
   if ((lane & 15) < S) my_ml = __ldcg(P.part_ml + (base + my_slot) * P.hq + head);
-  float v[8][VPL];   // rows of visual slots 0..3 and text slots 0..3
+  const int gv = min(static_cast<int>(guess & 0xffffu), 4), gt = min(static_cast<int>(guess >> 16), 4);
+  float v[8][VPL];   // rows of visual slots 0..3 and text slots 0..3, as far as the guess goes
 #pragma unroll
   for (int u = 0; u < 8; ++u) {
     const int s = u < 4 ? u : S + u - 4;
     const float* src = P.part_acc + ((base + s) * P.hq + head) * D + lane * VPL;
-    if (VPL == 4) {
-      const float4 a = __ldcg(reinterpret_cast<const float4*>(src));
-      v[u][0] = a.x, v[u][1] = a.y, v[u][2 % VPL] = a.z, v[u][3 % VPL] = a.w;
+    if ((u < 4 ? u : u - 4) < (u < 4 ? gv : gt)) {
+      if (VPL == 4) {
+        const float4 a = __ldcg(reinterpret_cast<const float4*>(src));
+        v[u][0] = a.x, v[u][1] = a.y, v[u][2 % VPL] = a.z, v[u][3 % VPL] = a.w;
+      } else {
+        const float2 a = __ldcg(reinterpret_cast<const float2*>(src));
+        v[u][0] = a.x, v[u][1] = a.y;
+      }
     } else {
-      const float2 a = __ldcg(reinterpret_cast<const float2*>(src));
-      v[u][0] = a.x, v[u][1] = a.y;
+#pragma unroll
+      for (int e = 0; e < VPL; ++e) v[u][e] = 0.f;
     }
   }
   const int nv = sq.len_vis > 0 ? static_cast<int>(both & 0xffffu) : 0;
   const int nt = static_cast<int>(both >> 16);
-  if (nv > 16 || nt > 16) {
+  if (nv > 16 || nt > 16 || min(nv, 4) > gv || min(nt, 4) > gt) {   // more pieces than guessed: the general path
     merge_row<D>(P, layer, si, head, sq, lane, -1);
     return;
   }
@@ -712,14 +727,17 @@ __global__ void merge_kernel(const __grid_constant__ Params P) {
       for (int e = 0; e < VPL; ++e) acc[e] = fmaf(v[u][e], w, acc[e]);
     }
   }
-  // rows beyond the first four of a stream: four of either stream per round of loads
-  for (int s0 = 4; s0 < max(nv, nt); s0 += 4) {
-    float r[8][VPL];
+  // rows beyond the first four of a stream: the rest of one stream per round of loads (at most 16
+  // per stream here), so a row cut into many pieces costs two rounds, not one per four pieces
+#pragma unroll 1
+  for (int t = 0; t < 2; ++t) {
+    const int n = t ? nt : nv, first = 4;
+    if (n <= first) continue;
+    float r[12][VPL];
 #pragma unroll
-    for (int u = 0; u < 8; ++u) {
-      const int s = s0 + (u & 3), t = u >> 2;
-      const bool have = s < (t ? nt : nv);
-      const float* src = P.part_acc + ((base + (t ? S : 0) + (have ? s : 0)) * P.hq + head) * D + lane * VPL;
+    for (int u = 0; u < 12; ++u) {
+      const int s = first + u;
+      const float* src = P.part_acc + ((base + (t ? S : 0) + (s < n ? s : 0)) * P.hq + head) * D + lane * VPL;
       if (VPL == 4) {
         const float4 a = __ldcg(reinterpret_cast<const float4*>(src));
         r[u][0] = a.x, r[u][1] = a.y, r[u][2 % VPL] = a.z, r[u][3 % VPL] = a.w;
@@ -729,10 +747,10 @@ __global__ void merge_kernel(const __grid_constant__ Params P) {
       }
     }
 #pragma unroll
-    for (int u = 0; u < 8; ++u) {
-      const int s = s0 + (u & 3), t = u >> 2;
+    for (int u = 0; u < 12; ++u) {
+      const int s = first + u;
       const float w = __shfl_sync(0xffffffffu, my_w, (t ? 16 : 0) + (s & 15));
-      if (s < (t ? nt : nv) && w > 0.f) {
+      if (s < n && w > 0.f) {
 #pragma unroll
         for (int e = 0; e < VPL; ++e) acc[e] = fmaf(r[u][e], w, acc[e]);
       }
