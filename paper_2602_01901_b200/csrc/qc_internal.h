@@ -88,7 +88,8 @@ struct Patch {
 // Static partition of one attention launch, as the kernel that plans a step ahead needs it.
 struct LaunchDesc {
   int32_t pos_begin, pos_end;
-  int32_t part_q, part_k, part_vw, part_workers, part_row_cost, pad;
+  int32_t part_q, part_k, part_vw, part_workers, part_row_cost;
+  int32_t merge_wide;   // a row of the launch may leave more than four partial rows of its visual stream
 };
 static_assert(sizeof(LaunchDesc) == 32, "LaunchDesc layout");
 constexpr int kMaxPlanLaunches = 128;   // launches of a step that can be planned ahead (a launch per layer fits)
@@ -167,6 +168,7 @@ struct Params {
                                      // Q Cache) are taken from the step's inputs by the attention worker (or the
                                      // merge warp) that meets the end of the layer's text stream, which also stores
                                      // them: no append launch, nothing of a layer is touched before its own launch
+  int32_t merge_wide;                // merge: rows may have more than four partial rows of the visual stream
   int32_t debug_drop_tile;           // test hook: every worker of an attention launch leaves out the copy of its first
                                      // tile and waits for it with a short limit (nothing in flight, nothing faults)
   int32_t extra_key_leader;          // merge only, >= 0: the rows also take the step's new token as one more key,

@@ -644,12 +644,15 @@ __global__ void __launch_bounds__(kThreads, 1) attend_kernel(const __grid_consta
 // rounds of loads (counts, then (max, sum) pairs, then rows).  When a row has at most 16 partials
 // per stream (the common case: a launch per layer leaves a handful) everything is requested in
 // one round instead: the counts, the pairs of the first 16 slots of either stream (lanes 0..15 /
-// 16..31) and the first rows (up to four) of either stream that a guess at the counts names; what
-// the counts then rule out is ignored, and what they add beyond four is one more round per stream
+// 16..31) and the rows that a guess at the counts names (up to 4 or 16 of the visual stream, 4 of the
+// text stream); what the counts then rule out is ignored, rows beyond those take one more round
 // (eight visual rows in the first round were measured slower: rows never written are not in the
 // L2).  The step's sequence descriptor is read ahead of the wait for the
 // attention kernel (it was written when the step began).
-template <int D>
+// NVIS = 0: the general path alone (few registers: a launch per step merges every layer's rows);
+// NVIS = 4 / 16: the one-round path with up to NVIS visual rows in the first round (the host knows
+// from the partition whether a row of the launch can leave more than four).
+template <int D, int NVIS>
 __global__ void merge_kernel(const __grid_constant__ Params P) {
   constexpr int VPL = D / 32;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -661,34 +664,34 @@ __global__ void merge_kernel(const __grid_constant__ Params P) {
   const int layer = P.layer_begin + idx / (P.hq * P.n_seqs);
   StepSeq sq{};
   if (live) sq = P.seqs[si];
-  const bool fast = P.part_static && P.extra_key_leader < 0 && P.slots_per_stream >= 4;
   const size_t row = (static_cast<size_t>(layer) * P.max_seqs + si) * P.hq + head;
   // A guess at the row's piece counts, read while the attention kernel may still run: its workers
   // record the counts when they start a row, and the entry keeps the previous step's counts until
   // then, which are nearly always the same.  The guess only decides which rows the first round of
   // loads asks for (rows never written are not in the L2); the counts used are read after the wait.
   uint32_t guess = 0;
-  if (live && fast) guess = __ldcg(reinterpret_cast<const uint32_t*>(P.row_slots + 2 * row));
+  if (NVIS > 0 && live) guess = __ldcg(reinterpret_cast<const uint32_t*>(P.row_slots + 2 * row));
   pdl_wait();
   pdl_launch_dependents();
   if (!live) return;
-  if (!fast) {
+  if (NVIS == 0) {
     merge_row<D>(P, layer, si, head, sq, lane, P.extra_key_leader);
     return;
   }
+  constexpr int NV1 = NVIS > 0 ? NVIS : 1;   // visual rows of the first round
   const int S = P.slots_per_stream;
   const size_t base = (static_cast<size_t>(layer) * P.max_seqs + si) * P.max_slots;
   const uint32_t both = __ldcg(reinterpret_cast<const uint32_t*>(P.row_slots + 2 * row));
   const int my_slot = lane < 16 ? lane : S + lane - 16;
   float2 my_ml = make_float2(-INFINITY, 0.f);
   if ((lane & 15) < S) my_ml = __ldcg(P.part_ml + (base + my_slot) * P.hq + head);
-  const int gv = min(static_cast<int>(guess & 0xffffu), 4), gt = min(static_cast<int>(guess >> 16), 4);
-  float v[8][VPL];   // rows of visual slots 0..3 and text slots 0..3, as far as the guess goes
+  const int gv = min(min(static_cast<int>(guess & 0xffffu), NV1), S), gt = min(static_cast<int>(guess >> 16), 4);
+  float v[NV1 + 4][VPL];   // rows of visual slots 0..NV1-1 and text slots 0..3, as far as the guess goes
 #pragma unroll
-  for (int u = 0; u < 8; ++u) {
-    const int s = u < 4 ? u : S + u - 4;
+  for (int u = 0; u < NV1 + 4; ++u) {
+    const int s = u < NV1 ? u : S + u - NV1;
     const float* src = P.part_acc + ((base + s) * P.hq + head) * D + lane * VPL;
-    if ((u < 4 ? u : u - 4) < (u < 4 ? gv : gt)) {
+    if ((u < NV1 ? u : u - NV1) < (u < NV1 ? gv : gt)) {
       if (VPL == 4) {
         const float4 a = __ldcg(reinterpret_cast<const float4*>(src));
         v[u][0] = a.x, v[u][1] = a.y, v[u][2 % VPL] = a.z, v[u][3 % VPL] = a.w;
@@ -703,7 +706,7 @@ __global__ void merge_kernel(const __grid_constant__ Params P) {
   }
   const int nv = sq.len_vis > 0 ? static_cast<int>(both & 0xffffu) : 0;
   const int nt = static_cast<int>(both >> 16);
-  if (nv > 16 || nt > 16 || min(nv, 4) > gv || min(nt, 4) > gt) {   // more pieces than guessed: the general path
+  if (nv > 16 || nt > 16 || min(nv, NV1) > gv || min(nt, 4) > gt) {   // more pieces than guessed (or than this path holds)
     merge_row<D>(P, layer, si, head, sq, lane, -1);
     return;
   }
@@ -720,18 +723,18 @@ __global__ void merge_kernel(const __grid_constant__ Params P) {
 #pragma unroll
   for (int e = 0; e < VPL; ++e) acc[e] = 0.f;
 #pragma unroll
-  for (int u = 0; u < 8; ++u) {
-    const float w = __shfl_sync(0xffffffffu, my_w, u < 4 ? u : 12 + u);   // lanes 0..3 and 16..19
+  for (int u = 0; u < NV1 + 4; ++u) {
+    const float w = __shfl_sync(0xffffffffu, my_w, u < NV1 ? u : 16 + u - NV1);   // lanes 0..15: visual slots, 16..: text slots
     if (w > 0.f) {
 #pragma unroll
       for (int e = 0; e < VPL; ++e) acc[e] = fmaf(v[u][e], w, acc[e]);
     }
   }
-  // rows beyond the first four of a stream: the rest of one stream per round of loads (at most 16
-  // per stream here), so a row cut into many pieces costs two rounds, not one per four pieces
+  // rows beyond the first round's (visual rows past NV1, text rows past four): the rest of a stream
+  // in one more round of loads
 #pragma unroll 1
-  for (int t = 0; t < 2; ++t) {
-    const int n = t ? nt : nv, first = 4;
+  for (int t = (NV1 >= 16 ? 1 : 0); t < 2; ++t) {
+    const int n = t ? nt : nv, first = t ? 4 : NV1;
     if (n <= first) continue;
     float r[12][VPL];
 #pragma unroll
@@ -833,9 +836,17 @@ cudaError_t launch_merge(const Params& p, cudaStream_t stream) {
   if (n <= 0) return cudaSuccess;
   const int warps_per_block = 8;
   const int blocks = (n + warps_per_block - 1) / warps_per_block;
-  if (p.d == 128)
-    return launch_pdl(merge_kernel<128>, dim3(blocks), dim3(warps_per_block * 32), 0, stream, p);
-  return launch_pdl(merge_kernel<64>, dim3(blocks), dim3(warps_per_block * 32), 0, stream, p);
+  const dim3 grid(blocks), block(warps_per_block * 32);
+  // the one-round path needs the recorded piece counts of the static partition and no extra key
+  const bool one_round = p.part_static && p.extra_key_leader < 0 && p.slots_per_stream >= 4;
+  if (p.d == 128) {
+    if (!one_round) return launch_pdl(merge_kernel<128, 0>, grid, block, 0, stream, p);
+    if (p.merge_wide) return launch_pdl(merge_kernel<128, 16>, grid, block, 0, stream, p);
+    return launch_pdl(merge_kernel<128, 4>, grid, block, 0, stream, p);
+  }
+  if (!one_round) return launch_pdl(merge_kernel<64, 0>, grid, block, 0, stream, p);
+  if (p.merge_wide) return launch_pdl(merge_kernel<64, 16>, grid, block, 0, stream, p);
+  return launch_pdl(merge_kernel<64, 4>, grid, block, 0, stream, p);
 }
 
 cudaError_t launch_prefill_scatter(const Params& p, const int32_t* tok_seq, const int32_t* tok_stream,

@@ -1139,6 +1139,7 @@ int run_group(qc_cache* c, Params& p, size_t gi, const LaunchList& launches, boo
     p.part_vw = one.part_vw;
     p.part_workers = one.part_workers;
     p.part_row_cost = one.part_row_cost;
+    p.merge_wide = one.merge_wide;
     p.part_tiles = 0;
   }
   if (wait_in) QC_CUDA(cudaStreamWaitEvent(stream, wait_in, 0));
@@ -1396,6 +1397,7 @@ int decode_step_core(qc_cache* c, int32_t n_seqs, const int32_t* seq_ids, const 
     L.part_k = static_cast<int32_t>(k);
     L.part_workers = static_cast<int32_t>((vw + k - 1) / k);
     L.part_q = static_cast<int32_t>(q);
+    L.merge_wide = (static_cast<int64_t>(pmax_v) * g.w_max_v + q - 1) / q + 1 > 4 ? 1 : 0;
     return L;
   };
   LaunchList launches;
