@@ -300,20 +300,24 @@ class _Arms:
     def run_host(self, n):
         """n steps through qc_decode_step_host with pinned host buffers; returns tokens/s inputs."""
         torch = self.torch
-        dev_in = _gen_inputs(self.w, self.step, n, self.dev, self.seq_offset)
+        warm = 3   # untimed: the entry point's launch plan, copy streams and events are made on its first call
+        dev_in = _gen_inputs(self.w, self.step, warm + n, self.dev, self.seq_offset)
         host_in = [tuple(t.cpu().pin_memory() for t in step) for step in dev_in]
         host_out = torch.empty(self.out.shape, dtype=torch.bfloat16).pin_memory()
         del dev_in
+        for i in range(warm):
+            self.s.decode_step_host(self.ids, *host_in[i], host_out)
         self.barrier()
         g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         g0.record()
-        for i in range(n):
+        for i in range(warm, warm + n):
             self.s.decode_step_host(self.ids, *host_in[i], host_out)   # returns after the copy back has finished
         g1.record()
         self.barrier()
         ms = self.group.max_over_ranks(g0.elapsed_time(g1)) / n
-        self.step += n
-        return {"ms_per_step": ms, "h2d": sum(t.numel() * 2 for t in host_in[0]), "d2h": host_out.numel() * 2}
+        self.step += warm + n
+        return {"ms_per_step": ms, "h2d": sum(t.numel() * 2 for t in host_in[0]), "d2h": host_out.numel() * 2,
+                "context_first": self.w.n_prompt + self.step - n + 1, "context_last": self.w.n_prompt + self.step}
 
     def check_output(self):
         checksum = float(self.out.float().abs().sum().item())
@@ -355,6 +359,7 @@ def measure_workload(args, w, mode, group, local_rank, world, rank, K, W_, Ke, e
     prof = kp["prof"]
     n_launch = max(1, prof.attend_kernel_launches)
     kernel_gbs = prof.kv_bytes_read / (prof.attend_kernel_ms / 1e3) / 1e9
+    host = a.run_host(Ke)                       # next to the headline steps: nearly the same contexts
     a.set(ONE_LAUNCH)
     a.run(3, timed=False)
     one = a.run(K)
@@ -384,9 +389,6 @@ def measure_workload(args, w, mode, group, local_rank, world, rank, K, W_, Ke, e
             "context": [lc["context_first"], lc["context_last"]],
             "note": "the in-order step through qc_decode_begin + one qc_decode_layer per layer (each call gets only "
                     "that layer's q/k/v and also appends them: one more small launch per layer)"}
-    a.set(IN_ORDER)
-    a.run(3, timed=False)
-    host = a.run_host(Ke)
     st = a.close()
     tokens = w.batch * world
     res = {
@@ -407,7 +409,8 @@ def measure_workload(args, w, mode, group, local_rank, world, rank, K, W_, Ke, e
                        "kernel_gb_per_s": one_gbs, "frac": one_gbs / peak, "context": [one["context_first"], one["context_last"]],
                        "note": "all layers in one attention launch: needs every layer's q/k/v before the step starts"},
         "e2e": {"value": tokens / (host["ms_per_step"] / 1e3), "unit": UNIT, "h2d_bytes_per_step": host["h2d"],
-                "d2h_bytes_per_step": host["d2h"], "steps": Ke, "ms_per_step": host["ms_per_step"]},
+                "d2h_bytes_per_step": host["d2h"], "steps": Ke, "ms_per_step": host["ms_per_step"],
+                "context": [host["context_first"], host["context_last"]]},
         "kv_saved": {"token_exact": 1 - st.kv_bytes_stored / st.kv_bytes_all_full,
                      "paged": 1 - st.kv_bytes_stored_paged / st.kv_bytes_all_full_paged,
                      "bytes_stored": st.kv_bytes_stored, "bytes_all_full": st.kv_bytes_all_full,

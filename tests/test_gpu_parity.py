@@ -529,6 +529,10 @@ FULL_CASES = [
     ("llava15_7b", qc.QC_MODE_GLA, 16, "in_order"),
     ("llava_next_2048_lazy22", qc.QC_MODE_GLA, 16, "in_order"),
     ("llava_next_2048_lazy22", qc.QC_MODE_VLA_QC, 16, "in_order"),
+    # the host-buffer entry point (four launch groups of lazy blocks, copies overlapped)
+    ("llava15_7b", qc.QC_MODE_VLA_QC, 16, "host"),
+    ("qwen2vl_gqa", qc.QC_MODE_GLA, 16, "host"),
+    ("long_video_pruned", qc.QC_MODE_VLA_QC, 16, "host"),
 ]
 
 
@@ -557,9 +561,17 @@ def test_full_size_sampled(case):
     bi = torch.tensor([t[1] for t in samples], device=s.device)
     hi = torch.tensor([t[2] for t in samples], device=s.device)
     worst = (0.0, 0.0)
+    if launches == "host":
+        h_out = torch.empty(out.shape, dtype=torch.bfloat16).pin_memory()
+        h_lse = torch.empty(lse.shape, dtype=torch.float32).pin_memory()
     for step in range(w.decode_steps):
         q, k, v = W.decode_qkv_torch(w, step, s.device)
-        s.decode_step(ids, q, k, v, out, lse)
+        if launches == "host":
+            s.decode_step_host(ids, q.cpu().pin_memory(), k.cpu().pin_memory(), v.cpu().pin_memory(), h_out, h_lse)
+            out.copy_(h_out)
+            lse.copy_(h_lse)
+        else:
+            s.decode_step(ids, q, k, v, out, lse)
         model.decode_step(list(range(w.batch)))
         refs = [o.advance() for o in oracles]
         if step in schedule:
